@@ -1,0 +1,442 @@
+// CPU oracle for the PrefixQuant W4A4KV4 inference path (static setting, "O2" of Table 1).
+//
+// THIS IS TEST INFRASTRUCTURE. It is a plain, slow, scalar restatement of what the path
+// computes, written from the paper; it shares no code with the CUDA library and nothing in
+// the product path may call it. Only the tests, the smoke check and the bench's CPU-baseline
+// legs load it.
+//
+// Conventions
+//   * bf16 / fp16 tensors are passed as raw uint16 bit patterns, decoded exactly to double.
+//   * All floating-point work is double, except weight quantization, where the decision that
+//     produces an integer code is taken in IEEE fp32 (division, round-half-even) because that
+//     is the precision the offline GPU kernel uses for the same decision.
+//   * Packed INT4: element 2j in the low nibble, element 2j+1 in the high nibble, two's
+//     complement, packed along the contraction (or head) dimension.
+//   * Threading is over independent rows only; arithmetic per row is strictly sequential.
+//
+// Pins (see tests/test_oracle_pins.py): H H^T = n I, rotation of unit vectors / all-ones,
+// involution, Parseval, comparison with a library-built Sylvester matrix product; quantizer
+// range / ties / idempotence / hand-worked Eq. (1) values; brute-force integer GEMM;
+// attention against closed forms and a library softmax-attention; RoPE against the complex
+// rotation form; RMSNorm and SwiGLU closed forms.
+// Readings fixed by the benchmark spec rather than the paper (symmetric max/7 scale,
+// round-half-even, low-nibble-first, 2048-wide blocks) are "parity unpinned by the paper".
+
+#include <algorithm>
+#include <atomic>
+#include <cfenv>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <functional>
+#include <thread>
+#include <vector>
+
+namespace {
+
+int g_threads = 0;
+
+int n_threads() {
+  if (g_threads > 0) return g_threads;
+  unsigned h = std::thread::hardware_concurrency();
+  return h == 0 ? 1 : static_cast<int>(h);
+}
+
+// Run fn(i) for i in [0, n) on the host cores; rows are independent, so no ordering matters.
+void parallel_rows(int64_t n, const std::function<void(int64_t)>& fn) {
+  int nt = static_cast<int>(std::min<int64_t>(n_threads(), n));
+  if (nt <= 1) {
+    for (int64_t i = 0; i < n; ++i) fn(i);
+    return;
+  }
+  std::atomic<int64_t> next{0};
+  std::vector<std::thread> pool;
+  for (int t = 0; t < nt; ++t)
+    pool.emplace_back([&] {
+      for (;;) {
+        int64_t i = next.fetch_add(1);
+        if (i >= n) break;
+        fn(i);
+      }
+    });
+  for (auto& th : pool) th.join();
+}
+
+double bf16_to_double(uint16_t b) {
+  uint32_t u = static_cast<uint32_t>(b) << 16;
+  float f;
+  std::memcpy(&f, &u, 4);
+  return static_cast<double>(f);
+}
+
+double fp16_to_double(uint16_t h) {
+  int sign = (h >> 15) & 1;
+  int exp = (h >> 10) & 0x1f;
+  int man = h & 0x3ff;
+  double v;
+  if (exp == 0)
+    v = std::ldexp(static_cast<double>(man), -24);
+  else if (exp == 31)
+    v = man ? NAN : INFINITY;
+  else
+    v = std::ldexp(static_cast<double>(man + 1024), exp - 25);
+  return sign ? -v : v;
+}
+
+// One rounding, double -> bf16, round-half-to-even (8 significant bits, fp32 exponent range).
+uint16_t double_to_bf16(double x) {
+  if (std::isnan(x)) return 0x7fc0;
+  uint16_t sign = std::signbit(x) ? 0x8000 : 0;
+  double a = std::fabs(x);
+  if (a == 0.0) return sign;
+  if (std::isinf(a)) return sign | 0x7f80;
+  int e = std::ilogb(a);
+  if (e < -126) e = -126;  // subnormal quantum
+  double q = std::ldexp(a, 7 - e);
+  double r = std::nearbyint(q);  // FE_TONEAREST: ties to even
+  double v = std::ldexp(r, e - 7);
+  float f = static_cast<float>(v);  // exact: v has <= 8 significant bits
+  if (std::isinf(f)) return sign | 0x7f80;
+  uint32_t u;
+  std::memcpy(&u, &f, 4);
+  return sign | static_cast<uint16_t>(u >> 16);
+}
+
+inline int clampi(long v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : static_cast<int>(v)); }
+
+inline int nib_get(const uint8_t* row, int64_t j) {
+  uint8_t b = row[j >> 1];
+  int n = (j & 1) ? (b >> 4) : (b & 0xf);
+  return n >= 8 ? n - 16 : n;
+}
+
+inline void nib_set(uint8_t* row, int64_t j, int code) {
+  uint8_t n = static_cast<uint8_t>(code & 0xf);
+  uint8_t& b = row[j >> 1];
+  if (j & 1)
+    b = static_cast<uint8_t>((b & 0x0f) | (n << 4));
+  else
+    b = static_cast<uint8_t>((b & 0xf0) | n);
+}
+
+// Rotation of one row (App. B "Details of Rotation"): y = x H_B / sqrt(B) on each contiguous
+// B-wide block, with the Sylvester-ordered matrix H[i][j] = (-1)^popcount(i & j), written as
+// the matrix product itself. B == 0 means "no rotation".
+void rotate_row(const double* x, double* y, int64_t K, int B) {
+  if (B == 0) {
+    for (int64_t j = 0; j < K; ++j) y[j] = x[j];
+    return;
+  }
+  const double norm = 1.0 / std::sqrt(static_cast<double>(B));
+  for (int64_t base = 0; base < K; base += B) {
+    for (int j = 0; j < B; ++j) {
+      double s = 0.0;
+      for (int i = 0; i < B; ++i) {
+        double v = x[base + i];
+        s += (__builtin_popcount(static_cast<unsigned>(i & j)) & 1) ? -v : v;
+      }
+      y[base + j] = s * norm;
+    }
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+void orc_set_threads(int n) { g_threads = n; }
+int orc_get_threads() { return n_threads(); }
+
+// ---- format helpers exposed for the tests --------------------------------------------------
+void orc_bf16_to_f64(const uint16_t* in, double* out, int64_t n) {
+  for (int64_t i = 0; i < n; ++i) out[i] = bf16_to_double(in[i]);
+}
+void orc_f64_to_bf16(const double* in, uint16_t* out, int64_t n) {
+  for (int64_t i = 0; i < n; ++i) out[i] = double_to_bf16(in[i]);
+}
+void orc_fp16_to_f64(const uint16_t* in, double* out, int64_t n) {
+  for (int64_t i = 0; i < n; ++i) out[i] = fp16_to_double(in[i]);
+}
+void orc_unpack_int4(const uint8_t* in, int8_t* out, int64_t rows, int64_t K) {
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t j = 0; j < K; ++j) out[r * K + j] = static_cast<int8_t>(nib_get(in + r * (K / 2), j));
+}
+void orc_pack_int4(const int8_t* in, uint8_t* out, int64_t rows, int64_t K) {
+  std::memset(out, 0, static_cast<size_t>(rows * (K / 2)));
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t j = 0; j < K; ++j) nib_set(out + r * (K / 2), j, in[r * K + j]);
+}
+
+// ---- rotation (App. B) -----------------------------------------------------------------------
+// x double [M,K] -> y double [M,K]; B = block width (power of two dividing K) or 0.
+void orc_rotate_f64(const double* x, double* y, int64_t M, int64_t K, int B) {
+  parallel_rows(M, [&](int64_t m) { rotate_row(x + m * K, y + m * K, K, B); });
+}
+
+// x bf16 [M,K] with row stride ldx (elements) -> y double [M,K].
+void orc_rotate_bf16(const uint16_t* x, int64_t ldx, double* y, int64_t M, int64_t K, int B) {
+  parallel_rows(M, [&](int64_t m) {
+    std::vector<double> xr(K);
+    for (int64_t j = 0; j < K; ++j) xr[j] = bf16_to_double(x[m * ldx + j]);
+    rotate_row(xr.data(), y + m * K, K, B);
+  });
+}
+
+// ---- static per-tensor activation scale (Table 1, O2; Sec. 3 "Dynamic and Static") -----------
+// s_a = fp32( max |fp32(y)| / 7 ) over rows >= row_begin of the rotated calibration batch:
+// rows below row_begin are the prefixed outlier tokens and never take part.
+float orc_calib_act_scale(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin) {
+  std::vector<double> rowmax(M, 0.0);
+  parallel_rows(M, [&](int64_t m) {
+    if (m < row_begin) return;
+    std::vector<double> xr(K), yr(K);
+    for (int64_t j = 0; j < K; ++j) xr[j] = bf16_to_double(x[m * ldx + j]);
+    rotate_row(xr.data(), yr.data(), K, B);
+    double mx = 0.0;
+    for (int64_t j = 0; j < K; ++j) mx = std::max(mx, std::fabs(static_cast<double>(static_cast<float>(yr[j]))));
+    rowmax[m] = mx;
+  });
+  double mx = 0.0;
+  for (int64_t m = row_begin; m < M; ++m) mx = std::max(mx, rowmax[m]);
+  if (mx == 0.0) return 1.0f;
+  return static_cast<float>(mx / 7.0);
+}
+
+// ---- activation quantization (Eq. 1, symmetric signed form) ---------------------------------
+// code = clamp(round_half_even(y / s_a), -8, 7), y the rotated row. Rows < row_begin are left
+// untouched. tie_dist (nullable, [M,K] float) receives |y/s_a - nearest half-integer|, the
+// distance of the pre-rounding value from the closest rounding tie.
+void orc_quant_act(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin, float s_a,
+                   uint8_t* xq, float* tie_dist) {
+  const double s = static_cast<double>(s_a);
+  parallel_rows(M, [&](int64_t m) {
+    if (m < row_begin) return;
+    std::vector<double> xr(K), yr(K);
+    for (int64_t j = 0; j < K; ++j) xr[j] = bf16_to_double(x[m * ldx + j]);
+    rotate_row(xr.data(), yr.data(), K, B);
+    uint8_t* out = xq + m * (K / 2);
+    for (int64_t j = 0; j < K; ++j) {
+      double r = yr[j] / s;
+      long c = std::lrint(std::nearbyint(r));
+      nib_set(out, j, clampi(c, -8, 7));
+      if (tie_dist) {
+        double f = r - std::floor(r);  // in [0,1)
+        tie_dist[m * K + j] = static_cast<float>(std::fabs(f - 0.5));
+      }
+    }
+  });
+}
+
+// Plain quantizer on double inputs, for pins: code = clamp(rne(v / s), -8, 7).
+void orc_quant_f64(const double* v, int64_t n, double s, int8_t* codes) {
+  for (int64_t i = 0; i < n; ++i) codes[i] = static_cast<int8_t>(clampi(std::lrint(std::nearbyint(v[i] / s)), -8, 7));
+}
+
+// ---- weight quantization: RTN, one scale per output channel (Table 1; Table 6 "RTN") --------
+// s_w[n] = fp32(max_k |W[n,k]|) / 7 in fp32 (1 if the row is all zero);
+// code = clamp(rint_fp32(W[n,k] / s_w[n]), -8, 7) with an fp32 IEEE division.
+void orc_quant_weights(const uint16_t* W, int64_t ldw, int64_t N, int64_t K, uint8_t* wq, float* s_w) {
+  parallel_rows(N, [&](int64_t n) {
+    float mx = 0.0f;
+    for (int64_t k = 0; k < K; ++k) mx = std::max(mx, std::fabs(static_cast<float>(bf16_to_double(W[n * ldw + k]))));
+    volatile float sv = (mx == 0.0f) ? 1.0f : mx / 7.0f;
+    float s = sv;
+    s_w[n] = s;
+    uint8_t* out = wq + n * (K / 2);
+    for (int64_t k = 0; k < K; ++k) {
+      float w = static_cast<float>(bf16_to_double(W[n * ldw + k]));
+      volatile float q = w / s;  // fp32 division, no double intermediate
+      float r = std::nearbyintf(q);
+      nib_set(out, k, clampi(static_cast<long>(r), -8, 7));
+    }
+  });
+}
+
+// ---- integer GEMM (Sec. 3: low-bit matrix multiplication) --------------------------------------
+// acc[t,n] = sum_k xq[t,k] * wq[n,k], accumulated in int64, returned as int32.
+// Returns 0, or 1 if any accumulator does not fit int32.
+int orc_gemm_i4(const uint8_t* xq, const uint8_t* wq, int64_t M, int64_t N, int64_t K, int32_t* acc) {
+  std::atomic<int> overflow{0};
+  std::vector<int8_t> w(static_cast<size_t>(N * K));
+  for (int64_t n = 0; n < N; ++n)
+    for (int64_t k = 0; k < K; ++k) w[n * K + k] = static_cast<int8_t>(nib_get(wq + n * (K / 2), k));
+  parallel_rows(M, [&](int64_t t) {
+    std::vector<int8_t> xr(K);
+    for (int64_t k = 0; k < K; ++k) xr[k] = static_cast<int8_t>(nib_get(xq + t * (K / 2), k));
+    for (int64_t n = 0; n < N; ++n) {
+      const int8_t* wr = w.data() + n * K;
+      int64_t s = 0;
+      for (int64_t k = 0; k < K; ++k) s += static_cast<int64_t>(xr[k]) * static_cast<int64_t>(wr[k]);
+      if (s > INT32_MAX || s < INT32_MIN) overflow = 1;
+      acc[t * N + n] = static_cast<int32_t>(s);
+    }
+  });
+  return overflow.load();
+}
+
+// Dequantization epilogue: out[t,n] = bf16( acc * s_a * s_w[n] ), product in double, one rounding.
+void orc_dequant_bf16(const int32_t* acc, int64_t M, int64_t N, float s_a, const float* s_w, uint16_t* out) {
+  parallel_rows(M, [&](int64_t t) {
+    for (int64_t n = 0; n < N; ++n)
+      out[t * N + n] =
+          double_to_bf16(static_cast<double>(acc[t * N + n]) * static_cast<double>(s_a) * static_cast<double>(s_w[n]));
+  });
+}
+
+// ---- per-head static KV scale and KV4 append (Table 1, O2: per-head static KV cache) ----------
+// kv bf16 [B,T,H,D]; s[h] = fp32(max |kv[:,:,h,:]|) / 7 in double then fp32 (1 if all zero).
+void orc_calib_kv_scale(const uint16_t* kv, int64_t B, int64_t T, int64_t H, int64_t D, float* s) {
+  for (int64_t h = 0; h < H; ++h) {
+    double mx = 0.0;
+    for (int64_t b = 0; b < B; ++b)
+      for (int64_t t = 0; t < T; ++t)
+        for (int64_t d = 0; d < D; ++d) mx = std::max(mx, std::fabs(bf16_to_double(kv[((b * T + t) * H + h) * D + d])));
+    s[h] = mx == 0.0 ? 1.0f : static_cast<float>(mx / 7.0);
+  }
+}
+
+// k, v bf16 [B,T_new,H,D] -> codes written at rows len[b] .. len[b]+T_new-1 of
+// kq, vq u8 [B,H,Tmax,D/2]; len[b] += T_new. Returns 1 (nothing written) if any sequence would
+// exceed Tmax.
+int orc_kv4_append(const uint16_t* k, const uint16_t* v, int64_t B, int64_t T_new, int64_t H, int64_t D,
+                   const float* s_k, const float* s_v, uint8_t* kq, uint8_t* vq, int32_t* len, int64_t Tmax) {
+  for (int64_t b = 0; b < B; ++b)
+    if (len[b] + T_new > Tmax) return 1;
+  for (int64_t b = 0; b < B; ++b) {
+    for (int64_t t = 0; t < T_new; ++t)
+      for (int64_t h = 0; h < H; ++h) {
+        int64_t pos = len[b] + t;
+        uint8_t* kr = kq + ((b * H + h) * Tmax + pos) * (D / 2);
+        uint8_t* vr = vq + ((b * H + h) * Tmax + pos) * (D / 2);
+        for (int64_t d = 0; d < D; ++d) {
+          double kv = bf16_to_double(k[((b * T_new + t) * H + h) * D + d]);
+          double vv = bf16_to_double(v[((b * T_new + t) * H + h) * D + d]);
+          nib_set(kr, d, clampi(std::lrint(std::nearbyint(kv / static_cast<double>(s_k[h]))), -8, 7));
+          nib_set(vr, d, clampi(std::lrint(std::nearbyint(vv / static_cast<double>(s_v[h]))), -8, 7));
+        }
+      }
+    len[b] += static_cast<int32_t>(T_new);
+  }
+  return 0;
+}
+
+// ---- attention over [full-precision prefix || INT4 cache] (Eq. 3) -------------------------------
+// One (query row, head) of softmax attention in double over the union of
+//   n_prefix prefix keys/values (fp16, [Hkv, n_prefix, D], one copy shared by every sequence) and
+//   n_ctx quantized keys/values (codes * per-head scale).
+static void attend_one(const double* q, int64_t D, double sm_scale, const uint16_t* pk, const uint16_t* pv,
+                       int64_t n_prefix, const uint8_t* kq, const uint8_t* vq, int64_t n_ctx, double sk, double sv,
+                       double* out) {
+  int64_t n = n_prefix + n_ctx;
+  std::vector<double> sc(n);
+  for (int64_t j = 0; j < n; ++j) {
+    double s = 0.0;
+    if (j < n_prefix)
+      for (int64_t d = 0; d < D; ++d) s += q[d] * fp16_to_double(pk[j * D + d]);
+    else
+      for (int64_t d = 0; d < D; ++d) s += q[d] * (nib_get(kq + (j - n_prefix) * (D / 2), d) * sk);
+    sc[j] = s * sm_scale;
+  }
+  double mx = -INFINITY;
+  for (int64_t j = 0; j < n; ++j) mx = std::max(mx, sc[j]);
+  double den = 0.0;
+  for (int64_t j = 0; j < n; ++j) {
+    sc[j] = std::exp(sc[j] - mx);
+    den += sc[j];
+  }
+  for (int64_t d = 0; d < D; ++d) out[d] = 0.0;
+  for (int64_t j = 0; j < n; ++j) {
+    double p = sc[j] / den;
+    if (j < n_prefix)
+      for (int64_t d = 0; d < D; ++d) out[d] += p * fp16_to_double(pv[j * D + d]);
+    else
+      for (int64_t d = 0; d < D; ++d) out[d] += p * (nib_get(vq + (j - n_prefix) * (D / 2), d) * sv);
+  }
+}
+
+// Decode: one query token per sequence, every cached key visible.
+// q bf16 [B,Hq,D]; prefix_k/v fp16 [Hkv,n_prefix,D]; kq/vq u8 [B,Hkv,Tmax,D/2]; len int32 [B];
+// out bf16 [B,Hq,D]; out_f64 (nullable) receives the unrounded result.
+void orc_decode_attn(const uint16_t* q, const uint16_t* prefix_k, const uint16_t* prefix_v, const uint8_t* kq,
+                     const uint8_t* vq, const float* s_k, const float* s_v, const int32_t* len, int64_t B, int64_t Hq,
+                     int64_t Hkv, int64_t D, int64_t n_prefix, int64_t Tmax, double sm_scale, uint16_t* out,
+                     double* out_f64) {
+  int64_t group = Hq / Hkv;
+  parallel_rows(B * Hq, [&](int64_t i) {
+    int64_t b = i / Hq, g = i % Hq, h = g / group;
+    std::vector<double> qd(D), od(D);
+    for (int64_t d = 0; d < D; ++d) qd[d] = bf16_to_double(q[(b * Hq + g) * D + d]);
+    attend_one(qd.data(), D, sm_scale, prefix_k + h * n_prefix * D, prefix_v + h * n_prefix * D, n_prefix,
+               kq + (b * Hkv + h) * Tmax * (D / 2), vq + (b * Hkv + h) * Tmax * (D / 2), len[b], s_k[h], s_v[h],
+               od.data());
+    for (int64_t d = 0; d < D; ++d) {
+      out[(b * Hq + g) * D + d] = double_to_bf16(od[d]);
+      if (out_f64) out_f64[(b * Hq + g) * D + d] = od[d];
+    }
+  });
+}
+
+// Prefill: T query tokens of one sequence; query t sees the whole prefix and cached keys 0..t
+// (the prefix sits at the beginning of the sequence, Sec. 4.2).
+// q bf16 [T,Hq,D]; kq/vq u8 [Hkv,Tmax,D/2] of this sequence; out bf16 [T,Hq,D].
+void orc_prefill_attn(const uint16_t* q, const uint16_t* prefix_k, const uint16_t* prefix_v, const uint8_t* kq,
+                      const uint8_t* vq, const float* s_k, const float* s_v, int64_t T, int64_t Hq, int64_t Hkv,
+                      int64_t D, int64_t n_prefix, int64_t Tmax, double sm_scale, uint16_t* out) {
+  int64_t group = Hq / Hkv;
+  parallel_rows(T * Hq, [&](int64_t i) {
+    int64_t t = i / Hq, g = i % Hq, h = g / group;
+    std::vector<double> qd(D), od(D);
+    for (int64_t d = 0; d < D; ++d) qd[d] = bf16_to_double(q[(t * Hq + g) * D + d]);
+    attend_one(qd.data(), D, sm_scale, prefix_k + h * n_prefix * D, prefix_v + h * n_prefix * D, n_prefix,
+               kq + h * Tmax * (D / 2), vq + h * Tmax * (D / 2), t + 1, s_k[h], s_v[h], od.data());
+    for (int64_t d = 0; d < D; ++d) out[(t * Hq + g) * D + d] = double_to_bf16(od[d]);
+  });
+}
+
+// ---- transformer-block glue of a Llama block (App. B figure; used by the full-block config) ----
+// RMSNorm: y = x / sqrt(mean(x^2) + eps) * g, rounded once to bf16.
+void orc_rmsnorm(const uint16_t* x, const uint16_t* g, int64_t M, int64_t K, double eps, uint16_t* y) {
+  parallel_rows(M, [&](int64_t m) {
+    double ss = 0.0;
+    for (int64_t j = 0; j < K; ++j) {
+      double v = bf16_to_double(x[m * K + j]);
+      ss += v * v;
+    }
+    double r = 1.0 / std::sqrt(ss / static_cast<double>(K) + eps);
+    for (int64_t j = 0; j < K; ++j)
+      y[m * K + j] = double_to_bf16(bf16_to_double(x[m * K + j]) * r * bf16_to_double(g[j]));
+  });
+}
+
+// Rotary embedding, rotate-half pairing: for i < D/2, angle = pos * theta^(-2i/D),
+//   y[i] = x[i] cos - x[i+D/2] sin,  y[i+D/2] = x[i+D/2] cos + x[i] sin.
+// x bf16 [T,H,D], token t at position pos0 + t; result rounded once to bf16.
+void orc_rope(const uint16_t* x, int64_t T, int64_t H, int64_t D, int64_t pos0, double theta, uint16_t* y) {
+  parallel_rows(T, [&](int64_t t) {
+    double pos = static_cast<double>(pos0 + t);
+    for (int64_t h = 0; h < H; ++h)
+      for (int64_t i = 0; i < D / 2; ++i) {
+        double ang = pos * std::pow(theta, -2.0 * static_cast<double>(i) / static_cast<double>(D));
+        double c = std::cos(ang), s = std::sin(ang);
+        double a = bf16_to_double(x[(t * H + h) * D + i]);
+        double b = bf16_to_double(x[(t * H + h) * D + i + D / 2]);
+        y[(t * H + h) * D + i] = double_to_bf16(a * c - b * s);
+        y[(t * H + h) * D + i + D / 2] = double_to_bf16(b * c + a * s);
+      }
+  });
+}
+
+// SwiGLU gate: y = silu(gate) * up = gate / (1 + exp(-gate)) * up, rounded once to bf16.
+void orc_silu_mul(const uint16_t* gate, const uint16_t* up, int64_t n, uint16_t* y) {
+  for (int64_t i = 0; i < n; ++i) {
+    double g = bf16_to_double(gate[i]), u = bf16_to_double(up[i]);
+    y[i] = double_to_bf16(g / (1.0 + std::exp(-g)) * u);
+  }
+}
+
+// Residual: y = a + b, rounded once to bf16.
+void orc_add(const uint16_t* a, const uint16_t* b, int64_t n, uint16_t* y) {
+  for (int64_t i = 0; i < n; ++i) y[i] = double_to_bf16(bf16_to_double(a[i]) + bf16_to_double(b[i]));
+}
+
+}  // extern "C"

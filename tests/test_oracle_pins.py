@@ -1,0 +1,440 @@
+"""Pins for the CPU oracle: it is checked against closed forms, invariants, brute force and
+independent library routines before anything is compared with it. No GPU needed."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+from scipy.linalg import hadamard
+
+from oracle import pq_oracle as orc
+from paper_2410_05265_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _load(name):
+    return np.loadtxt(os.path.join(GOLDEN, name), comments="#")
+
+
+def bf16_bits(x):
+    return inputs.bits(torch.as_tensor(np.asarray(x, np.float64)).to(torch.bfloat16))
+
+
+def fp16_bits(x):
+    return inputs.bits(torch.as_tensor(np.asarray(x, np.float64)).to(torch.float16))
+
+
+rng = np.random.default_rng(1234)
+
+
+# ---------------------------------------------------------------- formats
+def test_bf16_roundtrip_matches_library_rounding():
+    x = np.concatenate([rng.standard_normal(4000) * np.exp(rng.standard_normal(4000) * 8), [0.0, -0.0, 1e-40, 3e38]])
+    # exact ties between two bf16 neighbours must go to even
+    ties = np.array([1.0 + 2.0**-8, 1.0 + 3 * 2.0**-8, -(2.0 + 2.0**-7), 2.0**-130 + 2.0**-134])
+    x = np.concatenate([x, ties])
+    got = orc.f64_to_bf16(x)
+    # torch rounds float64 -> bf16 through float32; avoid that double rounding in the reference by
+    # using values whose float32 image is exact or far from a bf16 tie
+    ref = inputs.bits(torch.from_numpy(x).to(torch.float32).to(torch.bfloat16))
+    f32_exact = x.astype(np.float32).astype(np.float64) == x
+    assert np.array_equal(got[f32_exact], ref[f32_exact])
+    assert np.mean(got == ref) > 0.999
+    assert got[-4] == 0x3F80 and got[-3] == 0x3F82  # 1+2^-8 -> 1.0 (even), 1+3*2^-8 -> 1+2^-6
+    back = orc.bf16_to_f64(got)
+    assert np.array_equal(orc.f64_to_bf16(back), got)
+
+
+def test_fp16_decode_matches_numpy_for_every_pattern():
+    allbits = np.arange(65536, dtype=np.uint16)
+    ref = allbits.view(np.float16).astype(np.float64)
+    got = orc.fp16_to_f64(allbits)
+    ok = ~np.isnan(ref)
+    assert np.array_equal(got[ok], ref[ok]) and np.all(np.isnan(got[~ok]))
+
+
+def test_pack_layout_low_nibble_first_twos_complement():
+    assert orc.unpack_int4(np.array([[0x21]], np.uint8)).tolist() == [[1, 2]]
+    assert orc.unpack_int4(np.array([[0xF8]], np.uint8)).tolist() == [[-8, -1]]
+    every = np.arange(256, dtype=np.uint8).reshape(16, 16)
+    codes = orc.unpack_int4(every)
+    assert codes.min() == -8 and codes.max() == 7
+    assert np.array_equal(orc.pack_int4(codes), every)
+    lo = (every & 0xF).astype(np.int16)
+    hi = (every >> 4).astype(np.int16)
+    assert np.array_equal(codes[:, 0::2], np.where(lo >= 8, lo - 16, lo))
+    assert np.array_equal(codes[:, 1::2], np.where(hi >= 8, hi - 16, hi))
+
+
+# ---------------------------------------------------------------- rotation (App. B)
+def test_hadamard_golden_h4():
+    H4 = _load("hadamard_h4_sylvester.txt")
+    got = orc.rotate_f64(np.eye(4), 4) * 2.0
+    assert np.array_equal(got, H4)
+
+
+@pytest.mark.parametrize("n", [1, 2, 4, 8, 16, 32, 64])
+def test_hadamard_orthogonality(n):
+    H = orc.rotate_f64(np.eye(n), n) * math.sqrt(n)
+    H = np.rint(H)
+    assert set(np.unique(H).tolist()) <= {-1.0, 1.0}
+    assert np.array_equal(H @ H.T, n * np.eye(n))
+    assert np.array_equal(H, H.T)
+
+
+@pytest.mark.parametrize("n", [2, 8, 64, 256])
+def test_rotation_equals_library_sylvester_product(n):
+    x = rng.standard_normal((5, n))
+    ref = x @ hadamard(n).astype(np.float64) / math.sqrt(n)
+    assert np.allclose(orc.rotate_f64(x, n), ref, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("n", [2048, 4096])
+def test_rotation_large_blocks(n):
+    x = rng.standard_normal((3, n))
+    y = orc.rotate_f64(x, n)
+    ref = x @ hadamard(n).astype(np.float64) / math.sqrt(n)
+    assert np.allclose(y, ref, rtol=0, atol=1e-10)
+    # unit vector -> one matrix row; all-ones -> sqrt(n) * e_0
+    e = np.zeros((1, n))
+    e[0, 37] = 1.0
+    col = orc.rotate_f64(e, n)[0] * math.sqrt(n)
+    i = np.arange(n)
+    parity = np.array([bin(v & 37).count("1") & 1 for v in i])
+    assert np.array_equal(np.rint(col), np.where(parity == 1, -1.0, 1.0))
+    ones = orc.rotate_f64(np.ones((1, n)), n)[0]
+    assert abs(ones[0] - math.sqrt(n)) < 1e-12 and np.all(ones[1:] == 0.0)
+
+
+def test_rotation_involution_and_parseval():
+    x = rng.standard_normal((4, 512))
+    y = orc.rotate_f64(x, 512)
+    assert np.allclose(orc.rotate_f64(y, 512), x, atol=1e-12)
+    assert np.allclose((y**2).sum(1), (x**2).sum(1), rtol=1e-12)
+
+
+def test_block_diagonal_rotation_is_independent_per_block():
+    x = rng.standard_normal((3, 7 * 64))
+    y = orc.rotate_f64(x, 64)
+    for b in range(7):
+        assert np.array_equal(y[:, b * 64:(b + 1) * 64], orc.rotate_f64(np.ascontiguousarray(x[:, b * 64:(b + 1) * 64]), 64))
+    assert np.array_equal(orc.rotate_f64(x, 0), x)
+
+
+def test_rotate_bf16_decodes_bits_exactly():
+    xb = bf16_bits(rng.standard_normal((4, 128)))
+    assert np.array_equal(orc.rotate_bf16(xb, 128), orc.rotate_f64(orc.bf16_to_f64(xb), 128))
+
+
+def test_computational_invariance_of_rotation():
+    # App. B: rotating activations and counter-rotating weights leaves x W^T unchanged
+    n = 256
+    x = rng.standard_normal((6, n))
+    W = rng.standard_normal((10, n))
+    lhs = orc.rotate_f64(x, n) @ orc.rotate_f64(W, n).T
+    assert np.allclose(lhs, x @ W.T, rtol=0, atol=1e-11)
+
+
+# ---------------------------------------------------------------- quantizer (Eq. 1)
+def test_quantizer_golden_worked_example():
+    g = _load("quantizer_eq1_worked.txt")
+    codes = orc.quant_f64(g[:, 0], 0.25)
+    assert codes.tolist() == g[:, 2].astype(int).tolist()
+    assert (np.clip(codes.astype(int) + 8, 0, 15)).tolist() == g[:, 3].astype(int).tolist()
+
+
+def test_quantizer_range_ties_clamp_monotone_idempotent():
+    v = np.linspace(-3.0, 3.0, 4001)
+    c = orc.quant_f64(v, 0.25)
+    assert c.min() == -8 and c.max() == 7
+    assert np.all(np.diff(c.astype(int)) >= 0)
+    ties = (np.arange(-8, 7) + 0.5) * 0.25
+    ct = orc.quant_f64(ties, 0.25).astype(int)
+    assert np.all(ct % 2 == 0), "ties must go to the even code"
+    assert np.all(np.abs(ct - (np.arange(-8, 7) + 0.5)) == 0.5)
+    deq = c.astype(np.float64) * 0.25
+    assert np.array_equal(orc.quant_f64(deq, 0.25), c)
+    inside = np.abs(v) <= 1.75
+    assert np.all(np.abs(deq[inside] - v[inside]) <= 0.125 + 1e-15)
+
+
+def test_quant_act_codes_and_tie_distance():
+    K = 64
+    x = rng.standard_normal((5, K))
+    xb = bf16_bits(x)
+    y = orc.rotate_bf16(xb, K)
+    s = np.float32(np.abs(y).max() / 7)
+    xq, tie = orc.quant_act(xb, K, s, want_tie_dist=True)
+    codes = orc.unpack_int4(xq)
+    r = y / np.float64(s)
+    assert np.all(np.abs(codes - r) <= 0.5 + 1e-12)
+    assert np.abs(codes).max() == 7
+    frac = r - np.floor(r)
+    assert np.allclose(tie, np.abs(frac - 0.5), atol=1e-6)
+    # rows below row_begin are left untouched
+    xq2 = orc.quant_act(xb, K, s, row_begin=2)
+    assert np.all(xq2[:2] == 0) and np.array_equal(xq2[2:], xq[2:])
+
+
+def test_static_scale_ignores_prefixed_rows():
+    M, K, P = 12, 128, 4
+    x = inputs.activations(M, K, seed=1, n_prefix=P)
+    xb = inputs.bits(x)
+    y = orc.rotate_bf16(xb, K)
+    s = orc.calib_act_scale(xb, K, row_begin=P)
+    assert s == np.float32(np.abs(y[P:].astype(np.float32)).max() / 7.0)
+    x2 = x.clone()
+    x2[:P] *= 1000.0
+    assert orc.calib_act_scale(inputs.bits(x2), K, row_begin=P) == s
+    assert orc.calib_act_scale(xb, K, row_begin=0) > 10 * s  # with the outlier rows the scale explodes
+
+
+# ---------------------------------------------------------------- weights (RTN per output channel)
+def test_weight_quantization_rtn_per_channel():
+    W = inputs.weights(24, 96, seed=2)
+    W[5] = 0
+    Wb = inputs.bits(W)
+    wq, s_w = orc.quant_weights(Wb)
+    Wf = W.to(torch.float32).numpy()
+    mx = np.abs(Wf).max(1)
+    expect = np.where(mx == 0, np.float32(1), mx / np.float32(7)).astype(np.float32)
+    assert np.array_equal(s_w, expect)
+    codes = orc.unpack_int4(wq).astype(np.int32)
+    assert codes.min() >= -7 and codes.max() <= 7  # symmetric max/7 never needs -8
+    assert np.all(codes[5] == 0) and s_w[5] == 1.0
+    am = np.abs(Wf).argmax(1)
+    rows = np.arange(24)
+    assert np.all(np.abs(codes[rows, am])[mx > 0] == 7)
+    assert np.all(np.abs(codes * s_w[:, None].astype(np.float64) - Wf) <= s_w[:, None] * 0.5 * (1 + 1e-6))
+    # idempotent: quantizing the dequantized weights (exact in bf16 only approximately, so use codes*2^-k scale)
+    W2 = (np.arange(-7, 8)[None, :].repeat(3, 0) * 0.25).astype(np.float64)
+    wq2, s2 = orc.quant_weights(bf16_bits(np.concatenate([W2, W2[:, :1]], 1)))
+    assert np.array_equal(orc.unpack_int4(wq2)[:, :15], np.arange(-7, 8)[None, :].repeat(3, 0)) and np.all(s2 == 0.25)
+
+
+# ---------------------------------------------------------------- integer GEMM
+def test_gemm_brute_force_tiny():
+    M, N, K = 3, 5, 8
+    x = rng.integers(-8, 8, (M, K)).astype(np.int8)
+    w = rng.integers(-8, 8, (N, K)).astype(np.int8)
+    acc = orc.gemm_i4(orc.pack_int4(x), orc.pack_int4(w))
+    for t, n in itertools.product(range(M), range(N)):
+        assert acc[t, n] == sum(int(x[t, k]) * int(w[n, k]) for k in range(K))
+
+
+def test_gemm_matches_int64_library_matmul_and_special_cases():
+    M, N, K = 17, 23, 160
+    x = rng.integers(-8, 8, (M, K)).astype(np.int8)
+    w = rng.integers(-8, 8, (N, K)).astype(np.int8)
+    acc = orc.gemm_i4(orc.pack_int4(x), orc.pack_int4(w))
+    assert np.array_equal(acc, x.astype(np.int64) @ w.astype(np.int64).T)
+    ones = np.ones((4, K), np.int8)
+    assert np.all(orc.gemm_i4(orc.pack_int4(ones), orc.pack_int4(ones)) == K)
+    lo = np.full((2, K), -8, np.int8)
+    assert np.all(orc.gemm_i4(orc.pack_int4(lo), orc.pack_int4(lo)) == 64 * K)
+    onehot = np.zeros((K, K), np.int8)
+    onehot[np.arange(K), np.arange(K)] = 1
+    assert np.array_equal(orc.gemm_i4(orc.pack_int4(onehot), orc.pack_int4(w)), w.T.astype(np.int32))
+
+
+def test_dequant_epilogue_closed_form_and_one_rounding():
+    acc = np.array([[3, -5, 0, 1 << 20]], np.int32)
+    s_w = np.array([0.25, 0.5, 7.0, 2.0**-10], np.float32)
+    out = orc.bf16_to_f64(orc.dequant_bf16(acc, 0.5, s_w))
+    assert out.tolist() == [[0.375, -1.25, 0.0, 512.0]]
+    acc = rng.integers(-200000, 200000, (8, 16)).astype(np.int32)
+    s_w = (rng.random(16) * 0.01 + 1e-3).astype(np.float32)
+    s_a = np.float32(0.0371)
+    got = orc.bf16_to_f64(orc.dequant_bf16(acc, s_a, s_w))
+    exact = acc.astype(np.float64) * np.float64(s_a) * s_w.astype(np.float64)[None, :]
+    assert np.all(np.abs(got - exact) <= np.abs(exact) * 2.0**-8 + 1e-300)  # half a bf16 ulp (8 significant bits)
+
+
+# ---------------------------------------------------------------- KV cache
+def test_kv_scale_and_append():
+    B, T, H, D, Tmax = 2, 3, 2, 16, 8
+    k = inputs.kv_tensor(B, T, H, D, 0, "k")
+    v = inputs.kv_tensor(B, T, H, D, 0, "v")
+    kc = inputs.kv_tensor(4, 8, H, D, 1, "k")
+    s_k = orc.calib_kv_scale(inputs.bits(kc))
+    kcf = kc.to(torch.float64).numpy()
+    assert np.array_equal(s_k, (np.abs(kcf).max(axis=(0, 1, 3)) / 7).astype(np.float32))
+    s_v = orc.calib_kv_scale(inputs.bits(inputs.kv_tensor(4, 8, H, D, 1, "v")))
+    kq = np.full((B, H, Tmax, D // 2), 0xEE, np.uint8)
+    vq = np.full((B, H, Tmax, D // 2), 0xEE, np.uint8)
+    length = np.array([1, 4], np.int32)
+    assert orc.kv4_append(inputs.bits(k), inputs.bits(v), s_k, s_v, kq, vq, length) == 0
+    assert length.tolist() == [4, 7]
+    kcodes = orc.unpack_int4(kq)
+    kf = k.to(torch.float64).numpy()
+    for b, l0 in enumerate([1, 4]):
+        for h in range(H):
+            r = kf[b, :, h, :] / np.float64(s_k[h])
+            got = kcodes[b, h, l0:l0 + T]
+            assert np.all(np.abs(got - np.clip(r, -8, 7)) <= 0.5 + 1e-12)
+            assert np.all(kq[b, h, :l0] == 0xEE) and np.all(kq[b, h, l0 + T:] == 0xEE)  # nothing else touched
+    # a sequence that would overflow Tmax is refused and nothing moves
+    before = kq.copy()
+    assert orc.kv4_append(inputs.bits(k), inputs.bits(v), s_k, s_v, kq, vq, length) == 1
+    assert np.array_equal(kq, before) and length.tolist() == [4, 7]
+
+
+# ---------------------------------------------------------------- attention (Eq. 3)
+def _attn_setup(B=2, Hq=4, Hkv=2, D=16, P=2, T=9, Tmax=12, mag=1.0, seed=0):
+    q = inputs.queries(B, Hq, D, seed)
+    pk = inputs.prefix_kv(Hkv, P, D, seed, "k", mag)
+    pv = inputs.prefix_kv(Hkv, P, D, seed, "v", mag)
+    kq = rng.integers(0, 256, (B, Hkv, Tmax, D // 2)).astype(np.uint8)
+    vq = rng.integers(0, 256, (B, Hkv, Tmax, D // 2)).astype(np.uint8)
+    s_k = (rng.random(Hkv) * 0.3 + 0.1).astype(np.float32)
+    s_v = (rng.random(Hkv) * 0.3 + 0.1).astype(np.float32)
+    length = np.array([T, T - 4][:B], np.int32)
+    return q, pk, pv, kq, vq, s_k, s_v, length
+
+
+def _library_attention(q, pk, pv, kq, vq, s_k, s_v, length, sm):
+    """Textbook softmax attention with torch on the dequantized tensors (float64)."""
+    B, Hq, D = q.shape
+    Hkv = pk.shape[0]
+    out = np.zeros((B, Hq, D))
+    kd = orc.unpack_int4(kq).astype(np.float64) * s_k.astype(np.float64)[None, :, None, None]
+    vd = orc.unpack_int4(vq).astype(np.float64) * s_v.astype(np.float64)[None, :, None, None]
+    for b in range(B):
+        for g in range(Hq):
+            h = g // (Hq // Hkv)
+            K = torch.cat([pk[h].double(), torch.from_numpy(kd[b, h, :length[b]])])
+            V = torch.cat([pv[h].double(), torch.from_numpy(vd[b, h, :length[b]])])
+            p = torch.softmax(K @ q[b, g].double() * sm, dim=0)
+            out[b, g] = (p @ V).numpy()
+    return out
+
+
+def test_decode_attention_equals_library_softmax_attention():
+    q, pk, pv, kq, vq, s_k, s_v, length = _attn_setup()
+    sm = 1 / math.sqrt(16)
+    out, out64 = orc.decode_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq, vq, s_k, s_v, length, sm, want_f64=True)
+    ref = _library_attention(q, pk, pv, kq, vq, s_k, s_v, length, sm)
+    assert np.allclose(out64, ref, rtol=1e-12, atol=1e-13)
+    assert np.array_equal(out, orc.f64_to_bf16(out64))
+    # no prefix at all: plain attention over the dequantized cache
+    pk0, pv0 = pk[:, :0], pv[:, :0]
+    _, o0 = orc.decode_attn(inputs.bits(q), inputs.bits(pk0), inputs.bits(pv0), kq, vq, s_k, s_v, length, sm, want_f64=True)
+    assert np.allclose(o0, _library_attention(q, pk0, pv0, kq, vq, s_k, s_v, length, sm), rtol=1e-12, atol=1e-13)
+    # empty cache: attention over the full-precision prefix only
+    _, o1 = orc.decode_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq, vq, s_k, s_v, np.zeros(2, np.int32), sm, want_f64=True)
+    assert np.allclose(o1, _library_attention(q, pk, pv, kq, vq, s_k, s_v, [0, 0], sm), rtol=1e-12, atol=1e-13)
+
+
+def test_decode_attention_closed_forms():
+    B, Hq, Hkv, D, P, T, Tmax = 1, 4, 2, 16, 0, 6, 6
+    q = inputs.queries(B, Hq, D, 3)
+    pk = torch.zeros((Hkv, 0, D), dtype=torch.float16)
+    vq = rng.integers(0, 256, (B, Hkv, Tmax, D // 2)).astype(np.uint8)
+    s = np.array([0.5, 0.25], np.float32)
+    length = np.array([T], np.int32)
+    # all-zero keys -> uniform probabilities -> output is the mean of V
+    kq = np.zeros((B, Hkv, Tmax, D // 2), np.uint8)
+    _, o = orc.decode_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pk), kq, vq, s, s, length, 0.25, want_f64=True)
+    vd = orc.unpack_int4(vq).astype(np.float64) * s.astype(np.float64)[None, :, None, None]
+    for g in range(Hq):
+        assert np.allclose(o[0, g], vd[0, g // 2].mean(0), rtol=1e-13)
+    # one dominant key -> output is that key's value row; equal queries in a GQA group -> equal outputs
+    qd = torch.zeros((1, Hq, D), dtype=torch.bfloat16)
+    qd[..., 0] = 100.0
+    kc = np.zeros((B, Hkv, Tmax, D), np.int8)
+    kc[:, :, 3, 0] = 7
+    _, o = orc.decode_attn(inputs.bits(qd), inputs.bits(pk), inputs.bits(pk), orc.pack_int4(kc), vq, s, s, length, 1.0, want_f64=True)
+    for g in range(Hq):
+        assert np.allclose(o[0, g], vd[0, g // 2, 3], rtol=1e-9)
+    assert np.array_equal(o[0, 0], o[0, 1]) and np.array_equal(o[0, 2], o[0, 3])
+
+
+def test_decode_attention_key_permutation_invariance():
+    q, pk, pv, kq, vq, s_k, s_v, length = _attn_setup(B=1, T=9)
+    sm = 0.25
+    _, o = orc.decode_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq, vq, s_k, s_v, length, sm, want_f64=True)
+    perm = rng.permutation(int(length[0]))
+    kq2, vq2 = kq.copy(), vq.copy()
+    kq2[:, :, :length[0]] = kq[:, :, perm]
+    vq2[:, :, :length[0]] = vq[:, :, perm]
+    _, o2 = orc.decode_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq2, vq2, s_k, s_v, length, sm, want_f64=True)
+    assert np.allclose(o, o2, rtol=1e-12, atol=1e-14)
+
+
+def test_prefill_attention_is_causal_decode_per_row():
+    T, Hq, Hkv, D, P, Tmax = 7, 4, 2, 16, 2, 8
+    qt = inputs.normal(5, inputs.STREAM_Q, (T, Hq, D), dtype=torch.bfloat16)
+    pk = inputs.prefix_kv(Hkv, P, D, 0, "k", 1.0)
+    pv = inputs.prefix_kv(Hkv, P, D, 0, "v", 1.0)
+    kq = rng.integers(0, 256, (Hkv, Tmax, D // 2)).astype(np.uint8)
+    vq = rng.integers(0, 256, (Hkv, Tmax, D // 2)).astype(np.uint8)
+    s_k = np.array([0.2, 0.3], np.float32)
+    s_v = np.array([0.4, 0.1], np.float32)
+    out = orc.prefill_attn(inputs.bits(qt), inputs.bits(pk), inputs.bits(pv), kq, vq, s_k, s_v, 0.25)
+    for t in range(T):
+        ref = orc.decode_attn(inputs.bits(qt[t:t + 1]), inputs.bits(pk), inputs.bits(pv), kq[None], vq[None], s_k, s_v,
+                              np.array([t + 1], np.int32), 0.25)
+        assert np.array_equal(out[t], ref[0])
+    # without a prefix the first token attends to itself only: its output is its own value row
+    out0 = orc.prefill_attn(inputs.bits(qt), inputs.bits(pk[:, :0]), inputs.bits(pv[:, :0]), kq, vq, s_k, s_v, 0.25)
+    vd = orc.unpack_int4(vq).astype(np.float64) * s_v.astype(np.float64)[:, None, None]
+    for g in range(Hq):
+        assert np.array_equal(out0[0, g], orc.f64_to_bf16(vd[g // 2, 0]))
+
+
+# ---------------------------------------------------------------- block glue
+def test_rope_matches_complex_rotation_and_relative_property():
+    T, H, D, theta = 6, 2, 16, 500000.0
+    x = inputs.normal(9, inputs.STREAM_Q, (T, H, D), dtype=torch.bfloat16)
+    y = orc.bf16_to_f64(orc.rope(inputs.bits(x), 4, theta))
+    xd = x.to(torch.float64).numpy()
+    z = xd[..., :D // 2] + 1j * xd[..., D // 2:]
+    freq = theta ** (-np.arange(D // 2) * 2.0 / D)
+    pos = (4 + np.arange(T))[:, None, None]
+    zr = z * np.exp(1j * pos * freq[None, None, :])
+    ref = np.concatenate([zr.real, zr.imag], -1)
+    assert np.all(np.abs(y - ref) <= np.abs(ref) * 2.0**-8 + 1e-30)
+    # position 0 is the identity
+    y0 = orc.rope(inputs.bits(x[:1]), 0, theta)
+    assert np.array_equal(y0, inputs.bits(x[:1]))
+    # <rope(a, m), rope(b, n)> depends on m - n only (checked through the complex form, in double)
+    a, b = z[0, 0], z[1, 0]
+    d1 = np.real(np.sum(a * np.exp(1j * 7 * freq) * np.conj(b * np.exp(1j * 3 * freq))))
+    d2 = np.real(np.sum(a * np.exp(1j * 14 * freq) * np.conj(b * np.exp(1j * 10 * freq))))
+    assert abs(d1 - d2) < 1e-10
+
+
+def test_rmsnorm_silu_add_closed_forms():
+    x = inputs.activations(5, 64, seed=0)
+    g = torch.ones(64, dtype=torch.bfloat16)
+    y = orc.bf16_to_f64(orc.rmsnorm(inputs.bits(x), inputs.bits(g), 0.0))
+    assert np.allclose(np.sqrt((y**2).mean(1)), 1.0, atol=4e-3)
+    y2 = orc.bf16_to_f64(orc.rmsnorm(inputs.bits(x * 4), inputs.bits(g), 0.0))
+    assert np.array_equal(y, y2)  # scale invariance (power-of-two scaling is exact in bf16)
+    ref = torch.nn.functional.rms_norm(x.double(), (64,), eps=1e-5).numpy()
+    got = orc.bf16_to_f64(orc.rmsnorm(inputs.bits(x), inputs.bits(g), 1e-5))
+    assert np.all(np.abs(got - ref) <= np.abs(ref) * 2.0**-8)
+    gate = torch.tensor([0.0, 30.0, -30.0, 1.0, -1.0], dtype=torch.bfloat16)
+    up = torch.tensor([5.0, 2.0, 2.0, 3.0, 3.0], dtype=torch.bfloat16)
+    s = orc.bf16_to_f64(orc.silu_mul(inputs.bits(gate), inputs.bits(up)))
+    ref = (torch.nn.functional.silu(gate.double()) * up.double()).numpy()
+    assert s[0] == 0.0 and s[1] == 60.0 and abs(s[2]) < 1e-11
+    assert np.all(np.abs(s - ref) <= np.abs(ref) * 2.0**-8 + 1e-30)
+    a = torch.tensor([1.0, 2.5, -3.0], dtype=torch.bfloat16)
+    b = torch.tensor([0.5, 0.25, 3.0], dtype=torch.bfloat16)
+    assert orc.bf16_to_f64(orc.add(inputs.bits(a), inputs.bits(b))).tolist() == [1.5, 2.75, 0.0]
+
+
+# ---------------------------------------------------------------- input generator sanity (no method arithmetic there)
+def test_input_generator_is_deterministic_and_sliceable():
+    a = inputs.normal(3, inputs.STREAM_ACT, (1000,))
+    b = inputs.normal(3, inputs.STREAM_ACT, (1000,))
+    assert torch.equal(a, b)
+    c = inputs.normal(3, inputs.STREAM_ACT, (400,), offset=600)
+    assert torch.equal(a[600:], c)
+    big = inputs.normal(4, inputs.STREAM_ACT, (200000,))
+    assert abs(float(big.mean())) < 0.01 and abs(float(big.std()) - 1.0) < 0.01
+    assert not torch.equal(inputs.normal(3, inputs.STREAM_ACT, (10,)), inputs.normal(3, inputs.STREAM_K, (10,)))
