@@ -1,0 +1,148 @@
+/*
+ * pq.h — C ABI of the B200 (sm_100a) W4A4KV4 inference hot path of PrefixQuant in its static
+ * setting ("O2" in Table 1: per-channel weights, per-tensor static activations, per-head static
+ * KV cache), where the outlier tokens are prefixed and their K/V stay in full precision (Eq. 3).
+ *
+ * General rules
+ *   - Every tensor pointer is a DEVICE pointer on the device that was current at pq_create(),
+ *     owned by the caller. The library allocates only inside pq_create() (a few KB: a status
+ *     word and ticket counters) and frees only inside pq_destroy(). Scratch memory is a caller
+ *     buffer sized by the matching *_workspace_bytes() function.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return at once.
+ *     Argument errors are reported synchronously through the return value and enqueue nothing.
+ *     Errors found on the device (a bounded wait that ran out, a KV append past capacity) are
+ *     written to a status word read by pq_check().
+ *   - Nothing aborts, traps or prints. Every wait inside a kernel is bounded.
+ *   - One pq_ctx must not be used from two streams at the same time (ticket counters are shared).
+ *   - bf16 / fp16 tensors are raw 16-bit patterns. Packed INT4 tensors hold element 2j in the low
+ *     nibble and element 2j+1 in the high nibble of byte j, two's complement, packed along the
+ *     contraction (K) or head (D) dimension.
+ *   - The signed 4-bit code of a value v with step s is clamp(round_half_even(v / s), -8, 7): Eq. (1)
+ *     with N = 4 in its symmetric reading (zero-point fixed at 8, s = max|v| / 7).
+ */
+#ifndef PQ_H_
+#define PQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t pq_status;
+enum {
+  PQ_OK = 0,
+  PQ_ERR_INVALID_ARG = 1, /* null pointer, negative size, bad enum */
+  PQ_ERR_SHAPE = 2,       /* size outside what the kernels support, KV append past Tmax */
+  PQ_ERR_ALIGN = 3,       /* pointer or leading dimension not aligned as documented */
+  PQ_ERR_WORKSPACE = 4,   /* workspace missing or too small */
+  PQ_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed */
+  PQ_ERR_TIMEOUT = 6,     /* a bounded device-side wait ran out */
+  PQ_ERR_UNSUPPORTED = 7
+};
+
+typedef struct pq_ctx pq_ctx;
+
+/* Human-readable name of a status code (static storage). */
+const char* pq_status_string(pq_status s);
+
+/* Creates a context on the current device: caches the SM count, resolves the tensor-map encoder,
+ * allocates the device status word and the ticket counters. */
+pq_status pq_create(pq_ctx** out);
+pq_status pq_destroy(pq_ctx* ctx);
+
+/* Synchronizes `stream`, returns the device status word (PQ_OK if no kernel reported anything)
+ * and clears it. */
+pq_status pq_check(pq_ctx* ctx, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Offline weight quantization: round-to-nearest, one symmetric scale per output channel
+ * (Table 1 "per-channel" weights; the "RTN" row of Table 6; Eq. 1).
+ *   W    bf16 [N, K], row stride ldw elements (ldw >= K)
+ *   wq   u8   [N, K/2] packed codes (dense rows)
+ *   s_w  f32  [N]: s_w[n] = max_k |W[n,k]| / 7 in fp32 (1 for an all-zero row)
+ *   code = clamp(rint(W[n,k] / s_w[n]), -8, 7) with IEEE fp32 division.
+ * K must be even. */
+pq_status pq_quant_weights(pq_ctx* ctx, const void* W, int64_t N, int64_t K, int64_t ldw, uint8_t* wq, float* s_w,
+                           void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Online rotation (App. B, "Online Rotation": the Walsh-Hadamard transform applied to a linear
+ * layer's input) fused with the static per-tensor quantizer (Table 1, O2; Sec. 3 "Dynamic and
+ * Static") and the nibble pack.
+ * For every row t >= row_begin and every contiguous had_block-wide block of that row:
+ *     y = x_block * H / sqrt(had_block),  H[i][j] = (-1)^popcount(i & j)   (Sylvester order)
+ *     xq = pack(clamp(round_half_even(y / s_a), -8, 7))
+ *   x    bf16 [M, K], row stride ldx elements (even, >= K), base 4-byte aligned
+ *   xq   u8   [M, K/2] dense rows, base 16-byte aligned
+ *   s_a  f32 scalar on the device (static: calibrated offline, never recomputed here)
+ *   had_block: a power of two in [128, 8192] dividing K, or 0 for "no rotation" (K % 128 == 0).
+ * Rows below row_begin are the prefixed outlier tokens: they are neither read nor written. */
+pq_status pq_hadamard_quant_act(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                int64_t row_begin, const float* s_a, uint8_t* xq, void* stream);
+
+/* Calibration helper for the static activation scale: over rows >= row_begin of a calibration
+ * batch, *s_a = max(*s_a, max |y| / 7) with y the rotated rows as above. *s_a must be initialised
+ * by the caller (0 to start); several batches may be folded into it. The prefixed rows never
+ * take part (Sec. 5.5: isolating the >1e3 outliers is what makes the static scale usable). */
+pq_status pq_calib_act_scale(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                             int64_t row_begin, float* s_a, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * W4A4 linear layer (Sec. 3: low-bit matrix multiplication; Table 1, O2):
+ *     acc[t, n] = sum_k xq[t, k] * wq[n, k]          exact, int32
+ *     out[t, n] = bf16( acc[t, n] * s_a * s_w[n] )   for rows t >= row_begin
+ *   xq   u8 [M, K/2], wq u8 [N, K/2] dense packed rows, bases 16-byte aligned
+ *   s_a  f32 scalar (device), s_w f32 [N] (device)
+ *   out  bf16 [M, N], row stride ldo elements
+ *   acc_dbg  nullable int32 [M, N] dense: receives the raw accumulators (parity checks)
+ *   K % 32 == 0, K <= 65536. Output rows below row_begin are left untouched.
+ * Shapes with M - row_begin > 16 run on the tensor-core kernel (TMA + tcgen05, kind::i8);
+ * smaller M runs the weight-streaming kernel. No workspace is needed (ws may be NULL). */
+size_t pq_w4a4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+pq_status pq_w4a4_gemm(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
+                       void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int64_t row_begin, int32_t* acc_dbg,
+                       void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * KV cache with a full-precision prefix region and a 4-bit region (Sec. 4.2, Eq. 3; Table 1, O2:
+ * per-head static KV scales). All buffers are the caller's.
+ *   prefix_k, prefix_v  fp16 [Hkv, n_prefix, D]  K/V of the prefixed tokens, computed once by the
+ *                       full-precision model and shared by every sequence
+ *   kq, vq              u8 [B, Hkv, Tmax, D/2]   packed codes of the ordinary tokens
+ *   s_k, s_v            f32 [Hkv]                static per-head steps
+ *   len                 int32 [B] on the device  number of 4-bit entries of each sequence
+ * D must be 128; Hq a multiple of Hkv with Hq / Hkv <= 8. */
+typedef struct pq_kv4_cache {
+  const void* prefix_k;
+  const void* prefix_v;
+  uint8_t* kq;
+  uint8_t* vq;
+  const float* s_k;
+  const float* s_v;
+  int32_t* len;
+  int32_t B, Hq, Hkv, D, n_prefix, Tmax;
+} pq_kv4_cache;
+
+/* Quantize-on-write: k, v bf16 [B, T_new, Hkv, D] are quantized with s_k[h], s_v[h] and written at
+ * positions len[b] .. len[b]+T_new-1, then len[b] += T_new (on the device, in stream order).
+ * If any sequence would exceed Tmax nothing is written, len is unchanged and PQ_ERR_SHAPE is
+ * left in the status word. */
+pq_status pq_kv4_append(pq_ctx* ctx, const pq_kv4_cache* cache, const void* k, const void* v, int32_t T_new,
+                        void* stream);
+
+/* Decode attention, one query token per sequence, over [prefix || 4-bit cache] (Eq. 3):
+ *     score_j = q . K_j * sm_scale,  K_j = prefix_k[h, j] (j < n_prefix) or s_k[h] * code
+ *     out     = softmax(score) . V   with V_j = prefix_v[h, j] or s_v[h] * code
+ *   q, out  bf16 [B, Hq, D]; query head g reads KV head g / (Hq / Hkv)
+ *   ws      scratch of pq_decode_attn_workspace_bytes(cache) bytes, 16-byte aligned
+ * Every cached entry is visible (no mask). */
+size_t pq_decode_attn_workspace_bytes(const pq_kv4_cache* cache);
+pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, const void* q, void* out, float sm_scale,
+                                    void* ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PQ_H_ */

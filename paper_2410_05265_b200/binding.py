@@ -1,0 +1,219 @@
+"""Thin ctypes binding over the C-ABI CUDA library (argument marshalling only).
+
+Functions take torch CUDA tensors, pass their device pointers and the current torch stream to
+the library and raise ``PQError`` on a non-zero status. No step of the path runs in Python or
+torch; there is no CPU fallback: without the compiled library every call fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, c_char_p, c_float, c_int32, c_int64, c_size_t, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpq_b200.so")
+
+STATUS_NAMES = {
+    0: "PQ_OK", 1: "PQ_ERR_INVALID_ARG", 2: "PQ_ERR_SHAPE", 3: "PQ_ERR_ALIGN", 4: "PQ_ERR_WORKSPACE",
+    5: "PQ_ERR_CUDA", 6: "PQ_ERR_TIMEOUT", 7: "PQ_ERR_UNSUPPORTED",
+}
+
+EXPORTS = [
+    "pq_status_string", "pq_create", "pq_destroy", "pq_check", "pq_quant_weights", "pq_hadamard_quant_act",
+    "pq_calib_act_scale", "pq_w4a4_gemm_workspace_bytes", "pq_w4a4_gemm", "pq_kv4_append",
+    "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix",
+]
+
+
+class PQError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class KV4CacheStruct(Structure):
+    _fields_ = [
+        ("prefix_k", c_void_p), ("prefix_v", c_void_p), ("kq", c_void_p), ("vq", c_void_p),
+        ("s_k", c_void_p), ("s_v", c_void_p), ("len", c_void_p),
+        ("B", c_int32), ("Hq", c_int32), ("Hkv", c_int32), ("D", c_int32), ("n_prefix", c_int32), ("Tmax", c_int32),
+    ]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the compiled library; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2410_05265_b200.build` first")
+    lib = ctypes.CDLL(LIB_PATH)
+    lib.pq_status_string.restype = c_char_p
+    lib.pq_status_string.argtypes = [c_int32]
+    lib.pq_create.argtypes = [POINTER(c_void_p)]
+    lib.pq_destroy.argtypes = [c_void_p]
+    lib.pq_check.argtypes = [c_void_p, c_void_p]
+    lib.pq_quant_weights.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p]
+    lib.pq_hadamard_quant_act.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p,
+                                          c_void_p, c_void_p]
+    lib.pq_calib_act_scale.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p,
+                                       c_void_p]
+    lib.pq_w4a4_gemm_workspace_bytes.restype = c_size_t
+    lib.pq_w4a4_gemm_workspace_bytes.argtypes = [c_int64, c_int64, c_int64]
+    lib.pq_w4a4_gemm.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64,
+                                 c_int64, c_int64, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.pq_kv4_append.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_void_p, c_void_p, c_int32, c_void_p]
+    lib.pq_decode_attn_workspace_bytes.restype = c_size_t
+    lib.pq_decode_attn_workspace_bytes.argtypes = [POINTER(KV4CacheStruct)]
+    lib.pq_decode_attn_kv4_prefix.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_void_p, c_void_p, c_float, c_void_p,
+                                              c_size_t, c_void_p]
+    for name in EXPORTS:
+        getattr(lib, name)
+        if name not in ("pq_status_string", "pq_w4a4_gemm_workspace_bytes", "pq_decode_attn_workspace_bytes"):
+            getattr(lib, name).restype = c_int32
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    return c_void_p(t.data_ptr()) if t is not None else c_void_p(0)
+
+
+def _stream():
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ok(status: int, where: str):
+    if status != 0:
+        raise PQError(status, where)
+
+
+def _dev(t: torch.Tensor, dtype, name: str):
+    if not t.is_cuda or t.dtype != dtype:
+        raise TypeError(f"{name} must be a CUDA tensor of dtype {dtype}")
+    return t
+
+
+class KV4Cache:
+    """Caller-owned buffers of one layer's KV cache: fp16 prefix region + packed INT4 region."""
+
+    def __init__(self, prefix_k, prefix_v, kq, vq, s_k, s_v, length, Hq: int):
+        B, Hkv, Tmax, D2 = kq.shape
+        self.prefix_k, self.prefix_v, self.kq, self.vq = prefix_k, prefix_v, kq, vq
+        self.s_k, self.s_v, self.length = s_k, s_v, length
+        _dev(kq, torch.uint8, "kq"), _dev(vq, torch.uint8, "vq")
+        _dev(s_k, torch.float32, "s_k"), _dev(s_v, torch.float32, "s_v"), _dev(length, torch.int32, "length")
+        n_prefix = 0 if prefix_k is None else prefix_k.shape[1]
+        if n_prefix:
+            _dev(prefix_k, torch.float16, "prefix_k"), _dev(prefix_v, torch.float16, "prefix_v")
+            assert prefix_k.is_contiguous() and prefix_v.is_contiguous()
+        assert kq.is_contiguous() and vq.is_contiguous() and vq.shape == kq.shape
+        self.B, self.Hq, self.Hkv, self.D, self.n_prefix, self.Tmax = B, Hq, Hkv, D2 * 2, n_prefix, Tmax
+        self.struct = KV4CacheStruct(
+            prefix_k.data_ptr() if n_prefix else 0, prefix_v.data_ptr() if n_prefix else 0, kq.data_ptr(), vq.data_ptr(),
+            s_k.data_ptr(), s_v.data_ptr(), length.data_ptr(), B, Hq, Hkv, D2 * 2, n_prefix, Tmax,
+        )
+
+
+class Context:
+    """Owns one pq_ctx on the current CUDA device."""
+
+    def __init__(self):
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise RuntimeError("paper_2410_05265_b200 needs a CUDA device (sm_100a); there is no CPU path")
+        torch.cuda.init()
+        torch.empty(1, device="cuda")  # make sure the primary context exists
+        h = c_void_p()
+        _ok(self.lib.pq_create(ctypes.byref(h)), "pq_create")
+        self.h = h
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.pq_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def check(self):
+        """Synchronizes the current stream and raises if a kernel reported an error."""
+        _ok(self.lib.pq_check(self.h, _stream()), "pq_check")
+
+    def check_status(self) -> int:
+        return int(self.lib.pq_check(self.h, _stream()))
+
+    # ---- offline -----------------------------------------------------------------------------
+    def quant_weights(self, W: torch.Tensor):
+        _dev(W, torch.bfloat16, "W")
+        N, K = W.shape
+        assert W.stride(1) == 1
+        wq = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
+        s_w = torch.empty((N,), dtype=torch.float32, device=W.device)
+        _ok(self.lib.pq_quant_weights(self.h, _ptr(W), N, K, W.stride(0), _ptr(wq), _ptr(s_w), _stream()), "pq_quant_weights")
+        return wq, s_w
+
+    def calib_act_scale(self, x: torch.Tensor, had_block: int, row_begin: int = 0, s_a: torch.Tensor | None = None):
+        _dev(x, torch.bfloat16, "x")
+        M, K = x.shape
+        if s_a is None:
+            s_a = torch.zeros((1,), dtype=torch.float32, device=x.device)
+        _ok(self.lib.pq_calib_act_scale(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, _ptr(s_a), _stream()),
+            "pq_calib_act_scale")
+        return s_a
+
+    # ---- hot path ------------------------------------------------------------------------------
+    def hadamard_quant_act(self, x: torch.Tensor, had_block: int, s_a: torch.Tensor, row_begin: int = 0,
+                           out: torch.Tensor | None = None):
+        _dev(x, torch.bfloat16, "x"), _dev(s_a, torch.float32, "s_a")
+        M, K = x.shape
+        assert x.stride(1) == 1
+        if out is None:
+            out = torch.zeros((M, K // 2), dtype=torch.uint8, device=x.device)
+        _ok(self.lib.pq_hadamard_quant_act(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, _ptr(s_a), _ptr(out),
+                                           _stream()), "pq_hadamard_quant_act")
+        return out
+
+    def w4a4_gemm(self, xq: torch.Tensor, wq: torch.Tensor, s_a: torch.Tensor, s_w: torch.Tensor, row_begin: int = 0,
+                  out: torch.Tensor | None = None, acc_dbg: torch.Tensor | None = None):
+        _dev(xq, torch.uint8, "xq"), _dev(wq, torch.uint8, "wq")
+        _dev(s_a, torch.float32, "s_a"), _dev(s_w, torch.float32, "s_w")
+        M, K2 = xq.shape
+        N = wq.shape[0]
+        assert wq.shape[1] == K2 and xq.is_contiguous() and wq.is_contiguous()
+        if out is None:
+            out = torch.zeros((M, N), dtype=torch.bfloat16, device=xq.device)
+        if acc_dbg is not None:
+            _dev(acc_dbg, torch.int32, "acc_dbg")
+            assert acc_dbg.shape == (M, N) and acc_dbg.is_contiguous()
+        _ok(self.lib.pq_w4a4_gemm(self.h, _ptr(xq), _ptr(wq), _ptr(s_a), _ptr(s_w), _ptr(out), out.stride(0), M, N, K2 * 2,
+                                  row_begin, _ptr(acc_dbg), c_void_p(0), 0, _stream()), "pq_w4a4_gemm")
+        return out
+
+    def kv4_append(self, cache: KV4Cache, k: torch.Tensor, v: torch.Tensor):
+        _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v")
+        B, T_new, Hkv, D = k.shape
+        assert (B, Hkv, D) == (cache.B, cache.Hkv, cache.D) and v.shape == k.shape
+        assert k.is_contiguous() and v.is_contiguous()
+        _ok(self.lib.pq_kv4_append(self.h, ctypes.byref(cache.struct), _ptr(k), _ptr(v), T_new, _stream()), "pq_kv4_append")
+
+    def decode_attn_workspace(self, cache: KV4Cache) -> torch.Tensor:
+        n = int(self.lib.pq_decode_attn_workspace_bytes(ctypes.byref(cache.struct)))
+        return torch.empty((max(n, 16),), dtype=torch.uint8, device=cache.kq.device)
+
+    def decode_attn(self, cache: KV4Cache, q: torch.Tensor, sm_scale: float, ws: torch.Tensor,
+                    out: torch.Tensor | None = None):
+        _dev(q, torch.bfloat16, "q")
+        assert q.shape == (cache.B, cache.Hq, cache.D) and q.is_contiguous()
+        if out is None:
+            out = torch.empty_like(q)
+        _ok(self.lib.pq_decode_attn_kv4_prefix(self.h, ctypes.byref(cache.struct), _ptr(q), _ptr(out), float(sm_scale),
+                                               _ptr(ws), ws.numel(), _stream()), "pq_decode_attn_kv4_prefix")
+        return out

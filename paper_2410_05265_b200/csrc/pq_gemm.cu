@@ -1,0 +1,33 @@
+// Entry point of the W4A4 linear layer: argument checks and the choice between the tensor-core
+// kernel (prefill-shaped) and the weight-streaming kernel (decode-shaped).
+#include "pq_common.cuh"
+
+pq_status pq_gemm_tc_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
+                            void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st);
+pq_status pq_gemm_stream_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a,
+                                const float* s_w, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                                int32_t* acc_dbg, cudaStream_t st);
+
+extern "C" size_t pq_w4a4_gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
+
+extern "C" pq_status pq_w4a4_gemm(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a,
+                                  const float* s_w, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                                  int64_t row_begin, int32_t* acc_dbg, void* ws, size_t ws_bytes, void* stream) {
+  (void)ws;
+  (void)ws_bytes;
+  if (!ctx || !xq || !wq || !s_a || !s_w || !out) return PQ_ERR_INVALID_ARG;
+  if (M < 0 || N < 0 || K < 0 || row_begin < 0 || ldo < N) return PQ_ERR_INVALID_ARG;
+  if (K % 32 != 0 || K > 65536 || M > (1 << 30) || N > (1 << 30)) return PQ_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(xq) & 15) || (reinterpret_cast<uintptr_t>(wq) & 15) ||
+      (reinterpret_cast<uintptr_t>(out) & 1))
+    return PQ_ERR_ALIGN;
+  if (row_begin >= M || N == 0) return PQ_OK;
+  const int64_t m = M - row_begin;
+  const uint8_t* xq0 = xq + row_begin * (K / 2);
+  void* out0 = static_cast<__nv_bfloat16*>(out) + row_begin * ldo;
+  int32_t* dbg0 = acc_dbg ? acc_dbg + row_begin * N : nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (K == 0) return PQ_ERR_SHAPE;
+  if (m <= 16) return pq_gemm_stream_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st);
+  return pq_gemm_tc_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st);
+}

@@ -1,0 +1,138 @@
+// W4A4 GEMM for decode-shaped problems (at most 16 tokens): the packed weights are streamed
+// from HBM exactly once with 128-bit loads and the kernel is bound by that stream.
+//
+// One CTA owns 16 output channels; its 8 warps split K in 128-element steps and meet in shared
+// memory at the end. Each warp multiplies with the warp-level integer MMA (m16n8k32, s8): the 16
+// weight rows are the M side, up to 8 tokens the N side. A lane loads one 16-byte chunk (32 codes)
+// from two weight rows and from one token row, expands the nibbles to s8 values scaled by 16
+// (even-position codes in one word, odd-position codes in the next) and feeds word pairs to four
+// MMAs. Weights and tokens apply the same permutation of k inside a chunk, so the dot product is
+// unchanged; the factor 16*16 is shifted out exactly in the epilogue.
+#include "pq_common.cuh"
+
+namespace {
+
+constexpr int GS_WARPS = 8;
+constexpr int GS_THREADS = GS_WARPS * 32;
+constexpr int GS_CH = 16;     // output channels per CTA
+constexpr int GS_UNROLL = 4;  // K steps whose loads are in flight together
+
+__device__ __forceinline__ void mma_s8_16832(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                             uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void expand(const uint4& w, uint32_t (&o)[8]) {
+  o[0] = pq::nib_lo_x16(w.x), o[1] = pq::nib_hi_x16(w.x);
+  o[2] = pq::nib_lo_x16(w.y), o[3] = pq::nib_hi_x16(w.y);
+  o[4] = pq::nib_lo_x16(w.z), o[5] = pq::nib_hi_x16(w.z);
+  o[6] = pq::nib_lo_x16(w.w), o[7] = pq::nib_hi_x16(w.w);
+}
+
+// Streaming load of weight bytes that are used once: do not keep them in L1.
+__device__ __forceinline__ uint4 ld_stream(const uint8_t* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+template <bool TWO_GROUPS>
+__global__ void __launch_bounds__(GS_THREADS)
+    gemm_w4a4_stream_kernel(const uint8_t* __restrict__ xq, const uint8_t* __restrict__ wq,
+                            const float* __restrict__ s_a, const float* __restrict__ s_w,
+                            __nv_bfloat16* __restrict__ out, int64_t ldo, int M, int N, int K,
+                            int32_t* __restrict__ acc_dbg) {
+  __shared__ int red[GS_WARPS][GS_CH][16];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int n0 = blockIdx.x * GS_CH;
+  const int kbytes = K / 2;
+  const int n_steps = (K + 127) / 128;
+
+  const bool w0_ok = n0 + g < N, w1_ok = n0 + g + 8 < N;
+  const bool x0_ok = g < M, x1_ok = TWO_GROUPS && (g + 8 < M);
+  const uint8_t* w0p = wq + static_cast<int64_t>(n0 + g) * kbytes + t * 16;
+  const uint8_t* w1p = wq + static_cast<int64_t>(n0 + g + 8) * kbytes + t * 16;
+  const uint8_t* x0p = xq + static_cast<int64_t>(g) * kbytes + t * 16;
+  const uint8_t* x1p = xq + static_cast<int64_t>(g + 8) * kbytes + t * 16;
+
+  int c0[4] = {0, 0, 0, 0}, c1[4] = {0, 0, 0, 0};
+  const uint4 zero = make_uint4(0, 0, 0, 0);
+
+  for (int base = warp; base < n_steps; base += GS_WARPS * GS_UNROLL) {
+    uint4 wa[GS_UNROLL], wb[GS_UNROLL], xa[GS_UNROLL], xb[GS_UNROLL];
+#pragma unroll
+    for (int u = 0; u < GS_UNROLL; ++u) {
+      const int ks = base + u * GS_WARPS;
+      const int off = ks * 64;
+      const bool in_k = ks < n_steps && off + t * 16 < kbytes;
+      wa[u] = (in_k && w0_ok) ? ld_stream(w0p + off) : zero;
+      wb[u] = (in_k && w1_ok) ? ld_stream(w1p + off) : zero;
+      xa[u] = (in_k && x0_ok) ? __ldg(reinterpret_cast<const uint4*>(x0p + off)) : zero;
+      if (TWO_GROUPS) xb[u] = (in_k && x1_ok) ? __ldg(reinterpret_cast<const uint4*>(x1p + off)) : zero;
+    }
+#pragma unroll
+    for (int u = 0; u < GS_UNROLL; ++u) {
+      uint32_t ea[8], eb[8], ex[8];
+      expand(wa[u], ea);
+      expand(wb[u], eb);
+      expand(xa[u], ex);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) mma_s8_16832(c0, ea[2 * j], eb[2 * j], ea[2 * j + 1], eb[2 * j + 1], ex[2 * j], ex[2 * j + 1]);
+      if (TWO_GROUPS) {
+        expand(xb[u], ex);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          mma_s8_16832(c1, ea[2 * j], eb[2 * j], ea[2 * j + 1], eb[2 * j + 1], ex[2 * j], ex[2 * j + 1]);
+      }
+    }
+  }
+  // accumulator layout: c[0], c[1] -> channel g, tokens 2t, 2t+1; c[2], c[3] -> channel g+8
+  red[warp][g][2 * t] = c0[0];
+  red[warp][g][2 * t + 1] = c0[1];
+  red[warp][g + 8][2 * t] = c0[2];
+  red[warp][g + 8][2 * t + 1] = c0[3];
+  if (TWO_GROUPS) {
+    red[warp][g][8 + 2 * t] = c1[0];
+    red[warp][g][8 + 2 * t + 1] = c1[1];
+    red[warp][g + 8][8 + 2 * t] = c1[2];
+    red[warp][g + 8][8 + 2 * t + 1] = c1[3];
+  }
+  __syncthreads();
+  {
+    const int ch = threadIdx.x & 15, tok = threadIdx.x >> 4;  // 16 tokens x 16 channels = 256 threads
+    const int n = n0 + ch;
+    if (tok < M && n < N && (TWO_GROUPS || tok < 8)) {
+      int s = 0;
+#pragma unroll
+      for (int w = 0; w < GS_WARPS; ++w) s += red[w][ch][tok];
+      s >>= 8;  // exact: every product carries the factor 16*16
+      const float f = static_cast<float>(s) * (__ldg(s_a) * __ldg(s_w + n));
+      out[static_cast<int64_t>(tok) * ldo + n] = __float2bfloat16_rn(f);
+      if (acc_dbg) acc_dbg[static_cast<int64_t>(tok) * N + n] = s;
+    }
+  }
+}
+
+}  // namespace
+
+// Rows [0, M) of xq/out, M <= 16 (the caller has already applied row_begin).
+pq_status pq_gemm_stream_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
+                                void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg,
+                                cudaStream_t st) {
+  (void)ctx;
+  const int grid = static_cast<int>((N + GS_CH - 1) / GS_CH);
+  if (M <= 8)
+    gemm_w4a4_stream_kernel<false><<<grid, GS_THREADS, 0, st>>>(xq, wq, s_a, s_w, static_cast<__nv_bfloat16*>(out), ldo,
+                                                                static_cast<int>(M), static_cast<int>(N),
+                                                                static_cast<int>(K), acc_dbg);
+  else
+    gemm_w4a4_stream_kernel<true><<<grid, GS_THREADS, 0, st>>>(xq, wq, s_a, s_w, static_cast<__nv_bfloat16*>(out), ldo,
+                                                               static_cast<int>(M), static_cast<int>(N),
+                                                               static_cast<int>(K), acc_dbg);
+  return pq_launch_status();
+}

@@ -1,0 +1,226 @@
+// Online Walsh-Hadamard rotation of a linear layer's input (App. B, "Online Rotation") fused with
+// the static per-tensor INT4 quantizer (Table 1, O2; Eq. 1) and the nibble pack; the same
+// butterfly also serves the calibration helper that produces the static scale.
+//
+// A B-wide block (B = 2^LOGB) is transformed by B/64 threads, 64 values per thread, in two
+// register passes joined by one trip through shared memory:
+//   pass 1: thread u loads 32 bf16 pairs (coalesced 4-byte loads, 128 bytes per warp request) and
+//           holds index bits {i0} + the five top bits; six butterfly stages in registers.
+//   exchange: values go to shared memory (8-byte stores, 2 floats of padding per 128 so that the
+//           transposed reads hit 32 distinct banks).
+//   pass 2: thread u' holds index bits i1..i6 of one 128-element segment for one value of i0;
+//           the remaining stages run in registers (plus one lane-shuffle stage when B = 8192).
+//   quantize: clamp, add 1.5*2^23 (the FP add performs the round-half-even), take the low nibble;
+//           lane pairs swap half of their nibbles so that each thread stores 32 contiguous bytes.
+#include "pq_common.cuh"
+
+namespace {
+
+constexpr int HQ_THREADS = 256;
+constexpr int HQ_ELEMS = HQ_THREADS * 64;             // elements handled per CTA iteration
+constexpr int HQ_SMEM_FLOATS = HQ_ELEMS + HQ_ELEMS / 64;  // + 2 floats of padding per 128
+
+template <int LOGB, bool ROTATE, bool CALIB>
+__global__ void __launch_bounds__(HQ_THREADS, 2)
+    hadamard_quant_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int64_t n_rows, int64_t K,
+                          const float* __restrict__ s_a_in, uint8_t* __restrict__ xq, float* __restrict__ s_a_out) {
+  constexpr int B = 1 << LOGB;
+  constexpr int TPB = B / 64;                  // threads per block of the transform
+  constexpr int G = HQ_THREADS / TPB;          // blocks per CTA iteration
+  constexpr int BLK_FLOATS = B + B / 64;       // padded block footprint in shared memory
+  constexpr int RSTRIDE = 1 << (LOGB - 5);     // element distance between consecutive r
+  extern __shared__ __align__(16) float sm[];
+
+  const int tid = threadIdx.x;
+  const int blk_local = tid / TPB;
+  const int u = tid % TPB;
+  const int64_t blocks_per_row = K / B;
+  const int64_t total_blocks = n_rows * blocks_per_row;
+  const int64_t n_super = (total_blocks + G - 1) / G;
+  float* my = sm + blk_local * BLK_FLOATS;
+
+  const float norm = ROTATE ? __fdiv_rn(1.0f, __fsqrt_rn(static_cast<float>(B))) : 1.0f;
+  float inv = norm;
+  if (!CALIB) inv = __fdiv_rn(norm, __ldg(s_a_in));
+  float cal_max = 0.0f;
+
+  for (int64_t sb = blockIdx.x; sb < n_super; sb += gridDim.x) {
+    const int64_t gb = sb * G + blk_local;
+    const bool active = gb < total_blocks;
+    const int64_t row = active ? gb / blocks_per_row : 0;
+    const int64_t col0 = active ? (gb % blocks_per_row) * B : 0;
+
+    // ---- pass 1 --------------------------------------------------------------------------
+    float v[64];
+    {
+      const uint32_t* src = reinterpret_cast<const uint32_t*>(x + row * ldx + col0) + u;
+      uint32_t w[32];
+#pragma unroll
+      for (int r = 0; r < 32; ++r) w[r] = active ? __ldg(src + r * (RSTRIDE / 2)) : 0u;
+#pragma unroll
+      for (int r = 0; r < 32; ++r) {
+        float a = __uint_as_float(w[r] << 16);
+        float b = __uint_as_float(w[r] & 0xFFFF0000u);
+        if (ROTATE) {
+          v[2 * r] = a + b;
+          v[2 * r + 1] = a - b;
+        } else {
+          v[2 * r] = a;
+          v[2 * r + 1] = b;
+        }
+      }
+    }
+    if (ROTATE) {
+#pragma unroll
+      for (int s = 0; s < 5; ++s) {
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+          if ((r & (1 << s)) == 0) {
+            const int r2 = r | (1 << s);
+#pragma unroll
+            for (int p = 0; p < 2; ++p) {
+              float a = v[2 * r + p], b = v[2 * r2 + p];
+              v[2 * r + p] = a + b;
+              v[2 * r2 + p] = a - b;
+            }
+          }
+        }
+      }
+    }
+    // ---- exchange ------------------------------------------------------------------------
+#pragma unroll
+    for (int r = 0; r < 32; ++r) {
+      const int i = r * RSTRIDE + 2 * u;
+      *reinterpret_cast<float2*>(my + i + 2 * (i >> 7)) = make_float2(v[2 * r], v[2 * r + 1]);
+    }
+    __syncthreads();
+    const int seg = u >> 1, par = u & 1;
+    {
+      const float* src = my + seg * 130 + par;
+#pragma unroll
+      for (int q = 0; q < 64; ++q) v[q] = src[2 * q];
+    }
+    __syncthreads();
+    // ---- pass 2 --------------------------------------------------------------------------
+    if (ROTATE) {
+#pragma unroll
+      for (int j = 0; j < 6; ++j) {
+        if (j < LOGB - 6) {
+#pragma unroll
+          for (int q = 0; q < 64; ++q) {
+            if ((q & (1 << j)) == 0) {
+              const int q2 = q | (1 << j);
+              float a = v[q], b = v[q2];
+              v[q] = a + b;
+              v[q2] = a - b;
+            }
+          }
+        }
+      }
+      if (LOGB == 13) {  // index bit 7 lives in lane bit 1
+        const float sgn = (u & 2) ? -1.0f : 1.0f;
+#pragma unroll
+        for (int q = 0; q < 64; ++q) {
+          float o = __shfl_xor_sync(0xffffffffu, v[q], 2);
+          v[q] = fmaf(v[q], sgn, o);
+        }
+      }
+    }
+    if (CALIB) {
+      if (active) {
+#pragma unroll
+        for (int q = 0; q < 64; ++q) cal_max = fmaxf(cal_max, fabsf(v[q] * norm));
+      }
+    } else {
+      // ---- quantize and pack -----------------------------------------------------------------
+      uint32_t pw[16];
+#pragma unroll
+      for (int wd = 0; wd < 16; ++wd) {
+        uint32_t acc = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          float t = fminf(fmaxf(v[wd * 4 + b] * inv, -8.0f), 7.0f);
+          uint32_t bits = __float_as_uint(t + 12582912.0f);
+          acc |= (bits & 0xFu) << (8 * b);
+        }
+        pw[wd] = acc;
+      }
+      uint32_t fin[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        uint32_t send = par ? pw[j] : pw[8 + j];
+        uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
+        fin[j] = par ? (recv | (pw[8 + j] << 4)) : (pw[j] | (recv << 4));
+      }
+      if (active) {
+        uint4* dst = reinterpret_cast<uint4*>(xq + row * (K / 2) + (col0 + seg * 128) / 2 + par * 32);
+        dst[0] = make_uint4(fin[0], fin[1], fin[2], fin[3]);
+        dst[1] = make_uint4(fin[4], fin[5], fin[6], fin[7]);
+      }
+    }
+  }
+  if (CALIB) {
+    for (int o = 16; o > 0; o >>= 1) cal_max = fmaxf(cal_max, __shfl_xor_sync(0xffffffffu, cal_max, o));
+    if ((tid & 31) == 0 && cal_max > 0.0f)
+      atomicMax(reinterpret_cast<int*>(s_a_out), __float_as_int(__fdiv_rn(cal_max, 7.0f)));
+  }
+}
+
+template <int LOGB, bool ROTATE, bool CALIB>
+pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_t K, const float* s_a_in, uint8_t* xq,
+                 float* s_a_out, cudaStream_t st) {
+  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB>;
+  constexpr size_t smem = HQ_SMEM_FLOATS * sizeof(float);
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+    return PQ_ERR_CUDA;
+  constexpr int B = 1 << LOGB;
+  constexpr int G = HQ_THREADS / (B / 64);
+  int64_t n_super = (n_rows * (K / B) + G - 1) / G;
+  int64_t grid = n_super < 2LL * ctx->sm_count ? n_super : 2LL * ctx->sm_count;
+  kern<<<static_cast<int>(grid), HQ_THREADS, smem, st>>>(static_cast<const __nv_bfloat16*>(x), ldx, n_rows, K, s_a_in,
+                                                        xq, s_a_out);
+  return pq_launch_status();
+}
+
+template <bool CALIB>
+pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block, int64_t row_begin,
+                   const float* s_a_in, uint8_t* xq, float* s_a_out, void* stream) {
+  if (!ctx || !x || (!CALIB && (!s_a_in || !xq)) || (CALIB && !s_a_out)) return PQ_ERR_INVALID_ARG;
+  if (M < 0 || K <= 0 || ldx < K || row_begin < 0 || had_block < 0) return PQ_ERR_INVALID_ARG;
+  if (K % 128 != 0) return PQ_ERR_SHAPE;
+  if (had_block != 0) {
+    if ((had_block & (had_block - 1)) != 0 || had_block < 128 || had_block > 8192 || K % had_block != 0)
+      return PQ_ERR_SHAPE;
+  }
+  if ((ldx & 1) || (reinterpret_cast<uintptr_t>(x) & 3)) return PQ_ERR_ALIGN;
+  if (!CALIB && (reinterpret_cast<uintptr_t>(xq) & 15)) return PQ_ERR_ALIGN;
+  if (row_begin >= M) return PQ_OK;
+  const int64_t n_rows = M - row_begin;
+  const void* x0 = static_cast<const __nv_bfloat16*>(x) + row_begin * ldx;
+  uint8_t* xq0 = CALIB ? nullptr : xq + row_begin * (K / 2);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  switch (had_block) {
+    case 0: return launch<7, false, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 128: return launch<7, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 256: return launch<8, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 512: return launch<9, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 1024: return launch<10, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 2048: return launch<11, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 4096: return launch<12, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 8192: return launch<13, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    default: return PQ_ERR_SHAPE;
+  }
+}
+
+}  // namespace
+
+extern "C" pq_status pq_hadamard_quant_act(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx,
+                                           int had_block, int64_t row_begin, const float* s_a, uint8_t* xq,
+                                           void* stream) {
+  return dispatch<false>(ctx, x, M, K, ldx, had_block, row_begin, s_a, xq, nullptr, stream);
+}
+
+extern "C" pq_status pq_calib_act_scale(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                        int64_t row_begin, float* s_a, void* stream) {
+  return dispatch<true>(ctx, x, M, K, ldx, had_block, row_begin, nullptr, nullptr, s_a, stream);
+}

@@ -1,0 +1,265 @@
+"""GPU parity: every entry point of the C-ABI library against the CPU oracle on the same seeded
+inputs, element by element. Integer results bit-exact; tolerances as stated in helpers.py."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import pq_oracle as orc
+from paper_2410_05265_b200 import inputs
+from helpers import (assert_attn_close, assert_bf16_close, assert_codes_tie_tolerant, rand_codes, to_np)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2410_05265_b200 import binding
+
+    c = binding.Context()
+    yield c
+    c.check()
+    c.close()
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.view(dtype)
+    return t.cuda()
+
+
+# ------------------------------------------------------------------------------- a0 weights
+@pytest.mark.parametrize("N,K", [(64, 256), (301, 4096), (16, 14336)])
+def test_quant_weights_bit_exact(ctx, N, K):
+    W = inputs.weights(N, K, seed=2)
+    if N > 5:
+        W[5] = 0
+    wq_ref, sw_ref = orc.quant_weights(inputs.bits(W))
+    wq, s_w = ctx.quant_weights(W.cuda())
+    ctx.check()
+    assert np.array_equal(to_np(s_w), sw_ref)
+    assert np.array_equal(to_np(wq), wq_ref)
+
+
+# ------------------------------------------------------------------------------- a1 rotation + quantizer
+@pytest.mark.parametrize("M,K,B,row_begin", [
+    (5, 128, 128, 0), (37, 768, 256, 0), (19, 1024, 1024, 3), (70, 6144, 2048, 4), (33, 4096, 4096, 0),
+    (9, 8192, 8192, 1), (300, 4096, 4096, 4), (21, 384, 0, 2),
+])
+def test_hadamard_quant_act_matches_oracle(ctx, M, K, B, row_begin):
+    x = inputs.activations(M, K, seed=0, n_prefix=row_begin)
+    cal = inputs.activations(max(M, 16), K, seed=1, n_prefix=row_begin)
+    s_ref = orc.calib_act_scale(inputs.bits(cal), B, row_begin)
+    s_gpu = ctx.calib_act_scale(cal.cuda(), B, row_begin)
+    ctx.check()
+    assert abs(float(s_gpu[0]) - float(s_ref)) <= 2e-6 * float(s_ref)
+    s_a = torch.tensor([s_ref], dtype=torch.float32, device="cuda")
+    xq_ref, tie = orc.quant_act(inputs.bits(x), B, s_ref, row_begin, want_tie_dist=True)
+    out = torch.full((M, K // 2), 0x5A, dtype=torch.uint8, device="cuda")
+    ctx.hadamard_quant_act(x.cuda(), B, s_a, row_begin, out=out)
+    ctx.check()
+    got = to_np(out)
+    assert np.all(got[:row_begin] == 0x5A), "prefix rows must not be written"
+    n_mis = assert_codes_tie_tolerant(got[row_begin:], xq_ref[row_begin:], tie[row_begin:], "hadamard_quant_act")
+    assert n_mis <= max(2, int(2e-4 * x.numel()))
+    # isolation: the same rows quantize identically when the prefix rows are absent
+    if row_begin:
+        out2 = ctx.hadamard_quant_act(x[row_begin:].cuda().contiguous(), B, s_a)
+        assert torch.equal(out2, out[row_begin:])
+
+
+def test_hadamard_quant_prefix_outliers_never_set_scale(ctx):
+    x = inputs.activations(64, 4096, seed=1, n_prefix=4)
+    s1 = ctx.calib_act_scale(x.cuda(), 4096, 4)
+    x2 = x.clone()
+    x2[:4] *= 100.0
+    s2 = ctx.calib_act_scale(x2.cuda(), 4096, 4)
+    s0 = ctx.calib_act_scale(x.cuda(), 4096, 0)
+    ctx.check()
+    assert float(s1) == float(s2) and float(s0) > 5 * float(s1)
+
+
+# ------------------------------------------------------------------------------- a2 / a3 GEMM
+def _gemm_case(ctx, M, N, K, seed, row_begin=0, real_scales=True):
+    rng = np.random.default_rng(seed)
+    xq = rand_codes(rng, M, K)
+    wq = rand_codes(rng, N, K)
+    s_a = np.float32(0.0173)
+    s_w = (rng.random(N) * 0.004 + 0.001).astype(np.float32)
+    acc_ref = orc.gemm_i4(xq, wq)
+    out_ref = orc.dequant_bf16(acc_ref, s_a, s_w)
+    acc = torch.full((M, N), -77, dtype=torch.int32, device="cuda")
+    out = torch.full((M, N), 3.0, dtype=torch.bfloat16, device="cuda")
+    ctx.w4a4_gemm(dev(xq), dev(wq), torch.tensor([s_a], device="cuda"), dev(s_w), row_begin, out=out, acc_dbg=acc)
+    ctx.check()
+    acc = to_np(acc)
+    assert np.all(acc[:row_begin] == -77) and np.all(to_np(out[:row_begin].float()) == 3.0)
+    assert np.array_equal(acc[row_begin:], acc_ref[row_begin:]), "int32 accumulators must be bit-exact"
+    assert_bf16_close(inputs.bits(out)[row_begin:], out_ref[row_begin:], f"gemm {M}x{N}x{K}")
+
+
+@pytest.mark.parametrize("M,N,K", [
+    (128, 256, 128),     # one tile, one K block
+    (128, 256, 512),     # one tile, ring wraps
+    (256, 512, 4096),    # several tiles per CTA pipeline
+    (200, 264, 416),     # ragged M, N and K (K % 128 != 0)
+    (17, 40, 160),       # smallest tensor-core case, mostly padding
+    (333, 1000, 2048),
+])
+def test_gemm_prefill_shapes_bit_exact(ctx, M, N, K):
+    _gemm_case(ctx, M, N, K, seed=M + N + K)
+
+
+def test_gemm_many_tiles_persistent_schedule(ctx):
+    _gemm_case(ctx, 1024, 6144, 1024, seed=5)      # 192 tiles: CTAs take a second tile
+
+
+def test_gemm_row_begin_skips_prefix_rows(ctx):
+    _gemm_case(ctx, 260, 256, 256, seed=11, row_begin=4)
+    _gemm_case(ctx, 12, 64, 256, seed=12, row_begin=4)
+
+
+@pytest.mark.parametrize("M", [1, 4, 8, 9, 16])
+@pytest.mark.parametrize("N,K", [(48, 4096), (1024, 4096), (40, 160), (4096, 14336)])
+def test_gemm_decode_shapes_bit_exact(ctx, M, N, K):
+    if N * K > 1 << 24 and M not in (1, 16):
+        pytest.skip("large shape covered at M=1 and M=16")
+    _gemm_case(ctx, M, N, K, seed=M * 7 + N)
+
+
+def test_gemm_extreme_codes_fit_int32(ctx):
+    M, N, K = 128, 256, 28672
+    xq = np.full((M, K // 2), 0x88, np.uint8)   # every code -8
+    wq = np.full((N, K // 2), 0x88, np.uint8)
+    acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    ctx.w4a4_gemm(dev(xq), dev(wq), torch.ones(1, device="cuda"), torch.ones(N, device="cuda"), acc_dbg=acc)
+    ctx.check()
+    assert int(acc.min()) == int(acc.max()) == 64 * K
+
+
+# ------------------------------------------------------------------------------- a1 -> a2 (config 0)
+def test_linear_end_to_end_config0(ctx):
+    M, K, N = 256, 4096, 4096
+    x = inputs.activations(M, K, seed=0)
+    cal = inputs.activations(M, K, seed=1)
+    W = inputs.weights(N, K, seed=2)
+    s_ref = orc.calib_act_scale(inputs.bits(cal), K)
+    xq_ref, tie = orc.quant_act(inputs.bits(x), K, s_ref, want_tie_dist=True)
+    wq_ref, sw_ref = orc.quant_weights(inputs.bits(W))
+    out_ref = orc.dequant_bf16(orc.gemm_i4(xq_ref, wq_ref), s_ref, sw_ref)
+    s_a = torch.tensor([s_ref], device="cuda")
+    wq, s_w = ctx.quant_weights(W.cuda())
+    xq = ctx.hadamard_quant_act(x.cuda(), K, s_a)
+    out = ctx.w4a4_gemm(xq, wq, s_a, s_w)
+    ctx.check()
+    assert np.array_equal(to_np(wq), wq_ref) and np.array_equal(to_np(s_w), sw_ref)
+    n_mis = assert_codes_tie_tolerant(to_np(xq), xq_ref, tie, "config0 codes")
+    rows_clean = ~(orc.unpack_int4(to_np(xq)) != orc.unpack_int4(xq_ref)).any(axis=1)
+    assert rows_clean.sum() >= M - n_mis
+    assert_bf16_close(inputs.bits(out)[rows_clean], out_ref[rows_clean], "config0 output")
+    # a row with a counted tie mismatch moves by at most one product per mismatch
+    if n_mis:
+        g = orc.bf16_to_f64(inputs.bits(out)[~rows_clean])
+        r = orc.bf16_to_f64(out_ref[~rows_clean])
+        assert np.all(np.abs(g - r) <= n_mis * 8 * float(s_ref) * sw_ref.max() + 2e-3 + np.abs(r) * 2.0**-7)
+
+
+# ------------------------------------------------------------------------------- a4 / a5 KV cache
+def _kv_setup(B, Hq, Hkv, D, P, T, Tmax, mag, seed=0, lens=None):
+    k = inputs.kv_tensor(B, T, Hkv, D, seed, "k")
+    v = inputs.kv_tensor(B, T, Hkv, D, seed, "v")
+    s_k = orc.calib_kv_scale(inputs.bits(inputs.kv_tensor(2, 64, Hkv, D, 1, "k")))
+    s_v = orc.calib_kv_scale(inputs.bits(inputs.kv_tensor(2, 64, Hkv, D, 1, "v")))
+    pk = inputs.prefix_kv(Hkv, P, D, seed, "k", mag)
+    pv = inputs.prefix_kv(Hkv, P, D, seed, "v", mag)
+    q = inputs.queries(B, Hq, D, seed)
+    return k, v, s_k, s_v, pk, pv, q
+
+
+def _run_attention(ctx, B, Hq, Hkv, P, T, Tmax, mag, seed=0, start=None):
+    from paper_2410_05265_b200 import binding
+
+    D = 128
+    k, v, s_k, s_v, pk, pv, q = _kv_setup(B, Hq, Hkv, D, P, T, Tmax, mag, seed)
+    start = np.zeros(B, np.int32) if start is None else np.asarray(start, np.int32)
+    # oracle
+    kq_ref = np.full((B, Hkv, Tmax, D // 2), 0x11, np.uint8)
+    vq_ref = np.full((B, Hkv, Tmax, D // 2), 0x11, np.uint8)
+    len_ref = start.copy()
+    assert orc.kv4_append(inputs.bits(k), inputs.bits(v), s_k, s_v, kq_ref, vq_ref, len_ref) == 0
+    out_ref = orc.decode_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq_ref, vq_ref, s_k, s_v, len_ref,
+                              1 / math.sqrt(D))
+    # GPU
+    kq = torch.full((B, Hkv, Tmax, D // 2), 0x11, dtype=torch.uint8, device="cuda")
+    vq = torch.full((B, Hkv, Tmax, D // 2), 0x11, dtype=torch.uint8, device="cuda")
+    length = dev(start)
+    cache = binding.KV4Cache(pk.cuda() if P else None, pv.cuda() if P else None, kq, vq, dev(s_k), dev(s_v), length, Hq)
+    ctx.kv4_append(cache, k.cuda(), v.cuda())
+    ctx.check()
+    assert np.array_equal(to_np(length), len_ref)
+    assert np.array_equal(to_np(kq), kq_ref) and np.array_equal(to_np(vq), vq_ref), "KV4 codes must match bit for bit"
+    ws = ctx.decode_attn_workspace(cache)
+    out = ctx.decode_attn(cache, q.cuda(), 1 / math.sqrt(D), ws)
+    ctx.check()
+    worst = assert_attn_close(inputs.bits(out), out_ref, f"decode attention B{B} Hq{Hq} T{T} P{P} mag{mag}")
+    # a second call on the same cache must give the same bits (ticket counters reset themselves)
+    out2 = ctx.decode_attn(cache, q.cuda(), 1 / math.sqrt(D), ws)
+    assert torch.equal(out, out2)
+    return worst
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,P,T,Tmax,mag", [
+    (1, 4, 1, 0, 16, 16, 1.0),       # one block, no prefix
+    (2, 8, 2, 2, 100, 128, 1.0),     # ragged tail inside a 16-key block
+    (3, 32, 8, 4, 333, 400, 1.0),    # GQA 4, several splits
+    (2, 16, 2, 4, 1000, 1024, 50.0), # GQA 8, dominant prefix keys
+    (1, 8, 8, 1, 5, 64, 1.0),        # fewer keys than one block, MHA
+])
+def test_kv4_append_and_decode_attention(ctx, B, Hq, Hkv, P, T, Tmax, mag):
+    _run_attention(ctx, B, Hq, Hkv, P, T, Tmax, mag)
+
+
+def test_decode_attention_config3_variants(ctx):
+    # config 3 (prefix magnitude ~50 makes most heads one-hot on a prefix key), plus the variants
+    # that put the weight on the INT4 region: magnitude 1 and no prefix at all
+    for P, mag in [(4, 50.0), (4, 1.0), (0, 1.0)]:
+        _run_attention(ctx, 8, 32, 8, P, 4092, 4096, mag)
+
+
+def test_decode_attention_ragged_lengths_and_empty_cache(ctx):
+    # appending one token to sequences of different lengths, one of them empty
+    _run_attention(ctx, 4, 8, 2, 2, 1, 64, 1.0, start=[0, 5, 31, 63])
+    _run_attention(ctx, 2, 8, 2, 0, 3, 64, 1.0, start=[0, 40])
+
+
+def test_kv4_append_refuses_overflow(ctx):
+    from paper_2410_05265_b200 import binding
+
+    B, Hkv, D, Tmax = 2, 2, 128, 8
+    k = inputs.kv_tensor(B, 3, Hkv, D, 0, "k").cuda()
+    kq = torch.zeros((B, Hkv, Tmax, D // 2), dtype=torch.uint8, device="cuda")
+    vq = torch.zeros_like(kq)
+    length = torch.tensor([2, 6], dtype=torch.int32, device="cuda")
+    s = torch.ones(Hkv, device="cuda")
+    cache = binding.KV4Cache(None, None, kq, vq, s, s, length, 4)
+    ctx.kv4_append(cache, k, k)
+    assert ctx.check_status() == 2  # PQ_ERR_SHAPE, reported through the status word
+    assert length.tolist() == [2, 6] and int(kq.sum()) == 0
+    assert ctx.check_status() == 0  # the status word was cleared
+
+
+def test_argument_errors_are_synchronous(ctx):
+    from paper_2410_05265_b200.binding import PQError
+
+    x = torch.zeros((4, 96), dtype=torch.bfloat16, device="cuda")
+    s = torch.ones(1, device="cuda")
+    with pytest.raises(PQError):
+        ctx.hadamard_quant_act(x, 0, s)            # K % 128 != 0
+    x = torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(PQError):
+        ctx.hadamard_quant_act(x, 192, s)          # not a power of two
+    xq = torch.zeros((4, 24), dtype=torch.uint8, device="cuda")
+    with pytest.raises(PQError):
+        ctx.w4a4_gemm(xq, xq, s, torch.ones(4, device="cuda"))   # K = 48 not a multiple of 32
