@@ -1,0 +1,467 @@
+#!/usr/bin/env python
+"""Benchmark of the W4A4KV4 hot path.
+
+A step is one pass of the Llama-3-8B-shaped linear set at prefill (M = 2048 tokens, 4 of them
+prefixed outlier tokens that the W4A4 path skips): for each of the four distinct layer inputs one
+fused rotate+quantize call, then the W4A4 GEMMs (q|k|v and gate|up concatenated along N, o, down).
+The metric is integer tera-operations per second over the GEMM work of the step (2*M*N*K), the
+rotate+quantize kernels included in the time. Extra sections report the decode-shaped GEMMs and
+the KV4 decode attention in GB/s. `--impl reference` times the CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "w4a4_prefill_linear_set_tops"
+UNIT = "TOPS"
+M_TOKENS = 2048
+N_PREFIX = 4
+NOMINAL_INT8_TOPS = 4500.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def linear_launches():
+    """(name, N, K, had_block, input id) of the launches of one step; logical layers in the name."""
+    from paper_2410_05265_b200 import inputs
+
+    c = inputs.LLAMA3_8B
+    h, kv, f = c["hidden"], c["kv_dim"], c["ffn"]
+    return [
+        ("q|k|v", h + 2 * kv, h, h, 0),
+        ("o", h, h, h, 1),
+        ("gate|up", 2 * f, h, h, 2),
+        ("down", h, f, 2048, 3),
+    ]
+
+
+def step_ops(m_rows: int) -> float:
+    return sum(2.0 * m_rows * n * k for _, n, k, _, _ in linear_launches())
+
+
+def read_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], bf16=d["bf16_tflops"], bf16_sus=d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                    src="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sus=1400.0, src="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])), mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------- GPU arm
+def build_workload(ctx, device):
+    """Synthetic Llama-3-8B-shaped tensors, weights quantized offline, static scales calibrated on
+    the seed-1 batch over the non-prefix rows."""
+    import torch
+
+    from paper_2410_05265_b200 import inputs
+
+    L = linear_launches()
+    acts, scales, wqs, sws = [], [], [], []
+    for i, (name, N, K, had, inp) in enumerate(L):
+        x = inputs.activations(M_TOKENS, K, seed=0, n_prefix=N_PREFIX, layer=inp, device=device)
+        cal = inputs.activations(M_TOKENS, K, seed=1, n_prefix=N_PREFIX, layer=inp, device=device)
+        s_a = ctx.calib_act_scale(cal, had, N_PREFIX)
+        del cal
+        W = inputs.weights(N, K, seed=2 + i, device=device)
+        wq, s_w = ctx.quant_weights(W)
+        del W
+        acts.append(x), scales.append(s_a), wqs.append(wq), sws.append(s_w)
+    torch.cuda.synchronize()
+    return L, acts, scales, wqs, sws
+
+
+def run_gpu(args):
+    import torch
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+
+    from paper_2410_05265_b200 import binding, build as pq_build
+
+    if rank == 0:
+        pq_build.build()
+    if dist:
+        dist.barrier()
+    ctx = binding.Context()
+    L, acts, scales, wqs, sws = build_workload(ctx, device)
+    m_rows = M_TOKENS - N_PREFIX
+    xqs = [torch.zeros((M_TOKENS, K // 2), dtype=torch.uint8, device=device) for _, _, K, _, _ in L]
+    outs = [torch.zeros((M_TOKENS, N), dtype=torch.bfloat16, device=device) for _, N, _, _, _ in L]
+
+    def step(gemm_events=None):
+        for i, (name, N, K, had, inp) in enumerate(L):
+            ctx.hadamard_quant_act(acts[i], had, scales[i], N_PREFIX, out=xqs[i])
+            if gemm_events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            ctx.w4a4_gemm(xqs[i], wqs[i], scales[i], sws[i], N_PREFIX, out=outs[i])
+            if gemm_events is not None:
+                e1.record()
+                gemm_events.append((i, e0, e1))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    ctx.check()
+    # ---- timed region: device-resident inputs -------------------------------------------------
+    sampler = ClockSampler(local)
+    gemm_events = []
+    barrier()
+    sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        step(gemm_events)
+    t1.record()
+    barrier()
+    clocks = sampler.stop()
+    ctx.check()
+    ms = t0.elapsed_time(t1)
+    if dist:
+        tmax = torch.tensor([ms], device=device)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms = float(tmax.item())
+    ms_per_step = ms / args.steps
+    value = world * step_ops(m_rows) / (ms_per_step * 1e-3) / 1e12
+
+    gemm_ms = sum(e0.elapsed_time(e1) for _, e0, e1 in gemm_events)
+    per_shape = {}
+    for i, e0, e1 in gemm_events:
+        per_shape.setdefault(L[i][0], []).append(e0.elapsed_time(e1))
+    gemm_ops = args.steps * step_ops(m_rows)
+    peaks = read_peaks()
+    int8_peak = 2.0 * peaks["bf16_sus"]  # dense INT8 = 2x dense bf16 (nominal ratio 4.5 / 2.25 PFLOP/s)
+    achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
+    roofline = {
+        "kernel": "gemm_w4a4_tc_kernel", "bound": "tensor", "achieved": round(achieved, 1), "peak": round(int8_peak, 1),
+        "unit": "TOPS", "frac": round(achieved / int8_peak, 4), "traffic": None,
+        "peak_source": f"2 x bf16 sustained GEMM of {peaks['src']}", "frac_of_nominal_4500": round(achieved / NOMINAL_INT8_TOPS, 4),
+        "frac_of_2x_bf16_burst": round(achieved / (2.0 * peaks["bf16"]), 4),
+        "per_launch": {k: {"ms": round(statistics.mean(v), 4),
+                           "tops": round(2.0 * m_rows * next(n * kk for nm, n, kk, _, _ in L if nm == k) /
+                                         (statistics.mean(v) * 1e-3) / 1e12, 1)} for k, v in per_shape.items()},
+    }
+
+    # ---- end to end: host buffers in, host buffers out, through the same calls ----------------------
+    h_acts = [a.cpu().pin_memory() for a in acts]
+    h_outs = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in outs]
+    d_acts = [torch.empty_like(a) for a in acts]
+    h2d = sum(a.numel() * a.element_size() for a in h_acts)
+    d2h = sum(o.numel() * o.element_size() for o in h_outs)
+
+    def e2e_step():
+        for i, (name, N, K, had, inp) in enumerate(L):
+            d_acts[i].copy_(h_acts[i], non_blocking=True)
+            ctx.hadamard_quant_act(d_acts[i], had, scales[i], N_PREFIX, out=xqs[i])
+            ctx.w4a4_gemm(xqs[i], wqs[i], scales[i], sws[i], N_PREFIX, out=outs[i])
+            h_outs[i].copy_(outs[i], non_blocking=True)
+
+    e2e_steps = max(2, min(args.steps, 10))
+    e2e_step()
+    barrier()
+    w0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = time.perf_counter() - w0
+    if dist:
+        tmax = torch.tensor([e2e_s], device=device)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        e2e_s = float(tmax.item())
+    e2e_value = world * step_ops(m_rows) * e2e_steps / e2e_s / 1e12
+
+    sections, cpu_baseline = None, None
+    if rank == 0 and world == 1 and not args.no_sections:
+        sections = {}
+        try:
+            sections["decode_gemm"] = section_decode_gemm(ctx, device, peaks)
+            sections["decode_attention"] = section_decode_attention(ctx, device, peaks)
+        except Exception as e:  # sections never take the main line down
+            sections["error"] = repr(e)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = oracle_sample(16)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "s4 x s4 -> s32 (tcgen05 kind::i8 on 16*code), fp32 epilogue, bf16 out",
+            "data": "synthetic",
+            "config": {"workload": "configs[1]: Llama-3-8B linear set, prefill M=2048 (4 prefixed rows skipped), batch 1",
+                       "launches_per_step": "4 x hadamard_quant_act + 4 x w4a4_gemm (q|k|v and gate|up concatenated along N)",
+                       "l2": "inputs larger than L2: a step touches ~400 MB (weights 109 MB, activations 109 MB, outputs 176 MB) against 126 MB",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks, "roofline": roofline,
+            "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": args.steps * 2 * len(L),
+        }
+        if cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline
+        if sections:
+            line["sections"] = sections
+        print(json.dumps(line))
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def _graph_time(torch, fn, n_inner, reps=5):
+    """Captures n_inner calls of fn(i) in a CUDA graph and returns the best ms per call."""
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            for i in range(n_inner):
+                fn(i)
+        g.replay()
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1) / n_inner)
+    torch.cuda.current_stream().wait_stream(s)
+    return best
+
+
+def section_decode_gemm(ctx, device, peaks):
+    """configs[2]: M in {1,4,16} through the Llama-3-8B shapes; 8 distinct weight copies visited
+    round-robin (872 MB > L2) so the weights stream from HBM; 1000 calls in a CUDA graph."""
+    import torch
+
+    from paper_2410_05265_b200 import inputs
+
+    res = {}
+    n_copies = 8
+    for name, N, K, had, inp in linear_launches():
+        wq = torch.randint(0, 256, (n_copies, N, K // 2), dtype=torch.uint8, device=device)
+        s_w = torch.full((N,), 0.003, device=device)
+        s_a = torch.full((1,), 0.05, device=device)
+        for M in (1, 4, 16):
+            xq = torch.randint(0, 256, (M, K // 2), dtype=torch.uint8, device=device)
+            out = torch.zeros((M, N), dtype=torch.bfloat16, device=device)
+            ms = _graph_time(torch, lambda i: ctx.w4a4_gemm(xq, wq[i % n_copies], s_a, s_w, out=out), 1000)
+            by = N * K // 2 + N * 4 + M * K // 2 + M * N * 2
+            gbs = by / (ms * 1e-3) / 1e9
+            res[f"{name} M={M}"] = {"us": round(ms * 1e3, 3), "GB/s": round(gbs, 1), "frac_measured_hbm": round(gbs / peaks["hbm"], 3),
+                                    "frac_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 3)}
+        del wq
+    ctx.check()
+    return res
+
+
+def section_decode_attention(ctx, device, peaks):
+    """configs[3]: batch 8, 32 query / 8 KV heads, head_dim 128, 4 fp16 prefix entries + 4092 INT4
+    entries; 32 distinct cache layers (1.07 GB) visited round-robin; one append + one attention per step."""
+    import torch
+
+    from paper_2410_05265_b200 import binding, inputs
+
+    B, Hq, Hkv, D, P, T, Tmax, layers = 8, 32, 8, 128, 4, 4091, 4096, 32
+    pk = inputs.prefix_kv(Hkv, P, D, 0, "k", 50.0, device=device)
+    pv = inputs.prefix_kv(Hkv, P, D, 0, "v", 50.0, device=device)
+    s_k = torch.full((Hkv,), 4.5 / 7, device=device)
+    s_v = torch.full((Hkv,), 4.5 / 7, device=device)
+    caches = []
+    for _ in range(layers):
+        kq = torch.randint(0, 256, (B, Hkv, Tmax, D // 2), dtype=torch.uint8, device=device)
+        vq = torch.randint(0, 256, (B, Hkv, Tmax, D // 2), dtype=torch.uint8, device=device)
+        length = torch.full((B,), T, dtype=torch.int32, device=device)
+        caches.append(binding.KV4Cache(pk, pv, kq, vq, s_k, s_v, length, Hq))
+    q = inputs.queries(B, Hq, D, 0, device=device)
+    k1 = inputs.kv_tensor(B, 1, Hkv, D, 0, "k", device=device)
+    v1 = inputs.kv_tensor(B, 1, Hkv, D, 0, "v", device=device)
+    ws = ctx.decode_attn_workspace(caches[0])
+    out = torch.empty_like(q)
+    sm = 1 / math.sqrt(D)
+
+    def reset():
+        for c in caches:
+            c.length.fill_(T)
+
+    def both(i):
+        c = caches[i % layers]
+        ctx.kv4_append(c, k1, v1)
+        ctx.decode_attn(c, q, sm, ws, out=out)
+
+    def attn_only(i):
+        ctx.decode_attn(caches[i % layers], q, sm, ws, out=out)
+
+    def append_only(i):
+        ctx.kv4_append(caches[i % layers], k1, v1)
+
+    reset()
+    ms_attn = _graph_time(torch, attn_only, 320)
+    # each layer is appended to at most (3 + 32 * 7) / 32 + 1 < 9 times below: start low enough
+    for c in caches:
+        c.length.fill_(T - 40)
+    ms_app = _graph_time(torch, append_only, 32, reps=3)
+    for c in caches:
+        c.length.fill_(T - 40)
+    ms_both = _graph_time(torch, both, 32, reps=3)
+    ctx.check()
+    by = B * Hkv * (T + 1) * (D // 2) * 2 + Hkv * P * D * 2 * 2 + 2 * B * Hq * D * 2 + 2 * Hkv * 4
+    gbs = by / (ms_attn * 1e-3) / 1e9
+    return {"attention_us": round(ms_attn * 1e3, 3), "append_us": round(ms_app * 1e3, 3), "append+attention_us": round(ms_both * 1e3, 3),
+            "GB/s": round(gbs, 1), "frac_measured_hbm": round(gbs / peaks["hbm"], 3), "frac_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 3),
+            "bytes_per_step": by}
+
+
+# ------------------------------------------------------------------------------------- CPU oracle arms
+def oracle_sample(rows: int):
+    """Times the CPU oracle, as it stands, on `rows` non-prefix token rows of the same workload
+    through all seven linears (rotation, quantizer, integer GEMM, dequantization)."""
+    import numpy as np
+
+    from oracle import pq_oracle as orc
+    from paper_2410_05265_b200 import inputs
+
+    L = linear_launches()
+    prepared = []
+    rng = np.random.default_rng(0)
+    for i, (name, N, K, had, inp) in enumerate(L):
+        x = inputs.activations(N_PREFIX + rows, K, seed=0, n_prefix=N_PREFIX, layer=inp)
+        wq = rng.integers(0, 256, (N, K // 2)).astype(np.uint8)  # weight codes: offline work, not timed
+        s_w = np.full((N,), 0.003, np.float32)
+        prepared.append((inputs.bits(x), wq, s_w, K, had))
+    t0 = time.perf_counter()
+    for xb, wq, s_w, K, had in prepared:
+        s_a = np.float32(0.25)
+        xq = orc.quant_act(xb, had, s_a, N_PREFIX)
+        acc = orc.gemm_i4(xq[N_PREFIX:], wq)
+        orc.dequant_bf16(acc, s_a, s_w)
+    dt = time.perf_counter() - t0
+    return {"value": round(step_ops(rows) / dt / 1e12, 6), "unit": UNIT, "cores": orc.get_threads(), "kind": "oracle",
+            "sample": f"{rows} of {M_TOKENS - N_PREFIX} non-prefix token rows through all 7 linears (rotate, quantize, int GEMM, dequant)",
+            "seconds": round(dt, 2)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    rows = 4
+    for _ in range(args.warmup):
+        oracle_sample(1)
+    t0 = time.perf_counter()
+    last = None
+    for _ in range(args.steps):
+        last = oracle_sample(rows)
+    dt = time.perf_counter() - t0
+    value = step_ops(rows) * args.steps / dt / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": round(value, 6), "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(dt / args.steps * 1e3, 2), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64 / int64 (CPU oracle)", "data": "synthetic",
+        "config": {"workload": "configs[1]: Llama-3-8B linear set, prefill M=2048 (4 prefixed rows skipped), batch 1",
+                   "sample": f"each step = {rows} token rows through all 7 linears"},
+        "cpu_baseline": {"value": round(value, 6), "unit": UNIT, "cores": last["cores"], "kind": "oracle", "sample": last["sample"]},
+        "e2e": {"value": round(value, 6), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-sections", action="store_true", help="skip the decode GEMM / decode attention sections")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

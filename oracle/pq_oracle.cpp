@@ -7,9 +7,10 @@
 //
 // Conventions
 //   * bf16 / fp16 tensors are passed as raw uint16 bit patterns, decoded exactly to double.
-//   * All floating-point work is double, except weight quantization, where the decision that
-//     produces an integer code is taken in IEEE fp32 (division, round-half-even) because that
-//     is the precision the offline GPU kernel uses for the same decision.
+//   * All floating-point work is double, except weight and KV quantization, where the decision
+//     that produces an integer code is taken in IEEE fp32 (division, round-half-even) because
+//     that is the precision the GPU kernels use for the same decision (bf16 inputs, fp32 steps:
+//     exact ties of x / (max/7) do occur, and only an equal-precision decision is reproducible).
 //   * Packed INT4: element 2j in the low nibble, element 2j+1 in the high nibble, two's
 //     complement, packed along the contraction (or head) dimension.
 //   * Threading is over independent rows only; arithmetic per row is strictly sequential.
@@ -309,10 +310,13 @@ int orc_kv4_append(const uint16_t* k, const uint16_t* v, int64_t B, int64_t T_ne
         uint8_t* kr = kq + ((b * H + h) * Tmax + pos) * (D / 2);
         uint8_t* vr = vq + ((b * H + h) * Tmax + pos) * (D / 2);
         for (int64_t d = 0; d < D; ++d) {
-          double kv = bf16_to_double(k[((b * T_new + t) * H + h) * D + d]);
-          double vv = bf16_to_double(v[((b * T_new + t) * H + h) * D + d]);
-          nib_set(kr, d, clampi(std::lrint(std::nearbyint(kv / static_cast<double>(s_k[h]))), -8, 7));
-          nib_set(vr, d, clampi(std::lrint(std::nearbyint(vv / static_cast<double>(s_v[h]))), -8, 7));
+          // the code is decided in IEEE fp32 (bf16 input, fp32 step), the precision of the GPU kernel
+          float kf = static_cast<float>(bf16_to_double(k[((b * T_new + t) * H + h) * D + d]));
+          float vf = static_cast<float>(bf16_to_double(v[((b * T_new + t) * H + h) * D + d]));
+          volatile float qk = kf / s_k[h];
+          volatile float qv = vf / s_v[h];
+          nib_set(kr, d, clampi(static_cast<long>(std::nearbyintf(qk)), -8, 7));
+          nib_set(vr, d, clampi(static_cast<long>(std::nearbyintf(qv)), -8, 7));
         }
       }
     len[b] += static_cast<int32_t>(T_new);

@@ -175,8 +175,9 @@ __global__ void __launch_bounds__(N_THREADS, 1)
       for (int kb = 0; kb < n_kb; ++kb, ++it) {
         const uint32_t ps = it % N_PK, pph = (it / N_PK) & 1;
         const uint32_t ss = it % N_S8, sph = (it / N_S8) & 1;
-        if (bars->abort_flag || !pq::mbar_wait(&bars->pk_full[ps], pph) ||
-            !pq::mbar_wait(&bars->s8_empty[ss], sph ^ 1)) {
+        const bool stuck = bars->abort_flag || !pq::mbar_wait(&bars->pk_full[ps], pph) ||
+                           !pq::mbar_wait(&bars->s8_empty[ss], sph ^ 1);
+        if (__any_sync(0xffffffffu, stuck)) {  // warp-uniform decision
           ok = false;
           break;
         }
@@ -219,7 +220,8 @@ __global__ void __launch_bounds__(N_THREADS, 1)
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
       const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
       const uint32_t ab = tcount & 1, aph = (tcount >> 1) & 1;
-      if (bars->abort_flag || !pq::mbar_wait(&bars->acc_full[ab], aph)) {
+      const bool stuck = bars->abort_flag || !pq::mbar_wait(&bars->acc_full[ab], aph);
+      if (__any_sync(0xffffffffu, stuck)) {  // warp-uniform: the TMEM loads below are warp-collective
         ok = false;
         break;
       }

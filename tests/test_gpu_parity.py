@@ -189,8 +189,8 @@ def _run_attention(ctx, B, Hq, Hkv, P, T, Tmax, mag, seed=0, start=None):
     vq_ref = np.full((B, Hkv, Tmax, D // 2), 0x11, np.uint8)
     len_ref = start.copy()
     assert orc.kv4_append(inputs.bits(k), inputs.bits(v), s_k, s_v, kq_ref, vq_ref, len_ref) == 0
-    out_ref = orc.decode_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq_ref, vq_ref, s_k, s_v, len_ref,
-                              1 / math.sqrt(D))
+    _, out_ref = orc.decode_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq_ref, vq_ref, s_k, s_v, len_ref,
+                                 1 / math.sqrt(D), want_f64=True)
     # GPU
     kq = torch.full((B, Hkv, Tmax, D // 2), 0x11, dtype=torch.uint8, device="cuda")
     vq = torch.full((B, Hkv, Tmax, D // 2), 0x11, dtype=torch.uint8, device="cuda")

@@ -274,7 +274,7 @@ def test_kv_scale_and_append():
         for h in range(H):
             r = kf[b, :, h, :] / np.float64(s_k[h])
             got = kcodes[b, h, l0:l0 + T]
-            assert np.all(np.abs(got - np.clip(r, -8, 7)) <= 0.5 + 1e-12)
+            assert np.all(np.abs(got - np.clip(r, -8, 7)) <= 0.5 + 1e-6)  # decided in fp32
             assert np.all(kq[b, h, :l0] == 0xEE) and np.all(kq[b, h, l0 + T:] == 0xEE)  # nothing else touched
     # a sequence that would overflow Tmax is refused and nothing moves
     before = kq.copy()
