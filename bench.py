@@ -446,8 +446,67 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_case(args):
+    """Runs one kernel a few times on a small synthetic case (the command ncu captures are made with)."""
+    import torch
+
+    from paper_2410_05265_b200 import binding, inputs
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    ctx = binding.Context()
+    name, _, rest = args.case.partition(":")
+    dims = [int(v) for v in rest.split(",")] if rest else []
+    reps = args.steps
+    if name == "gemm":
+        M, N, K = dims or [2048, 28672, 4096]
+        xq = torch.randint(0, 256, (M, K // 2), dtype=torch.uint8, device=dev)
+        wq = torch.randint(0, 256, (N, K // 2), dtype=torch.uint8, device=dev)
+        s_a, s_w = torch.full((1,), 0.05, device=dev), torch.full((N,), 0.003, device=dev)
+        out = torch.zeros((M, N), dtype=torch.bfloat16, device=dev)
+        fn = lambda: ctx.w4a4_gemm(xq, wq, s_a, s_w, out=out)
+        work = 2.0 * M * N * K
+    elif name == "hadamard":
+        M, K, B = dims or [8192, 14336, 2048]
+        x = inputs.activations(M, K, seed=0, device=dev)
+        s_a = ctx.calib_act_scale(x, B)
+        out = torch.zeros((M, K // 2), dtype=torch.uint8, device=dev)
+        fn = lambda: ctx.hadamard_quant_act(x, B, s_a, out=out)
+        work = 2.5 * M * K
+    elif name == "attn":
+        B, Hq, Hkv, T, layers = dims or [8, 32, 8, 4092, 8]
+        D, P = 128, 4
+        pk = inputs.prefix_kv(Hkv, P, D, 0, "k", 50.0, device=dev)
+        pv = inputs.prefix_kv(Hkv, P, D, 0, "v", 50.0, device=dev)
+        s = torch.full((Hkv,), 4.5 / 7, device=dev)
+        caches = [binding.KV4Cache(pk, pv, torch.randint(0, 256, (B, Hkv, T + 4, D // 2), dtype=torch.uint8, device=dev),
+                                   torch.randint(0, 256, (B, Hkv, T + 4, D // 2), dtype=torch.uint8, device=dev), s, s,
+                                   torch.full((B,), T, dtype=torch.int32, device=dev), Hq) for _ in range(layers)]
+        q = inputs.queries(B, Hq, D, 0, device=dev)
+        ws = ctx.decode_attn_workspace(caches[0])
+        out = torch.empty_like(q)
+        it = iter(range(10**9))
+        fn = lambda: ctx.decode_attn(caches[next(it) % layers], q, 1 / math.sqrt(D), ws, out=out)
+        work = float(B * Hkv * T * D)
+    else:
+        raise SystemExit(f"unknown case {name}")
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ctx.check()
+    ms = e0.elapsed_time(e1) / reps
+    print(json.dumps({"case": args.case, "ms": round(ms, 5), "work_per_s": work / (ms * 1e-3)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--case", default=None, help="run one kernel on a small case: gemm:M,N,K | hadamard:M,K,B | attn:B,Hq,Hkv,T,layers")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
@@ -457,7 +516,9 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
-    if args.impl == "reference":
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)
