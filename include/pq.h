@@ -142,6 +142,33 @@ size_t pq_decode_attn_workspace_bytes(const pq_kv4_cache* cache);
 pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, const void* q, void* out, float sm_scale,
                                     void* ws, size_t ws_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Decode attention for callers that may not allocate. (The paper has no counterpart: this is a
+ * packaging variant of pq_decode_attn_kv4_prefix, same kernel, same arguments and result.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or unavailable - inside a
+ * region that must not synchronise the device, under a memory pool it does not own, in a plug-in
+ * that is handed buffers but no allocator, or in a start-up path that runs before an allocator
+ * exists. Such callers can create neither a pq_ctx (pq_create allocates) nor a workspace, so this
+ * entry point takes neither: the split partials and the ticket counters live in a fixed array
+ * inside the library's device image (8 MiB + 16 KiB, held by every GPU that loads the library
+ * until the process exits). The caller still passes the inputs and the output.
+ *
+ *   - Limits: B * Hkv <= 4096 and B * Hkv * splits * (Hq / Hkv) * 520 bytes <= 8 MiB, where
+ *     splits = min(32, Tmax / 64, 4 * SM count / (B * Hkv)), at least 1. Anything larger returns
+ *     PQ_ERR_WORKSPACE and enqueues nothing. Other argument rules are those of
+ *     pq_decode_attn_kv4_prefix.
+ *   - It calls no cudaMalloc, cudaFree or other allocating routine. The first call on each device
+ *     resolves the array's device address and reads the SM count (with that device current);
+ *     make that first call before any stream capture begins.
+ *   - Every call on a device shares the one array and the array keeps the previous call's
+ *     contents: the counters are cleared in stream order at the start of each call, the partials
+ *     are fully rewritten before they are read. Two calls that overlap on the GPU (different
+ *     streams, or different host threads without ordering) race on it and give wrong results;
+ *     issue them in one stream or order them yourself. */
+pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache, const void* q, void* out, float sm_scale,
+                                            void* stream);
+
 #ifdef __cplusplus
 }
 #endif

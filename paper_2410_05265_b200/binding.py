@@ -23,7 +23,7 @@ STATUS_NAMES = {
 EXPORTS = [
     "pq_status_string", "pq_create", "pq_destroy", "pq_check", "pq_quant_weights", "pq_hadamard_quant_act",
     "pq_calib_act_scale", "pq_w4a4_gemm_workspace_bytes", "pq_w4a4_gemm", "pq_kv4_append",
-    "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix",
+    "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix", "pq_decode_attn_kv4_prefix_noalloc",
 ]
 
 
@@ -71,6 +71,7 @@ def load_library() -> ctypes.CDLL:
     lib.pq_decode_attn_workspace_bytes.argtypes = [POINTER(KV4CacheStruct)]
     lib.pq_decode_attn_kv4_prefix.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_void_p, c_void_p, c_float, c_void_p,
                                               c_size_t, c_void_p]
+    lib.pq_decode_attn_kv4_prefix_noalloc.argtypes = [POINTER(KV4CacheStruct), c_void_p, c_void_p, c_float, c_void_p]
     for name in EXPORTS:
         getattr(lib, name)
         if name not in ("pq_status_string", "pq_w4a4_gemm_workspace_bytes", "pq_decode_attn_workspace_bytes"):
@@ -217,3 +218,16 @@ class Context:
         _ok(self.lib.pq_decode_attn_kv4_prefix(self.h, ctypes.byref(cache.struct), _ptr(q), _ptr(out), float(sm_scale),
                                                _ptr(ws), ws.numel(), _stream()), "pq_decode_attn_kv4_prefix")
         return out
+
+
+def decode_attn_noalloc(cache: KV4Cache, q: torch.Tensor, sm_scale: float, out: torch.Tensor) -> torch.Tensor:
+    """Decode attention through the entry point that allocates nothing: no Context and no
+    workspace are involved, the library's built-in scratch array is used instead. It exists for
+    callers that are handed buffers but may not allocate device memory themselves; `out` must
+    therefore be supplied. Calls on one device must not overlap on the GPU (they share the array).
+    The first call on a device should come before any CUDA-graph capture."""
+    _dev(q, torch.bfloat16, "q"), _dev(out, torch.bfloat16, "out")
+    assert q.shape == (cache.B, cache.Hq, cache.D) and q.is_contiguous() and out.shape == q.shape and out.is_contiguous()
+    _ok(load_library().pq_decode_attn_kv4_prefix_noalloc(ctypes.byref(cache.struct), _ptr(q), _ptr(out), float(sm_scale),
+                                                       _stream()), "pq_decode_attn_kv4_prefix_noalloc")
+    return out

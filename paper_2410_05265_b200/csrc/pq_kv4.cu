@@ -2,6 +2,8 @@
 // (Sec. 4.2, Eq. 3; Table 1, O2: per-head static KV scales).
 #include <math.h>
 
+#include <mutex>
+
 #include "pq_common.cuh"
 
 namespace {
@@ -424,5 +426,94 @@ extern "C" pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* 
   p.B = cache->B, p.Hq = cache->Hq, p.Hkv = cache->Hkv, p.G = G, p.n_prefix = cache->n_prefix, p.Tmax = cache->Tmax;
   dim3 grid(S, cache->Hkv, cache->B);
   decode_attn_kernel<<<grid, DA_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  return pq_launch_status();
+}
+
+// ================================================================================= no-allocation variant
+// Scratch of pq_decode_attn_kv4_prefix_noalloc: split partials followed by the ticket counters.
+// It lives in the loaded module, so every GPU that loads this library holds it until exit.
+namespace {
+constexpr size_t NA_PARTIAL_BYTES = size_t(8) << 20;  // 8 MiB of split partials
+constexpr int NA_MAX_BH = 4096;                       // sequences x KV heads
+constexpr size_t NA_TICKET_BYTES = (NA_MAX_BH + DA_TICKET0) * sizeof(uint32_t);
+}  // namespace
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NA_PARTIAL_BYTES + NA_TICKET_BYTES];
+
+namespace {
+struct NoAllocDevice {
+  bool ready;
+  unsigned char* scratch;  // device address of g_noalloc_scratch on this device
+  int sm_count;
+};
+NoAllocDevice g_na_dev[64];
+std::mutex g_na_mutex;
+
+int choose_splits_by_sm_count(int sm_count, const pq_kv4_cache* c) {
+  const int64_t bh = static_cast<int64_t>(c->B) * c->Hkv;
+  int64_t s = (4LL * sm_count) / (bh > 0 ? bh : 1);
+  const int64_t by_len = c->Tmax / 64;
+  if (s > by_len) s = by_len;
+  if (s > DA_MAX_SPLITS) s = DA_MAX_SPLITS;
+  if (s < 1) s = 1;
+  return static_cast<int>(s);
+}
+}  // namespace
+
+extern "C" pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache, const void* q, void* out,
+                                                       float sm_scale, void* stream) {
+  if (!q || !out) return PQ_ERR_INVALID_ARG;
+  pq_status st = check_cache(cache);
+  if (st != PQ_OK) return st;
+  if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 1)) return PQ_ERR_ALIGN;
+  if (cache->B == 0) return PQ_OK;
+  if (cache->B > 65535 || cache->Hkv > 65535) return PQ_ERR_SHAPE;
+  const int64_t bh = static_cast<int64_t>(cache->B) * cache->Hkv;
+  if (bh > NA_MAX_BH) return PQ_ERR_WORKSPACE;
+
+  // once per device, with that device current: the array's name is only a host-side handle, the
+  // kernel needs the device address the runtime resolves for it
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return PQ_ERR_CUDA;
+  NoAllocDevice nd;
+  {
+    std::lock_guard<std::mutex> lock(g_na_mutex);
+    if (!g_na_dev[dev].ready) {
+      void* ptr = nullptr;
+      int sms = 0;
+      if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return PQ_ERR_CUDA;
+      if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return PQ_ERR_CUDA;
+      g_na_dev[dev].scratch = static_cast<unsigned char*>(ptr);
+      g_na_dev[dev].sm_count = sms;
+      g_na_dev[dev].ready = true;
+    }
+    nd = g_na_dev[dev];
+  }
+  const int S = choose_splits_by_sm_count(nd.sm_count, cache);
+  const int G = cache->Hq / cache->Hkv;
+  const size_t need = static_cast<size_t>(bh) * S * G * (128 + 2) * sizeof(float);
+  if (need > NA_PARTIAL_BYTES) return PQ_ERR_WORKSPACE;
+
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  uint32_t* tickets = reinterpret_cast<uint32_t*>(nd.scratch + NA_PARTIAL_BYTES);
+  // the array keeps whatever the previous call left: the counters must start at zero
+  if (cudaMemsetAsync(tickets + DA_TICKET0, 0, static_cast<size_t>(bh) * sizeof(uint32_t), cs) != cudaSuccess)
+    return PQ_ERR_CUDA;
+  AttnParams p;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.prefix_k = static_cast<const __half*>(cache->prefix_k);
+  p.prefix_v = static_cast<const __half*>(cache->prefix_v);
+  p.kq = cache->kq;
+  p.vq = cache->vq;
+  p.s_k = cache->s_k;
+  p.s_v = cache->s_v;
+  p.len = cache->len;
+  p.ws_o = reinterpret_cast<float*>(nd.scratch);
+  p.ws_ml = p.ws_o + static_cast<size_t>(bh) * S * G * 128;
+  p.tickets = tickets;
+  p.sm_scale = sm_scale;
+  p.B = cache->B, p.Hq = cache->Hq, p.Hkv = cache->Hkv, p.G = G, p.n_prefix = cache->n_prefix, p.Tmax = cache->Tmax;
+  dim3 grid(S, cache->Hkv, cache->B);
+  decode_attn_kernel<<<grid, DA_THREADS, 0, cs>>>(p);
   return pq_launch_status();
 }
