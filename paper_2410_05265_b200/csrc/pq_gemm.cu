@@ -4,6 +4,8 @@
 
 pq_status pq_gemm_tc_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
                             void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st);
+pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
+                              void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st);
 pq_status pq_gemm_stream_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a,
                                 const float* s_w, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K,
                                 int32_t* acc_dbg, cudaStream_t st);
@@ -29,5 +31,5 @@ extern "C" pq_status pq_w4a4_gemm(pq_ctx* ctx, const uint8_t* xq, const uint8_t*
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (K == 0) return PQ_ERR_SHAPE;
   if (m <= 16) return pq_gemm_stream_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st);
-  return pq_gemm_tc_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st);
+  return pq_gemm_pair_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st);
 }
