@@ -12,8 +12,8 @@
 // Roles inside each CTA (24 warps):
 //   warp 0        TMA producer: packed A [128 x 64 B] and packed B half [128 x 64 B] per 128-wide
 //                 K block into a ring of landing buffers (own shared memory, own barriers).
-//   warps 8..23   unpack, in two groups that take alternate K blocks so that one group's barrier
-//                 and fence latency overlaps the other group's stores. A 16-byte packed chunk
+//   warps 8..23   unpack, in four groups that take K blocks in turn so that one group's barrier
+//                 hops and fence latency overlap the other groups' stores. A 16-byte packed chunk
 //                 (32 codes) becomes two 16-byte s8 chunks holding 16*code: `w & 0xF0F0F0F0` is
 //                 16*hi, `(w << 4) & 0xF0F0F0F0` is 16*lo. Even-position codes go to one chunk,
 //                 odd-position codes to the next; A and B use the same permutation of k inside a
@@ -39,21 +39,41 @@ constexpr int BN_CTA = 128;                 // weight rows expanded by each CTA
 constexpr int BK = 128;                     // K elements per stage
 constexpr int PK_ROW = BK / 2;              // packed bytes per row per stage
 constexpr int ROWS = BM_CTA + BN_CTA;       // operand rows per CTA per stage
-constexpr int N_PK = 3;                     // landing-buffer stages
-constexpr int N_S8 = 4;                     // operand-buffer stages
+#ifndef PQ_GEMM_N_PK
+#define PQ_GEMM_N_PK 4
+#endif
+#ifndef PQ_GEMM_N_S8
+#define PQ_GEMM_N_S8 4
+#endif
+#ifndef PQ_GEMM_EPI_BUFS
+#define PQ_GEMM_EPI_BUFS 1
+#endif
+#ifndef PQ_GEMM_UNPACK_WARPS
+#define PQ_GEMM_UNPACK_WARPS 16
+#endif
+#ifndef PQ_GEMM_GROUPS
+#define PQ_GEMM_GROUPS 4
+#endif
+constexpr int N_PK = PQ_GEMM_N_PK;          // landing-buffer stages
+constexpr int N_S8 = PQ_GEMM_N_S8;          // operand-buffer stages
+constexpr int EPI_BUFS = PQ_GEMM_EPI_BUFS;  // staging buffers per epilogue warp
 constexpr int PK_STAGE = ROWS * PK_ROW;     // 16 KB
 constexpr int S8_STAGE = ROWS * BK;         // 32 KB
 constexpr int S8_A = BM_CTA * BK;           // the A part of an operand stage
-constexpr int N_UNPACK_WARPS = 16;
-constexpr int N_GROUPS = 2;
+constexpr int N_UNPACK_WARPS = PQ_GEMM_UNPACK_WARPS;
+constexpr int N_GROUPS = PQ_GEMM_GROUPS;
 constexpr int GROUP_WARPS = N_UNPACK_WARPS / N_GROUPS;
+// A ring slot is always served by the same group, so no group can get a whole phase ahead of a
+// barrier it waits on (a parity wait cannot tell phase k from phase k+2).
+static_assert(N_PK % N_GROUPS == 0 && N_S8 % N_GROUPS == 0, "ring depths must be multiples of the group count");
+static_assert(N_UNPACK_WARPS % N_GROUPS == 0, "equal groups");
 constexpr int GROUP_THREADS = GROUP_WARPS * 32;
 constexpr int UNPACK_WARP0 = 8, EPI_WARP0 = 4;
 constexpr int N_THREADS = (UNPACK_WARP0 + N_UNPACK_WARPS) * 32;
 constexpr int TMEM_COLS = 512;              // two 256-column accumulators
 constexpr int EPI_COLS = 64;                // columns per TMA store (128 bytes of bf16)
 constexpr int EPI_BUF = 32 * EPI_COLS * 2;  // 4 KB: one warp's 32 rows x 64 columns
-constexpr int EPI_BYTES = 4 * 2 * EPI_BUF;  // two buffers per epilogue warp
+constexpr int EPI_BYTES = 4 * EPI_BUFS * EPI_BUF;
 constexpr int SCALE_BYTES = 4 * BN * 4;     // per-warp copy of s_a * s_w[n0 .. n0+255]
 
 struct __align__(8) Barriers {
@@ -100,14 +120,17 @@ __device__ __forceinline__ uint32_t map_to_cta(const void* p, uint32_t rank) {
   return r;
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  // default semantics on purpose: a cluster-scope release here waits for the CTA's TMA traffic in
+  // flight and costs more than the rest of the stage; the data this arrival publishes is the warp's
+  // own shared-memory stores, already ordered by the proxy fence before it
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_try_wait_local(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n"
       ".reg .pred p;\n"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
       "selp.u32 %0, 1, 0, p;\n"
       "}\n"
       : "=r"(ok)
@@ -117,12 +140,12 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
 }
 // Bounded wait (about a second of SM clocks); also gives up when the CTA's abort flag is raised.
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait_cluster(bar, parity)) return true;
+  if (mbar_try_wait_local(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 1024; ++i)
-      if (mbar_try_wait_cluster(bar, parity)) return true;
+      if (mbar_try_wait_local(bar, parity)) return true;
     if (*abort_flag) return false;
     if (clock64() - t0 > (1ll << 31)) return false;
   }
@@ -340,7 +363,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
     // ------------------------------------------------------------------ epilogue warps
     const int q = warp & 3;  // TMEM lane quarter this warp may access
     const float s_a = __ldg(p.s_a);
-    uint8_t* my_buf = epi_buf + q * 2 * EPI_BUF;
+    uint8_t* my_buf = epi_buf + q * EPI_BUFS * EPI_BUF;
     float* my_scale = scale_buf + q * BN;
     uint32_t tcount = 0, n_store = 0;
     bool ok = true;
@@ -375,9 +398,9 @@ __global__ void __launch_bounds__(N_THREADS, 1)
         }
         const int col0 = n0 + c * 32;
         if (p.tma_store) {
-          uint8_t* buf = my_buf + (n_store & 1) * EPI_BUF;
+          uint8_t* buf = my_buf + (n_store % EPI_BUFS) * EPI_BUF;
           if ((c & 1) == 0) {  // the store that last read this buffer is two stores back
-            if (lane == 0) bulk_wait_read<1>();
+            if (lane == 0) bulk_wait_read<EPI_BUFS - 1>();
             __syncwarp();
           }
 #pragma unroll
