@@ -135,7 +135,7 @@ pq_status pq_kv4_append(pq_ctx* ctx, const pq_kv4_cache* cache, const void* k, c
 /* Decode attention, one query token per sequence, over [prefix || 4-bit cache] (Eq. 3):
  *     score_j = q . K_j * sm_scale,  K_j = prefix_k[h, j] (j < n_prefix) or s_k[h] * code
  *     out     = softmax(score) . V   with V_j = prefix_v[h, j] or s_v[h] * code
- *   q, out  bf16 [B, Hq, D]; query head g reads KV head g / (Hq / Hkv)
+ *   q, out  bf16 [B, Hq, D] (q 16-byte, out 8-byte aligned); query head g reads KV head g / (Hq / Hkv)
  *   ws      scratch of pq_decode_attn_workspace_bytes(cache) bytes, 16-byte aligned
  * Every cached entry is visible (no mask). */
 size_t pq_decode_attn_workspace_bytes(const pq_kv4_cache* cache);

@@ -79,18 +79,26 @@ constexpr int DA_MAX_SPLITS = 32;
 constexpr int DA_MAX_PREFIX = 64;
 constexpr int DA_ROWS = 8;  // query heads per KV head the MMA tile can carry
 constexpr int DA_TICKET0 = 16;
+constexpr int DA_ROUND = 128;                     // keys staged per round (one half of the staging buffer)
+constexpr int DA_CHUNK = 64;                      // keys per bulk copy and per barrier
+constexpr int DA_CHUNKS = DA_ROUND / DA_CHUNK;
+constexpr int DA_HALF_BYTES = DA_ROUND * 64 * 2;  // packed K rows, then packed V rows
+constexpr int DA_SMEM_BYTES = 2 * DA_HALF_BYTES;  // 32 KB
+static_assert(DA_CHUNK == 16 * DA_WARPS, "one 16-key block per warp per chunk");
+static_assert(DA_SMEM_BYTES >= DA_WARPS * DA_ROWS * 128 * 4, "the staging area is reused for the per-warp partials");
 
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  const uint32_t z = 0;  // rows 8..15 of the A tile are padding
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(z), "r"(a2), "r"(z), "r"(b0), "r"(b1));
-}
+// D (+)= A * B, m16n8k16, fp16 inputs, fp32 accumulate. The short form leaves rows 8..15 of A zero.
 __device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
   const uint32_t z = 0;
   asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(z), "r"(a2), "r"(z), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_f16_16816_full(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                   uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 // (a & m) ^ c in one LOP3
 __device__ __forceinline__ uint32_t and_xor(uint32_t a, uint32_t m, uint32_t c) {
@@ -112,6 +120,22 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier.
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
+               "l"(src), "r"(bytes), "r"(pq::smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
 
 struct AttnParams {
   const __nv_bfloat16* q;
@@ -123,21 +147,33 @@ struct AttnParams {
   const float* s_k;
   const float* s_v;
   const int32_t* len;
-  float* ws_o;   // [B*Hkv, S, G, 128]
-  float* ws_ml;  // [B*Hkv, S, G, 2]
+  float* ws_o;   // [B*Hkv, S, G, 128] partial outputs, already in value units
+  float* ws_ml;  // [B*Hkv, S, G, 2]   running maximum (log2 units) and denominator
   uint32_t* tickets;
+  int32_t* status;  // device status word; null for the entry point that has no context
   float sm_scale;
   int B, Hq, Hkv, G, n_prefix, Tmax;
 };
 
-// Grid (splits, Hkv, B). A CTA streams its slice of one (sequence, KV head) cache row by row:
-// each warp takes 16-key blocks, computes the scores of the G query heads of the group with the
-// bf16 MMA (codes turned into bf16 by OR-ing them under an exponent; the resulting +136 offset
-// is removed through the row sum of q), runs an online softmax and accumulates P.V with the
-// fp16 MMA (codes turned into exact fp16 integers). The last CTA of a (sequence, head) merges the
-// splits, adds the full-precision prefix keys/values and writes bf16.
+// Grid (splits, Hkv, B). A CTA owns a slice of one (sequence, KV head) cache. One thread copies the
+// slice into shared memory with bulk asynchronous copies, 64 keys per copy and two rounds of 128
+// keys ahead of the warps, so the HBM stream starts with the first instructions and never waits
+// for arithmetic. Each warp takes one 16-key block of every 64-key chunk:
+//   scores   S[head, key] with the fp16 MMA, query heads on the 16-row side. Codes become fp16 in
+//            place under an exponent (one LOP3 for two codes: nibbles 0 and 2 of a 16-bit half give
+//            1032 + code, nibbles 1 and 3 give 1152 + 16 * code with no shift); the factor 16 is
+//            folded into q and the offsets into a per-head constant.
+//   softmax  online, in log2 units; the running maximum moves only when a block exceeds it.
+//   output   O^T = V^T P^T with the fp16 MMA, head dims on the 16-row side (no padded rows), codes
+//            made exact fp16 integers; P is rounded to fp16 and the denominator sums the same
+//            rounded values.
+// The CTA of split 0 also scores the full-precision prefix keys and folds them into its partial.
+// The last CTA of a (sequence, head) to finish merges the partials and writes bf16.
 __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParams p) {
-  __shared__ float sm_o[DA_WARPS][DA_ROWS][128];
+  extern __shared__ __align__(128) uint8_t da_stage[];  // two halves of [K rows | V rows] of one round
+  // the per-warp partial outputs reuse the staging area once the key loop is over
+  float (*sm_o)[DA_ROWS][128] = reinterpret_cast<float (*)[DA_ROWS][128]>(da_stage);
+  __shared__ __align__(8) uint64_t full[2][DA_CHUNKS];
   __shared__ float sm_ml[DA_WARPS][DA_ROWS][2];
   __shared__ float sm_pre[DA_ROWS][DA_MAX_PREFIX];
   __shared__ int is_last;
@@ -151,143 +187,213 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
   const int chunk = (((len_b + S - 1) / S) + 15) & ~15;
   const int t0 = split * chunk;
   const int t1 = min(len_b, t0 + chunk);
-
-  // ---- query fragments: register rho = 4m + k holds q[d], q[d+4] with d = 32t + 8m + k ----------
-  const bool row_ok = g < G;
-  const __nv_bfloat16* qrow = p.q + (static_cast<int64_t>(b) * p.Hq + h * G + (row_ok ? g : 0)) * 128;
-  uint32_t qa[16];
-  float qsum = 0.0f;
-  {
-    const uint4* q4 = reinterpret_cast<const uint4*>(qrow + 32 * t);
-#pragma unroll
-    for (int m = 0; m < 4; ++m) {
-      uint4 w = row_ok ? __ldg(q4 + m) : make_uint4(0, 0, 0, 0);  // 8 bf16: d = 32t + 8m + 0..7
-      const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        // element k is in word k/2, half k%2; element k+4 in word (k+4)/2, same half
-        const uint32_t lo = (k & 1) ? (ww[k >> 1] >> 16) : (ww[k >> 1] & 0xFFFFu);
-        const uint32_t hi = (k & 1) ? (ww[(k + 4) >> 1] >> 16) : (ww[(k + 4) >> 1] & 0xFFFFu);
-        qa[4 * m + k] = lo | (hi << 16);
-        qsum += __uint_as_float(lo << 16) + __uint_as_float(hi << 16);
-      }
-    }
-    qsum += __shfl_xor_sync(0xffffffffu, qsum, 1);
-    qsum += __shfl_xor_sync(0xffffffffu, qsum, 2);
-  }
-  const float scale2 = __ldg(p.s_k + h) * p.sm_scale * 1.4426950408889634f;  // scores in log2 units
-  const float bias = 136.0f * qsum * scale2;
-
   const uint8_t* kbase = p.kq + static_cast<int64_t>(bh) * p.Tmax * 64;
   const uint8_t* vbase = p.vq + static_cast<int64_t>(bh) * p.Tmax * 64;
 
-  float o[16][4];
-#pragma unroll
-  for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f;
-  float m_run = -INFINITY, l_run = 0.0f;
-
-  const uint4 z4 = make_uint4(0, 0, 0, 0);
-  const uint2 z2 = make_uint2(0, 0);
-  uint4 kc[2];
-  uint2 vc[4];
-  auto load_block = [&](int j0, uint4 (&kk)[2], uint2 (&vv)[4]) {
-#pragma unroll
-    for (int ti = 0; ti < 2; ++ti) {
-      const int key = j0 + 8 * ti + g;
-      kk[ti] = key < t1 ? __ldg(reinterpret_cast<const uint4*>(kbase + static_cast<int64_t>(key) * 64 + 16 * t)) : z4;
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int key = j0 + 2 * t + (i & 1) + 8 * (i >> 1);
-      vv[i] = key < t1 ? __ldg(reinterpret_cast<const uint2*>(vbase + static_cast<int64_t>(key) * 64 + 8 * g)) : z2;
+  // ---- staging: thread 0 issues the copies of a round; chunk c of a half has its own barrier. The
+  // first two rounds start before anything else so that the set-up below runs under them.
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2 * DA_CHUNKS; ++i) pq::mbar_init(&full[0][0] + i, 1);
+    pq::mbar_fence_init();
+  }
+  __syncthreads();
+  const uint32_t stage_addr = pq::smem_u32(da_stage);
+  const int n_rounds = t1 > t0 ? (t1 - t0 + DA_ROUND - 1) / DA_ROUND : 0;
+  auto issue_round = [&](int r) {
+    const uint32_t half = stage_addr + (r & 1) * DA_HALF_BYTES;
+    const int r0 = t0 + r * DA_ROUND;
+    for (int c = 0; c < DA_CHUNKS; ++c) {
+      const int k0 = r0 + c * DA_CHUNK;
+      if (k0 >= t1) break;
+      const uint32_t bytes = static_cast<uint32_t>(min(DA_CHUNK, t1 - k0)) * 64u;
+      uint64_t* bar = &full[r & 1][c];
+      pq::mbar_arrive_expect_tx(bar, 2 * bytes);
+      bulk_load(half + c * (DA_CHUNK * 64), kbase + static_cast<int64_t>(k0) * 64, bytes, bar);
+      bulk_load(half + DA_ROUND * 64 + c * (DA_CHUNK * 64), vbase + static_cast<int64_t>(k0) * 64, bytes, bar);
     }
   };
-
-  int j0 = t0 + 16 * warp;
-  if (j0 < t1) load_block(j0, kc, vc);
-  for (; j0 < t1; j0 += 16 * DA_WARPS) {
-    uint4 kn[2];
-    uint2 vn[4];
-    const int jn = j0 + 16 * DA_WARPS;
-    if (jn < t1) load_block(jn, kn, vn);
-
-    // ---- scores of 16 keys -----------------------------------------------------------------
-    float s[2][2];
+  if (threadIdx.x == 0) {
+    if (n_rounds > 0) issue_round(0);
+    if (n_rounds > 1) issue_round(1);
+  }
+  // ---- split 0 scores the full-precision prefix keys (fp32), in log2 units ---------------------------
+  if (split == 0) {
+    for (int pair = warp; pair < G * p.n_prefix; pair += DA_WARPS) {
+      const int r = pair / p.n_prefix, j = pair % p.n_prefix;
+      const __nv_bfloat16* qr = p.q + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128;
+      const __half* kr = p.prefix_k + (static_cast<int64_t>(h) * p.n_prefix + j) * 128;
+      float acc = 0.0f;
 #pragma unroll
-    for (int ti = 0; ti < 2; ++ti) {
-      const uint32_t ww[4] = {kc[ti].x, kc[ti].y, kc[ti].z, kc[ti].w};
-      float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      for (int i = 0; i < 4; ++i) acc += __bfloat162float(qr[lane + 32 * i]) * __half2float(kr[lane + 32 * i]);
+      for (int o2 = 16; o2 > 0; o2 >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o2);
+      if (lane == 0) sm_pre[r][j] = acc * p.sm_scale * 1.4426950408889634f;
+    }
+  }
+
+  // ---- query fragments (fp16 A operand of the score MMA, rows = query heads) ----------------------
+  // A 32-bit word of a packed key row holds the codes of dims 8W..8W+7; nibble i of its low half is
+  // dim 8W+i, nibble i of its high half dim 8W+4+i. Register 2j of a lane holds (q[D], q[D+4]) and
+  // register 2j+1 holds (q[D+1], q[D+5]) / 16 with D = 32t + 8(j>>1) + 2(j&1): the k columns
+  // 2t, 2t+1 and 2t+8, 2t+9 of score MMA j.
+  const bool row_ok = g < G;
+  uint32_t qa[16];
+  float q_even = 0.0f, q_odd = 0.0f;
+  {
+    const __nv_bfloat16* qrow = p.q + (static_cast<int64_t>(b) * p.Hq + h * G + (row_ok ? g : 0)) * 128;
+    const uint4* q4 = reinterpret_cast<const uint4*>(qrow + 32 * t);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        // registers rho = 2i, 2i+1: word m = rho / 4, shift k = rho % 4
-        const uint32_t b0 = and_xor(ww[(2 * i) >> 2] >> (4 * ((2 * i) & 3)), 0x000F000Fu, 0x43084308u);
-        const uint32_t b1 = and_xor(ww[(2 * i + 1) >> 2] >> (4 * ((2 * i + 1) & 3)), 0x000F000Fu, 0x43084308u);
-        mma_bf16_16816(c, qa[2 * i], qa[2 * i + 1], b0, b1);
+    for (int w = 0; w < 4; ++w) {
+      const uint4 v = row_ok ? __ldg(q4 + w) : make_uint4(0, 0, 0, 0);  // 8 bf16: d = 32t + 8w + 0..7
+      const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+      float f[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] = __uint_as_float((e & 1) ? (ww[e >> 1] & 0xFFFF0000u) : (ww[e >> 1] << 16));
+#pragma unroll
+      for (int jj = 0; jj < 2; ++jj) {  // score MMA j = 2w + jj uses nibbles 2jj and 2jj + 1
+        const int i0 = 2 * jj;
+        const __half2 a0 = __floats2half2_rn(f[i0], f[i0 + 4]);
+        const __half2 a2 = __floats2half2_rn(f[i0 + 1] * 0.0625f, f[i0 + 5] * 0.0625f);
+        qa[2 * (2 * w + jj)] = *reinterpret_cast<const uint32_t*>(&a0);
+        qa[2 * (2 * w + jj) + 1] = *reinterpret_cast<const uint32_t*>(&a2);
+        // the offsets are removed with the values the MMA really multiplies
+        const float2 e0 = __half22float2(a0), e1 = __half22float2(a2);
+        q_even += e0.x + e0.y;
+        q_odd += e1.x + e1.y;
       }
-      const int key = j0 + 8 * ti + 2 * t;
-      s[ti][0] = key < t1 ? c[0] * scale2 - bias : -INFINITY;
-      s[ti][1] = key + 1 < t1 ? c[1] * scale2 - bias : -INFINITY;
     }
-    float bm = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
-    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
-    const float m_new = fmaxf(m_run, bm);  // finite: key j0 of this block is valid for every row
-    const float alpha = ex2(m_run - m_new);
-    const float p00 = ex2(s[0][0] - m_new), p01 = ex2(s[0][1] - m_new);
-    const float p10 = ex2(s[1][0] - m_new), p11 = ex2(s[1][1] - m_new);
-    const uint32_t pa0 = pack_half2(p00, p01), pa2 = pack_half2(p10, p11);
-    {
-      // the denominator sums the same fp16-rounded probabilities the MMA multiplies with
-      const __half2 h0 = *reinterpret_cast<const __half2*>(&pa0), h1 = *reinterpret_cast<const __half2*>(&pa2);
-      const float2 f0 = __half22float2(h0), f1 = __half22float2(h1);
-      l_run = l_run * alpha + ((f0.x + f0.y) + (f1.x + f1.y));
-    }
-    if (__any_sync(0xffffffffu, alpha != 1.0f)) {
-#pragma unroll
-      for (int i = 0; i < 16; ++i) o[i][0] *= alpha, o[i][1] *= alpha;
-    }
-    m_run = m_new;
+    q_even += __shfl_xor_sync(0xffffffffu, q_even, 1);
+    q_even += __shfl_xor_sync(0xffffffffu, q_even, 2);
+    q_odd += __shfl_xor_sync(0xffffffffu, q_odd, 1);
+    q_odd += __shfl_xor_sync(0xffffffffu, q_odd, 2);
+  }
+  const float scale2 = __ldg(p.s_k + h) * p.sm_scale * 1.4426950408889634f;  // scores in log2 units
+  const float bias = (1032.0f * q_even + 1152.0f * q_odd) * scale2;
 
-    // ---- P.V for the 16 keys -----------------------------------------------------------------
-    // vc[0], vc[1]: keys 2t, 2t+1; vc[2], vc[3]: keys 2t+8, 2t+9; 16 nibbles each: d = 16g + 0..15
+  // Output accumulators of the transposed product: tile m holds, for this lane, o[m][0], o[m][1] =
+  // dim 16g+2m of heads 2t, 2t+1 and o[m][2], o[m][3] = 16 x dim 16g+2m+1 of the same heads.
+  float o[8][4];
 #pragma unroll
-    for (int pair = 0; pair < 2; ++pair) {
-      const uint32_t a0w = pair ? vc[0].y : vc[0].x, a1w = pair ? vc[1].y : vc[1].x;
-      const uint32_t b0w = pair ? vc[2].y : vc[2].x, b1w = pair ? vc[3].y : vc[3].x;
+  for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f;
+  float m_run = -INFINITY, l_run = 0.0f;  // of head g; the four lanes of a head keep the same m_run
+
+  // byte offsets of this lane's loads inside a staged 16-key block
+  const uint32_t k_off = g * 64 + 16 * t;             // key g (and g + 8): 32 codes at dims 32t..32t+31
+  const uint32_t v_off = (2 * t) * 64 + 8 * g;        // keys 2t, 2t+1, 2t+8, 2t+9: 16 codes at dims 16g..16g+15
+  bool timed_out = false;
+  for (int r = 0; r < n_rounds && !timed_out; ++r) {
+    const uint32_t ks = stage_addr + (r & 1) * DA_HALF_BYTES;
+    const int r0 = t0 + r * DA_ROUND;
+    for (int ch = 0; ch < DA_CHUNKS; ++ch) {
+      if (r0 + ch * DA_CHUNK >= t1) break;
+      if (!pq::mbar_wait(&full[r & 1][ch], (r >> 1) & 1)) {
+        timed_out = true;
+        break;
+      }
+      const int j0 = r0 + ch * DA_CHUNK + 16 * warp;  // this warp's 16-key block of the chunk
+      if (j0 >= t1) continue;
+      const uint32_t kb = ks + (j0 - r0) * 64, vb = kb + DA_ROUND * 64;
+      // Rows past the end of the slice were not copied; whatever the buffer holds there turns into
+      // finite fp16 values, and their probabilities are forced to zero below.
+      const uint4 kc0 = lds128(kb + k_off), kc1 = lds128(kb + k_off + 8 * 64);
+      const uint2 vc0 = lds64(vb + v_off), vc1 = lds64(vb + v_off + 64);
+      const uint2 vc2 = lds64(vb + v_off + 8 * 64), vc3 = lds64(vb + v_off + 9 * 64);
+      // ---- scores of 16 keys: S[head, key] for two tiles of 8 keys -----------------------------
+      float s[2][2];
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const uint32_t wa = __byte_perm(a0w, a1w, half ? 0x7632 : 0x5410);
-        const uint32_t wb = __byte_perm(b0w, b1w, half ? 0x7632 : 0x5410);
+      for (int ti = 0; ti < 2; ++ti) {
+        const uint32_t ww[4] = {ti ? kc1.x : kc0.x, ti ? kc1.y : kc0.y, ti ? kc1.z : kc0.z, ti ? kc1.w : kc0.w};
+        float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-        for (int n = 0; n < 4; ++n) {
-          const uint32_t f0 = hsub2_u32(and_xor(wa >> (4 * n), 0x000F000Fu, 0x64086408u), 0x64086408u);
-          const uint32_t f1 = hsub2_u32(and_xor(wb >> (4 * n), 0x000F000Fu, 0x64086408u), 0x64086408u);
-          mma_f16_16816(o[pair * 8 + half * 4 + n], pa0, pa2, f0, f1);
+        for (int w = 0; w < 4; ++w) {
+          const uint32_t hi8 = ww[w] >> 8;
+          mma_f16_16816(c, qa[4 * w], qa[4 * w + 1], and_xor(ww[w], 0x000F000Fu, 0x64086408u),
+                        and_xor(ww[w], 0x00F000F0u, 0x64806480u));
+          mma_f16_16816(c, qa[4 * w + 2], qa[4 * w + 3], and_xor(hi8, 0x000F000Fu, 0x64086408u),
+                        and_xor(hi8, 0x00F000F0u, 0x64806480u));
+        }
+        s[ti][0] = fmaf(c[0], scale2, -bias);
+        s[ti][1] = fmaf(c[1], scale2, -bias);
+      }
+      if (j0 + 16 > t1) {  // ragged last block
+#pragma unroll
+        for (int ti = 0; ti < 2; ++ti) {
+          const int key = j0 + 8 * ti + 2 * t;
+          if (key >= t1) s[ti][0] = -INFINITY;
+          if (key + 1 >= t1) s[ti][1] = -INFINITY;
         }
       }
+      // ---- online softmax; the running maximum moves only when a score of the block exceeds it ---
+      const float lm = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
+      if (__any_sync(0xffffffffu, lm > m_run)) {
+        float bm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, 1));
+        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
+        const float m_new = fmaxf(m_run, bm);  // finite: key j0 of this block is valid for every row
+        const float alpha = ex2(m_run - m_new);
+        m_run = m_new;
+        l_run *= alpha;
+        // this lane's accumulators belong to heads 2t and 2t+1, whose factors live in lanes 8t and 8t+4
+        const float a_lo = __shfl_sync(0xffffffffu, alpha, 8 * t), a_hi = __shfl_sync(0xffffffffu, alpha, 8 * t + 4);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i][0] *= a_lo, o[i][1] *= a_hi, o[i][2] *= a_lo, o[i][3] *= a_hi;
+      }
+      const uint32_t pb0 = pack_half2(ex2(s[0][0] - m_run), ex2(s[0][1] - m_run));
+      const uint32_t pb1 = pack_half2(ex2(s[1][0] - m_run), ex2(s[1][1] - m_run));
+      {
+        // the denominator sums the same fp16-rounded probabilities the MMA multiplies with
+        const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&pb0));
+        const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&pb1));
+        l_run += (f0.x + f0.y) + (f1.x + f1.y);
+      }
+      // ---- O^T += V^T P^T: rows = head dims, columns = query heads ------------------------------
+      // A merged word pairs the same four dims of two neighbouring keys; its nibbles 0 and 2 give
+      // exact codes, nibbles 1 and 3 give 16 * code (rows g+8 of the tile, rescaled at the end).
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        const uint32_t sel = (q4 & 1) ? 0x7632u : 0x5410u;
+        const uint32_t ya = __byte_perm(q4 < 2 ? vc0.x : vc0.y, q4 < 2 ? vc1.x : vc1.y, sel);
+        const uint32_t yb = __byte_perm(q4 < 2 ? vc2.x : vc2.y, q4 < 2 ? vc3.x : vc3.y, sel);
+        const uint32_t ya8 = ya >> 8, yb8 = yb >> 8;
+        mma_f16_16816_full(o[2 * q4], hsub2_u32(and_xor(ya, 0x000F000Fu, 0x64086408u), 0x64086408u),
+                           hsub2_u32(and_xor(ya, 0x00F000F0u, 0x64806480u), 0x64806480u),
+                           hsub2_u32(and_xor(yb, 0x000F000Fu, 0x64086408u), 0x64086408u),
+                           hsub2_u32(and_xor(yb, 0x00F000F0u, 0x64806480u), 0x64806480u), pb0, pb1);
+        mma_f16_16816_full(o[2 * q4 + 1], hsub2_u32(and_xor(ya8, 0x000F000Fu, 0x64086408u), 0x64086408u),
+                           hsub2_u32(and_xor(ya8, 0x00F000F0u, 0x64806480u), 0x64806480u),
+                           hsub2_u32(and_xor(yb8, 0x000F000Fu, 0x64086408u), 0x64086408u),
+                           hsub2_u32(and_xor(yb8, 0x00F000F0u, 0x64806480u), 0x64806480u), pb0, pb1);
+      }
     }
-    kc[0] = kn[0], kc[1] = kn[1];
-    vc[0] = vn[0], vc[1] = vn[1], vc[2] = vn[2], vc[3] = vn[3];
+    if (r + 2 < n_rounds) {  // the half is free once every warp is past it
+      __syncthreads();
+      if (threadIdx.x == 0) issue_round(r + 2);
+    }
   }
+  if (timed_out && lane == 0 && p.status) pq::report(p.status, PQ_ERR_TIMEOUT);
+  __syncthreads();  // the staging area becomes the per-warp partial outputs
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
 
-  // ---- merge the warps of this CTA -----------------------------------------------------------
-  if (row_ok) {
+  // ---- merge the warps of this CTA (and, in split 0, the prefix keys) into one partial ------------
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      sm_o[warp][g][32 * t + i] = o[i][0];       // column 2t   -> d = 16*(2t)   + i
-      sm_o[warp][g][32 * t + 16 + i] = o[i][1];  // column 2t+1 -> d = 16*(2t+1) + i
+  for (int hh = 0; hh < 2; ++hh) {
+    const int head = 2 * t + hh;
+    if (head < G) {
+#pragma unroll
+      for (int m = 0; m < 8; ++m)
+        *reinterpret_cast<float2*>(&sm_o[warp][head][16 * g + 2 * m]) = make_float2(o[m][hh], o[m][2 + hh] * 0.0625f);
     }
-    if (t == 0) sm_ml[warp][g][0] = m_run, sm_ml[warp][g][1] = l_run;
   }
+  if (row_ok && t == 0) sm_ml[warp][g][0] = m_run, sm_ml[warp][g][1] = l_run;
   __syncthreads();
   {
     const int d = threadIdx.x;  // 128 threads <-> 128 head-dim elements
+    const float sv = __ldg(p.s_v + h);
+    const int n_pre = split == 0 ? p.n_prefix : 0;
     for (int r = 0; r < G; ++r) {
       float m = -INFINITY;
 #pragma unroll
       for (int w = 0; w < DA_WARPS; ++w) m = fmaxf(m, sm_ml[w][r][0]);
+      for (int j = 0; j < n_pre; ++j) m = fmaxf(m, sm_pre[r][j]);
       float acc = 0.0f, l = 0.0f;
 #pragma unroll
       for (int w = 0; w < DA_WARPS; ++w) {
@@ -296,9 +402,15 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
         acc += sm_o[w][r][d] * e;
         l += sm_ml[w][r][1] * e;
       }
+      acc *= sv;  // codes -> values; the prefix values below are already in value units
+      for (int j = 0; j < n_pre; ++j) {
+        const float e = ex2(sm_pre[r][j] - m);
+        acc = fmaf(e, __half2float(p.prefix_v[(static_cast<int64_t>(h) * p.n_prefix + j) * 128 + d]), acc);
+        l += e;
+      }
       const int64_t slot = (static_cast<int64_t>(bh) * S + split) * G + r;
       p.ws_o[slot * 128 + d] = acc;
-      if (d == 0) p.ws_ml[slot * 2] = m, p.ws_ml[slot * 2 + 1] = l;
+      if (d == 0) *reinterpret_cast<float2*>(p.ws_ml + slot * 2) = make_float2(m, l);
     }
   }
   __threadfence();
@@ -308,48 +420,76 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
   if (!is_last) return;
   __threadfence();
 
-  // ---- last CTA of this (sequence, KV head): prefix scores, then the final merge ---------------
-  const float l2e = 1.4426950408889634f;
-  for (int pair = warp; pair < G * p.n_prefix; pair += DA_WARPS) {
-    const int r = pair / p.n_prefix, j = pair % p.n_prefix;
-    const __nv_bfloat16* qr = p.q + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128;
-    const __half* kr = p.prefix_k + (static_cast<int64_t>(h) * p.n_prefix + j) * 128;
-    float acc = 0.0f;
+  // ---- last CTA of this (sequence, KV head): merge the S partials --------------------------------
+  // One L2 round trip: every (m, l) pair and the first eight partial columns of each thread are
+  // requested together; the weights are computed while the columns are in flight.
+  float* part_m = reinterpret_cast<float*>(da_stage);  // [S][G]; the staging area is free again
+  float* part_l = part_m + DA_MAX_SPLITS * DA_ROWS;
+  float* part_w = part_l + DA_MAX_SPLITS * DA_ROWS;
+  float* head_l = part_w + DA_MAX_SPLITS * DA_ROWS;    // [G]
+  for (int i = threadIdx.x; i < S * G; i += DA_THREADS) {
+    const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.ws_ml) + static_cast<int64_t>(bh) * S * G + i);
+    part_m[i] = ml.x, part_l[i] = ml.y;
+  }
+  const float4* wo = reinterpret_cast<const float4*>(p.ws_o) + static_cast<int64_t>(bh) * S * G * 32;
+  const int n_items = G * 32;  // (head, group of four dims)
+  float4 pre[8];
+  {
+    const int item = threadIdx.x, r = item >> 5, c4 = item & 31;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) acc += __bfloat162float(qr[lane + 32 * i]) * __half2float(kr[lane + 32 * i]);
-    for (int o2 = 16; o2 > 0; o2 >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o2);
-    if (lane == 0) sm_pre[r][j] = acc * p.sm_scale * l2e;
+    for (int sp = 0; sp < 8; ++sp)
+      pre[sp] = (item < n_items && sp < S) ? __ldcg(wo + (sp * G + r) * 32 + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   __syncthreads();
-  {
-    const int d = threadIdx.x;
-    const float sv = __ldg(p.s_v + h);
-    for (int r = 0; r < G; ++r) {
-      float m = -INFINITY;
-      for (int sp = 0; sp < S; ++sp) m = fmaxf(m, __ldcg(p.ws_ml + ((static_cast<int64_t>(bh) * S + sp) * G + r) * 2));
-      for (int j = 0; j < p.n_prefix; ++j) m = fmaxf(m, sm_pre[r][j]);
-      float acc = 0.0f, l = 0.0f;
-      if (m != -INFINITY) {
-        for (int sp = 0; sp < S; ++sp) {
-          const int64_t slot = (static_cast<int64_t>(bh) * S + sp) * G + r;
-          const float ms = __ldcg(p.ws_ml + slot * 2);
-          if (ms == -INFINITY) continue;
-          const float e = ex2(ms - m);
-          acc += __ldcg(p.ws_o + slot * 128 + d) * e;
-          l += __ldcg(p.ws_ml + slot * 2 + 1) * e;
-        }
-        acc *= sv;
-        for (int j = 0; j < p.n_prefix; ++j) {
-          const float e = ex2(sm_pre[r][j] - m);
-          acc += e * __half2float(p.prefix_v[(static_cast<int64_t>(h) * p.n_prefix + j) * 128 + d]);
-          l += e;
+  if (threadIdx.x < G) {
+    const int r = threadIdx.x;
+    float m = -INFINITY;
+    for (int sp = 0; sp < S; ++sp) m = fmaxf(m, part_m[sp * G + r]);
+    float l = 0.0f;
+    for (int sp = 0; sp < S; ++sp) {
+      const float ms = part_m[sp * G + r];
+      const float e = ms == -INFINITY ? 0.0f : ex2(ms - m);  // also covers m == -inf (nothing cached, no prefix)
+      part_w[sp * G + r] = e;
+      l += part_l[sp * G + r] * e;
+    }
+    head_l[r] = l;
+  }
+  __syncthreads();
+  for (int item = threadIdx.x; item < n_items; item += DA_THREADS) {
+    const int r = item >> 5, c4 = item & 31;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int sp0 = 0; sp0 < S; sp0 += 8) {
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int sp = sp0 + u;
+        if (sp < S) {
+          const float4 v = (sp0 == 0 && item == static_cast<int>(threadIdx.x)) ? pre[u] : __ldcg(wo + (sp * G + r) * 32 + c4);
+          const float w = part_w[sp * G + r];
+          acc.x = fmaf(v.x, w, acc.x), acc.y = fmaf(v.y, w, acc.y), acc.z = fmaf(v.z, w, acc.z), acc.w = fmaf(v.w, w, acc.w);
         }
       }
-      const float res = l > 0.0f ? acc / l : 0.0f;
-      p.out[(static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + d] = __float2bfloat16_rn(res);
     }
+    const float l = head_l[r];
+    const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+    uint2 packed;
+    packed.x = *reinterpret_cast<const uint32_t*>(&lo), packed.y = *reinterpret_cast<const uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p.out + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + 4 * c4) = packed;
   }
   if (threadIdx.x == 0) p.tickets[DA_TICKET0 + bh] = 0;
+}
+
+// The kernel needs the dynamic shared-memory attribute set once per device (this allocates nothing).
+bool set_attn_smem() {
+  static bool done[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  if (!done[dev]) {
+    if (cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) != cudaSuccess)
+      return false;
+    done[dev] = true;
+  }
+  return true;
 }
 
 int choose_splits(const pq_ctx* ctx, const pq_kv4_cache* c) {
@@ -401,7 +541,7 @@ extern "C" pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* 
   if (!ctx || !q || !out) return PQ_ERR_INVALID_ARG;
   pq_status st = check_cache(cache);
   if (st != PQ_OK) return st;
-  if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 1)) return PQ_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 7)) return PQ_ERR_ALIGN;
   if (cache->B == 0) return PQ_OK;
   if (static_cast<int64_t>(cache->B) * cache->Hkv > PQ_N_TICKETS - DA_TICKET0 || cache->B > 65535 || cache->Hkv > 65535)
     return PQ_ERR_SHAPE;
@@ -422,10 +562,12 @@ extern "C" pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* 
   p.ws_o = static_cast<float*>(ws);
   p.ws_ml = p.ws_o + static_cast<size_t>(cache->B) * cache->Hkv * S * G * 128;
   p.tickets = ctx->d_tickets;
+  p.status = ctx->d_status;
   p.sm_scale = sm_scale;
   p.B = cache->B, p.Hq = cache->Hq, p.Hkv = cache->Hkv, p.G = G, p.n_prefix = cache->n_prefix, p.Tmax = cache->Tmax;
   dim3 grid(S, cache->Hkv, cache->B);
-  decode_attn_kernel<<<grid, DA_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  if (!set_attn_smem()) return PQ_ERR_CUDA;
+  decode_attn_kernel<<<grid, DA_THREADS, DA_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(p);
   return pq_launch_status();
 }
 
@@ -464,7 +606,7 @@ extern "C" pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache
   if (!q || !out) return PQ_ERR_INVALID_ARG;
   pq_status st = check_cache(cache);
   if (st != PQ_OK) return st;
-  if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 1)) return PQ_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 7)) return PQ_ERR_ALIGN;
   if (cache->B == 0) return PQ_OK;
   if (cache->B > 65535 || cache->Hkv > 65535) return PQ_ERR_SHAPE;
   const int64_t bh = static_cast<int64_t>(cache->B) * cache->Hkv;
@@ -511,9 +653,11 @@ extern "C" pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache
   p.ws_o = reinterpret_cast<float*>(nd.scratch);
   p.ws_ml = p.ws_o + static_cast<size_t>(bh) * S * G * 128;
   p.tickets = tickets;
+  p.status = nullptr;
   p.sm_scale = sm_scale;
   p.B = cache->B, p.Hq = cache->Hq, p.Hkv = cache->Hkv, p.G = G, p.n_prefix = cache->n_prefix, p.Tmax = cache->Tmax;
   dim3 grid(S, cache->Hkv, cache->B);
-  decode_attn_kernel<<<grid, DA_THREADS, 0, cs>>>(p);
+  if (!set_attn_smem()) return PQ_ERR_CUDA;
+  decode_attn_kernel<<<grid, DA_THREADS, DA_SMEM_BYTES, cs>>>(p);
   return pq_launch_status();
 }
