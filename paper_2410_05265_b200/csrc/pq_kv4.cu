@@ -61,14 +61,19 @@ __global__ void __launch_bounds__(AP_THREADS)
       *reinterpret_cast<uint4*>((which ? vq : kq) + dst) = make_uint4(o[0], o[1], o[2], o[3]);
     }
   }
-  // the last CTA to finish advances the lengths (every other CTA has read them by then)
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+  // the last CTA to finish advances the lengths (every other CTA has read them by then); a lone
+  // CTA, the usual case at decode, needs no ticket
+  if (gridDim.x > 1) {
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+  } else if (threadIdx.x == 0) {
+    last = 1;
+  }
   __syncthreads();
   if (last) {
     for (int b = threadIdx.x; b < B; b += AP_THREADS) len[b] += T_new;
-    if (threadIdx.x == 0) *ticket = 0;
+    if (threadIdx.x == 0 && gridDim.x > 1) *ticket = 0;
   }
 }
 
@@ -167,7 +172,7 @@ struct AttnParams {
 //   output   O^T = V^T P^T with the fp16 MMA, head dims on the 16-row side (no padded rows), codes
 //            made exact fp16 integers; P is rounded to fp16 and the denominator sums the same
 //            rounded values.
-// The CTA of split 0 also scores the full-precision prefix keys and folds them into its partial.
+// The CTA of the last split also scores the full-precision prefix keys and folds them into its partial.
 // The last CTA of a (sequence, head) to finish merges the partials and writes bf16.
 __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParams p) {
   extern __shared__ __align__(128) uint8_t da_stage[];  // two halves of [K rows | V rows] of one round
@@ -216,17 +221,33 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
     if (n_rounds > 0) issue_round(0);
     if (n_rounds > 1) issue_round(1);
   }
-  // ---- split 0 scores the full-precision prefix keys (fp32), in log2 units ---------------------------
-  if (split == 0) {
-    for (int pair = warp; pair < G * p.n_prefix; pair += DA_WARPS) {
-      const int r = pair / p.n_prefix, j = pair % p.n_prefix;
-      const __nv_bfloat16* qr = p.q + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128;
-      const __half* kr = p.prefix_k + (static_cast<int64_t>(h) * p.n_prefix + j) * 128;
+  // ---- the last split (its slice is the shortest) scores the full-precision prefix keys in fp32, in
+  // log2 units: eight lanes per (head, prefix key) pair, 16 dims each, every load issued at once
+  const bool has_prefix = split == S - 1 && p.n_prefix > 0;
+  if (has_prefix) {
+    const int n_pairs = G * p.n_prefix, sub = threadIdx.x & 7;
+    for (int pair0 = 0; pair0 < n_pairs; pair0 += DA_THREADS / 8) {
+      const int pair = pair0 + (threadIdx.x >> 3);
+      const bool ok = pair < n_pairs;
+      const int r = ok ? pair / p.n_prefix : 0, j = ok ? pair % p.n_prefix : 0;
+      const uint4* qr = reinterpret_cast<const uint4*>(p.q + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + 16 * sub);
+      const uint4* kr = reinterpret_cast<const uint4*>(p.prefix_k + (static_cast<int64_t>(h) * p.n_prefix + j) * 128 + 16 * sub);
+      const uint4 qv[2] = {__ldg(qr), __ldg(qr + 1)}, kv[2] = {__ldg(kr), __ldg(kr + 1)};
       float acc = 0.0f;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) acc += __bfloat162float(qr[lane + 32 * i]) * __half2float(kr[lane + 32 * i]);
-      for (int o2 = 16; o2 > 0; o2 >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o2);
-      if (lane == 0) sm_pre[r][j] = acc * p.sm_scale * 1.4426950408889634f;
+      for (int i = 0; i < 2; ++i) {
+        const uint32_t qw[4] = {qv[i].x, qv[i].y, qv[i].z, qv[i].w}, kw[4] = {kv[i].x, kv[i].y, kv[i].z, kv[i].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 kf = __half22float2(*reinterpret_cast<const __half2*>(&kw[e]));
+          acc = fmaf(__uint_as_float(qw[e] << 16), kf.x, acc);
+          acc = fmaf(__uint_as_float(qw[e] & 0xFFFF0000u), kf.y, acc);
+        }
+      }
+      acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+      acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+      acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+      if (ok && sub == 0) sm_pre[r][j] = acc * p.sm_scale * 1.4426950408889634f;
     }
   }
 
@@ -373,7 +394,7 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
 
-  // ---- merge the warps of this CTA (and, in split 0, the prefix keys) into one partial ------------
+  // ---- merge the warps of this CTA (and, in the last split, the prefix keys) into one partial ------------
 #pragma unroll
   for (int hh = 0; hh < 2; ++hh) {
     const int head = 2 * t + hh;
@@ -388,7 +409,7 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
   {
     const int d = threadIdx.x;  // 128 threads <-> 128 head-dim elements
     const float sv = __ldg(p.s_v + h);
-    const int n_pre = split == 0 ? p.n_prefix : 0;
+    const int n_pre = has_prefix ? p.n_prefix : 0;
     for (int r = 0; r < G; ++r) {
       float m = -INFINITY;
 #pragma unroll
@@ -509,6 +530,7 @@ pq_status check_cache(const pq_kv4_cache* c) {
   if (c->D != 128 || c->Hq % c->Hkv != 0 || c->Hq / c->Hkv > DA_ROWS || c->n_prefix > DA_MAX_PREFIX)
     return PQ_ERR_SHAPE;
   if ((reinterpret_cast<uintptr_t>(c->kq) & 15) || (reinterpret_cast<uintptr_t>(c->vq) & 15)) return PQ_ERR_ALIGN;
+  if (c->n_prefix > 0 && (reinterpret_cast<uintptr_t>(c->prefix_k) & 15)) return PQ_ERR_ALIGN;
   return PQ_OK;
 }
 
