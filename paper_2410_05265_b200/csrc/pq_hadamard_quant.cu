@@ -51,7 +51,9 @@ __global__ void __launch_bounds__(HQ_THREADS, 2)
     const int64_t col0 = active ? (gb % blocks_per_row) * B : 0;
 
     // ---- pass 1 --------------------------------------------------------------------------
-    float v[64];
+    // V[r] = (x[2u + r*RSTRIDE], x[2u+1 + r*RSTRIDE]) after the stage on index bit 0; the other five
+    // stages combine whole pairs, two fp32 additions per instruction.
+    float2 V[32];
     {
       const uint32_t* src = reinterpret_cast<const uint32_t*>(x + row * ldx + col0) + u;
       uint32_t w[32];
@@ -59,15 +61,8 @@ __global__ void __launch_bounds__(HQ_THREADS, 2)
       for (int r = 0; r < 32; ++r) w[r] = active ? __ldg(src + r * (RSTRIDE / 2)) : 0u;
 #pragma unroll
       for (int r = 0; r < 32; ++r) {
-        float a = __uint_as_float(w[r] << 16);
-        float b = __uint_as_float(w[r] & 0xFFFF0000u);
-        if (ROTATE) {
-          v[2 * r] = a + b;
-          v[2 * r + 1] = a - b;
-        } else {
-          v[2 * r] = a;
-          v[2 * r + 1] = b;
-        }
+        const float a = __uint_as_float(w[r] << 16), b = __uint_as_float(w[r] & 0xFFFF0000u);
+        V[r] = ROTATE ? make_float2(a + b, a - b) : make_float2(a, b);
       }
     }
     if (ROTATE) {
@@ -77,12 +72,9 @@ __global__ void __launch_bounds__(HQ_THREADS, 2)
         for (int r = 0; r < 32; ++r) {
           if ((r & (1 << s)) == 0) {
             const int r2 = r | (1 << s);
-#pragma unroll
-            for (int p = 0; p < 2; ++p) {
-              float a = v[2 * r + p], b = v[2 * r2 + p];
-              v[2 * r + p] = a + b;
-              v[2 * r2 + p] = a - b;
-            }
+            const float2 a = V[r], b = V[r2];
+            V[r] = __fadd2_rn(a, b);
+            V[r2] = __ffma2_rn(b, make_float2(-1.0f, -1.0f), a);
           }
         }
       }
@@ -91,59 +83,69 @@ __global__ void __launch_bounds__(HQ_THREADS, 2)
 #pragma unroll
     for (int r = 0; r < 32; ++r) {
       const int i = r * RSTRIDE + 2 * u;
-      *reinterpret_cast<float2*>(my + i + 2 * (i >> 7)) = make_float2(v[2 * r], v[2 * r + 1]);
+      *reinterpret_cast<float2*>(my + i + 2 * (i >> 7)) = V[r];
     }
     __syncthreads();
     const int seg = u >> 1, par = u & 1;
+    // ---- pass 2: W[q] = (v[q], v[q + 32]); stages on index bits 1..5 of the segment combine pairs,
+    // the stage on bit 6 works inside a pair ---------------------------------------------------
+    float2 W[32];
     {
       const float* src = my + seg * 130 + par;
 #pragma unroll
-      for (int q = 0; q < 64; ++q) v[q] = src[2 * q];
+      for (int q = 0; q < 32; ++q) W[q] = make_float2(src[2 * q], src[2 * q + 64]);
     }
     __syncthreads();
-    // ---- pass 2 --------------------------------------------------------------------------
     if (ROTATE) {
 #pragma unroll
-      for (int j = 0; j < 6; ++j) {
+      for (int j = 0; j < 5; ++j) {
         if (j < LOGB - 6) {
 #pragma unroll
-          for (int q = 0; q < 64; ++q) {
+          for (int q = 0; q < 32; ++q) {
             if ((q & (1 << j)) == 0) {
               const int q2 = q | (1 << j);
-              float a = v[q], b = v[q2];
-              v[q] = a + b;
-              v[q2] = a - b;
+              const float2 a = W[q], b = W[q2];
+              W[q] = __fadd2_rn(a, b);
+              W[q2] = __ffma2_rn(b, make_float2(-1.0f, -1.0f), a);
             }
           }
         }
       }
+      if (LOGB - 6 > 5) {
+#pragma unroll
+        for (int q = 0; q < 32; ++q) W[q] = make_float2(W[q].x + W[q].y, W[q].x - W[q].y);
+      }
       if (LOGB == 13) {  // index bit 7 lives in lane bit 1
         const float sgn = (u & 2) ? -1.0f : 1.0f;
 #pragma unroll
-        for (int q = 0; q < 64; ++q) {
-          float o = __shfl_xor_sync(0xffffffffu, v[q], 2);
-          v[q] = fmaf(v[q], sgn, o);
+        for (int q = 0; q < 32; ++q) {
+          const float ox = __shfl_xor_sync(0xffffffffu, W[q].x, 2), oy = __shfl_xor_sync(0xffffffffu, W[q].y, 2);
+          W[q] = make_float2(fmaf(W[q].x, sgn, ox), fmaf(W[q].y, sgn, oy));
         }
       }
     }
     if (CALIB) {
       if (active) {
 #pragma unroll
-        for (int q = 0; q < 64; ++q) cal_max = fmaxf(cal_max, fabsf(v[q] * norm));
+        for (int q = 0; q < 32; ++q) cal_max = fmaxf(cal_max, fmaxf(fabsf(W[q].x * norm), fabsf(W[q].y * norm)));
       }
     } else {
       // ---- quantize and pack -----------------------------------------------------------------
-      uint32_t pw[16];
+      // y * inv + 1.5 * 2^23: the fp32 addition rounds half to even and leaves the integer in the low
+      // mantissa bits; clamped as an integer, the low byte is the code as an s8.
+      const float2 inv2 = make_float2(inv, inv), magic2 = make_float2(12582912.0f, 12582912.0f);
+      uint32_t pw[16];  // word wd: codes of v[4wd .. 4wd+3], one nibble per byte
 #pragma unroll
-      for (int wd = 0; wd < 16; ++wd) {
-        uint32_t acc = 0;
+      for (int wd = 0; wd < 8; ++wd) {
+        int lo[4], hi[4];
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
-          float t = fminf(fmaxf(v[wd * 4 + b] * inv, -8.0f), 7.0f);
-          uint32_t bits = __float_as_uint(t + 12582912.0f);
-          acc |= (bits & 0xFu) << (8 * b);
+          const float2 tq = __ffma2_rn(W[4 * wd + b], inv2, magic2);
+          lo[b] = max(min(__float_as_int(tq.x), 0x4B400007), 0x4B3FFFF8);
+          hi[b] = max(min(__float_as_int(tq.y), 0x4B400007), 0x4B3FFFF8);
         }
-        pw[wd] = acc;
+        pw[wd] = __byte_perm(__byte_perm(lo[0], lo[1], 0x0040), __byte_perm(lo[2], lo[3], 0x0040), 0x5410) & 0x0F0F0F0Fu;
+        pw[wd + 8] = __byte_perm(__byte_perm(hi[0], hi[1], 0x0040), __byte_perm(hi[2], hi[3], 0x0040), 0x5410) & 0x0F0F0F0Fu;
       }
       uint32_t fin[8];
 #pragma unroll
