@@ -16,12 +16,13 @@
 
 namespace {
 
-constexpr int HQ_THREADS = 256;
+constexpr int HQ_THREADS = 128;
+constexpr int HQ_CTAS_PER_SM = 5;         // 33 KB of shared memory and about 11K registers each
 constexpr int HQ_ELEMS = HQ_THREADS * 64;             // elements handled per CTA iteration
 constexpr int HQ_SMEM_FLOATS = HQ_ELEMS + HQ_ELEMS / 64;  // + 2 floats of padding per 128
 
 template <int LOGB, bool ROTATE, bool CALIB>
-__global__ void __launch_bounds__(HQ_THREADS, 2)
+__global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
     hadamard_quant_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int64_t n_rows, int64_t K,
                           const float* __restrict__ s_a_in, uint8_t* __restrict__ xq, float* __restrict__ s_a_out) {
   constexpr int B = 1 << LOGB;
@@ -178,7 +179,8 @@ pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_
   constexpr int B = 1 << LOGB;
   constexpr int G = HQ_THREADS / (B / 64);
   int64_t n_super = (n_rows * (K / B) + G - 1) / G;
-  int64_t grid = n_super < 2LL * ctx->sm_count ? n_super : 2LL * ctx->sm_count;
+  const int64_t resident = static_cast<int64_t>(HQ_CTAS_PER_SM) * ctx->sm_count;
+  int64_t grid = n_super < resident ? n_super : resident;
   kern<<<static_cast<int>(grid), HQ_THREADS, smem, st>>>(static_cast<const __nv_bfloat16*>(x), ldx, n_rows, K, s_a_in,
                                                         xq, s_a_out);
   return pq_launch_status();
