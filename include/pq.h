@@ -143,6 +143,27 @@ pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, cons
                                     void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Element-wise glue of a Llama transformer block around the quantized linears (the block of the
+ * rotation figure in App. B: RMSNorm -> linears -> rotary embedding -> attention -> SwiGLU, with
+ * residual connections). bf16 in, fp32 arithmetic (fp64 angles), one rounding to bf16 out. Every
+ * pointer is 16-byte aligned and every leading dimension a multiple of 8 elements.
+ *
+ *   pq_rmsnorm       y[t,:] = x[t,:] / sqrt(mean(x[t,:]^2) + eps) * g      x, y [M,K], g [K]; K % 8 == 0, K <= 16384
+ *   pq_rope          rotate-half pairing, head dim D = 128: for i < 64 and token t at position pos0 + t,
+ *                    angle = (pos0 + t) * theta^(-2i/D), y[i] = x[i] cos - x[i+64] sin,
+ *                    y[i+64] = x[i+64] cos + x[i] sin       x, y [T,H,D] dense; y may alias x
+ *   pq_silu_mul      y = gate / (1 + exp(-gate)) * up        gate, up [M,F] with row stride ld_in (the two
+ *                    halves of a concatenated gate|up GEMM output), y [M,F] with row stride ldy; F % 8 == 0
+ *   pq_residual_add  y = a + b over n elements, n % 8 == 0; y may alias a or b */
+pq_status pq_rmsnorm(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, const void* g, float eps, void* y,
+                     int64_t ldy, void* stream);
+pq_status pq_rope(pq_ctx* ctx, const void* x, int64_t T, int32_t H, int32_t D, int64_t pos0, double theta, void* y,
+                  void* stream);
+pq_status pq_silu_mul(pq_ctx* ctx, const void* gate, const void* up, int64_t M, int64_t F, int64_t ld_in, void* y,
+                      int64_t ldy, void* stream);
+pq_status pq_residual_add(pq_ctx* ctx, const void* a, const void* b, void* y, int64_t n, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Decode attention for callers that may not allocate. (The paper has no counterpart: this is a
  * packaging variant of pq_decode_attn_kv4_prefix, same kernel, same arguments and result.)
  *

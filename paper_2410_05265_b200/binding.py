@@ -8,7 +8,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import POINTER, Structure, c_char_p, c_float, c_int32, c_int64, c_size_t, c_void_p
+from ctypes import POINTER, Structure, c_char_p, c_double, c_float, c_int32, c_int64, c_size_t, c_void_p
 
 import torch
 
@@ -24,6 +24,7 @@ EXPORTS = [
     "pq_status_string", "pq_create", "pq_destroy", "pq_check", "pq_quant_weights", "pq_hadamard_quant_act",
     "pq_calib_act_scale", "pq_w4a4_gemm_workspace_bytes", "pq_w4a4_gemm", "pq_kv4_append",
     "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix", "pq_decode_attn_kv4_prefix_noalloc",
+    "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add",
 ]
 
 
@@ -72,6 +73,10 @@ def load_library() -> ctypes.CDLL:
     lib.pq_decode_attn_kv4_prefix.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_void_p, c_void_p, c_float, c_void_p,
                                               c_size_t, c_void_p]
     lib.pq_decode_attn_kv4_prefix_noalloc.argtypes = [POINTER(KV4CacheStruct), c_void_p, c_void_p, c_float, c_void_p]
+    lib.pq_rmsnorm.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_float, c_void_p, c_int64, c_void_p]
+    lib.pq_rope.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_int32, c_int64, c_double, c_void_p, c_void_p]
+    lib.pq_silu_mul.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p]
+    lib.pq_residual_add.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p]
     for name in EXPORTS:
         getattr(lib, name)
         if name not in ("pq_status_string", "pq_w4a4_gemm_workspace_bytes", "pq_decode_attn_workspace_bytes"):
@@ -217,6 +222,45 @@ class Context:
             out = torch.empty_like(q)
         _ok(self.lib.pq_decode_attn_kv4_prefix(self.h, ctypes.byref(cache.struct), _ptr(q), _ptr(out), float(sm_scale),
                                                _ptr(ws), ws.numel(), _stream()), "pq_decode_attn_kv4_prefix")
+        return out
+
+
+    # ---- transformer-block glue -----------------------------------------------------------------
+    def rmsnorm(self, x: torch.Tensor, g: torch.Tensor, eps: float = 1e-5, out: torch.Tensor | None = None):
+        _dev(x, torch.bfloat16, "x"), _dev(g, torch.bfloat16, "g")
+        M, K = x.shape
+        assert x.stride(1) == 1 and g.numel() == K
+        if out is None:
+            out = torch.empty((M, K), dtype=torch.bfloat16, device=x.device)
+        _ok(self.lib.pq_rmsnorm(self.h, _ptr(x), M, K, x.stride(0), _ptr(g), float(eps), _ptr(out), out.stride(0),
+                                _stream()), "pq_rmsnorm")
+        return out
+
+    def rope(self, x: torch.Tensor, pos0: int, theta: float, out: torch.Tensor | None = None):
+        _dev(x, torch.bfloat16, "x")
+        T, H, D = x.shape
+        assert x.is_contiguous()
+        if out is None:
+            out = torch.empty_like(x)
+        _ok(self.lib.pq_rope(self.h, _ptr(x), T, H, D, int(pos0), float(theta), _ptr(out), _stream()), "pq_rope")
+        return out
+
+    def silu_mul(self, gate: torch.Tensor, up: torch.Tensor, out: torch.Tensor | None = None):
+        _dev(gate, torch.bfloat16, "gate"), _dev(up, torch.bfloat16, "up")
+        M, F = gate.shape
+        assert up.shape == (M, F) and gate.stride(1) == 1 and up.stride(1) == 1 and gate.stride(0) == up.stride(0)
+        if out is None:
+            out = torch.empty((M, F), dtype=torch.bfloat16, device=gate.device)
+        _ok(self.lib.pq_silu_mul(self.h, _ptr(gate), _ptr(up), M, F, gate.stride(0), _ptr(out), out.stride(0), _stream()),
+            "pq_silu_mul")
+        return out
+
+    def residual_add(self, a: torch.Tensor, b: torch.Tensor, out: torch.Tensor | None = None):
+        _dev(a, torch.bfloat16, "a"), _dev(b, torch.bfloat16, "b")
+        assert a.shape == b.shape and a.is_contiguous() and b.is_contiguous()
+        if out is None:
+            out = torch.empty_like(a)
+        _ok(self.lib.pq_residual_add(self.h, _ptr(a), _ptr(b), _ptr(out), a.numel(), _stream()), "pq_residual_add")
         return out
 
 

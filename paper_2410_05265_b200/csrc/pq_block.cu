@@ -1,0 +1,203 @@
+// Element-wise glue of a Llama transformer block around the W4A4 linears and the KV4 attention
+// (App. B places the rotations inside such a block): RMSNorm, rotary embedding, SwiGLU gate and
+// residual addition. Each kernel reads bf16, computes in fp32 (angles in fp64) and rounds once to
+// bf16, so every tensor that crosses HBM is a bf16 tensor. All are bound by HBM bandwidth.
+#include <math.h>
+
+#include "pq_common.cuh"
+
+namespace {
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// ---- RMSNorm: y = x * rsqrt(mean(x^2) + eps) * g; one CTA per row, the row is read once ---------
+constexpr int RN_THREADS = 256;
+constexpr int RN_MAX_VEC = 8;  // 8-element vectors per thread kept in registers: K <= 256 * 8 * 8 = 16384
+
+__global__ void __launch_bounds__(RN_THREADS)
+    rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const __nv_bfloat16* __restrict__ g, float eps,
+                   __nv_bfloat16* __restrict__ y, int64_t ldy, int64_t M, int K) {
+  __shared__ float red[RN_THREADS / 32];
+  __shared__ float s_r;
+  const int n_vec = K / 8;
+  for (int64_t row = blockIdx.x; row < M; row += gridDim.x) {
+    const uint4* xr = reinterpret_cast<const uint4*>(x + row * ldx);
+    uint4 v[RN_MAX_VEC];
+    float ss = 0.0f;
+#pragma unroll
+    for (int i = 0; i < RN_MAX_VEC; ++i) {
+      const int j = threadIdx.x + i * RN_THREADS;
+      v[i] = j < n_vec ? __ldg(xr + j) : make_uint4(0, 0, 0, 0);
+      const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) ss = fmaf(bf16_lo(w[e]), bf16_lo(w[e]), fmaf(bf16_hi(w[e]), bf16_hi(w[e]), ss));
+    }
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float t = 0.0f;
+      for (int i = 0; i < RN_THREADS / 32; ++i) t += red[i];
+      s_r = 1.0f / sqrtf(t / static_cast<float>(K) + eps);
+    }
+    __syncthreads();
+    const float r = s_r;
+    uint4* yr = reinterpret_cast<uint4*>(y + row * ldy);
+    const uint4* gr = reinterpret_cast<const uint4*>(g);
+#pragma unroll
+    for (int i = 0; i < RN_MAX_VEC; ++i) {
+      const int j = threadIdx.x + i * RN_THREADS;
+      if (j < n_vec) {
+        const uint4 gv = __ldg(gr + j);
+        const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w}, gw[4] = {gv.x, gv.y, gv.z, gv.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[e] = pack_bf16(bf16_lo(w[e]) * r * bf16_lo(gw[e]), bf16_hi(w[e]) * r * bf16_hi(gw[e]));
+        yr[j] = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// ---- rotary embedding, rotate-half pairing, head_dim 128 -----------------------------------------
+// One CTA per token: 64 threads build cos/sin of pos * theta^(-2i/128) in fp64 (positions reach the
+// thousands, where an fp32 angle already costs a visible part of a bf16 ulp), then every thread
+// rotates 8-element vectors of the token's heads.
+constexpr int RP_THREADS = 128;
+
+__global__ void __launch_bounds__(RP_THREADS)
+    rope_kernel(const __nv_bfloat16* x, __nv_bfloat16* y, int64_t T, int H, int64_t pos0,
+                double log2_theta) {
+  __shared__ float cs[64], sn[64];
+  for (int64_t t = blockIdx.x; t < T; t += gridDim.x) {
+    if (threadIdx.x < 64) {
+      const double inv_freq = exp2(-2.0 * static_cast<double>(threadIdx.x) / 128.0 * log2_theta);
+      double s, c;
+      sincos(static_cast<double>(pos0 + t) * inv_freq, &s, &c);
+      cs[threadIdx.x] = static_cast<float>(c), sn[threadIdx.x] = static_cast<float>(s);
+    }
+    __syncthreads();
+    // a work item = (head, group of 8 consecutive i in [0, 64)): reads x[i..i+7] and x[64+i..64+i+7]
+    for (int item = threadIdx.x; item < H * 8; item += RP_THREADS) {
+      const int hd = item >> 3, i0 = (item & 7) * 8;
+      const __nv_bfloat16* px = x + (t * H + hd) * 128;
+      __nv_bfloat16* py = y + (t * H + hd) * 128;
+      const uint4 a = *reinterpret_cast<const uint4*>(px + i0), b = *reinterpret_cast<const uint4*>(px + 64 + i0);  // y may alias x
+      const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+      uint32_t oa[4], ob[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float c0 = cs[i0 + 2 * e], s0 = sn[i0 + 2 * e], c1 = cs[i0 + 2 * e + 1], s1 = sn[i0 + 2 * e + 1];
+        const float a0 = bf16_lo(aw[e]), a1 = bf16_hi(aw[e]), b0 = bf16_lo(bw[e]), b1 = bf16_hi(bw[e]);
+        oa[e] = pack_bf16(a0 * c0 - b0 * s0, a1 * c1 - b1 * s1);
+        ob[e] = pack_bf16(b0 * c0 + a0 * s0, b1 * c1 + a1 * s1);
+      }
+      *reinterpret_cast<uint4*>(py + i0) = make_uint4(oa[0], oa[1], oa[2], oa[3]);
+      *reinterpret_cast<uint4*>(py + 64 + i0) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+    }
+    __syncthreads();
+  }
+}
+
+// ---- SwiGLU gate: y = gate / (1 + exp(-gate)) * up ------------------------------------------------
+constexpr int EW_THREADS = 256;
+
+__global__ void __launch_bounds__(EW_THREADS)
+    silu_mul_kernel(const __nv_bfloat16* __restrict__ gate, const __nv_bfloat16* __restrict__ up, int64_t ld_in,
+                    __nv_bfloat16* __restrict__ y, int64_t ldy, int64_t M, int F) {
+  const int vec_per_row = F / 8;
+  const int64_t n_vec = M * vec_per_row;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * EW_THREADS + threadIdx.x; i < n_vec;
+       i += static_cast<int64_t>(gridDim.x) * EW_THREADS) {
+    const int64_t row = i / vec_per_row;
+    const int col = static_cast<int>(i % vec_per_row) * 8;
+    const uint4 gv = __ldg(reinterpret_cast<const uint4*>(gate + row * ld_in + col));
+    const uint4 uv = __ldg(reinterpret_cast<const uint4*>(up + row * ld_in + col));
+    const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w}, uw[4] = {uv.x, uv.y, uv.z, uv.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float g0 = bf16_lo(gw[e]), g1 = bf16_hi(gw[e]);
+      o[e] = pack_bf16(g0 / (1.0f + expf(-g0)) * bf16_lo(uw[e]), g1 / (1.0f + expf(-g1)) * bf16_hi(uw[e]));
+    }
+    *reinterpret_cast<uint4*>(y + row * ldy + col) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+// ---- residual: y = a + b -----------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+    add_kernel(const __nv_bfloat16* a, const __nv_bfloat16* b, __nv_bfloat16* y,
+               int64_t n_vec) {
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * EW_THREADS + threadIdx.x; i < n_vec;
+       i += static_cast<int64_t>(gridDim.x) * EW_THREADS) {
+    const uint4 av = reinterpret_cast<const uint4*>(a)[i], bv = reinterpret_cast<const uint4*>(b)[i];  // y may alias a or b
+    const uint32_t aw[4] = {av.x, av.y, av.z, av.w}, bw[4] = {bv.x, bv.y, bv.z, bv.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) o[e] = pack_bf16(bf16_lo(aw[e]) + bf16_lo(bw[e]), bf16_hi(aw[e]) + bf16_hi(bw[e]));
+    reinterpret_cast<uint4*>(y)[i] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+int grid_for(pq_ctx* ctx, int64_t work_items, int per_cta) {
+  int64_t g = (work_items + per_cta - 1) / per_cta;
+  const int64_t cap = 16LL * ctx->sm_count;
+  return static_cast<int>(g < 1 ? 1 : (g > cap ? cap : g));
+}
+
+}  // namespace
+
+extern "C" pq_status pq_rmsnorm(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, const void* g, float eps,
+                                void* y, int64_t ldy, void* stream) {
+  if (!ctx || !x || !g || !y) return PQ_ERR_INVALID_ARG;
+  if (M < 0 || K <= 0 || ldx < K || ldy < K) return PQ_ERR_INVALID_ARG;
+  if (K % 8 != 0 || K > RN_THREADS * RN_MAX_VEC * 8) return PQ_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(g) || !aligned16(y) || ldx % 8 != 0 || ldy % 8 != 0) return PQ_ERR_ALIGN;
+  if (M == 0) return PQ_OK;
+  rmsnorm_kernel<<<grid_for(ctx, M, 1), RN_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(x), ldx, static_cast<const __nv_bfloat16*>(g), eps,
+      static_cast<__nv_bfloat16*>(y), ldy, M, static_cast<int>(K));
+  return pq_launch_status();
+}
+
+extern "C" pq_status pq_rope(pq_ctx* ctx, const void* x, int64_t T, int32_t H, int32_t D, int64_t pos0, double theta,
+                             void* y, void* stream) {
+  if (!ctx || !x || !y) return PQ_ERR_INVALID_ARG;
+  if (T < 0 || H <= 0 || pos0 < 0 || !(theta > 1.0)) return PQ_ERR_INVALID_ARG;
+  if (D != 128) return PQ_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(y)) return PQ_ERR_ALIGN;
+  if (T == 0) return PQ_OK;
+  rope_kernel<<<grid_for(ctx, T, 1), RP_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(y), T, H, pos0, log2(theta));
+  return pq_launch_status();
+}
+
+extern "C" pq_status pq_silu_mul(pq_ctx* ctx, const void* gate, const void* up, int64_t M, int64_t F, int64_t ld_in,
+                                 void* y, int64_t ldy, void* stream) {
+  if (!ctx || !gate || !up || !y) return PQ_ERR_INVALID_ARG;
+  if (M < 0 || F <= 0 || ld_in < F || ldy < F) return PQ_ERR_INVALID_ARG;
+  if (F % 8 != 0 || F > (1 << 30)) return PQ_ERR_SHAPE;
+  if (!aligned16(gate) || !aligned16(up) || !aligned16(y) || ld_in % 8 != 0 || ldy % 8 != 0) return PQ_ERR_ALIGN;
+  if (M == 0) return PQ_OK;
+  silu_mul_kernel<<<grid_for(ctx, M * (F / 8), EW_THREADS), EW_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(gate), static_cast<const __nv_bfloat16*>(up), ld_in,
+      static_cast<__nv_bfloat16*>(y), ldy, M, static_cast<int>(F));
+  return pq_launch_status();
+}
+
+extern "C" pq_status pq_residual_add(pq_ctx* ctx, const void* a, const void* b, void* y, int64_t n, void* stream) {
+  if (!ctx || !a || !b || !y || n < 0) return PQ_ERR_INVALID_ARG;
+  if (n % 8 != 0) return PQ_ERR_SHAPE;
+  if (!aligned16(a) || !aligned16(b) || !aligned16(y)) return PQ_ERR_ALIGN;
+  if (n == 0) return PQ_OK;
+  add_kernel<<<grid_for(ctx, n / 8, EW_THREADS), EW_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(a), static_cast<const __nv_bfloat16*>(b), static_cast<__nv_bfloat16*>(y), n / 8);
+  return pq_launch_status();
+}

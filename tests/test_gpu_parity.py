@@ -263,3 +263,42 @@ def test_argument_errors_are_synchronous(ctx):
     xq = torch.zeros((4, 24), dtype=torch.uint8, device="cuda")
     with pytest.raises(PQError):
         ctx.w4a4_gemm(xq, xq, s, torch.ones(4, device="cuda"))   # K = 48 not a multiple of 32
+
+
+# ------------------------------------------------------------------------------- a6 block glue
+@pytest.mark.parametrize("M,K", [(5, 128), (37, 4096), (9, 8192), (3, 16384)])
+def test_rmsnorm_matches_oracle(ctx, M, K):
+    x = inputs.activations(M, K, seed=0)
+    g = (1.0 + 0.1 * inputs.weights(1, K, seed=7)[0] / 0.02 * 0.1).to(torch.bfloat16)
+    ref = orc.rmsnorm(inputs.bits(x), inputs.bits(g))
+    got = ctx.rmsnorm(x.cuda(), g.cuda())
+    ctx.check()
+    assert_bf16_close(inputs.bits(got), ref, "rmsnorm")
+
+
+@pytest.mark.parametrize("T,H,pos0", [(3, 2, 0), (33, 9, 4), (5, 72, 4090)])
+def test_rope_matches_oracle(ctx, T, H, pos0):
+    x = inputs.kv_tensor(1, T, H, 128, 0, "k")[0]
+    ref = orc.rope(inputs.bits(x), pos0, 500000.0)
+    got = ctx.rope(x.cuda().contiguous(), pos0, 500000.0)
+    ctx.check()
+    assert_bf16_close(inputs.bits(got), ref, "rope")
+    xin = x.cuda().contiguous()
+    ctx.rope(xin, pos0, 500000.0, out=xin)  # in place
+    assert torch.equal(xin, got)
+
+
+def test_silu_mul_and_residual_match_oracle(ctx):
+    M, F = 19, 1024
+    gu = (inputs.activations(M, 2 * F, seed=3) * 2).to(torch.bfloat16)
+    gate, up = gu[:, :F], gu[:, F:]
+    ref = orc.silu_mul(inputs.bits(gate.contiguous()), inputs.bits(up.contiguous()))
+    gud = gu.cuda()
+    got = ctx.silu_mul(gud[:, :F], gud[:, F:])
+    ctx.check()
+    assert_bf16_close(inputs.bits(got), ref, "silu_mul")
+    a, b = inputs.activations(M, F, seed=4), inputs.activations(M, F, seed=5)
+    ref = orc.add(inputs.bits(a), inputs.bits(b))
+    got = ctx.residual_add(a.cuda(), b.cuda())
+    ctx.check()
+    assert np.array_equal(inputs.bits(got), ref), "a + b in fp32 rounds exactly like the oracle"
