@@ -142,6 +142,15 @@ size_t pq_decode_attn_workspace_bytes(const pq_kv4_cache* cache);
 pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, const void* q, void* out, float sm_scale,
                                     void* ws, size_t ws_bytes, void* stream);
 
+/* Causal prefill attention of one sequence over [prefix || 4-bit cache] (Sec. 4.2, Eq. 3): query
+ * token t sees every prefixed key and the cached keys 0..t of sequence `seq` (the cache rows must
+ * already hold the T tokens: call pq_kv4_append first).
+ *     out[t, g, :] = softmax_j(q[t, g, :] . K_j * sm_scale) . V   over j in prefix and j <= t
+ *   q, out  bf16 [T, Hq, D] dense, 4-byte aligned; D = 128; Hq / Hkv in {1, 2, 4, 8}; T <= Tmax;
+ *   n_prefix <= 64; prefix_k, prefix_v, kq, vq 16-byte aligned. No workspace. */
+pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, int32_t seq, const void* q, int32_t T,
+                                     void* out, float sm_scale, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Element-wise glue of a Llama transformer block around the quantized linears (the block of the
  * rotation figure in App. B: RMSNorm -> linears -> rotary embedding -> attention -> SwiGLU, with

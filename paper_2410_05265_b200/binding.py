@@ -24,7 +24,7 @@ EXPORTS = [
     "pq_status_string", "pq_create", "pq_destroy", "pq_check", "pq_quant_weights", "pq_hadamard_quant_act",
     "pq_calib_act_scale", "pq_w4a4_gemm_workspace_bytes", "pq_w4a4_gemm", "pq_kv4_append",
     "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix", "pq_decode_attn_kv4_prefix_noalloc",
-    "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add",
+    "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add", "pq_prefill_attn_kv4_prefix",
 ]
 
 
@@ -73,6 +73,8 @@ def load_library() -> ctypes.CDLL:
     lib.pq_decode_attn_kv4_prefix.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_void_p, c_void_p, c_float, c_void_p,
                                               c_size_t, c_void_p]
     lib.pq_decode_attn_kv4_prefix_noalloc.argtypes = [POINTER(KV4CacheStruct), c_void_p, c_void_p, c_float, c_void_p]
+    lib.pq_prefill_attn_kv4_prefix.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_int32, c_void_p, c_int32, c_void_p, c_float,
+                                               c_void_p]
     lib.pq_rmsnorm.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_float, c_void_p, c_int64, c_void_p]
     lib.pq_rope.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_int32, c_int64, c_double, c_void_p, c_void_p]
     lib.pq_silu_mul.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p]
@@ -224,6 +226,16 @@ class Context:
                                                _ptr(ws), ws.numel(), _stream()), "pq_decode_attn_kv4_prefix")
         return out
 
+
+    def prefill_attn(self, cache: KV4Cache, seq: int, q: torch.Tensor, sm_scale: float, out: torch.Tensor | None = None):
+        _dev(q, torch.bfloat16, "q")
+        T = q.shape[0]
+        assert q.shape == (T, cache.Hq, cache.D) and q.is_contiguous()
+        if out is None:
+            out = torch.empty_like(q)
+        _ok(self.lib.pq_prefill_attn_kv4_prefix(self.h, ctypes.byref(cache.struct), int(seq), _ptr(q), T, _ptr(out),
+                                                float(sm_scale), _stream()), "pq_prefill_attn_kv4_prefix")
+        return out
 
     # ---- transformer-block glue -----------------------------------------------------------------
     def rmsnorm(self, x: torch.Tensor, g: torch.Tensor, eps: float = 1e-5, out: torch.Tensor | None = None):

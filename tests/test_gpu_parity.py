@@ -8,7 +8,7 @@ import torch
 
 from oracle import pq_oracle as orc
 from paper_2410_05265_b200 import inputs
-from helpers import (assert_attn_close, assert_bf16_close, assert_codes_tie_tolerant, rand_codes, to_np)
+from helpers import (assert_attn_close, assert_bf16_close, assert_codes_tie_tolerant, bf16_ulp, rand_codes, to_np)
 
 pytestmark = pytest.mark.gpu
 
@@ -302,3 +302,36 @@ def test_silu_mul_and_residual_match_oracle(ctx):
     got = ctx.residual_add(a.cuda(), b.cuda())
     ctx.check()
     assert np.array_equal(inputs.bits(got), ref), "a + b in fp32 rounds exactly like the oracle"
+
+
+@pytest.mark.parametrize("T,Hq,Hkv,P,mag", [(1, 8, 1, 4, 1.0), (37, 8, 2, 4, 50.0), (150, 4, 1, 0, 1.0), (200, 16, 2, 3, 1.0),
+                                            (70, 2, 2, 64, 1.0), (96, 4, 2, 4, 1.0)])
+def test_prefill_attention_matches_oracle(ctx, T, Hq, Hkv, P, mag):
+    from paper_2410_05265_b200 import binding
+
+    D, Tmax, B = 128, T + 11, 2
+    k = inputs.kv_tensor(B, T, Hkv, D, 0, "k")
+    v = inputs.kv_tensor(B, T, Hkv, D, 0, "v")
+    s_k, s_v = orc.calib_kv_scale(inputs.bits(k)), orc.calib_kv_scale(inputs.bits(v))
+    kq_ref = np.zeros((B, Hkv, Tmax, D // 2), np.uint8)
+    vq_ref = np.zeros_like(kq_ref)
+    orc.kv4_append(inputs.bits(k), inputs.bits(v), s_k, s_v, kq_ref, vq_ref, np.zeros(B, np.int32))
+    pk = inputs.prefix_kv(Hkv, max(P, 1), D, 0, "k", mag)[:, :P].contiguous()
+    pv = inputs.prefix_kv(Hkv, max(P, 1), D, 0, "v", mag)[:, :P].contiguous()
+    seq = 1
+    q = inputs.kv_tensor(1, T, Hq, D, 3, "k")[0].contiguous()
+    ref = orc.prefill_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq_ref[seq], vq_ref[seq], s_k, s_v,
+                           1 / math.sqrt(D))
+    cache = binding.KV4Cache(pk.cuda() if P else None, pv.cuda() if P else None, dev(kq_ref), dev(vq_ref), dev(s_k), dev(s_v),
+                             torch.full((B,), T, dtype=torch.int32, device="cuda"), Hq)
+    out = torch.full((T, Hq, D), 7.0, dtype=torch.bfloat16, device="cuda")
+    ctx.prefill_attn(cache, seq, q.cuda(), 1 / math.sqrt(D), out=out)
+    ctx.check()
+    got = orc.bf16_to_f64(inputs.bits(out))
+    r = orc.bf16_to_f64(ref)
+    vmax = np.abs(r).max(axis=-1, keepdims=True)
+    # the stated attention tolerance on the computed value, plus the bf16 store rounding of both sides
+    # (half an ulp each: the oracle's prefill result is only available rounded)
+    tol = 2e-3 * vmax + bf16_ulp(r) + 1e-30
+    bad = np.abs(got - r) > tol
+    assert not bad.any(), f"{bad.sum()} of {bad.size} outside tolerance; worst {np.max(np.abs(got - r) / np.maximum(vmax, 1e-30))}"
