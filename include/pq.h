@@ -125,12 +125,22 @@ typedef struct pq_kv4_cache {
   int32_t B, Hq, Hkv, D, n_prefix, Tmax;
 } pq_kv4_cache;
 
+/* Calibration helper for the static per-head KV steps (Table 1, O2): over a calibration batch
+ * x bf16 [n_tok, Hkv, D] with ld_tok elements between tokens, s[h] = max(s[h], max |x[:, h, :]| / 7).
+ * s must be initialised by the caller (0 to start); K and V are calibrated by separate calls. */
+pq_status pq_calib_kv_scale(pq_ctx* ctx, const void* x, int64_t n_tok, int32_t Hkv, int32_t D, int64_t ld_tok, float* s,
+                            void* stream);
+
 /* Quantize-on-write: k, v bf16 [B, T_new, Hkv, D] are quantized with s_k[h], s_v[h] and written at
  * positions len[b] .. len[b]+T_new-1, then len[b] += T_new (on the device, in stream order).
  * If any sequence would exceed Tmax nothing is written, len is unchanged and PQ_ERR_SHAPE is
  * left in the status word. */
 pq_status pq_kv4_append(pq_ctx* ctx, const pq_kv4_cache* cache, const void* k, const void* v, int32_t T_new,
                         void* stream);
+/* The same with ld_tok elements between consecutive tokens of k and of v (ld_tok >= Hkv * D, a multiple
+ * of 8): the k and v parts of a concatenated q|k|v projection output are appended without a copy. */
+pq_status pq_kv4_append_strided(pq_ctx* ctx, const pq_kv4_cache* cache, const void* k, const void* v, int32_t T_new,
+                                int64_t ld_tok, void* stream);
 
 /* Decode attention, one query token per sequence, over [prefix || 4-bit cache] (Eq. 3):
  *     score_j = q . K_j * sm_scale,  K_j = prefix_k[h, j] (j < n_prefix) or s_k[h] * code
@@ -146,10 +156,11 @@ pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, cons
  * token t sees every prefixed key and the cached keys 0..t of sequence `seq` (the cache rows must
  * already hold the T tokens: call pq_kv4_append first).
  *     out[t, g, :] = softmax_j(q[t, g, :] . K_j * sm_scale) . V   over j in prefix and j <= t
- *   q, out  bf16 [T, Hq, D] dense, 4-byte aligned; D = 128; Hq / Hkv in {1, 2, 4, 8}; T <= Tmax;
+ *   q  bf16 [T, Hq, D] with ldq elements between tokens (the q part of a concatenated q|k|v output),
+ *   out bf16 [T, Hq, D] dense, both 4-byte aligned; D = 128; Hq / Hkv in {1, 2, 4, 8}; T <= Tmax;
  *   n_prefix <= 64; prefix_k, prefix_v, kq, vq 16-byte aligned. No workspace. */
-pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, int32_t seq, const void* q, int32_t T,
-                                     void* out, float sm_scale, void* stream);
+pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, int32_t seq, const void* q, int64_t ldq,
+                                     int32_t T, void* out, float sm_scale, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Element-wise glue of a Llama transformer block around the quantized linears (the block of the
@@ -160,14 +171,16 @@ pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, int
  *   pq_rmsnorm       y[t,:] = x[t,:] / sqrt(mean(x[t,:]^2) + eps) * g      x, y [M,K], g [K]; K % 8 == 0, K <= 16384
  *   pq_rope          rotate-half pairing, head dim D = 128: for i < 64 and token t at position pos0 + t,
  *                    angle = (pos0 + t) * theta^(-2i/D), y[i] = x[i] cos - x[i+64] sin,
- *                    y[i+64] = x[i+64] cos + x[i] sin       x, y [T,H,D] dense; y may alias x
+ *                    y[i+64] = x[i+64] cos + x[i] sin       x, y [T,H,D] with ld elements between tokens
+ *                    (ld >= H*D, so the q and k heads of a concatenated q|k|v output are rotated in one
+ *                    call); y may alias x
  *   pq_silu_mul      y = gate / (1 + exp(-gate)) * up        gate, up [M,F] with row stride ld_in (the two
  *                    halves of a concatenated gate|up GEMM output), y [M,F] with row stride ldy; F % 8 == 0
  *   pq_residual_add  y = a + b over n elements, n % 8 == 0; y may alias a or b */
 pq_status pq_rmsnorm(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, const void* g, float eps, void* y,
                      int64_t ldy, void* stream);
-pq_status pq_rope(pq_ctx* ctx, const void* x, int64_t T, int32_t H, int32_t D, int64_t pos0, double theta, void* y,
-                  void* stream);
+pq_status pq_rope(pq_ctx* ctx, const void* x, int64_t T, int32_t H, int32_t D, int64_t ld, int64_t pos0, double theta,
+                  void* y, void* stream);
 pq_status pq_silu_mul(pq_ctx* ctx, const void* gate, const void* up, int64_t M, int64_t F, int64_t ld_in, void* y,
                       int64_t ldy, void* stream);
 pq_status pq_residual_add(pq_ctx* ctx, const void* a, const void* b, void* y, int64_t n, void* stream);

@@ -24,7 +24,7 @@ EXPORTS = [
     "pq_status_string", "pq_create", "pq_destroy", "pq_check", "pq_quant_weights", "pq_hadamard_quant_act",
     "pq_calib_act_scale", "pq_w4a4_gemm_workspace_bytes", "pq_w4a4_gemm", "pq_kv4_append",
     "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix", "pq_decode_attn_kv4_prefix_noalloc",
-    "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add", "pq_prefill_attn_kv4_prefix",
+    "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add", "pq_prefill_attn_kv4_prefix", "pq_kv4_append_strided", "pq_calib_kv_scale",
 ]
 
 
@@ -73,10 +73,12 @@ def load_library() -> ctypes.CDLL:
     lib.pq_decode_attn_kv4_prefix.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_void_p, c_void_p, c_float, c_void_p,
                                               c_size_t, c_void_p]
     lib.pq_decode_attn_kv4_prefix_noalloc.argtypes = [POINTER(KV4CacheStruct), c_void_p, c_void_p, c_float, c_void_p]
-    lib.pq_prefill_attn_kv4_prefix.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_int32, c_void_p, c_int32, c_void_p, c_float,
+    lib.pq_calib_kv_scale.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_int32, c_int64, c_void_p, c_void_p]
+    lib.pq_kv4_append_strided.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_void_p, c_void_p, c_int32, c_int64, c_void_p]
+    lib.pq_prefill_attn_kv4_prefix.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_int32, c_void_p, c_int64, c_int32, c_void_p, c_float,
                                                c_void_p]
     lib.pq_rmsnorm.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_float, c_void_p, c_int64, c_void_p]
-    lib.pq_rope.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_int32, c_int64, c_double, c_void_p, c_void_p]
+    lib.pq_rope.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_int32, c_int64, c_int64, c_double, c_void_p, c_void_p]
     lib.pq_silu_mul.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p]
     lib.pq_residual_add.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p]
     for name in EXPORTS:
@@ -209,8 +211,25 @@ class Context:
         _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v")
         B, T_new, Hkv, D = k.shape
         assert (B, Hkv, D) == (cache.B, cache.Hkv, cache.D) and v.shape == k.shape
-        assert k.is_contiguous() and v.is_contiguous()
-        _ok(self.lib.pq_kv4_append(self.h, ctypes.byref(cache.struct), _ptr(k), _ptr(v), T_new, _stream()), "pq_kv4_append")
+        if k.is_contiguous() and v.is_contiguous():
+            _ok(self.lib.pq_kv4_append(self.h, ctypes.byref(cache.struct), _ptr(k), _ptr(v), T_new, _stream()), "pq_kv4_append")
+            return
+        # column slices of a wider matrix (the k and v parts of a q|k|v projection output)
+        ld = k.stride(1)
+        for t in (k, v):
+            assert t.stride(3) == 1 and t.stride(2) == D and t.stride(1) == ld and (B == 1 or t.stride(0) == T_new * ld)
+        _ok(self.lib.pq_kv4_append_strided(self.h, ctypes.byref(cache.struct), _ptr(k), _ptr(v), T_new, ld, _stream()),
+            "pq_kv4_append_strided")
+
+    def calib_kv_scale(self, x: torch.Tensor, s: torch.Tensor | None = None) -> torch.Tensor:
+        """x bf16 [n_tok, Hkv, D] (token stride free): folds max|x|/7 per head into s (created as zeros)."""
+        _dev(x, torch.bfloat16, "x")
+        n_tok, Hkv, D = x.shape
+        assert x.stride(2) == 1 and x.stride(1) == D
+        if s is None:
+            s = torch.zeros((Hkv,), dtype=torch.float32, device=x.device)
+        _ok(self.lib.pq_calib_kv_scale(self.h, _ptr(x), n_tok, Hkv, D, x.stride(0), _ptr(s), _stream()), "pq_calib_kv_scale")
+        return s
 
     def decode_attn_workspace(self, cache: KV4Cache) -> torch.Tensor:
         n = int(self.lib.pq_decode_attn_workspace_bytes(ctypes.byref(cache.struct)))
@@ -230,10 +249,11 @@ class Context:
     def prefill_attn(self, cache: KV4Cache, seq: int, q: torch.Tensor, sm_scale: float, out: torch.Tensor | None = None):
         _dev(q, torch.bfloat16, "q")
         T = q.shape[0]
-        assert q.shape == (T, cache.Hq, cache.D) and q.is_contiguous()
+        assert q.shape == (T, cache.Hq, cache.D) and q.stride(2) == 1 and q.stride(1) == cache.D
         if out is None:
-            out = torch.empty_like(q)
-        _ok(self.lib.pq_prefill_attn_kv4_prefix(self.h, ctypes.byref(cache.struct), int(seq), _ptr(q), T, _ptr(out),
+            out = torch.empty((T, cache.Hq, cache.D), dtype=q.dtype, device=q.device)
+        assert out.is_contiguous()
+        _ok(self.lib.pq_prefill_attn_kv4_prefix(self.h, ctypes.byref(cache.struct), int(seq), _ptr(q), q.stride(0), T, _ptr(out),
                                                 float(sm_scale), _stream()), "pq_prefill_attn_kv4_prefix")
         return out
 
@@ -251,10 +271,11 @@ class Context:
     def rope(self, x: torch.Tensor, pos0: int, theta: float, out: torch.Tensor | None = None):
         _dev(x, torch.bfloat16, "x")
         T, H, D = x.shape
-        assert x.is_contiguous()
+        assert x.stride(2) == 1 and x.stride(1) == D
         if out is None:
-            out = torch.empty_like(x)
-        _ok(self.lib.pq_rope(self.h, _ptr(x), T, H, D, int(pos0), float(theta), _ptr(out), _stream()), "pq_rope")
+            out = torch.empty((T, H, D), dtype=x.dtype, device=x.device)
+        assert out.stride() == x.stride() or (out.is_contiguous() and x.is_contiguous())
+        _ok(self.lib.pq_rope(self.h, _ptr(x), T, H, D, x.stride(0), int(pos0), float(theta), _ptr(out), _stream()), "pq_rope")
         return out
 
     def silu_mul(self, gate: torch.Tensor, up: torch.Tensor, out: torch.Tensor | None = None):

@@ -72,7 +72,7 @@ __global__ void __launch_bounds__(RN_THREADS)
 constexpr int RP_THREADS = 128;
 
 __global__ void __launch_bounds__(RP_THREADS)
-    rope_kernel(const __nv_bfloat16* x, __nv_bfloat16* y, int64_t T, int H, int64_t pos0,
+    rope_kernel(const __nv_bfloat16* x, __nv_bfloat16* y, int64_t T, int H, int64_t ld, int64_t pos0,
                 double log2_theta) {
   __shared__ float cs[64], sn[64];
   for (int64_t t = blockIdx.x; t < T; t += gridDim.x) {
@@ -86,8 +86,8 @@ __global__ void __launch_bounds__(RP_THREADS)
     // a work item = (head, group of 8 consecutive i in [0, 64)): reads x[i..i+7] and x[64+i..64+i+7]
     for (int item = threadIdx.x; item < H * 8; item += RP_THREADS) {
       const int hd = item >> 3, i0 = (item & 7) * 8;
-      const __nv_bfloat16* px = x + (t * H + hd) * 128;
-      __nv_bfloat16* py = y + (t * H + hd) * 128;
+      const __nv_bfloat16* px = x + t * ld + hd * 128;
+      __nv_bfloat16* py = y + t * ld + hd * 128;
       const uint4 a = *reinterpret_cast<const uint4*>(px + i0), b = *reinterpret_cast<const uint4*>(px + 64 + i0);  // y may alias x
       const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
       uint32_t oa[4], ob[4];
@@ -145,6 +145,23 @@ __global__ void __launch_bounds__(EW_THREADS)
   }
 }
 
+// ---- calibration helper: per-head static KV step = max |x| / 7 over a calibration batch ------------
+__global__ void __launch_bounds__(EW_THREADS)
+    calib_kv_scale_kernel(const __nv_bfloat16* __restrict__ x, int64_t n_tok, int Hkv, int64_t ld_tok,
+                          float* __restrict__ s) {
+  const int lane = threadIdx.x & 31;
+  const int64_t n_rows = n_tok * Hkv;  // one warp per (token, head) row of 128 values
+  for (int64_t row = (static_cast<int64_t>(blockIdx.x) * EW_THREADS + threadIdx.x) >> 5; row < n_rows;
+       row += (static_cast<int64_t>(gridDim.x) * EW_THREADS) >> 5) {
+    const int64_t tok = row / Hkv;
+    const int h = static_cast<int>(row % Hkv);
+    const uint2 w = __ldg(reinterpret_cast<const uint2*>(x + tok * ld_tok + h * 128) + lane);
+    float m = fmaxf(fmaxf(fabsf(bf16_lo(w.x)), fabsf(bf16_hi(w.x))), fmaxf(fabsf(bf16_lo(w.y)), fabsf(bf16_hi(w.y))));
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0 && m > 0.0f) atomicMax(reinterpret_cast<int*>(s + h), __float_as_int(__fdiv_rn(m, 7.0f)));
+  }
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 int grid_for(pq_ctx* ctx, int64_t work_items, int per_cta) {
   int64_t g = (work_items + per_cta - 1) / per_cta;
@@ -167,15 +184,15 @@ extern "C" pq_status pq_rmsnorm(pq_ctx* ctx, const void* x, int64_t M, int64_t K
   return pq_launch_status();
 }
 
-extern "C" pq_status pq_rope(pq_ctx* ctx, const void* x, int64_t T, int32_t H, int32_t D, int64_t pos0, double theta,
-                             void* y, void* stream) {
+extern "C" pq_status pq_rope(pq_ctx* ctx, const void* x, int64_t T, int32_t H, int32_t D, int64_t ld, int64_t pos0,
+                             double theta, void* y, void* stream) {
   if (!ctx || !x || !y) return PQ_ERR_INVALID_ARG;
-  if (T < 0 || H <= 0 || pos0 < 0 || !(theta > 1.0)) return PQ_ERR_INVALID_ARG;
+  if (T < 0 || H <= 0 || pos0 < 0 || !(theta > 1.0) || ld < static_cast<int64_t>(H) * 128) return PQ_ERR_INVALID_ARG;
   if (D != 128) return PQ_ERR_SHAPE;
-  if (!aligned16(x) || !aligned16(y)) return PQ_ERR_ALIGN;
+  if (!aligned16(x) || !aligned16(y) || ld % 8 != 0) return PQ_ERR_ALIGN;
   if (T == 0) return PQ_OK;
   rope_kernel<<<grid_for(ctx, T, 1), RP_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(y), T, H, pos0, log2(theta));
+      static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(y), T, H, ld, pos0, log2(theta));
   return pq_launch_status();
 }
 
@@ -199,5 +216,17 @@ extern "C" pq_status pq_residual_add(pq_ctx* ctx, const void* a, const void* b, 
   if (n == 0) return PQ_OK;
   add_kernel<<<grid_for(ctx, n / 8, EW_THREADS), EW_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const __nv_bfloat16*>(a), static_cast<const __nv_bfloat16*>(b), static_cast<__nv_bfloat16*>(y), n / 8);
+  return pq_launch_status();
+}
+
+extern "C" pq_status pq_calib_kv_scale(pq_ctx* ctx, const void* x, int64_t n_tok, int32_t Hkv, int32_t D, int64_t ld_tok,
+                                       float* s, void* stream) {
+  if (!ctx || !x || !s) return PQ_ERR_INVALID_ARG;
+  if (n_tok < 0 || Hkv <= 0 || ld_tok < static_cast<int64_t>(Hkv) * 128) return PQ_ERR_INVALID_ARG;
+  if (D != 128) return PQ_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(x) & 7) || ld_tok % 4 != 0) return PQ_ERR_ALIGN;
+  if (n_tok == 0) return PQ_OK;
+  calib_kv_scale_kernel<<<grid_for(ctx, n_tok * Hkv, EW_THREADS / 32), EW_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(x), n_tok, Hkv, ld_tok, s);
   return pq_launch_status();
 }

@@ -15,7 +15,7 @@ constexpr int AP_THREADS = 256;
 __global__ void __launch_bounds__(AP_THREADS)
     kv4_append_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, uint8_t* __restrict__ kq,
                       uint8_t* __restrict__ vq, const float* __restrict__ s_k, const float* __restrict__ s_v,
-                      int32_t* __restrict__ len, int B, int T_new, int Hkv, int Tmax, int32_t* status,
+                      int32_t* __restrict__ len, int B, int T_new, int Hkv, int Tmax, int64_t ld_tok, int32_t* status,
                       uint32_t* ticket) {
   __shared__ int bad;
   __shared__ int last;
@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(AP_THREADS)
     const int64_t bt = bth / Hkv;
     const int t = static_cast<int>(bt % T_new), b = static_cast<int>(bt / T_new);
     const int64_t pos = len[b] + t;
-    const int64_t src = bth * 128 + part * 32;
+    const int64_t src = bt * ld_tok + h * 128 + part * 32;
     const int64_t dst = ((static_cast<int64_t>(b) * Hkv + h) * Tmax + pos) * 64 + part * 16;
 #pragma unroll
     for (int which = 0; which < 2; ++which) {
@@ -536,20 +536,27 @@ pq_status check_cache(const pq_kv4_cache* c) {
 
 }  // namespace
 
-extern "C" pq_status pq_kv4_append(pq_ctx* ctx, const pq_kv4_cache* cache, const void* k, const void* v,
-                                   int32_t T_new, void* stream) {
+extern "C" pq_status pq_kv4_append_strided(pq_ctx* ctx, const pq_kv4_cache* cache, const void* k, const void* v,
+                                           int32_t T_new, int64_t ld_tok, void* stream) {
   if (!ctx || !k || !v || T_new < 0) return PQ_ERR_INVALID_ARG;
   pq_status st = check_cache(cache);
   if (st != PQ_OK) return st;
-  if ((reinterpret_cast<uintptr_t>(k) & 15) || (reinterpret_cast<uintptr_t>(v) & 15)) return PQ_ERR_ALIGN;
+  if (ld_tok < static_cast<int64_t>(cache->Hkv) * 128) return PQ_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(k) & 15) || (reinterpret_cast<uintptr_t>(v) & 15) || ld_tok % 8 != 0) return PQ_ERR_ALIGN;
   if (T_new == 0 || cache->B == 0) return PQ_OK;
   const int64_t n_units = static_cast<int64_t>(cache->B) * T_new * cache->Hkv * 4;
   int64_t grid = (n_units + AP_THREADS - 1) / AP_THREADS;
   if (grid > 8LL * ctx->sm_count) grid = 8LL * ctx->sm_count;
   kv4_append_kernel<<<static_cast<int>(grid), AP_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v), cache->kq, cache->vq, cache->s_k,
-      cache->s_v, cache->len, cache->B, T_new, cache->Hkv, cache->Tmax, ctx->d_status, ctx->d_tickets);
+      cache->s_v, cache->len, cache->B, T_new, cache->Hkv, cache->Tmax, ld_tok, ctx->d_status, ctx->d_tickets);
   return pq_launch_status();
+}
+
+extern "C" pq_status pq_kv4_append(pq_ctx* ctx, const pq_kv4_cache* cache, const void* k, const void* v,
+                                   int32_t T_new, void* stream) {
+  if (!cache) return PQ_ERR_INVALID_ARG;
+  return pq_kv4_append_strided(ctx, cache, k, v, T_new, static_cast<int64_t>(cache->Hkv) * 128, stream);
 }
 
 extern "C" size_t pq_decode_attn_workspace_bytes(const pq_kv4_cache* cache) {

@@ -60,7 +60,8 @@ __device__ __forceinline__ uint32_t byte_to_h2(uint32_t b) {
 __device__ __forceinline__ uint32_t tile_off(int r, int c) { return static_cast<uint32_t>(r * 256 + ((c ^ (r & 7)) << 4)); }
 
 struct PrefillParams {
-  const __nv_bfloat16* q;   // [T, Hq, 128]
+  const __nv_bfloat16* q;   // [T, Hq, 128] with ldq elements between tokens
+  int64_t ldq;
   __nv_bfloat16* out;       // [T, Hq, 128]
   const __half* prefix_k;   // [Hkv, n_prefix, 128]
   const __half* prefix_v;
@@ -130,8 +131,8 @@ __global__ void __launch_bounds__(32 * G) prefill_attn_kernel(const PrefillParam
   uint32_t qa[8][4];
   {
     const int r0 = min(tok0 + g, p.T - 1), r1 = min(tok0 + g + 8, p.T - 1);
-    const uint32_t* q0 = reinterpret_cast<const uint32_t*>(p.q + (static_cast<int64_t>(r0) * p.Hq + head) * 128);
-    const uint32_t* q1 = reinterpret_cast<const uint32_t*>(p.q + (static_cast<int64_t>(r1) * p.Hq + head) * 128);
+    const uint32_t* q0 = reinterpret_cast<const uint32_t*>(p.q + static_cast<int64_t>(r0) * p.ldq + head * 128);
+    const uint32_t* q1 = reinterpret_cast<const uint32_t*>(p.q + static_cast<int64_t>(r1) * p.ldq + head * 128);
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
       const uint32_t w[4] = {__ldg(q0 + ks * 8 + t), __ldg(q1 + ks * 8 + t), __ldg(q0 + ks * 8 + 4 + t), __ldg(q1 + ks * 8 + 4 + t)};
@@ -300,9 +301,10 @@ pq_status launch_prefill(const PrefillParams& p, cudaStream_t st) {
 
 }  // namespace
 
-extern "C" pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* c, int32_t seq, const void* q, int32_t T,
-                                                void* out, float sm_scale, void* stream) {
+extern "C" pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* c, int32_t seq, const void* q, int64_t ldq,
+                                                int32_t T, void* out, float sm_scale, void* stream) {
   if (!ctx || !c || !q || !out || !c->kq || !c->vq || !c->s_k || !c->s_v) return PQ_ERR_INVALID_ARG;
+  if (ldq < static_cast<int64_t>(c->Hq) * 128 || (ldq & 1)) return PQ_ERR_INVALID_ARG;
   if (T < 0 || seq < 0 || seq >= c->B || c->Hkv <= 0 || c->Hq <= 0 || c->n_prefix < 0) return PQ_ERR_INVALID_ARG;
   if (c->n_prefix > 0 && (!c->prefix_k || !c->prefix_v)) return PQ_ERR_INVALID_ARG;
   if (c->D != 128 || c->Hq % c->Hkv != 0 || T > c->Tmax || c->n_prefix > PA_KEYS || c->Hkv > 65535) return PQ_ERR_SHAPE;
@@ -315,6 +317,7 @@ extern "C" pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache*
   if (T == 0) return PQ_OK;
   PrefillParams p;
   p.q = static_cast<const __nv_bfloat16*>(q);
+  p.ldq = ldq;
   p.out = static_cast<__nv_bfloat16*>(out);
   p.prefix_k = static_cast<const __half*>(c->prefix_k);
   p.prefix_v = static_cast<const __half*>(c->prefix_v);
