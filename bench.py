@@ -253,6 +253,7 @@ def run_gpu(args):
         try:
             sections["decode_gemm"] = section_decode_gemm(ctx, device, peaks)
             sections["decode_attention"] = section_decode_attention(ctx, device, peaks)
+            sections["block_llama3_70b_prefill4096"] = section_block(ctx, device, peaks)
         except Exception as e:  # sections never take the main line down
             sections["error"] = repr(e)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -390,6 +391,65 @@ def section_decode_attention(ctx, device, peaks):
     return {"attention_us": round(ms_attn * 1e3, 3), "append_us": round(ms_app * 1e3, 3), "append+attention_us": round(ms_both * 1e3, 3),
             "GB/s": round(gbs, 1), "frac_measured_hbm": round(gbs / peaks["hbm"], 3), "frac_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 3),
             "bytes_per_step": by}
+
+
+def section_block(ctx, device, peaks):
+    """configs[4]: one Llama-3-70B-shaped W4A4KV4 block at prefill, 4096 ordinary tokens after 4 prefixed
+    tokens whose K/V sit in the cache in fp16; static scales from a seed-1 calibration pass."""
+    import torch
+
+    from paper_2410_05265_b200 import block, inputs
+
+    c = inputs.LLAMA3_70B
+    T, P, D = 4096, 4, c["head_dim"]
+    shape = block.BlockShape(hidden=c["hidden"], n_q_heads=c["n_q_heads"], n_kv_heads=c["n_kv_heads"], ffn=c["ffn"])
+    qd, kvd = shape.q_dim, shape.kv_dim
+    mk = lambda n, k, seed: inputs.weights(n, k, seed=seed, device=device)
+    blk = block.Block(ctx, shape, mk(qd + 2 * kvd, shape.hidden, 2), mk(shape.hidden, qd, 3), mk(2 * shape.ffn, shape.hidden, 4),
+                      mk(shape.hidden, shape.ffn, 5), torch.ones(shape.hidden, dtype=torch.bfloat16, device=device),
+                      torch.ones(shape.hidden, dtype=torch.bfloat16, device=device),
+                      inputs.prefix_kv(c["n_kv_heads"], P, D, 0, "k", 50.0, device=device),
+                      inputs.prefix_kv(c["n_kv_heads"], P, D, 0, "v", 50.0, device=device), t_max=T)
+    torch.cuda.synchronize()
+    blk.forward(inputs.activations(T, shape.hidden, seed=1, device=device), calibrate=True)
+    x = inputs.activations(T, shape.hidden, seed=0, device=device)
+    for _ in range(3):
+        blk.forward(x)
+    ctx.check()
+    reps = 10
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        blk.forward(x)
+    e1.record()
+    torch.cuda.synchronize()
+    ctx.check()
+    ms = e0.elapsed_time(e1) / reps
+    # per-stage share: one more pass with an event after every stage
+    marks = []
+
+    def tap(name, t):
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record()
+        marks.append((name, ev))
+
+    start = torch.cuda.Event(enable_timing=True)
+    start.record()
+    blk.forward(x, tap=tap)
+    torch.cuda.synchronize()
+    stages, prev = {}, start
+    for name, ev in marks:
+        if name in ("vq", "y"):
+            continue
+        stages[name] = round(prev.elapsed_time(ev), 4)
+        prev = ev
+    gemm_ops = 2.0 * T * shape.hidden * (qd + 2 * kvd + qd + 2 * shape.ffn + shape.ffn)
+    attn_flops = 4.0 * D * c["n_q_heads"] * (T * (T + 1) / 2 + T * P)
+    gemm_ms = sum(stages[k] for k in ("qkv", "o", "gu", "d"))
+    return {"tokens_per_s": round(T / (ms * 1e-3), 1), "ms": round(ms, 4), "tokens": T, "n_prefix": P,
+            "gemm_TOPS": round(gemm_ops / (gemm_ms * 1e-3) / 1e12, 1), "gemm_share": round(gemm_ms / sum(stages.values()), 3),
+            "attention_TFLOPS": round(attn_flops / (stages["attn"] * 1e-3) / 1e12, 1), "stage_ms": stages,
+            "launches": block.Block.LAUNCHES_PER_FORWARD}
 
 
 # ------------------------------------------------------------------------------------- CPU oracle arms
