@@ -40,7 +40,9 @@ __device__ __forceinline__ uint4 ld_stream(const uint8_t* p) {
   return v;
 }
 
-template <bool TWO_GROUPS>
+// HALF_ROWS: the CTA owns 8 output channels instead of 16 (rows 8..15 of the MMA tile stay zero), which
+// doubles the CTA count of narrow layers.
+template <bool TWO_GROUPS, bool HALF_ROWS>
 __global__ void __launch_bounds__(GS_THREADS)
     gemm_w4a4_stream_kernel(const uint8_t* __restrict__ xq, const uint8_t* __restrict__ wq,
                             const float* __restrict__ s_a, const float* __restrict__ s_w,
@@ -49,11 +51,12 @@ __global__ void __launch_bounds__(GS_THREADS)
   __shared__ int red[GS_WARPS][GS_CH][16];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int n0 = blockIdx.x * GS_CH;
+  constexpr int CH = HALF_ROWS ? GS_CH / 2 : GS_CH;  // output channels of this CTA
+  const int n0 = blockIdx.x * CH;
   const int kbytes = K / 2;
   const int n_steps = (K + 127) / 128;
 
-  const bool w0_ok = n0 + g < N, w1_ok = n0 + g + 8 < N;
+  const bool w0_ok = n0 + g < N, w1_ok = !HALF_ROWS && n0 + g + 8 < N;
   const bool x0_ok = g < M, x1_ok = TWO_GROUPS && (g + 8 < M);
   const uint8_t* w0p = wq + static_cast<int64_t>(n0 + g) * kbytes + t * 16;
   const uint8_t* w1p = wq + static_cast<int64_t>(n0 + g + 8) * kbytes + t * 16;
@@ -63,6 +66,11 @@ __global__ void __launch_bounds__(GS_THREADS)
   int c0[4] = {0, 0, 0, 0}, c1[4] = {0, 0, 0, 0};
   const uint4 zero = make_uint4(0, 0, 0, 0);
 
+  // The weights are static, the activations and the output may belong to the kernel before this one
+  // in the stream: let the next kernel start early, fetch the first weight chunks, and only then wait
+  // for the previous kernel (programmatic dependent launch; both instructions do nothing without it).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  bool first = true;
   for (int base = warp; base < n_steps; base += GS_WARPS * GS_UNROLL) {
     uint4 wa[GS_UNROLL], wb[GS_UNROLL], xa[GS_UNROLL], xb[GS_UNROLL];
 #pragma unroll
@@ -72,6 +80,16 @@ __global__ void __launch_bounds__(GS_THREADS)
       const bool in_k = ks < n_steps && off + t * 16 < kbytes;
       wa[u] = (in_k && w0_ok) ? ld_stream(w0p + off) : zero;
       wb[u] = (in_k && w1_ok) ? ld_stream(w1p + off) : zero;
+    }
+    if (first) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      first = false;
+    }
+#pragma unroll
+    for (int u = 0; u < GS_UNROLL; ++u) {
+      const int ks = base + u * GS_WARPS;
+      const int off = ks * 64;
+      const bool in_k = ks < n_steps && off + t * 16 < kbytes;
       xa[u] = (in_k && x0_ok) ? __ldg(reinterpret_cast<const uint4*>(x0p + off)) : zero;
       if (TWO_GROUPS) xb[u] = (in_k && x1_ok) ? __ldg(reinterpret_cast<const uint4*>(x1p + off)) : zero;
     }
@@ -91,6 +109,7 @@ __global__ void __launch_bounds__(GS_THREADS)
       }
     }
   }
+  if (first) asm volatile("griddepcontrol.wait;" ::: "memory");  // a warp without any K step
   // accumulator layout: c[0], c[1] -> channel g, tokens 2t, 2t+1; c[2], c[3] -> channel g+8
   red[warp][g][2 * t] = c0[0];
   red[warp][g][2 * t + 1] = c0[1];
@@ -106,7 +125,7 @@ __global__ void __launch_bounds__(GS_THREADS)
   {
     const int ch = threadIdx.x & 15, tok = threadIdx.x >> 4;  // 16 tokens x 16 channels = 256 threads
     const int n = n0 + ch;
-    if (tok < M && n < N && (TWO_GROUPS || tok < 8)) {
+    if (tok < M && n < N && ch < CH && (TWO_GROUPS || tok < 8)) {
       int s = 0;
 #pragma unroll
       for (int w = 0; w < GS_WARPS; ++w) s += red[w][ch][tok];
@@ -121,18 +140,36 @@ __global__ void __launch_bounds__(GS_THREADS)
 }  // namespace
 
 // Rows [0, M) of xq/out, M <= 16 (the caller has already applied row_begin).
+template <bool TWO, bool HALF>
+static pq_status launch_stream(const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w, void* out,
+                               int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st) {
+  const int ch = HALF ? GS_CH / 2 : GS_CH;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>((N + ch - 1) / ch));
+  cfg.blockDim = dim3(GS_THREADS);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  // the kernel may start while its predecessor in the stream drains; it waits for it on the device
+  // before it touches anything but the weights
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, gemm_w4a4_stream_kernel<TWO, HALF>, xq, wq, s_a, s_w, static_cast<__nv_bfloat16*>(out), ldo,
+                         static_cast<int>(M), static_cast<int>(N), static_cast<int>(K), acc_dbg) != cudaSuccess)
+    return PQ_ERR_CUDA;
+  return pq_launch_status();
+}
+
 pq_status pq_gemm_stream_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
                                 void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg,
                                 cudaStream_t st) {
-  (void)ctx;
-  const int grid = static_cast<int>((N + GS_CH - 1) / GS_CH);
+  // 16 channels per CTA when that still gives every SM several CTAs, else 8 (only for up to 8 tokens:
+  // with two token groups the narrower CTA repeats too much of the activation expansion)
+  const bool half = M <= 8 && (N + GS_CH - 1) / GS_CH < 4LL * ctx->sm_count;
   if (M <= 8)
-    gemm_w4a4_stream_kernel<false><<<grid, GS_THREADS, 0, st>>>(xq, wq, s_a, s_w, static_cast<__nv_bfloat16*>(out), ldo,
-                                                                static_cast<int>(M), static_cast<int>(N),
-                                                                static_cast<int>(K), acc_dbg);
-  else
-    gemm_w4a4_stream_kernel<true><<<grid, GS_THREADS, 0, st>>>(xq, wq, s_a, s_w, static_cast<__nv_bfloat16*>(out), ldo,
-                                                               static_cast<int>(M), static_cast<int>(N),
-                                                               static_cast<int>(K), acc_dbg);
-  return pq_launch_status();
+    return half ? launch_stream<false, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st)
+                : launch_stream<false, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st);
+  return launch_stream<true, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st);
 }
