@@ -548,6 +548,19 @@ def run_case(args):
         it = iter(range(10**9))
         fn = lambda: ctx.decode_attn(caches[next(it) % layers], q, 1 / math.sqrt(D), ws, out=out)
         work = float(B * Hkv * T * D)
+    elif name == "prefill":
+        T, Hq, Hkv = dims or [4096, 64, 8]
+        D, P = 128, 4
+        pk = inputs.prefix_kv(Hkv, P, D, 0, "k", 50.0, device=dev)
+        pv = inputs.prefix_kv(Hkv, P, D, 0, "v", 50.0, device=dev)
+        s = torch.full((Hkv,), 4.5 / 7, device=dev)
+        cache = binding.KV4Cache(pk, pv, torch.randint(0, 256, (1, Hkv, T, D // 2), dtype=torch.uint8, device=dev),
+                                 torch.randint(0, 256, (1, Hkv, T, D // 2), dtype=torch.uint8, device=dev), s, s,
+                                 torch.full((1,), T, dtype=torch.int32, device=dev), Hq)
+        q = inputs.kv_tensor(1, T, Hq, D, 0, "k", device=dev)[0].contiguous()
+        out = torch.empty_like(q)
+        fn = lambda: ctx.prefill_attn(cache, 0, q, 1 / math.sqrt(D), out=out)
+        work = 4.0 * D * Hq * (T * (T + 1) / 2 + T * P)
     else:
         raise SystemExit(f"unknown case {name}")
     for _ in range(3):
@@ -566,7 +579,7 @@ def run_case(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--case", default=None, help="run one kernel on a small case: gemm:M,N,K | hadamard:M,K,B | attn:B,Hq,Hkv,T,layers")
+    ap.add_argument("--case", default=None, help="run one kernel on a small case: gemm:M,N,K | hadamard:M,K,B | attn:B,Hq,Hkv,T,layers | prefill:T,Hq,Hkv")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
