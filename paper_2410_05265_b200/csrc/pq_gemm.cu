@@ -1,11 +1,11 @@
 // Entry point of the W4A4 linear layer: argument checks and the choice between the tensor-core
-// kernel (prefill-shaped) and the weight-streaming kernel (decode-shaped).
+// kernels (prefill-shaped) and the weight-streaming kernel (decode-shaped).
 #include "pq_common.cuh"
 
-pq_status pq_gemm_tc_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
-                            void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st);
 pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
                               void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st);
+pq_status pq_gemm_pair_ts_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
+                                 void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st);
 pq_status pq_gemm_stream_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a,
                                 const float* s_w, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K,
                                 int32_t* acc_dbg, cudaStream_t st);
@@ -31,5 +31,10 @@ extern "C" pq_status pq_w4a4_gemm(pq_ctx* ctx, const uint8_t* xq, const uint8_t*
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (K == 0) return PQ_ERR_SHAPE;
   if (m <= 16) return pq_gemm_stream_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st);
+  // Two CTA-pair kernels: with the token operand in shared memory the accumulator is double-buffered
+  // and the epilogue is free, which wins for short K; with the token operand in tensor memory the
+  // expansion costs a third less shared-memory traffic, which wins once a tile's K loop is long enough
+  // to hide the single accumulator's epilogue (measured crossover near K = 8192).
+  if (K >= 8192) return pq_gemm_pair_ts_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st);
   return pq_gemm_pair_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st);
 }

@@ -107,6 +107,8 @@ def _gemm_case(ctx, M, N, K, seed, row_begin=0, real_scales=True):
     (200, 264, 416),     # ragged M, N and K (K % 128 != 0)
     (17, 40, 160),       # smallest tensor-core case, mostly padding
     (333, 1000, 2048),
+    (300, 520, 8192),    # long K: the kernel that keeps the token operand in tensor memory
+    (257, 256, 14336),
 ])
 def test_gemm_prefill_shapes_bit_exact(ctx, M, N, K):
     _gemm_case(ctx, M, N, K, seed=M + N + K)
