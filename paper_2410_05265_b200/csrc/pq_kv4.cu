@@ -90,7 +90,7 @@ constexpr int DA_CHUNKS = DA_ROUND / DA_CHUNK;
 constexpr int DA_HALF_BYTES = DA_ROUND * 64 * 2;  // packed K rows, then packed V rows
 constexpr int DA_SMEM_BYTES = 2 * DA_HALF_BYTES;  // 32 KB
 static_assert(DA_CHUNK == 16 * DA_WARPS, "one 16-key block per warp per chunk");
-static_assert(DA_SMEM_BYTES >= DA_WARPS * DA_ROWS * 128 * 4, "the staging area is reused for the per-warp partials");
+static_assert(DA_SMEM_BYTES >= (DA_WARPS + 1) * DA_ROWS * 128 * 4, "the staging area is reused for the partials");
 
 // D (+)= A * B, m16n8k16, fp16 inputs, fp32 accumulate. The short form leaves rows 8..15 of A zero.
 __device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
@@ -142,6 +142,27 @@ __device__ __forceinline__ uint2 lds64(uint32_t a) {
   return v;
 }
 
+// ---- thread-block cluster helpers (distributed shared memory) --------------------------------------
+__device__ __forceinline__ void cluster_arrive_wait() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_cta(uint32_t smem_addr, int rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ float2 ld_cluster_f2(uint32_t a) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a));
+  return v;
+}
+
 struct AttnParams {
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
@@ -174,10 +195,16 @@ struct AttnParams {
 //            rounded values.
 // The CTA of the last split also scores the full-precision prefix keys and folds them into its partial.
 // The last CTA of a (sequence, head) to finish merges the partials and writes bf16.
+// CLUSTER: the splits of a (sequence, head) form one thread-block cluster and merge their partials
+// through distributed shared memory (no workspace, no ticket); otherwise the partials go through the
+// caller's workspace and the last CTA to finish merges them.
+template <bool CLUSTER>
 __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParams p) {
   extern __shared__ __align__(128) uint8_t da_stage[];  // two halves of [K rows | V rows] of one round
   // the per-warp partial outputs reuse the staging area once the key loop is over
   float (*sm_o)[DA_ROWS][128] = reinterpret_cast<float (*)[DA_ROWS][128]>(da_stage);
+  float* cl_o = reinterpret_cast<float*>(da_stage + DA_WARPS * DA_ROWS * 128 * 4);  // [G][128]: this CTA's partial (cluster mode)
+  __shared__ float2 cl_ml[DA_ROWS];
   __shared__ __align__(8) uint64_t full[2][DA_CHUNKS];
   __shared__ float sm_ml[DA_WARPS][DA_ROWS][2];
   __shared__ float sm_pre[DA_ROWS][DA_MAX_PREFIX];
@@ -429,10 +456,55 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
         acc = fmaf(e, __half2float(p.prefix_v[(static_cast<int64_t>(h) * p.n_prefix + j) * 128 + d]), acc);
         l += e;
       }
-      const int64_t slot = (static_cast<int64_t>(bh) * S + split) * G + r;
-      p.ws_o[slot * 128 + d] = acc;
-      if (d == 0) *reinterpret_cast<float2*>(p.ws_ml + slot * 2) = make_float2(m, l);
+      if (CLUSTER) {
+        cl_o[r * 128 + d] = acc;
+        if (d == 0) cl_ml[r] = make_float2(m, l);
+      } else {
+        const int64_t slot = (static_cast<int64_t>(bh) * S + split) * G + r;
+        p.ws_o[slot * 128 + d] = acc;
+        if (d == 0) *reinterpret_cast<float2*>(p.ws_ml + slot * 2) = make_float2(m, l);
+      }
     }
+  }
+  if (CLUSTER) {
+    // every split's partial is in its CTA's shared memory; thread i of the cluster takes (head, four
+    // dims) item i and reads the S partials through distributed shared memory, all loads at once
+    cluster_arrive_wait();
+    const int item = split * DA_THREADS + threadIdx.x;  // split == rank in the cluster
+    if (item < G * 32) {
+      const int r = item >> 5, c4 = item & 31;
+      const uint32_t o_addr = pq::smem_u32(cl_o + r * 128 + 4 * c4), ml_addr = pq::smem_u32(cl_ml + r);
+      float4 v[8];
+      float2 ml[8];
+#pragma unroll
+      for (int sp = 0; sp < 8; ++sp) {
+        if (sp < S) {
+          v[sp] = ld_cluster_f4(map_cta(o_addr, sp));
+          ml[sp] = ld_cluster_f2(map_cta(ml_addr, sp));
+        } else {
+          v[sp] = make_float4(0.f, 0.f, 0.f, 0.f);
+          ml[sp] = make_float2(-INFINITY, 0.f);
+        }
+      }
+      float m = -INFINITY;
+#pragma unroll
+      for (int sp = 0; sp < 8; ++sp) m = fmaxf(m, ml[sp].x);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float l = 0.0f;
+#pragma unroll
+      for (int sp = 0; sp < 8; ++sp) {
+        const float w = ml[sp].x == -INFINITY ? 0.0f : ex2(ml[sp].x - m);
+        acc.x = fmaf(v[sp].x, w, acc.x), acc.y = fmaf(v[sp].y, w, acc.y), acc.z = fmaf(v[sp].z, w, acc.z), acc.w = fmaf(v[sp].w, w, acc.w);
+        l = fmaf(ml[sp].y, w, l);
+      }
+      const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+      uint2 packed;
+      packed.x = *reinterpret_cast<const uint32_t*>(&lo), packed.y = *reinterpret_cast<const uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(p.out + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + 4 * c4) = packed;
+    }
+    cluster_arrive_wait();  // no CTA leaves while a peer may still read its shared memory
+    return;
   }
   __threadfence();
   __syncthreads();
@@ -506,7 +578,10 @@ bool set_attn_smem() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
   if (!done[dev]) {
-    if (cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) != cudaSuccess)
+    if (cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) !=
+            cudaSuccess)
       return false;
     done[dev] = true;
   }
@@ -576,7 +651,11 @@ extern "C" pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* 
     return PQ_ERR_SHAPE;
   if (!ws || ws_bytes < pq_decode_attn_workspace_bytes(cache)) return PQ_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(ws) & 15) return PQ_ERR_ALIGN;
-  const int S = choose_splits(ctx, cache);
+  int S = choose_splits(ctx, cache);
+  // With enough (sequence, head) pairs, eight splits already fill the GPU: the splits then form one
+  // cluster and merge through distributed shared memory (the workspace and the tickets stay unused).
+  const bool cluster = static_cast<int64_t>(cache->B) * cache->Hkv * 8 >= 2LL * ctx->sm_count;
+  if (cluster && S > 8) S = 8;
   const int G = cache->Hq / cache->Hkv;
   AttnParams p;
   p.q = static_cast<const __nv_bfloat16*>(q);
@@ -596,7 +675,23 @@ extern "C" pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* 
   p.B = cache->B, p.Hq = cache->Hq, p.Hkv = cache->Hkv, p.G = G, p.n_prefix = cache->n_prefix, p.Tmax = cache->Tmax;
   dim3 grid(S, cache->Hkv, cache->B);
   if (!set_attn_smem()) return PQ_ERR_CUDA;
-  decode_attn_kernel<<<grid, DA_THREADS, DA_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(p);
+  if (cluster) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(DA_THREADS);
+    cfg.dynamicSmemBytes = DA_SMEM_BYTES;
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, decode_attn_kernel<true>, p) != cudaSuccess) return PQ_ERR_CUDA;
+    return pq_launch_status();
+  }
+  decode_attn_kernel<false><<<grid, DA_THREADS, DA_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(p);
   return pq_launch_status();
 }
 
@@ -687,6 +782,6 @@ extern "C" pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache
   p.B = cache->B, p.Hq = cache->Hq, p.Hkv = cache->Hkv, p.G = G, p.n_prefix = cache->n_prefix, p.Tmax = cache->Tmax;
   dim3 grid(S, cache->Hkv, cache->B);
   if (!set_attn_smem()) return PQ_ERR_CUDA;
-  decode_attn_kernel<<<grid, DA_THREADS, DA_SMEM_BYTES, cs>>>(p);
+  decode_attn_kernel<false><<<grid, DA_THREADS, DA_SMEM_BYTES, cs>>>(p);
   return pq_launch_status();
 }
