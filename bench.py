@@ -59,6 +59,21 @@ def read_peaks():
     return dict(hbm=6650.0, bf16=1590.0, bf16_sus=1400.0, src="fallback")
 
 
+def job_throughput(ms_local: float, steps: int, units_per_step_per_rank: float, world: int, dist=None, device=None):
+    """Whole-job figures of a replicated (weak-scaling) run: every rank processes the same number of
+    units per step, the job's step time is the slowest rank's, the value is all ranks' units over it.
+    Returns (ms_per_step, units_per_second). With dist given, the maximum is taken over the ranks."""
+    ms = float(ms_local)
+    if dist is not None and world > 1:
+        import torch
+
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / steps
+    return ms_per_step, world * units_per_step_per_rank / (ms_per_step * 1e-3)
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -193,13 +208,8 @@ def run_gpu(args):
     barrier()
     clocks = sampler.stop()
     ctx.check()
-    ms = t0.elapsed_time(t1)
-    if dist:
-        tmax = torch.tensor([ms], device=device)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
-    ms_per_step = ms / args.steps
-    value = world * step_ops(m_rows) / (ms_per_step * 1e-3) / 1e12
+    ms_per_step, ops_per_s = job_throughput(t0.elapsed_time(t1), args.steps, step_ops(m_rows), world, dist, device)
+    value = ops_per_s / 1e12
 
     gemm_ms = sum(e0.elapsed_time(e1) for _, e0, e1 in gemm_events)
     per_shape = {}
