@@ -1,8 +1,10 @@
 // Causal prefill attention over [full-precision prefix || INT4 cache] (Sec. 4.2, Eq. 3): query t of a
 // sequence sees every prefixed key and the cached keys 0..t of the same sequence.
 //
-// Grid (query tiles, KV heads). A CTA owns 16 consecutive query tokens of the G query heads that
-// share one KV head; warp g holds head g's 16 x 128 query tile as fp16 MMA fragments. Keys are
+// Grid (query tiles, KV heads, head groups). A CTA owns 16 consecutive query tokens of up to four of
+// the query heads that share one KV head (four warps: two such CTAs fit an SM, which hides the
+// softmax phases of one behind the MMAs of the other); warp g holds one head's 16 x 128 query tile as
+// fp16 MMA fragments. Keys are
 // walked in blocks of 64: the packed rows are fetched one block ahead into registers, expanded to
 // exact fp16 integers (the per-head steps s_k, s_v are folded into the score scale and the final
 // normalisation) and stored as swizzled [key][dim] tiles that ldmatrix turns into MMA operands.
@@ -122,7 +124,7 @@ __global__ void __launch_bounds__(32 * G) prefill_attn_kernel(const PrefillParam
   const int h = blockIdx.y;
   const int tile = gridDim.x - 1 - blockIdx.x;  // long tiles first
   const int tok0 = tile * PA_TOK;
-  const int head = h * G + warp;
+  const int head = h * p.G + blockIdx.z * G + warp;  // G = heads of this CTA, p.G = heads per KV head
   const int n_ctx = min(p.T, tok0 + PA_TOK);     // cached keys any row of this tile may see
   const int n_blocks = (n_ctx + PA_KEYS - 1) / PA_KEYS;
   const bool has_prefix = p.n_prefix > 0;
@@ -294,7 +296,7 @@ pq_status launch_prefill(const PrefillParams& p, cudaStream_t st) {
       return PQ_ERR_CUDA;
     attr_set[dev] = true;
   }
-  dim3 grid((p.T + PA_TOK - 1) / PA_TOK, p.Hkv);
+  dim3 grid((p.T + PA_TOK - 1) / PA_TOK, p.Hkv, p.G / G);
   prefill_attn_kernel<G><<<grid, 32 * G, smem, st>>>(p);
   return pq_launch_status();
 }
@@ -333,6 +335,6 @@ extern "C" pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache*
     case 1: return launch_prefill<1>(p, st);
     case 2: return launch_prefill<2>(p, st);
     case 4: return launch_prefill<4>(p, st);
-    default: return launch_prefill<8>(p, st);
+    default: return launch_prefill<4>(p, st);  // eight heads per KV head: two CTAs of four warps, two CTAs per SM
   }
 }
