@@ -268,7 +268,7 @@ def run_gpu(args):
         except Exception as e:  # sections never take the main line down
             sections["error"] = repr(e)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu_baseline = oracle_sample(16)
+        cpu_baseline = oracle_sample(384)  # about 10-15 s of host work
 
     if rank == 0:
         line = {
