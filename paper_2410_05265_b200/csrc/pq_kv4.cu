@@ -84,6 +84,7 @@ constexpr int DA_MAX_SPLITS = 32;
 constexpr int DA_MAX_PREFIX = 64;
 constexpr int DA_ROWS = 8;  // query heads per KV head the MMA tile can carry
 constexpr int DA_TICKET0 = 16;
+constexpr float DA_HEADROOM = 15.0f;  // log2 units a score may exceed the reference exponent before it is moved
 constexpr int DA_ROUND = 128;                     // keys staged per round (one half of the staging buffer)
 constexpr int DA_CHUNK = 64;                      // keys per bulk copy and per barrier
 constexpr int DA_CHUNKS = DA_ROUND / DA_CHUNK;
@@ -92,23 +93,19 @@ constexpr int DA_SMEM_BYTES = 2 * DA_HALF_BYTES;  // 32 KB
 static_assert(DA_CHUNK == 16 * DA_WARPS, "one 16-key block per warp per chunk");
 static_assert(DA_SMEM_BYTES >= (DA_WARPS + 1) * DA_ROWS * 128 * 4, "the staging area is reused for the partials");
 
-// D (+)= A * B, m16n8k16, fp16 inputs, fp32 accumulate. The short form leaves rows 8..15 of A zero.
-__device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  const uint32_t z = 0;
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(z), "r"(a2), "r"(z), "r"(b0), "r"(b1));
-}
+// D (+)= A * B, m16n8k16, fp16 inputs, fp32 accumulate.
 __device__ __forceinline__ void mma_f16_16816_full(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                    uint32_t b0, uint32_t b1) {
   asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-// (a & m) ^ c in one LOP3
-__device__ __forceinline__ uint32_t and_xor(uint32_t a, uint32_t m, uint32_t c) {
+// (a & M) ^ C in one LOP3; the constants are immediates of the instruction stream, so the compiler is
+// free to keep them wherever it likes instead of re-creating register copies next to every use
+template <uint32_t M, uint32_t C>
+__device__ __forceinline__ uint32_t and_xor(uint32_t a) {
   uint32_t d;
-  asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(a), "r"(m), "r"(c));  // (a & b) ^ c
+  asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(a), "n"(M), "n"(C));  // (a & b) ^ c
   return d;
 }
 __device__ __forceinline__ uint32_t hsub2_u32(uint32_t a, uint32_t b) {
@@ -280,11 +277,11 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
 
   // ---- query fragments (fp16 A operand of the score MMA, rows = query heads) ----------------------
   // A 32-bit word of a packed key row holds the codes of dims 8W..8W+7; nibble i of its low half is
-  // dim 8W+i, nibble i of its high half dim 8W+4+i. Register 2j of a lane holds (q[D], q[D+4]) and
-  // register 2j+1 holds (q[D+1], q[D+5]) / 16 with D = 32t + 8(j>>1) + 2(j&1): the k columns
+  // dim 8W+i, nibble i of its high half dim 8W+4+i. Fragment j of a lane holds (q[D], q[D+4]) in its first and
+  // (q[D+1], q[D+5]) / 16 in its third register with D = 32t + 8(j>>1) + 2(j&1): the k columns
   // 2t, 2t+1 and 2t+8, 2t+9 of score MMA j.
   const bool row_ok = g < G;
-  uint32_t qa[16];
+  uint32_t qa[8][4];  // whole A fragments (rows 8..15 zero) so that each MMA finds its operand tuple in place
   float q_even = 0.0f, q_odd = 0.0f;
   {
     const __nv_bfloat16* qrow = p.q + (static_cast<int64_t>(b) * p.Hq + h * G + (row_ok ? g : 0)) * 128;
@@ -301,8 +298,10 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
         const int i0 = 2 * jj;
         const __half2 a0 = __floats2half2_rn(f[i0], f[i0 + 4]);
         const __half2 a2 = __floats2half2_rn(f[i0 + 1] * 0.0625f, f[i0 + 5] * 0.0625f);
-        qa[2 * (2 * w + jj)] = *reinterpret_cast<const uint32_t*>(&a0);
-        qa[2 * (2 * w + jj) + 1] = *reinterpret_cast<const uint32_t*>(&a2);
+        qa[2 * w + jj][0] = *reinterpret_cast<const uint32_t*>(&a0);
+        qa[2 * w + jj][1] = 0u;
+        qa[2 * w + jj][2] = *reinterpret_cast<const uint32_t*>(&a2);
+        qa[2 * w + jj][3] = 0u;
         // the offsets are removed with the values the MMA really multiplies
         const float2 e0 = __half22float2(a0), e1 = __half22float2(a2);
         q_even += e0.x + e0.y;
@@ -354,10 +353,10 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
           const uint32_t hi8 = ww[w] >> 8;
-          mma_f16_16816(c, qa[4 * w], qa[4 * w + 1], and_xor(ww[w], 0x000F000Fu, 0x64086408u),
-                        and_xor(ww[w], 0x00F000F0u, 0x64806480u));
-          mma_f16_16816(c, qa[4 * w + 2], qa[4 * w + 3], and_xor(hi8, 0x000F000Fu, 0x64086408u),
-                        and_xor(hi8, 0x00F000F0u, 0x64806480u));
+          mma_f16_16816_full(c, qa[2 * w][0], qa[2 * w][1], qa[2 * w][2], qa[2 * w][3],
+                             and_xor<0x000F000Fu, 0x64086408u>(ww[w]), and_xor<0x00F000F0u, 0x64806480u>(ww[w]));
+          mma_f16_16816_full(c, qa[2 * w + 1][0], qa[2 * w + 1][1], qa[2 * w + 1][2], qa[2 * w + 1][3],
+                             and_xor<0x000F000Fu, 0x64086408u>(hi8), and_xor<0x00F000F0u, 0x64806480u>(hi8));
         }
         s[ti][0] = fmaf(c[0], scale2, -bias);
         s[ti][1] = fmaf(c[1], scale2, -bias);
@@ -370,9 +369,11 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
           if (key + 1 >= t1) s[ti][1] = -INFINITY;
         }
       }
-      // ---- online softmax; the running maximum moves only when a score of the block exceeds it ---
+      // ---- online softmax against a reference exponent m_run that moves only when a score exceeds it by
+      // more than DA_HEADROOM (probabilities then stay below 2^15, well inside fp16 and fp32 range; the
+      // reference is just a common exponent, the merges below rescale by it) -------------------------
       const float lm = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-      if (__any_sync(0xffffffffu, lm > m_run)) {
+      if (__any_sync(0xffffffffu, lm > m_run + DA_HEADROOM)) {
         float bm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, 1));
         bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
         const float m_new = fmaxf(m_run, bm);  // finite: key j0 of this block is valid for every row
@@ -401,14 +402,14 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
         const uint32_t ya = __byte_perm(q4 < 2 ? vc0.x : vc0.y, q4 < 2 ? vc1.x : vc1.y, sel);
         const uint32_t yb = __byte_perm(q4 < 2 ? vc2.x : vc2.y, q4 < 2 ? vc3.x : vc3.y, sel);
         const uint32_t ya8 = ya >> 8, yb8 = yb >> 8;
-        mma_f16_16816_full(o[2 * q4], hsub2_u32(and_xor(ya, 0x000F000Fu, 0x64086408u), 0x64086408u),
-                           hsub2_u32(and_xor(ya, 0x00F000F0u, 0x64806480u), 0x64806480u),
-                           hsub2_u32(and_xor(yb, 0x000F000Fu, 0x64086408u), 0x64086408u),
-                           hsub2_u32(and_xor(yb, 0x00F000F0u, 0x64806480u), 0x64806480u), pb0, pb1);
-        mma_f16_16816_full(o[2 * q4 + 1], hsub2_u32(and_xor(ya8, 0x000F000Fu, 0x64086408u), 0x64086408u),
-                           hsub2_u32(and_xor(ya8, 0x00F000F0u, 0x64806480u), 0x64806480u),
-                           hsub2_u32(and_xor(yb8, 0x000F000Fu, 0x64086408u), 0x64086408u),
-                           hsub2_u32(and_xor(yb8, 0x00F000F0u, 0x64806480u), 0x64806480u), pb0, pb1);
+        mma_f16_16816_full(o[2 * q4], hsub2_u32(and_xor<0x000F000Fu, 0x64086408u>(ya), 0x64086408u),
+                           hsub2_u32(and_xor<0x00F000F0u, 0x64806480u>(ya), 0x64806480u),
+                           hsub2_u32(and_xor<0x000F000Fu, 0x64086408u>(yb), 0x64086408u),
+                           hsub2_u32(and_xor<0x00F000F0u, 0x64806480u>(yb), 0x64806480u), pb0, pb1);
+        mma_f16_16816_full(o[2 * q4 + 1], hsub2_u32(and_xor<0x000F000Fu, 0x64086408u>(ya8), 0x64086408u),
+                           hsub2_u32(and_xor<0x00F000F0u, 0x64806480u>(ya8), 0x64806480u),
+                           hsub2_u32(and_xor<0x000F000Fu, 0x64086408u>(yb8), 0x64086408u),
+                           hsub2_u32(and_xor<0x00F000F0u, 0x64806480u>(yb8), 0x64806480u), pb0, pb1);
       }
     }
     if (r + 2 < n_rounds) {  // the half is free once every warp is past it
