@@ -225,6 +225,8 @@ __global__ void __launch_bounds__(N_THREADS, 1)
   float* scale_buf = reinterpret_cast<float*>(epi_buf + EPI_BYTES);
   Barriers* bars = reinterpret_cast<Barriers*>(reinterpret_cast<uint8_t*>(scale_buf) + SCALE_BYTES);
 
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // operands and output may belong to the previous kernel
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
@@ -568,13 +570,17 @@ pq_status pq_gemm_pair_ts_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* 
   cfg.blockDim = dim3(N_THREADS);
   cfg.dynamicSmemBytes = SMEM_BYTES;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // the kernel may be launched while its predecessor drains; it waits for it on the device before it
+  // reads or writes anything (griddepcontrol.wait at its top), which hides the launch itself
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   if (cudaLaunchKernelEx(&cfg, gemm_w4a4_pair_ts_kernel, ta, tb, to, p) != cudaSuccess) return PQ_ERR_CUDA;
   return pq_launch_status();
 }

@@ -31,6 +31,8 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
   constexpr int BLK_FLOATS = B + B / 64;       // padded block footprint in shared memory
   constexpr int RSTRIDE = 1 << (LOGB - 5);     // element distance between consecutive r
   extern __shared__ __align__(16) float sm[];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // input, scale and output may belong to the previous kernel
 
   const int tid = threadIdx.x;
   const int blk_local = tid / TPB;
@@ -188,8 +190,19 @@ pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_
   int64_t n_super = (n_rows * (K / B) + G - 1) / G;
   const int64_t resident = static_cast<int64_t>(HQ_CTAS_PER_SM) * ctx->sm_count;
   int64_t grid = n_super < resident ? n_super : resident;
-  kern<<<static_cast<int>(grid), HQ_THREADS, smem, st>>>(static_cast<const __nv_bfloat16*>(x), ldx, n_rows, K, s_a_in,
-                                                        xq, s_a_out);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(grid));
+  cfg.blockDim = dim3(HQ_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  // may be launched while the previous kernel drains; waits for it on the device before touching memory
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x), ldx, n_rows, K, s_a_in, xq, s_a_out) != cudaSuccess)
+    return PQ_ERR_CUDA;
   return pq_launch_status();
 }
 
