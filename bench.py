@@ -268,7 +268,7 @@ def run_gpu(args):
         except Exception as e:  # sections never take the main line down
             sections["error"] = repr(e)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu_baseline = oracle_sample(384)  # about 10-15 s of host work
+        cpu_baseline = oracle_sample(1536)  # about 10-15 s of host work on 16 cores
 
     if rank == 0:
         line = {
@@ -592,7 +592,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", default=None, help="run one kernel on a small case: gemm:M,N,K | hadamard:M,K,B | attn:B,Hq,Hkv,T,layers | prefill:T,Hq,Hkv")
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sections", action="store_true", help="skip the decode GEMM / decode attention sections")
