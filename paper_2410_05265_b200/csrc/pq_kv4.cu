@@ -117,6 +117,13 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   __half2 h = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&h);
 }
+// 8x8 transpose of 16-bit elements across the warp: lane (g, t) gives row g, columns 2t, 2t+1 and
+// receives row g, columns 2t, 2t+1 of the transposed matrix.
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -178,25 +185,30 @@ struct AttnParams {
   int B, Hq, Hkv, G, n_prefix, Tmax;
 };
 
-// Grid (splits, Hkv, B). A CTA owns a slice of one (sequence, KV head) cache. One thread copies the
-// slice into shared memory with bulk asynchronous copies, 64 keys per copy and two rounds of 128
-// keys ahead of the warps, so the HBM stream starts with the first instructions and never waits
-// for arithmetic. Each warp takes one 16-key block of every 64-key chunk:
-//   scores   S[head, key] with the fp16 MMA, query heads on the 16-row side. Codes become fp16 in
-//            place under an exponent (one LOP3 for two codes: nibbles 0 and 2 of a 16-bit half give
-//            1032 + code, nibbles 1 and 3 give 1152 + 16 * code with no shift); the factor 16 is
-//            folded into q and the offsets into a per-head constant.
-//   softmax  online, in log2 units; the running maximum moves only when a block exceeds it.
-//   output   O^T = V^T P^T with the fp16 MMA, head dims on the 16-row side (no padded rows), codes
-//            made exact fp16 integers; P is rounded to fp16 and the denominator sums the same
-//            rounded values.
+// Grid (splits, Hkv, B). The cache of one (sequence, KV head) is cut into rounds of 128 keys; split s
+// takes the rounds s, s + S, s + 2S, ... so that where its first rounds lie does not depend on the
+// sequence length: their bulk copies into shared memory start with the first instructions, before
+// len[b] has come back from memory (a round past the end is copied all the same when it lies inside
+// the cache allocation, and is then ignored). Two rounds are in flight ahead of the warps, 64 keys
+// per copy and barrier, issued by one lane of the warp that owns the barrier.
+// Each warp takes one 16-key block of every 64-key chunk:
+//   scores   S^T[key, head] with the fp16 MMA, keys on the 16-row side (every operand register is
+//            useful). Codes become fp16 in place under an exponent (one LOP3 for two codes: nibbles
+//            0 and 2 of a 16-bit half give 1032 + code, nibbles 1 and 3 give 1152 + 16 * code with
+//            no shift); the factor 16 is folded into q and the offsets into a per-head constant.
+//   softmax  in log2 units against a per-head reference exponent that moves only when a score
+//            exceeds it by more than DA_HEADROOM; the reference and the offset constant are one
+//            FFMA operand. P is rounded to fp16 and transposed to the operand layout of the next
+//            MMA by movmatrix.
+//   output   O^T = V^T P^T with the fp16 MMA, head dims on the 16-row side, codes made exact fp16
+//            integers; one more MMA with a matrix of ones sums the same rounded P into the
+//            denominator.
 // The CTA of the last split also scores the full-precision prefix keys and folds them into its partial.
-// The last CTA of a (sequence, head) to finish merges the partials and writes bf16.
 // CLUSTER: the splits of a (sequence, head) form one thread-block cluster and merge their partials
 // through distributed shared memory (no workspace, no ticket); otherwise the partials go through the
 // caller's workspace and the last CTA to finish merges them.
 template <bool CLUSTER>
-__global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnParams p) {
   extern __shared__ __align__(128) uint8_t da_stage[];  // two halves of [K rows | V rows] of one round
   // the per-warp partial outputs reuse the staging area once the key loop is over
   float (*sm_o)[DA_ROWS][128] = reinterpret_cast<float (*)[DA_ROWS][128]>(da_stage);
@@ -211,43 +223,74 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int G = p.G;
   const int bh = b * p.Hkv + h;
-  int len_b = p.len[b];
-  len_b = len_b < 0 ? 0 : (len_b > p.Tmax ? p.Tmax : len_b);
-  const int chunk = (((len_b + S - 1) / S) + 15) & ~15;
-  const int t0 = split * chunk;
-  const int t1 = min(len_b, t0 + chunk);
   const uint8_t* kbase = p.kq + static_cast<int64_t>(bh) * p.Tmax * 64;
   const uint8_t* vbase = p.vq + static_cast<int64_t>(bh) * p.Tmax * 64;
-
-  // ---- staging: thread 0 issues the copies of a round; chunk c of a half has its own barrier. The
-  // first two rounds start before anything else so that the set-up below runs under them.
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < 2 * DA_CHUNKS; ++i) pq::mbar_init(&full[0][0] + i, 1);
-    pq::mbar_fence_init();
-  }
-  __syncthreads();
   const uint32_t stage_addr = pq::smem_u32(da_stage);
-  const int n_rounds = t1 > t0 ? (t1 - t0 + DA_ROUND - 1) / DA_ROUND : 0;
-  auto issue_round = [&](int r) {
-    const uint32_t half = stage_addr + (r & 1) * DA_HALF_BYTES;
-    const int r0 = t0 + r * DA_ROUND;
-    for (int c = 0; c < DA_CHUNKS; ++c) {
-      const int k0 = r0 + c * DA_CHUNK;
-      if (k0 >= t1) break;
-      const uint32_t bytes = static_cast<uint32_t>(min(DA_CHUNK, t1 - k0)) * 64u;
-      uint64_t* bar = &full[r & 1][c];
-      pq::mbar_arrive_expect_tx(bar, 2 * bytes);
-      bulk_load(half + c * (DA_CHUNK * 64), kbase + static_cast<int64_t>(k0) * 64, bytes, bar);
-      bulk_load(half + DA_ROUND * 64 + c * (DA_CHUNK * 64), vbase + static_cast<int64_t>(k0) * 64, bytes, bar);
-    }
-  };
-  if (threadIdx.x == 0) {
-    if (n_rounds > 0) issue_round(0);
-    if (n_rounds > 1) issue_round(1);
-  }
-  // ---- the last split (its slice is the shortest) scores the full-precision prefix keys in fp32, in
-  // log2 units: eight lanes per (head, prefix key) pair, 16 dims each, every load issued at once
+
+  // ---- every small load of the set-up goes out before the first bulk copy: behind the copies of all
+  // the CTAs it would wait for megabytes of cache to be served first
+  const bool row_ok = g < G;
   const bool has_prefix = split == S - 1 && p.n_prefix > 0;
+  uint4 q_raw[4];  // 32 bf16 of query head g: dims 32t .. 32t+31
+  {
+    const uint4* q4 = reinterpret_cast<const uint4*>(p.q + (static_cast<int64_t>(b) * p.Hq + h * G + (row_ok ? g : 0)) * 128 + 32 * t);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) q_raw[w] = row_ok ? __ldg(q4 + w) : make_uint4(0, 0, 0, 0);
+  }
+  int len_b = __ldg(p.len + b);
+  const float s_k_h = __ldg(p.s_k + h);
+  // prefix values of this thread's head dim, so that the merge after the key loop does not wait for
+  // them (keys past the eighth are read there)
+  __half pv_early[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    pv_early[j] = (has_prefix && j < p.n_prefix) ? __ldg(p.prefix_v + (static_cast<int64_t>(h) * p.n_prefix + j) * 128 + threadIdx.x)
+                                                 : __float2half(0.0f);
+
+  // the operands of the first 16 (head, prefix key) pairs (all of them for a 4-token prefix under 4 heads)
+  uint4 pre_q[2] = {}, pre_k[2] = {};
+  if (has_prefix) {
+    const int pair = threadIdx.x >> 3, sub = threadIdx.x & 7;
+    const bool ok = pair < G * p.n_prefix;
+    const int r = ok ? pair / p.n_prefix : 0, j = ok ? pair % p.n_prefix : 0;
+    const uint4* qr = reinterpret_cast<const uint4*>(p.q + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + 16 * sub);
+    const uint4* kr = reinterpret_cast<const uint4*>(p.prefix_k + (static_cast<int64_t>(h) * p.n_prefix + j) * 128 + 16 * sub);
+    pre_q[0] = __ldg(qr), pre_q[1] = __ldg(qr + 1), pre_k[0] = __ldg(kr), pre_k[1] = __ldg(kr + 1);
+  }
+
+  // ---- staging. Warp w owns the barrier of chunk (w & 1) of half (w >> 1): its lane 0 initialises it
+  // and issues every copy that completes on it. Local round i of this split is the global round
+  // split + i * S; the rounds 0 and 1 are requested before the length is known when they lie inside
+  // the allocation as a whole.
+  static_assert(DA_WARPS == 2 * DA_CHUNKS, "one warp per (half, chunk) barrier");
+  const int my_half = warp >> 1, my_chunk = warp & 1;
+  auto round_key0 = [&](int i) { return (split + i * S) * DA_ROUND; };
+  auto speculated = [&](int i) { return round_key0(i) + DA_ROUND <= p.Tmax; };  // i = 0, 1 only
+  auto issue_chunk = [&](int i, int c, int n_keys) {  // lane 0 of the owning warp
+    const uint32_t half = stage_addr + (i & 1) * DA_HALF_BYTES;
+    const int k0 = round_key0(i) + c * DA_CHUNK;
+    const uint32_t bytes = static_cast<uint32_t>(n_keys) * 64u;
+    uint64_t* bar = &full[i & 1][c];
+    pq::mbar_arrive_expect_tx(bar, 2 * bytes);
+    bulk_load(half + c * (DA_CHUNK * 64), kbase + static_cast<int64_t>(k0) * 64, bytes, bar);
+    bulk_load(half + DA_ROUND * 64 + c * (DA_CHUNK * 64), vbase + static_cast<int64_t>(k0) * 64, bytes, bar);
+  };
+  if (lane == 0) {
+    pq::mbar_init(&full[my_half][my_chunk], 1);
+    pq::mbar_fence_init();
+    if (speculated(my_half)) issue_chunk(my_half, my_chunk, DA_CHUNK);
+  }
+  __syncthreads();  // every barrier is initialised (all warps are still together here: this costs nothing)
+  len_b = len_b < 0 ? 0 : (len_b > p.Tmax ? p.Tmax : len_b);
+  const int t1 = len_b;
+  const int n_rounds_all = (len_b + DA_ROUND - 1) / DA_ROUND;
+  const int n_rounds = n_rounds_all > split ? (n_rounds_all - split + S - 1) / S : 0;  // of this split
+  if (lane == 0 && !speculated(my_half) && my_half < n_rounds) {
+    const int k0 = round_key0(my_half) + my_chunk * DA_CHUNK;
+    if (k0 < t1) issue_chunk(my_half, my_chunk, min(DA_CHUNK, t1 - k0));
+  }
+  // ---- the last split (it never has more rounds than the others) scores the full-precision prefix keys in fp32, in
+  // log2 units: eight lanes per (head, prefix key) pair, 16 dims each, every load issued at once
   if (has_prefix) {
     const int n_pairs = G * p.n_prefix, sub = threadIdx.x & 7;
     for (int pair0 = 0; pair0 < n_pairs; pair0 += DA_THREADS / 8) {
@@ -256,7 +299,9 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
       const int r = ok ? pair / p.n_prefix : 0, j = ok ? pair % p.n_prefix : 0;
       const uint4* qr = reinterpret_cast<const uint4*>(p.q + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + 16 * sub);
       const uint4* kr = reinterpret_cast<const uint4*>(p.prefix_k + (static_cast<int64_t>(h) * p.n_prefix + j) * 128 + 16 * sub);
-      const uint4 qv[2] = {__ldg(qr), __ldg(qr + 1)}, kv[2] = {__ldg(kr), __ldg(kr + 1)};
+      const bool early = pair0 == 0;
+      const uint4 qv[2] = {early ? pre_q[0] : __ldg(qr), early ? pre_q[1] : __ldg(qr + 1)};
+      const uint4 kv[2] = {early ? pre_k[0] : __ldg(kr), early ? pre_k[1] : __ldg(kr + 1)};
       float acc = 0.0f;
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
@@ -275,20 +320,17 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
     }
   }
 
-  // ---- query fragments (fp16 A operand of the score MMA, rows = query heads) ----------------------
+  // ---- query fragments (fp16 B operand of the score MMA: k = head dims, n = query heads) ----------
   // A 32-bit word of a packed key row holds the codes of dims 8W..8W+7; nibble i of its low half is
   // dim 8W+i, nibble i of its high half dim 8W+4+i. Fragment j of a lane holds (q[D], q[D+4]) in its first and
-  // (q[D+1], q[D+5]) / 16 in its third register with D = 32t + 8(j>>1) + 2(j&1): the k columns
+  // (q[D+1], q[D+5]) / 16 in its second register with D = 32t + 8(j>>1) + 2(j&1), of head g: the k rows
   // 2t, 2t+1 and 2t+8, 2t+9 of score MMA j.
-  const bool row_ok = g < G;
-  uint32_t qa[8][4];  // whole A fragments (rows 8..15 zero) so that each MMA finds its operand tuple in place
+  uint32_t qb[8][2];
   float q_even = 0.0f, q_odd = 0.0f;
   {
-    const __nv_bfloat16* qrow = p.q + (static_cast<int64_t>(b) * p.Hq + h * G + (row_ok ? g : 0)) * 128;
-    const uint4* q4 = reinterpret_cast<const uint4*>(qrow + 32 * t);
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
-      const uint4 v = row_ok ? __ldg(q4 + w) : make_uint4(0, 0, 0, 0);  // 8 bf16: d = 32t + 8w + 0..7
+      const uint4 v = q_raw[w];  // 8 bf16: d = 32t + 8w + 0..7
       const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
       float f[8];
 #pragma unroll
@@ -298,10 +340,8 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
         const int i0 = 2 * jj;
         const __half2 a0 = __floats2half2_rn(f[i0], f[i0 + 4]);
         const __half2 a2 = __floats2half2_rn(f[i0 + 1] * 0.0625f, f[i0 + 5] * 0.0625f);
-        qa[2 * w + jj][0] = *reinterpret_cast<const uint32_t*>(&a0);
-        qa[2 * w + jj][1] = 0u;
-        qa[2 * w + jj][2] = *reinterpret_cast<const uint32_t*>(&a2);
-        qa[2 * w + jj][3] = 0u;
+        qb[2 * w + jj][0] = *reinterpret_cast<const uint32_t*>(&a0);
+        qb[2 * w + jj][1] = *reinterpret_cast<const uint32_t*>(&a2);
         // the offsets are removed with the values the MMA really multiplies
         const float2 e0 = __half22float2(a0), e1 = __half22float2(a2);
         q_even += e0.x + e0.y;
@@ -313,15 +353,22 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
     q_odd += __shfl_xor_sync(0xffffffffu, q_odd, 1);
     q_odd += __shfl_xor_sync(0xffffffffu, q_odd, 2);
   }
-  const float scale2 = __ldg(p.s_k + h) * p.sm_scale * 1.4426950408889634f;  // scores in log2 units
-  const float bias = (1032.0f * q_even + 1152.0f * q_odd) * scale2;
+  const float scale2 = s_k_h * p.sm_scale * 1.4426950408889634f;  // scores in log2 units
+  // The score tile of a lane is (keys g, g + 8) x (heads 2t, 2t + 1): it needs the offset constants of
+  // those two heads, which the lanes 8t and 8t + 4 hold.
+  const float bias_g = (1032.0f * q_even + 1152.0f * q_odd) * scale2;
+  const float bias0 = __shfl_sync(0xffffffffu, bias_g, 8 * t), bias1 = __shfl_sync(0xffffffffu, bias_g, 8 * t + 4);
+  // Reference exponents of heads 2t and 2t + 1 (the same in all lanes of equal t). A head that does not
+  // exist keeps a huge one: its probabilities are zero and it never asks for a move.
+  float m0 = 2 * t < G ? -INFINITY : 1e30f, m1 = 2 * t + 1 < G ? -INFINITY : 1e30f;
+  float bm0 = bias0 + m0, bm1 = bias1 + m1;  // what is subtracted from a raw score
 
   // Output accumulators of the transposed product: tile m holds, for this lane, o[m][0], o[m][1] =
   // dim 16g+2m of heads 2t, 2t+1 and o[m][2], o[m][3] = 16 x dim 16g+2m+1 of the same heads.
   float o[8][4];
 #pragma unroll
   for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f;
-  float m_run = -INFINITY, l_run = 0.0f;  // of head g; the four lanes of a head keep the same m_run
+  float lacc[4] = {0.0f, 0.0f, 0.0f, 0.0f};  // [0], [1]: denominators of heads 2t, 2t+1
 
   // byte offsets of this lane's loads inside a staged 16-key block
   const uint32_t k_off = g * 64 + 16 * t;             // key g (and g + 8): 32 codes at dims 32t..32t+31
@@ -329,70 +376,94 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
   bool timed_out = false;
   for (int r = 0; r < n_rounds && !timed_out; ++r) {
     const uint32_t ks = stage_addr + (r & 1) * DA_HALF_BYTES;
-    const int r0 = t0 + r * DA_ROUND;
-    for (int ch = 0; ch < DA_CHUNKS; ++ch) {
-      if (r0 + ch * DA_CHUNK >= t1) break;
-      if (!pq::mbar_wait(&full[r & 1][ch], (r >> 1) & 1)) {
-        timed_out = true;
-        break;
-      }
-      const int j0 = r0 + ch * DA_CHUNK + 16 * warp;  // this warp's 16-key block of the chunk
-      if (j0 >= t1) continue;
-      const uint32_t kb = ks + (j0 - r0) * 64, vb = kb + DA_ROUND * 64;
-      // Rows past the end of the slice were not copied; whatever the buffer holds there turns into
-      // finite fp16 values, and their probabilities are forced to zero below.
+    const int r0 = round_key0(r);
+    // A warp takes one 16-key block of each of the two chunks of a round, in one pass: two independent
+    // instruction streams to interleave. A block past the end of the sequence is computed all the
+    // same on whatever the buffer holds (any code pattern is a finite fp16 value) with all its
+    // probabilities forced to zero.
+    if (!pq::mbar_wait(&full[r & 1][0], (r >> 1) & 1) ||
+        (r0 + DA_CHUNK < t1 && !pq::mbar_wait(&full[r & 1][1], (r >> 1) & 1))) {
+      timed_out = true;
+      break;
+    }
+    float c[2][4];  // raw scores: [0], [1] = key g x heads 2t, 2t+1; [2], [3] = key g + 8 x the same heads
+    bool dead_lo[2], dead_hi[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int j0 = r0 + u * DA_CHUNK + 16 * warp;
+      const uint32_t kb = ks + (j0 - r0) * 64;
+      dead_lo[u] = j0 + g >= t1, dead_hi[u] = j0 + 8 + g >= t1;
       const uint4 kc0 = lds128(kb + k_off), kc1 = lds128(kb + k_off + 8 * 64);
+      // ---- scores of 16 keys x 8 heads: two accumulation chains over the eight 16-dim steps -------
+      float ca[4] = {0.0f, 0.0f, 0.0f, 0.0f}, cb[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      const uint32_t wl[4] = {kc0.x, kc0.y, kc0.z, kc0.w}, wh[4] = {kc1.x, kc1.y, kc1.z, kc1.w};
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const uint32_t wl8 = wl[w] >> 8, wh8 = wh[w] >> 8;
+        mma_f16_16816_full(ca, and_xor<0x000F000Fu, 0x64086408u>(wl[w]), and_xor<0x000F000Fu, 0x64086408u>(wh[w]),
+                           and_xor<0x00F000F0u, 0x64806480u>(wl[w]), and_xor<0x00F000F0u, 0x64806480u>(wh[w]),
+                           qb[2 * w][0], qb[2 * w][1]);
+        mma_f16_16816_full(cb, and_xor<0x000F000Fu, 0x64086408u>(wl8), and_xor<0x000F000Fu, 0x64086408u>(wh8),
+                           and_xor<0x00F000F0u, 0x64806480u>(wl8), and_xor<0x00F000F0u, 0x64806480u>(wh8),
+                           qb[2 * w + 1][0], qb[2 * w + 1][1]);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) c[u][i] = ca[i] + cb[i];
+    }
+    // ---- softmax against the reference exponents: e = log2 of the probability ----------------------
+    float e[2][4];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      e[u][0] = dead_lo[u] ? -INFINITY : fmaf(c[u][0], scale2, -bm0);
+      e[u][1] = dead_lo[u] ? -INFINITY : fmaf(c[u][1], scale2, -bm1);
+      e[u][2] = dead_hi[u] ? -INFINITY : fmaf(c[u][2], scale2, -bm0);
+      e[u][3] = dead_hi[u] ? -INFINITY : fmaf(c[u][3], scale2, -bm1);
+    }
+    // A reference moves only when a score exceeds it by more than DA_HEADROOM (probabilities then stay
+    // below 2^15, well inside fp16 and fp32 range; the reference is just a common exponent, the
+    // merges below rescale by it). The first pass of a warp always takes this path (e = +inf).
+    const float e_max = fmaxf(fmaxf(fmaxf(e[0][0], e[0][1]), fmaxf(e[0][2], e[0][3])), fmaxf(fmaxf(e[1][0], e[1][1]), fmaxf(e[1][2], e[1][3])));
+    if (__any_sync(0xffffffffu, e_max > DA_HEADROOM)) {
+      float s[2][4];
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        s[u][0] = dead_lo[u] ? -INFINITY : fmaf(c[u][0], scale2, -bias0);
+        s[u][1] = dead_lo[u] ? -INFINITY : fmaf(c[u][1], scale2, -bias1);
+        s[u][2] = dead_hi[u] ? -INFINITY : fmaf(c[u][2], scale2, -bias0);
+        s[u][3] = dead_hi[u] ? -INFINITY : fmaf(c[u][3], scale2, -bias1);
+      }
+      // maxima of heads 2t, 2t+1 over the 32 keys of this pass: over the eight lanes of equal t
+      float x0 = fmaxf(fmaxf(s[0][0], s[0][2]), fmaxf(s[1][0], s[1][2])), x1 = fmaxf(fmaxf(s[0][1], s[0][3]), fmaxf(s[1][1], s[1][3]));
+#pragma unroll
+      for (int d = 4; d < 32; d <<= 1) {
+        x0 = fmaxf(x0, __shfl_xor_sync(0xffffffffu, x0, d));
+        x1 = fmaxf(x1, __shfl_xor_sync(0xffffffffu, x1, d));
+      }
+      // a warp whose 32 keys all lie past the end keeps its reference (-inf - -inf would not be a number)
+      const float n0 = fmaxf(m0, x0), n1 = fmaxf(m1, x1);
+      const float a_lo = n0 == -INFINITY ? 1.0f : ex2(m0 - n0), a_hi = n1 == -INFINITY ? 1.0f : ex2(m1 - n1);
+      m0 = n0, m1 = n1;
+      bm0 = bias0 + m0, bm1 = bias1 + m1;
+      lacc[0] *= a_lo, lacc[1] *= a_hi, lacc[2] *= a_lo, lacc[3] *= a_hi;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) o[i][0] *= a_lo, o[i][1] *= a_hi, o[i][2] *= a_lo, o[i][3] *= a_hi;
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        e[u][0] = n0 == -INFINITY ? -INFINITY : s[u][0] - m0, e[u][1] = n1 == -INFINITY ? -INFINITY : s[u][1] - m1;
+        e[u][2] = n0 == -INFINITY ? -INFINITY : s[u][2] - m0, e[u][3] = n1 == -INFINITY ? -INFINITY : s[u][3] - m1;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int j0 = r0 + u * DA_CHUNK + 16 * warp;
+      const uint32_t vb = ks + (j0 - r0) * 64 + DA_ROUND * 64;
       const uint2 vc0 = lds64(vb + v_off), vc1 = lds64(vb + v_off + 64);
       const uint2 vc2 = lds64(vb + v_off + 8 * 64), vc3 = lds64(vb + v_off + 9 * 64);
-      // ---- scores of 16 keys: S[head, key] for two tiles of 8 keys -----------------------------
-      float s[2][2];
-#pragma unroll
-      for (int ti = 0; ti < 2; ++ti) {
-        const uint32_t ww[4] = {ti ? kc1.x : kc0.x, ti ? kc1.y : kc0.y, ti ? kc1.z : kc0.z, ti ? kc1.w : kc0.w};
-        float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          const uint32_t hi8 = ww[w] >> 8;
-          mma_f16_16816_full(c, qa[2 * w][0], qa[2 * w][1], qa[2 * w][2], qa[2 * w][3],
-                             and_xor<0x000F000Fu, 0x64086408u>(ww[w]), and_xor<0x00F000F0u, 0x64806480u>(ww[w]));
-          mma_f16_16816_full(c, qa[2 * w + 1][0], qa[2 * w + 1][1], qa[2 * w + 1][2], qa[2 * w + 1][3],
-                             and_xor<0x000F000Fu, 0x64086408u>(hi8), and_xor<0x00F000F0u, 0x64806480u>(hi8));
-        }
-        s[ti][0] = fmaf(c[0], scale2, -bias);
-        s[ti][1] = fmaf(c[1], scale2, -bias);
-      }
-      if (j0 + 16 > t1) {  // ragged last block
-#pragma unroll
-        for (int ti = 0; ti < 2; ++ti) {
-          const int key = j0 + 8 * ti + 2 * t;
-          if (key >= t1) s[ti][0] = -INFINITY;
-          if (key + 1 >= t1) s[ti][1] = -INFINITY;
-        }
-      }
-      // ---- online softmax against a reference exponent m_run that moves only when a score exceeds it by
-      // more than DA_HEADROOM (probabilities then stay below 2^15, well inside fp16 and fp32 range; the
-      // reference is just a common exponent, the merges below rescale by it) -------------------------
-      const float lm = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-      if (__any_sync(0xffffffffu, lm > m_run + DA_HEADROOM)) {
-        float bm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, 1));
-        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
-        const float m_new = fmaxf(m_run, bm);  // finite: key j0 of this block is valid for every row
-        const float alpha = ex2(m_run - m_new);
-        m_run = m_new;
-        l_run *= alpha;
-        // this lane's accumulators belong to heads 2t and 2t+1, whose factors live in lanes 8t and 8t+4
-        const float a_lo = __shfl_sync(0xffffffffu, alpha, 8 * t), a_hi = __shfl_sync(0xffffffffu, alpha, 8 * t + 4);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) o[i][0] *= a_lo, o[i][1] *= a_hi, o[i][2] *= a_lo, o[i][3] *= a_hi;
-      }
-      const uint32_t pb0 = pack_half2(ex2(s[0][0] - m_run), ex2(s[0][1] - m_run));
-      const uint32_t pb1 = pack_half2(ex2(s[1][0] - m_run), ex2(s[1][1] - m_run));
-      {
-        // the denominator sums the same fp16-rounded probabilities the MMA multiplies with
-        const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&pb0));
-        const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&pb1));
-        l_run += (f0.x + f0.y) + (f1.x + f1.y);
-      }
+      // P in fp16, transposed from (key, head pair) to the (key pair, head) layout of an MMA B operand
+      const uint32_t pb0 = movmatrix_trans(pack_half2(ex2(e[u][0]), ex2(e[u][1])));
+      const uint32_t pb1 = movmatrix_trans(pack_half2(ex2(e[u][2]), ex2(e[u][3])));
+      // the denominator sums the same fp16-rounded probabilities the output MMA multiplies with
+      mma_f16_16816_full(lacc, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, pb0, pb1);
       // ---- O^T += V^T P^T: rows = head dims, columns = query heads ------------------------------
       // A merged word pairs the same four dims of two neighbouring keys; its nibbles 0 and 2 give
       // exact codes, nibbles 1 and 3 give 16 * code (rows g+8 of the tile, rescaled at the end).
@@ -414,13 +485,22 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
     }
     if (r + 2 < n_rounds) {  // the half is free once every warp is past it
       __syncthreads();
-      if (threadIdx.x == 0) issue_round(r + 2);
+      if (lane == 0 && my_half == (r & 1)) {
+        const int k0 = round_key0(r + 2) + my_chunk * DA_CHUNK;
+        if (k0 < t1) issue_chunk(r + 2, my_chunk, min(DA_CHUNK, t1 - k0));
+      }
     }
   }
+  // a round requested ahead of the length and then not needed must still have landed before the
+  // staging area is reused
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+    for (int c = 0; c < DA_CHUNKS; ++c)
+      if (speculated(i) && !timed_out && (i >= n_rounds || round_key0(i) + c * DA_CHUNK >= t1) &&
+          !pq::mbar_wait(&full[i][c], 0))
+        timed_out = true;
   if (timed_out && lane == 0 && p.status) pq::report(p.status, PQ_ERR_TIMEOUT);
   __syncthreads();  // the staging area becomes the per-warp partial outputs
-  l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-  l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
 
   // ---- merge the warps of this CTA (and, in the last split, the prefix keys) into one partial ------------
 #pragma unroll
@@ -432,7 +512,10 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
         *reinterpret_cast<float2*>(&sm_o[warp][head][16 * g + 2 * m]) = make_float2(o[m][hh], o[m][2 + hh] * 0.0625f);
     }
   }
-  if (row_ok && t == 0) sm_ml[warp][g][0] = m_run, sm_ml[warp][g][1] = l_run;
+  if (g == 0) {
+    if (2 * t < G) sm_ml[warp][2 * t][0] = m0, sm_ml[warp][2 * t][1] = lacc[0];
+    if (2 * t + 1 < G) sm_ml[warp][2 * t + 1][0] = m1, sm_ml[warp][2 * t + 1][1] = lacc[1];
+  }
   __syncthreads();
   {
     const int d = threadIdx.x;  // 128 threads <-> 128 head-dim elements
@@ -452,7 +535,15 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attn_kernel(const AttnParam
         l += sm_ml[w][r][1] * e;
       }
       acc *= sv;  // codes -> values; the prefix values below are already in value units
-      for (int j = 0; j < n_pre; ++j) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (j < n_pre) {
+          const float e = ex2(sm_pre[r][j] - m);
+          acc = fmaf(e, __half2float(pv_early[j]), acc);
+          l += e;
+        }
+      }
+      for (int j = 8; j < n_pre; ++j) {
         const float e = ex2(sm_pre[r][j] - m);
         acc = fmaf(e, __half2float(p.prefix_v[(static_cast<int64_t>(h) * p.n_prefix + j) * 128 + d]), acc);
         l += e;
