@@ -113,7 +113,7 @@ pq_status pq_w4a4_gemm(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const 
  *   kq, vq              u8 [B, Hkv, Tmax, D/2]   packed codes of the ordinary tokens
  *   s_k, s_v            f32 [Hkv]                static per-head steps
  *   len                 int32 [B] on the device  number of 4-bit entries of each sequence
- * D must be 128; Hq a multiple of Hkv with Hq / Hkv <= 8; kq, vq and prefix_k 16-byte aligned. */
+ * D must be 128; Hq a multiple of Hkv with Hq / Hkv <= 8; kq, vq, prefix_k and prefix_v 16-byte aligned. */
 typedef struct pq_kv4_cache {
   const void* prefix_k;
   const void* prefix_v;

@@ -91,7 +91,8 @@ constexpr int DA_CHUNKS = DA_ROUND / DA_CHUNK;
 constexpr int DA_HALF_BYTES = DA_ROUND * 64 * 2;  // packed K rows, then packed V rows
 constexpr int DA_SMEM_BYTES = 2 * DA_HALF_BYTES;  // 32 KB
 static_assert(DA_CHUNK == 16 * DA_WARPS, "one 16-key block per warp per chunk");
-static_assert(DA_SMEM_BYTES >= (DA_WARPS + 1) * DA_ROWS * 128 * 4, "the staging area is reused for the partials");
+constexpr int DA_SO_STRIDE = 136;                 // floats per (warp, head) row of the per-warp partial outputs
+static_assert(DA_SMEM_BYTES >= (DA_WARPS * DA_SO_STRIDE + 128) * DA_ROWS * 4, "the staging area is reused for the partials");
 
 // D (+)= A * B, m16n8k16, fp16 inputs, fp32 accumulate.
 __device__ __forceinline__ void mma_f16_16816_full(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -211,8 +212,10 @@ template <bool CLUSTER>
 __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnParams p) {
   extern __shared__ __align__(128) uint8_t da_stage[];  // two halves of [K rows | V rows] of one round
   // the per-warp partial outputs reuse the staging area once the key loop is over
-  float (*sm_o)[DA_ROWS][128] = reinterpret_cast<float (*)[DA_ROWS][128]>(da_stage);
-  float* cl_o = reinterpret_cast<float*>(da_stage + DA_WARPS * DA_ROWS * 128 * 4);  // [G][128]: this CTA's partial (cluster mode)
+  // [warp][head][DA_SO_STRIDE]; head dim d = 16a + 2b + c sits at 16b + 2a + c and the rows are padded so
+  // that the 32 lanes of a store cover all banks (a lane holds dims 16g + 2m, +1 of the heads 2t, 2t+1)
+  float* sm_o = reinterpret_cast<float*>(da_stage);
+  float* cl_o = reinterpret_cast<float*>(da_stage + DA_WARPS * DA_ROWS * DA_SO_STRIDE * 4);  // [G][128]: this CTA's partial (cluster mode)
   __shared__ float2 cl_ml[DA_ROWS];
   __shared__ __align__(8) uint64_t full[2][DA_CHUNKS];
   __shared__ float sm_ml[DA_WARPS][DA_ROWS][2];
@@ -238,14 +241,15 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
     for (int w = 0; w < 4; ++w) q_raw[w] = row_ok ? __ldg(q4 + w) : make_uint4(0, 0, 0, 0);
   }
   int len_b = __ldg(p.len + b);
-  const float s_k_h = __ldg(p.s_k + h);
-  // prefix values of this thread's head dim, so that the merge after the key loop does not wait for
-  // them (keys past the eighth are read there)
-  __half pv_early[8];
+  const float s_k_h = __ldg(p.s_k + h), s_v_h = __ldg(p.s_v + h);
+  // prefix values of the four head dims this thread merges after the key loop, so that the merge does
+  // not wait for them (keys past the fourth are read there)
+  uint2 pv_early[4];
 #pragma unroll
-  for (int j = 0; j < 8; ++j)
-    pv_early[j] = (has_prefix && j < p.n_prefix) ? __ldg(p.prefix_v + (static_cast<int64_t>(h) * p.n_prefix + j) * 128 + threadIdx.x)
-                                                 : __float2half(0.0f);
+  for (int j = 0; j < 4; ++j)
+    pv_early[j] = (has_prefix && j < p.n_prefix)
+                      ? __ldg(reinterpret_cast<const uint2*>(p.prefix_v + (static_cast<int64_t>(h) * p.n_prefix + j) * 128) + lane)
+                      : make_uint2(0u, 0u);
 
   // the operands of the first 16 (head, prefix key) pairs (all of them for a 4-token prefix under 4 heads)
   uint4 pre_q[2] = {}, pre_k[2] = {};
@@ -509,7 +513,8 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
     if (head < G) {
 #pragma unroll
       for (int m = 0; m < 8; ++m)
-        *reinterpret_cast<float2*>(&sm_o[warp][head][16 * g + 2 * m]) = make_float2(o[m][hh], o[m][2 + hh] * 0.0625f);
+        *reinterpret_cast<float2*>(sm_o + (warp * DA_ROWS + head) * DA_SO_STRIDE + 16 * m + 2 * g) =
+            make_float2(o[m][hh], o[m][2 + hh] * 0.0625f);
     }
   }
   if (g == 0) {
@@ -518,43 +523,47 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   }
   __syncthreads();
   {
-    const int d = threadIdx.x;  // 128 threads <-> 128 head-dim elements
-    const float sv = __ldg(p.s_v + h);
+    // warp w takes the heads w, w + 4; lane c4 of it the head dims 4 c4 .. 4 c4 + 3
     const int n_pre = has_prefix ? p.n_prefix : 0;
-    for (int r = 0; r < G; ++r) {
+    const int c4 = lane;
+    const int qpos = 16 * ((2 * c4) & 7) + 2 * (c4 >> 2);  // dims 4 c4, +1 here, dims 4 c4 + 2, +3 sixteen floats on
+    for (int r = warp; r < G; r += DA_WARPS) {
       float m = -INFINITY;
 #pragma unroll
       for (int w = 0; w < DA_WARPS; ++w) m = fmaxf(m, sm_ml[w][r][0]);
       for (int j = 0; j < n_pre; ++j) m = fmaxf(m, sm_pre[r][j]);
-      float acc = 0.0f, l = 0.0f;
+      float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+      float l = 0.0f;
 #pragma unroll
       for (int w = 0; w < DA_WARPS; ++w) {
         const float mw = sm_ml[w][r][0];
         const float e = mw == -INFINITY ? 0.0f : ex2(mw - m);
-        acc += sm_o[w][r][d] * e;
-        l += sm_ml[w][r][1] * e;
+        const float* src = sm_o + (w * DA_ROWS + r) * DA_SO_STRIDE + qpos;
+        const float2 lo = *reinterpret_cast<const float2*>(src), hi = *reinterpret_cast<const float2*>(src + 16);
+        acc.x = fmaf(lo.x, e, acc.x), acc.y = fmaf(lo.y, e, acc.y), acc.z = fmaf(hi.x, e, acc.z), acc.w = fmaf(hi.y, e, acc.w);
+        l = fmaf(sm_ml[w][r][1], e, l);
       }
-      acc *= sv;  // codes -> values; the prefix values below are already in value units
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if (j < n_pre) {
-          const float e = ex2(sm_pre[r][j] - m);
-          acc = fmaf(e, __half2float(pv_early[j]), acc);
-          l += e;
-        }
-      }
-      for (int j = 8; j < n_pre; ++j) {
+      // codes -> values; the prefix values below are already in value units
+      acc.x *= s_v_h, acc.y *= s_v_h, acc.z *= s_v_h, acc.w *= s_v_h;
+      for (int j = 0; j < n_pre; ++j) {
         const float e = ex2(sm_pre[r][j] - m);
-        acc = fmaf(e, __half2float(p.prefix_v[(static_cast<int64_t>(h) * p.n_prefix + j) * 128 + d]), acc);
+        uint2 pv = make_uint2(0u, 0u);
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj)
+          if (j == jj) pv = pv_early[jj];
+        if (j >= 4) pv = __ldg(reinterpret_cast<const uint2*>(p.prefix_v + (static_cast<int64_t>(h) * p.n_prefix + j) * 128) + c4);
+        const float2 v01 = __half22float2(*reinterpret_cast<const __half2*>(&pv.x));
+        const float2 v23 = __half22float2(*reinterpret_cast<const __half2*>(&pv.y));
+        acc.x = fmaf(e, v01.x, acc.x), acc.y = fmaf(e, v01.y, acc.y), acc.z = fmaf(e, v23.x, acc.z), acc.w = fmaf(e, v23.y, acc.w);
         l += e;
       }
       if (CLUSTER) {
-        cl_o[r * 128 + d] = acc;
-        if (d == 0) cl_ml[r] = make_float2(m, l);
+        *reinterpret_cast<float4*>(cl_o + r * 128 + 4 * c4) = acc;
+        if (c4 == 0) cl_ml[r] = make_float2(m, l);
       } else {
         const int64_t slot = (static_cast<int64_t>(bh) * S + split) * G + r;
-        p.ws_o[slot * 128 + d] = acc;
-        if (d == 0) *reinterpret_cast<float2*>(p.ws_ml + slot * 2) = make_float2(m, l);
+        *reinterpret_cast<float4*>(p.ws_o + slot * 128 + 4 * c4) = acc;
+        if (c4 == 0) *reinterpret_cast<float2*>(p.ws_ml + slot * 2) = make_float2(m, l);
       }
     }
   }
@@ -697,7 +706,8 @@ pq_status check_cache(const pq_kv4_cache* c) {
   if (c->D != 128 || c->Hq % c->Hkv != 0 || c->Hq / c->Hkv > DA_ROWS || c->n_prefix > DA_MAX_PREFIX)
     return PQ_ERR_SHAPE;
   if ((reinterpret_cast<uintptr_t>(c->kq) & 15) || (reinterpret_cast<uintptr_t>(c->vq) & 15)) return PQ_ERR_ALIGN;
-  if (c->n_prefix > 0 && (reinterpret_cast<uintptr_t>(c->prefix_k) & 15)) return PQ_ERR_ALIGN;
+  if (c->n_prefix > 0 && ((reinterpret_cast<uintptr_t>(c->prefix_k) & 15) || (reinterpret_cast<uintptr_t>(c->prefix_v) & 15)))
+    return PQ_ERR_ALIGN;
   return PQ_OK;
 }
 
