@@ -88,8 +88,10 @@ constexpr float DA_HEADROOM = 15.0f;  // log2 units a score may exceed the refer
 constexpr int DA_ROUND = 128;                     // keys staged per round (one half of the staging buffer)
 constexpr int DA_CHUNK = 64;                      // keys per bulk copy and per barrier
 constexpr int DA_CHUNKS = DA_ROUND / DA_CHUNK;
-constexpr int DA_HALF_BYTES = DA_ROUND * 64 * 2;  // packed K rows, then packed V rows
-constexpr int DA_SMEM_BYTES = 2 * DA_HALF_BYTES;  // 32 KB
+constexpr int DA_SLOTS = 2;                       // rounds of staging per CTA
+constexpr int DA_EARLY = 1;                       // rounds requested at kernel entry
+constexpr int DA_HALF_BYTES = DA_ROUND * 64 * 2;  // one slot: packed K rows, then packed V rows
+constexpr int DA_SMEM_BYTES = DA_SLOTS * DA_HALF_BYTES;  // 32 KB
 static_assert(DA_CHUNK == 16 * DA_WARPS, "one 16-key block per warp per chunk");
 constexpr int DA_SO_STRIDE = 136;                 // floats per (warp, head) row of the per-warp partial outputs
 static_assert(DA_SMEM_BYTES >= (DA_WARPS * DA_SO_STRIDE + 128) * DA_ROWS * 4, "the staging area is reused for the partials");
@@ -190,7 +192,7 @@ struct AttnParams {
 // takes the rounds s, s + S, s + 2S, ... so that where its first rounds lie does not depend on the
 // sequence length: their bulk copies into shared memory start with the first instructions, before
 // len[b] has come back from memory (a round past the end is copied all the same when it lies inside
-// the cache allocation, and is then ignored). Two rounds are in flight ahead of the warps, 64 keys
+// the cache allocation, and is then ignored). Three rounds are in flight ahead of the warps, 64 keys
 // per copy and barrier, issued by one lane of the warp that owns the barrier.
 // Each warp takes one 16-key block of every 64-key chunk:
 //   scores   S^T[key, head] with the fp16 MMA, keys on the 16-row side (every operand register is
@@ -210,14 +212,14 @@ struct AttnParams {
 // caller's workspace and the last CTA to finish merges them.
 template <bool CLUSTER>
 __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnParams p) {
-  extern __shared__ __align__(128) uint8_t da_stage[];  // two halves of [K rows | V rows] of one round
+  extern __shared__ __align__(128) uint8_t da_stage[];  // DA_SLOTS slots of [K rows | V rows] of one round
   // the per-warp partial outputs reuse the staging area once the key loop is over
   // [warp][head][DA_SO_STRIDE]; head dim d = 16a + 2b + c sits at 16b + 2a + c and the rows are padded so
   // that the 32 lanes of a store cover all banks (a lane holds dims 16g + 2m, +1 of the heads 2t, 2t+1)
   float* sm_o = reinterpret_cast<float*>(da_stage);
   float* cl_o = reinterpret_cast<float*>(da_stage + DA_WARPS * DA_ROWS * DA_SO_STRIDE * 4);  // [G][128]: this CTA's partial (cluster mode)
   __shared__ float2 cl_ml[DA_ROWS];
-  __shared__ __align__(8) uint64_t full[2][DA_CHUNKS];
+  __shared__ __align__(8) uint64_t full[DA_SLOTS][DA_CHUNKS];
   __shared__ float sm_ml[DA_WARPS][DA_ROWS][2];
   __shared__ float sm_pre[DA_ROWS][DA_MAX_PREFIX];
   __shared__ int is_last;
@@ -262,36 +264,37 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
     pre_q[0] = __ldg(qr), pre_q[1] = __ldg(qr + 1), pre_k[0] = __ldg(kr), pre_k[1] = __ldg(kr + 1);
   }
 
-  // ---- staging. Warp w owns the barrier of chunk (w & 1) of half (w >> 1): its lane 0 initialises it
-  // and issues every copy that completes on it. Local round i of this split is the global round
-  // split + i * S; the rounds 0 and 1 are requested before the length is known when they lie inside
-  // the allocation as a whole.
-  static_assert(DA_WARPS == 2 * DA_CHUNKS, "one warp per (half, chunk) barrier");
-  const int my_half = warp >> 1, my_chunk = warp & 1;
+  // ---- staging. Barrier n = 2 * slot + chunk belongs to warp n % 4: its lane 0 initialises it and
+  // issues every copy that completes on it. Local round i of this split is the global round
+  // split + i * S and uses slot i % DA_SLOTS; the first DA_EARLY rounds are requested before the length
+  // is known when they lie inside the allocation as a whole.
   auto round_key0 = [&](int i) { return (split + i * S) * DA_ROUND; };
-  auto speculated = [&](int i) { return round_key0(i) + DA_ROUND <= p.Tmax; };  // i = 0, 1 only
+  auto speculated = [&](int i) { return round_key0(i) + DA_ROUND <= p.Tmax; };  // i < DA_EARLY only
   auto issue_chunk = [&](int i, int c, int n_keys) {  // lane 0 of the owning warp
-    const uint32_t half = stage_addr + (i & 1) * DA_HALF_BYTES;
+    const uint32_t slot = stage_addr + (i % DA_SLOTS) * DA_HALF_BYTES;
     const int k0 = round_key0(i) + c * DA_CHUNK;
     const uint32_t bytes = static_cast<uint32_t>(n_keys) * 64u;
-    uint64_t* bar = &full[i & 1][c];
+    uint64_t* bar = &full[i % DA_SLOTS][c];
     pq::mbar_arrive_expect_tx(bar, 2 * bytes);
-    bulk_load(half + c * (DA_CHUNK * 64), kbase + static_cast<int64_t>(k0) * 64, bytes, bar);
-    bulk_load(half + DA_ROUND * 64 + c * (DA_CHUNK * 64), vbase + static_cast<int64_t>(k0) * 64, bytes, bar);
+    bulk_load(slot + c * (DA_CHUNK * 64), kbase + static_cast<int64_t>(k0) * 64, bytes, bar);
+    bulk_load(slot + DA_ROUND * 64 + c * (DA_CHUNK * 64), vbase + static_cast<int64_t>(k0) * 64, bytes, bar);
   };
   if (lane == 0) {
-    pq::mbar_init(&full[my_half][my_chunk], 1);
+    for (int n = warp; n < DA_SLOTS * DA_CHUNKS; n += DA_WARPS) pq::mbar_init(&full[0][0] + n, 1);
     pq::mbar_fence_init();
-    if (speculated(my_half)) issue_chunk(my_half, my_chunk, DA_CHUNK);
+    for (int n = warp; n < DA_EARLY * DA_CHUNKS; n += DA_WARPS)
+      if (speculated(n / DA_CHUNKS)) issue_chunk(n / DA_CHUNKS, n % DA_CHUNKS, DA_CHUNK);
   }
   __syncthreads();  // every barrier is initialised (all warps are still together here: this costs nothing)
   len_b = len_b < 0 ? 0 : (len_b > p.Tmax ? p.Tmax : len_b);
   const int t1 = len_b;
   const int n_rounds_all = (len_b + DA_ROUND - 1) / DA_ROUND;
   const int n_rounds = n_rounds_all > split ? (n_rounds_all - split + S - 1) / S : 0;  // of this split
-  if (lane == 0 && !speculated(my_half) && my_half < n_rounds) {
-    const int k0 = round_key0(my_half) + my_chunk * DA_CHUNK;
-    if (k0 < t1) issue_chunk(my_half, my_chunk, min(DA_CHUNK, t1 - k0));
+  if (lane == 0) {
+    for (int n = warp; n < DA_EARLY * DA_CHUNKS; n += DA_WARPS) {
+      const int i = n / DA_CHUNKS, k0 = round_key0(i) + (n % DA_CHUNKS) * DA_CHUNK;
+      if (!speculated(i) && i < n_rounds && k0 < t1) issue_chunk(i, n % DA_CHUNKS, min(DA_CHUNK, t1 - k0));
+    }
   }
   // ---- the last split (it never has more rounds than the others) scores the full-precision prefix keys in fp32, in
   // log2 units: eight lanes per (head, prefix key) pair, 16 dims each, every load issued at once
@@ -379,16 +382,22 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   const uint32_t v_off = (2 * t) * 64 + 8 * g;        // keys 2t, 2t+1, 2t+8, 2t+9: 16 codes at dims 16g..16g+15
   bool timed_out = false;
   for (int r = 0; r < n_rounds && !timed_out; ++r) {
-    const uint32_t ks = stage_addr + (r & 1) * DA_HALF_BYTES;
+    const uint32_t ks = stage_addr + (r % DA_SLOTS) * DA_HALF_BYTES;
     const int r0 = round_key0(r);
+    const uint32_t parity = (r / DA_SLOTS) & 1;
     // A warp takes one 16-key block of each of the two chunks of a round, in one pass: two independent
     // instruction streams to interleave. A block past the end of the sequence is computed all the
     // same on whatever the buffer holds (any code pattern is a finite fp16 value) with all its
     // probabilities forced to zero.
-    if (!pq::mbar_wait(&full[r & 1][0], (r >> 1) & 1) ||
-        (r0 + DA_CHUNK < t1 && !pq::mbar_wait(&full[r & 1][1], (r >> 1) & 1))) {
+    if (!pq::mbar_wait(&full[r % DA_SLOTS][0], parity) || (r0 + DA_CHUNK < t1 && !pq::mbar_wait(&full[r % DA_SLOTS][1], parity))) {
       timed_out = true;
       break;
+    }
+    if (r == 0 && lane == 0) {  // the remaining slots are requested once the first data is here
+      for (int n = DA_EARLY * DA_CHUNKS + warp; n < DA_SLOTS * DA_CHUNKS; n += DA_WARPS) {
+        const int i = n / DA_CHUNKS, k0 = round_key0(i) + (n % DA_CHUNKS) * DA_CHUNK;
+        if (i < n_rounds && k0 < t1) issue_chunk(i, n % DA_CHUNKS, min(DA_CHUNK, t1 - k0));
+      }
     }
     float c[2][4];  // raw scores: [0], [1] = key g x heads 2t, 2t+1; [2], [3] = key g + 8 x the same heads
     bool dead_lo[2], dead_hi[2];
@@ -487,18 +496,19 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
                            hsub2_u32(and_xor<0x00F000F0u, 0x64806480u>(yb8), 0x64806480u), pb0, pb1);
       }
     }
-    if (r + 2 < n_rounds) {  // the half is free once every warp is past it
+    if (r + DA_SLOTS < n_rounds) {  // the slot is free once every warp is past it
       __syncthreads();
-      if (lane == 0 && my_half == (r & 1)) {
-        const int k0 = round_key0(r + 2) + my_chunk * DA_CHUNK;
-        if (k0 < t1) issue_chunk(r + 2, my_chunk, min(DA_CHUNK, t1 - k0));
+      for (int c = 0; c < DA_CHUNKS; ++c) {
+        const int k0 = round_key0(r + DA_SLOTS) + c * DA_CHUNK;
+        if (lane == 0 && warp == ((r % DA_SLOTS) * DA_CHUNKS + c) % DA_WARPS && k0 < t1)
+          issue_chunk(r + DA_SLOTS, c, min(DA_CHUNK, t1 - k0));
       }
     }
   }
   // a round requested ahead of the length and then not needed must still have landed before the
   // staging area is reused
 #pragma unroll
-  for (int i = 0; i < 2; ++i)
+  for (int i = 0; i < DA_EARLY; ++i)
     for (int c = 0; c < DA_CHUNKS; ++c)
       if (speculated(i) && !timed_out && (i >= n_rounds || round_key0(i) + c * DA_CHUNK >= t1) &&
           !pq::mbar_wait(&full[i][c], 0))
