@@ -17,7 +17,7 @@
 //
 // Pins (see tests/test_oracle_pins.py): H H^T = n I, rotation of unit vectors / all-ones,
 // involution, Parseval, comparison with a library-built Sylvester matrix product; quantizer
-// range / ties / idempotence / hand-worked Eq. (1) values; brute-force integer GEMM;
+// range / ties / idempotence / hand-worked Eq. (1) values (4-bit and 8-bit); brute-force integer GEMMs;
 // attention against closed forms and a library softmax-attention; RoPE against the complex
 // rotation form; RMSNorm and SwiGLU closed forms.
 // Readings fixed by the benchmark spec rather than the paper (symmetric max/7 scale,
@@ -282,6 +282,54 @@ void orc_dequant_bf16(const int32_t* acc, int64_t M, int64_t N, float s_a, const
       out[t * N + n] =
           double_to_bf16(static_cast<double>(acc[t * N + n]) * static_cast<double>(s_a) * static_cast<double>(s_w[n]));
   });
+}
+
+// ---- 8-bit activations (the W4A8KV4 precision of Sec. 5.1; Eq. 1 with N = 8, static per-tensor) -----
+// s_a = fp32( max |fp32(y)| / 127 ) over rows >= row_begin of the rotated calibration batch.
+float orc_calib_act_scale8(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin) {
+  double mx = 0.0;
+  std::vector<double> xr(K), yr(K);
+  for (int64_t m = row_begin; m < M; ++m) {
+    for (int64_t j = 0; j < K; ++j) xr[j] = bf16_to_double(x[m * ldx + j]);
+    rotate_row(xr.data(), yr.data(), K, B);
+    for (int64_t j = 0; j < K; ++j) mx = std::max(mx, std::fabs(static_cast<double>(static_cast<float>(yr[j]))));
+  }
+  if (mx == 0.0) return 1.0f;
+  return static_cast<float>(mx / 127.0);
+}
+
+// code = clamp(round_half_even(y / s_a), -128, 127), one signed byte per element, y the rotated row.
+// Rows < row_begin are left untouched; tie_dist as in orc_quant_act.
+void orc_quant_act8(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin, float s_a,
+                    int8_t* xq, float* tie_dist) {
+  const double s = static_cast<double>(s_a);
+  parallel_rows(M, [&](int64_t m) {
+    if (m < row_begin) return;
+    std::vector<double> xr(K), yr(K);
+    for (int64_t j = 0; j < K; ++j) xr[j] = bf16_to_double(x[m * ldx + j]);
+    rotate_row(xr.data(), yr.data(), K, B);
+    for (int64_t j = 0; j < K; ++j) {
+      double r = yr[j] / s;
+      xq[m * K + j] = static_cast<int8_t>(clampi(std::lrint(std::nearbyint(r)), -128, 127));
+      if (tie_dist) tie_dist[m * K + j] = static_cast<float>(std::fabs(r - std::floor(r) - 0.5));
+    }
+  });
+}
+
+// acc[t,n] = sum_k xq[t,k] * wq[n,k] with 8-bit activation codes and packed 4-bit weight codes,
+// accumulated in int64, returned as int32. Returns 0, or 1 if any accumulator does not fit int32.
+int orc_gemm_i8i4(const int8_t* xq, const uint8_t* wq, int64_t M, int64_t N, int64_t K, int32_t* acc) {
+  std::atomic<int> overflow{0};
+  parallel_rows(M, [&](int64_t t) {
+    for (int64_t n = 0; n < N; ++n) {
+      int64_t s = 0;
+      for (int64_t k = 0; k < K; ++k)
+        s += static_cast<int64_t>(xq[t * K + k]) * static_cast<int64_t>(nib_get(wq + n * (K / 2), k));
+      if (s > INT32_MAX || s < INT32_MIN) overflow = 1;
+      acc[t * N + n] = static_cast<int32_t>(s);
+    }
+  });
+  return overflow.load();
 }
 
 // ---- per-head static KV scale and KV4 append (Table 1, O2: per-head static KV cache) ----------

@@ -148,6 +148,41 @@ def quant_f64(v: np.ndarray, s: float) -> np.ndarray:
     return out
 
 
+def calib_act_scale8(x_bits: np.ndarray, block: int, row_begin: int = 0) -> np.float32:
+    """Static per-tensor step of 8-bit activations: max |rotated x| / 127 over rows >= row_begin."""
+    x_bits = _u16(x_bits)
+    M, K = x_bits.shape
+    f = lib().orc_calib_act_scale8
+    f.restype = c_float
+    return np.float32(f(_p(x_bits, c_uint16), c_int64(K), c_int64(M), c_int64(K), c_int(block), c_int64(row_begin)))
+
+
+def quant_act8(x_bits: np.ndarray, block: int, s_a, row_begin: int = 0, want_tie_dist: bool = False):
+    """Returns int8 codes [M,K] (rows < row_begin zero) and, optionally, the tie distances."""
+    x_bits = _u16(x_bits)
+    M, K = x_bits.shape
+    xq = np.zeros((M, K), np.int8)
+    tie = np.full((M, K), 0.5, np.float32) if want_tie_dist else None
+    lib().orc_quant_act8(
+        _p(x_bits, c_uint16), c_int64(K), c_int64(M), c_int64(K), c_int(block), c_int64(row_begin),
+        c_float(float(s_a)), _p(xq, c_int8), _p(tie, c_float) if want_tie_dist else None,
+    )
+    return (xq, tie) if want_tie_dist else xq
+
+
+def gemm_i8i4(xq8: np.ndarray, wq: np.ndarray) -> np.ndarray:
+    """int8 activation codes [M,K] x packed 4-bit weight codes [N,K/2] -> exact int32 [M,N]."""
+    xq8 = np.ascontiguousarray(xq8, np.int8)
+    wq = np.ascontiguousarray(wq, np.uint8)
+    M, K = xq8.shape
+    N = wq.shape[0]
+    assert wq.shape[1] * 2 == K
+    acc = np.empty((M, N), np.int32)
+    if lib().orc_gemm_i8i4(_p(xq8, c_int8), _p(wq, c_uint8), c_int64(M), c_int64(N), c_int64(K), _p(acc, c_int32)):
+        raise OverflowError("accumulator does not fit int32")
+    return acc
+
+
 # ---- weights ---------------------------------------------------------------------------------------
 def quant_weights(w_bits: np.ndarray):
     w_bits = _u16(w_bits)

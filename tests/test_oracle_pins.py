@@ -240,6 +240,64 @@ def test_gemm_matches_int64_library_matmul_and_special_cases():
     assert np.array_equal(orc.gemm_i4(orc.pack_int4(onehot), orc.pack_int4(w)), w.T.astype(np.int32))
 
 
+# ---------------------------------------------------------------- 8-bit activations (W4A8)
+def test_quant_act8_hand_values_ties_clamp_and_scale():
+    # no rotation, step 0.25: value / 0.25 decides the code by hand (Eq. 1 with N = 8, ties to even)
+    vals = np.array([0.0, 0.125, 0.375, 0.625, -0.125, -0.375, 1.0, 31.75, 31.875, 40.0, -32.0, -32.125, -50.0, 0.3, -0.3, 7.8125])
+    want = np.array([0, 0, 2, 2, 0, -2, 4, 127, 127, 127, -128, -128, -128, 1, -1, 31])
+    x = np.tile(vals, (2, 8))  # K = 128
+    got = orc.quant_act8(bf16_bits(x), 0, 0.25)
+    assert got.dtype == np.int8 and np.array_equal(got, np.tile(want, (2, 8)))
+    # idempotent on its own grid, monotone, full range reached
+    grid = np.arange(-128, 128, dtype=np.float64)[None, :] * 0.25
+    assert np.array_equal(orc.quant_act8(bf16_bits(grid), 0, 0.25)[0], np.arange(-128, 128))
+    v = np.sort(rng.uniform(-40, 40, (1, 256)), axis=1)
+    c = orc.quant_act8(bf16_bits(v), 0, 0.25).astype(int)
+    assert np.all(np.diff(c) >= 0) and c.min() == -128 and c.max() == 127
+    # the static step is max / 127 of the rotated rows at and after row_begin
+    M, K, P = 6, 128, 2
+    xb = inputs.bits(inputs.activations(M, K, seed=3, n_prefix=P))
+    y = orc.rotate_bf16(xb, K)
+    s = orc.calib_act_scale8(xb, K, row_begin=P)
+    assert s == np.float32(np.abs(y[P:].astype(np.float32)).max() / 127.0)
+    assert orc.calib_act_scale8(bf16_bits(np.zeros((2, K))), K) == 1.0
+    # rotated case: within half a step of y / s, the largest element takes +-127, rows below row_begin stay zero
+    q, tie = orc.quant_act8(xb, K, s, row_begin=P, want_tie_dist=True)
+    r = y / np.float64(s)
+    assert np.all(q[:P] == 0) and np.all(np.abs(q[P:] - r[P:]) <= 0.5 + 1e-9) and np.abs(q).max() == 127
+    assert np.allclose(tie[P:], np.abs(r[P:] - np.floor(r[P:]) - 0.5), atol=1e-6)
+    # eight more bits of resolution than the 4-bit code of the same tensor: the 4-bit code is the 8-bit one regrouped
+    s4 = orc.calib_act_scale(xb, K, row_begin=P)
+    assert np.isclose(float(s4) / float(s), 127.0 / 7.0, rtol=1e-6)
+
+
+def test_gemm_i8i4_brute_force_and_library_matmul():
+    M, N, K = 3, 5, 8
+    x = rng.integers(-128, 128, (M, K)).astype(np.int8)
+    w = rng.integers(-8, 8, (N, K)).astype(np.int8)
+    acc = orc.gemm_i8i4(x, orc.pack_int4(w))
+    for t, n in itertools.product(range(M), range(N)):
+        assert acc[t, n] == sum(int(x[t, k]) * int(w[n, k]) for k in range(K))
+    M, N, K = 9, 21, 192
+    x = rng.integers(-128, 128, (M, K)).astype(np.int8)
+    w = rng.integers(-8, 8, (N, K)).astype(np.int8)
+    # nibbles unpacked here with numpy, not with the oracle's own routine
+    pk = orc.pack_int4(w)
+    lo, hi = (pk & 0xF).astype(np.int64), (pk >> 4).astype(np.int64)
+    w_np = np.stack([np.where(lo > 7, lo - 16, lo), np.where(hi > 7, hi - 16, hi)], -1).reshape(N, K)
+    assert np.array_equal(w_np, w)
+    assert np.array_equal(orc.gemm_i8i4(x, pk), x.astype(np.int64) @ w_np.T)
+    # a transposed or swapped operand shows up: one-hot rows pick weight columns, extremes hit the bound
+    onehot = np.zeros((K, K), np.int8)
+    onehot[np.arange(K), np.arange(K)] = 1
+    assert np.array_equal(orc.gemm_i8i4(onehot, pk), w.T.astype(np.int32))
+    lo8, lo4 = np.full((2, K), -128, np.int8), np.full((3, K), -8, np.int8)
+    assert np.all(orc.gemm_i8i4(lo8, orc.pack_int4(lo4)) == 1024 * K)
+    # 4-bit activations are a special case: the same codes as bytes give the W4A4 accumulator
+    x4 = rng.integers(-8, 8, (M, K)).astype(np.int8)
+    assert np.array_equal(orc.gemm_i8i4(x4, pk), orc.gemm_i4(orc.pack_int4(x4), pk))
+
+
 def test_dequant_epilogue_closed_form_and_one_rounding():
     acc = np.array([[3, -5, 0, 1 << 20]], np.int32)
     s_w = np.array([0.25, 0.5, 7.0, 2.0**-10], np.float32)
