@@ -106,6 +106,22 @@ pq_status pq_w4a4_gemm(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const 
                        void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * W4A8 linear layer (the W4A8KV4 precision of Sec. 5.1; Eq. 1 with N = 8; static per-tensor
+ * activations as in Table 1, O2). The same pipeline with one signed byte per activation code:
+ *     xq8 = clamp(round_half_even(y / s_a), -128, 127)     y the rotated row, as above
+ *     *s_a = max(*s_a, max |y| / 127)                      calibration helper
+ *     acc[t, n] = sum_k xq8[t, k] * wq[n, k]   exact, int32;   out[t, n] = bf16(acc * s_a * s_w[n])
+ *   xq8  s8 [M, K] dense rows, base 16-byte aligned; every other argument as in the 4-bit calls.
+ * The GEMM runs on the tensor-core kernel for every M (the token bytes go to the MMA operand
+ * buffer untouched, only the weights are expanded); K % 32 == 0, K <= 65536. */
+pq_status pq_hadamard_quant_act8(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                 int64_t row_begin, const float* s_a, int8_t* xq8, void* stream);
+pq_status pq_calib_act_scale8(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                              int64_t row_begin, float* s_a, void* stream);
+pq_status pq_w4a8_gemm(pq_ctx* ctx, const int8_t* xq8, const uint8_t* wq, const float* s_a, const float* s_w, void* out,
+                       int64_t ldo, int64_t M, int64_t N, int64_t K, int64_t row_begin, int32_t* acc_dbg, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * KV cache with a full-precision prefix region and a 4-bit region (Sec. 4.2, Eq. 3; Table 1, O2:
  * per-head static KV scales). All buffers are the caller's.
  *   prefix_k, prefix_v  fp16 [Hkv, n_prefix, D]  K/V of the prefixed tokens, computed once by the

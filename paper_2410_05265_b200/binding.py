@@ -25,6 +25,7 @@ EXPORTS = [
     "pq_calib_act_scale", "pq_w4a4_gemm_workspace_bytes", "pq_w4a4_gemm", "pq_kv4_append",
     "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix", "pq_decode_attn_kv4_prefix_noalloc",
     "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add", "pq_prefill_attn_kv4_prefix", "pq_kv4_append_strided", "pq_calib_kv_scale",
+    "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm",
 ]
 
 
@@ -81,6 +82,10 @@ def load_library() -> ctypes.CDLL:
     lib.pq_rope.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_int32, c_int64, c_int64, c_double, c_void_p, c_void_p]
     lib.pq_silu_mul.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p]
     lib.pq_residual_add.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p]
+    lib.pq_hadamard_quant_act8.argtypes = lib.pq_hadamard_quant_act.argtypes
+    lib.pq_calib_act_scale8.argtypes = lib.pq_calib_act_scale.argtypes
+    lib.pq_w4a8_gemm.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int64,
+                                 c_int64, c_void_p, c_void_p]
     for name in EXPORTS:
         getattr(lib, name)
         if name not in ("pq_status_string", "pq_w4a4_gemm_workspace_bytes", "pq_decode_attn_workspace_bytes"):
@@ -205,6 +210,44 @@ class Context:
             assert acc_dbg.shape == (M, N) and acc_dbg.is_contiguous()
         _ok(self.lib.pq_w4a4_gemm(self.h, _ptr(xq), _ptr(wq), _ptr(s_a), _ptr(s_w), _ptr(out), out.stride(0), M, N, K2 * 2,
                                   row_begin, _ptr(acc_dbg), c_void_p(0), 0, _stream()), "pq_w4a4_gemm")
+        return out
+
+    # ---- W4A8: 8-bit activation codes, one signed byte per element (Sec. 5.1) -------------------------
+    def calib_act_scale8(self, x: torch.Tensor, had_block: int, row_begin: int = 0, s_a: torch.Tensor | None = None):
+        _dev(x, torch.bfloat16, "x")
+        M, K = x.shape
+        if s_a is None:
+            s_a = torch.zeros((1,), dtype=torch.float32, device=x.device)
+        _ok(self.lib.pq_calib_act_scale8(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, _ptr(s_a), _stream()),
+            "pq_calib_act_scale8")
+        return s_a
+
+    def hadamard_quant_act8(self, x: torch.Tensor, had_block: int, s_a: torch.Tensor, row_begin: int = 0,
+                            out: torch.Tensor | None = None):
+        _dev(x, torch.bfloat16, "x"), _dev(s_a, torch.float32, "s_a")
+        M, K = x.shape
+        assert x.stride(1) == 1
+        if out is None:
+            out = torch.zeros((M, K), dtype=torch.int8, device=x.device)
+        _dev(out, torch.int8, "out")
+        _ok(self.lib.pq_hadamard_quant_act8(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, _ptr(s_a), _ptr(out),
+                                            _stream()), "pq_hadamard_quant_act8")
+        return out
+
+    def w4a8_gemm(self, xq8: torch.Tensor, wq: torch.Tensor, s_a: torch.Tensor, s_w: torch.Tensor, row_begin: int = 0,
+                  out: torch.Tensor | None = None, acc_dbg: torch.Tensor | None = None):
+        _dev(xq8, torch.int8, "xq8"), _dev(wq, torch.uint8, "wq")
+        _dev(s_a, torch.float32, "s_a"), _dev(s_w, torch.float32, "s_w")
+        M, K = xq8.shape
+        N = wq.shape[0]
+        assert wq.shape[1] * 2 == K and xq8.is_contiguous() and wq.is_contiguous()
+        if out is None:
+            out = torch.zeros((M, N), dtype=torch.bfloat16, device=xq8.device)
+        if acc_dbg is not None:
+            _dev(acc_dbg, torch.int32, "acc_dbg")
+            assert acc_dbg.shape == (M, N) and acc_dbg.is_contiguous()
+        _ok(self.lib.pq_w4a8_gemm(self.h, _ptr(xq8), _ptr(wq), _ptr(s_a), _ptr(s_w), _ptr(out), out.stride(0), M, N, K,
+                                  row_begin, _ptr(acc_dbg), _stream()), "pq_w4a8_gemm")
         return out
 
     def kv4_append(self, cache: KV4Cache, k: torch.Tensor, v: torch.Tensor):

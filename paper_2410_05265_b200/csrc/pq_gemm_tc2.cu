@@ -27,6 +27,12 @@
 //                 factor exactly, scale, round to bf16, stage 32 x 64 blocks in swizzled shared
 //                 memory and write them with TMA stores (clipped at the matrix edge).
 //
+// A8 (the W4A8 precision, Sec. 5.1): the token operand already is s8. A second producer lane
+// (warp 2) copies its 128 x 128-byte box straight into the operand stage with a 128-byte-swizzling
+// tensor map; only the weight rows go through the landing ring and the unpack warps, which then
+// write the codes in their natural order (low nibble first) to match the untouched token bytes.
+// The accumulator carries one factor 16 instead of two.
+//
 // Every mbarrier wait is bounded; when one runs out the CTA raises an abort flag, every role of
 // the CTA drains, the peer's waits run out in turn, and PQ_ERR_TIMEOUT is reported.
 #include "pq_common.cuh"
@@ -83,6 +89,7 @@ struct __align__(8) Barriers {
   uint64_t acc_full[2];     // likewise
   uint64_t acc_empty[2];    // leader CTA only: 4 epilogue warps of each CTA
   uint64_t drain;
+  uint64_t a_full[N_S8];    // A8 only: the token box of an operand stage has landed (own CTA)
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -200,6 +207,7 @@ __device__ __forceinline__ void bulk_wait_read() {
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+template <bool A8>
 __global__ void __launch_bounds__(N_THREADS, 1)
     gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                           const __grid_constant__ CUtensorMap tmap_out, const GemmParams p) {
@@ -234,6 +242,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
       pq::mbar_init(&bars->acc_full[i], 1);
       pq::mbar_init(&bars->acc_empty[i], 8);
     }
+    for (int i = 0; i < N_S8; ++i) pq::mbar_init(&bars->a_full[i], 1);
     pq::mbar_init(&bars->drain, 1);
     bars->abort_flag = 0;
     pq::mbar_fence_init();
@@ -266,9 +275,14 @@ __global__ void __launch_bounds__(N_THREADS, 1)
             ok = false;
             break;
           }
-          pq::mbar_arrive_expect_tx(&bars->pk_full[s], PK_STAGE);
-          pq::tma_load_2d(pk_buf + s * PK_STAGE, &tmap_a, kb * PK_ROW, m_row, &bars->pk_full[s]);
-          pq::tma_load_2d(pk_buf + s * PK_STAGE + BM_CTA * PK_ROW, &tmap_b, kb * PK_ROW, n_row, &bars->pk_full[s]);
+          if (A8) {
+            pq::mbar_arrive_expect_tx(&bars->pk_full[s], BN_CTA * PK_ROW);
+            pq::tma_load_2d(pk_buf + s * PK_STAGE, &tmap_b, kb * PK_ROW, n_row, &bars->pk_full[s]);
+          } else {
+            pq::mbar_arrive_expect_tx(&bars->pk_full[s], PK_STAGE);
+            pq::tma_load_2d(pk_buf + s * PK_STAGE, &tmap_a, kb * PK_ROW, m_row, &bars->pk_full[s]);
+            pq::tma_load_2d(pk_buf + s * PK_STAGE + BM_CTA * PK_ROW, &tmap_b, kb * PK_ROW, n_row, &bars->pk_full[s]);
+          }
         }
       }
       if (!ok) {
@@ -277,6 +291,30 @@ __global__ void __launch_bounds__(N_THREADS, 1)
         // let the copies this thread started land before the CTA can exit
         const uint32_t first = it > N_PK ? it - N_PK : 0;
         for (uint32_t j = first; j < it; ++j) pq::mbar_wait(&bars->pk_full[j % N_PK], (j / N_PK) & 1);
+      }
+    }
+  } else if (A8 && warp == 2) {
+    // ------------------------------------------------------------------ token-operand producer (A8)
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+        const int m_row = (tile % p.tiles_m) * (2 * BM_CTA) + rank * BM_CTA;
+        for (int kb = 0; kb < n_kb; ++kb, ++it) {
+          const uint32_t s = it % N_S8, ph = (it / N_S8) & 1;
+          if (!wait_bar(&bars->s8_empty[s], ph ^ 1, abort_flag)) {
+            ok = false;
+            break;
+          }
+          pq::mbar_arrive_expect_tx(&bars->a_full[s], S8_A);
+          pq::tma_load_2d(s8_buf + s * S8_STAGE, &tmap_a, kb * BK, m_row, &bars->a_full[s]);
+        }
+      }
+      if (!ok) {
+        bars->abort_flag = 1;
+        pq::report(p.status, PQ_ERR_TIMEOUT);
+        const uint32_t first = it > N_S8 ? it - N_S8 : 0;
+        for (uint32_t j = first; j < it; ++j) pq::mbar_wait(&bars->a_full[j % N_S8], (j / N_S8) & 1);
       }
     }
   } else if (warp == 1) {
@@ -335,8 +373,8 @@ __global__ void __launch_bounds__(N_THREADS, 1)
         break;
       }
       const uint8_t* src = pk_buf + ps * PK_STAGE;
-      uint8_t* dst = s8_buf + ss * S8_STAGE;
-      constexpr int UNITS = ROWS * 4;  // one unit = one 16-byte packed chunk
+      uint8_t* dst = s8_buf + ss * S8_STAGE + (A8 ? S8_A : 0);  // A8: only the weight rows are expanded
+      constexpr int UNITS = (A8 ? BN_CTA : ROWS) * 4;  // one unit = one 16-byte packed chunk
 #pragma unroll
       for (int i = 0; i < UNITS / GROUP_THREADS; ++i) {
         const int unit = i * GROUP_THREADS + gt;
@@ -345,12 +383,27 @@ __global__ void __launch_bounds__(N_THREADS, 1)
         uint4 lo, hi;
         lo.x = pq::nib_lo_x16(w.x), lo.y = pq::nib_lo_x16(w.y), lo.z = pq::nib_lo_x16(w.z), lo.w = pq::nib_lo_x16(w.w);
         hi.x = pq::nib_hi_x16(w.x), hi.y = pq::nib_hi_x16(w.y), hi.z = pq::nib_hi_x16(w.z), hi.w = pq::nib_hi_x16(w.w);
+        if (A8) {
+          // natural order: byte 2i of a word pair is the low nibble of packed byte i, byte 2i+1 its high nibble
+          const uint4 c0 = make_uint4(__byte_perm(lo.x, hi.x, 0x5140), __byte_perm(lo.x, hi.x, 0x7362),
+                                      __byte_perm(lo.y, hi.y, 0x5140), __byte_perm(lo.y, hi.y, 0x7362));
+          const uint4 c1 = make_uint4(__byte_perm(lo.z, hi.z, 0x5140), __byte_perm(lo.z, hi.z, 0x7362),
+                                      __byte_perm(lo.w, hi.w, 0x5140), __byte_perm(lo.w, hi.w, 0x7362));
+          lo = c0, hi = c1;
+        }
         uint8_t* drow = dst + row * BK;
         const int sw = row & 7;
         *reinterpret_cast<uint4*>(drow + (((2 * j) ^ sw) << 4)) = lo;
         *reinterpret_cast<uint4*>(drow + (((2 * j + 1) ^ sw) << 4)) = hi;
       }
       pq::fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async proxy
+      if (A8) {  // the stage is complete only with this CTA's token box in place
+        const bool late = !wait_bar(&bars->a_full[ss], sph, abort_flag);
+        if (__any_sync(0xffffffffu, late)) {
+          ok = false;
+          break;
+        }
+      }
       __syncwarp();
       if (lane == 0) {
         mbar_arrive_cluster(map_to_cta(&bars->s8_full[ss], 0));
@@ -363,6 +416,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
     }
   } else if (warp >= EPI_WARP0) {
     // ------------------------------------------------------------------ epilogue warps
+    constexpr int SHIFT = A8 ? 4 : 8;  // the factors 16 the expanded codes carry
     const int q = warp & 3;  // TMEM lane quarter this warp may access
     const float s_a = __ldg(p.s_a);
     uint8_t* my_buf = epi_buf + q * EPI_BUFS * EPI_BUF;
@@ -410,14 +464,14 @@ __global__ void __launch_bounds__(N_THREADS, 1)
             const float4 sa = *reinterpret_cast<const float4*>(my_scale + c * 32 + g * 8);
             const float4 sb = *reinterpret_cast<const float4*>(my_scale + c * 32 + g * 8 + 4);
             const int b = g * 8;
-            const __nv_bfloat162 p0 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 0]) >> 8) * sa.x,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 1]) >> 8) * sa.y);
-            const __nv_bfloat162 p1 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 2]) >> 8) * sa.z,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 3]) >> 8) * sa.w);
-            const __nv_bfloat162 p2 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 4]) >> 8) * sb.x,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 5]) >> 8) * sb.y);
-            const __nv_bfloat162 p3 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 6]) >> 8) * sb.z,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 7]) >> 8) * sb.w);
+            const __nv_bfloat162 p0 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 0]) >> SHIFT) * sa.x,
+                                                            static_cast<float>(static_cast<int32_t>(r[b + 1]) >> SHIFT) * sa.y);
+            const __nv_bfloat162 p1 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 2]) >> SHIFT) * sa.z,
+                                                            static_cast<float>(static_cast<int32_t>(r[b + 3]) >> SHIFT) * sa.w);
+            const __nv_bfloat162 p2 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 4]) >> SHIFT) * sb.x,
+                                                            static_cast<float>(static_cast<int32_t>(r[b + 5]) >> SHIFT) * sb.y);
+            const __nv_bfloat162 p3 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 6]) >> SHIFT) * sb.z,
+                                                            static_cast<float>(static_cast<int32_t>(r[b + 7]) >> SHIFT) * sb.w);
             const int chunk = (c & 1) * 4 + g;  // 16-byte chunk inside the 128-byte staging row
             *reinterpret_cast<uint4*>(buf + lane * 128 + ((chunk ^ (lane & 7)) << 4)) =
                 make_uint4(*reinterpret_cast<const uint32_t*>(&p0), *reinterpret_cast<const uint32_t*>(&p1),
@@ -438,13 +492,13 @@ __global__ void __launch_bounds__(N_THREADS, 1)
             const int col = col0 + i;
             if (col < p.N)
               p.out[static_cast<int64_t>(row) * p.ldo + col] =
-                  __float2bfloat16_rn(static_cast<float>(static_cast<int32_t>(r[i]) >> 8) * my_scale[c * 32 + i]);
+                  __float2bfloat16_rn(static_cast<float>(static_cast<int32_t>(r[i]) >> SHIFT) * my_scale[c * 32 + i]);
           }
         }
         if (p.acc_dbg && row < p.M) {
           for (int i = 0; i < 32; ++i) {
             const int col = col0 + i;
-            if (col < p.N) p.acc_dbg[static_cast<int64_t>(row) * p.N + col] = static_cast<int32_t>(r[i]) >> 8;
+            if (col < p.N) p.acc_dbg[static_cast<int64_t>(row) * p.N + col] = static_cast<int32_t>(r[i]) >> SHIFT;
           }
         }
       }
@@ -482,6 +536,19 @@ bool make_packed_map(pq_ctx* ctx, CUtensorMap* map, const uint8_t* base, int64_t
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map over a dense s8 matrix [rows, K]; box = [128 rows, 128 bytes] landing in the 128-byte-swizzled
+// K-major layout the MMA descriptors read.
+bool make_s8_map(pq_ctx* ctx, CUtensorMap* map, const uint8_t* base, int64_t rows, int64_t K) {
+  cuuint64_t gdim[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
+  cuuint64_t gstride[1] = {static_cast<cuuint64_t>(K)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), static_cast<cuuint32_t>(BM_CTA)};
+  cuuint32_t estr[2] = {1, 1};
+  return reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+             map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), gdim, gstride, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Tensor map over the bf16 output [M, N] with row pitch ldo; box = [32 rows, 64 columns], 128-byte swizzle.
 bool make_out_map(pq_ctx* ctx, CUtensorMap* map, void* out, int64_t M, int64_t N, int64_t ldo) {
   cuuint64_t gdim[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(M)};
@@ -497,11 +564,13 @@ bool make_out_map(pq_ctx* ctx, CUtensorMap* map, void* out, int64_t M, int64_t N
 }  // namespace
 
 // Launches the CTA-pair kernel on rows [0, M) of xq/out (the caller has already applied row_begin).
+// a8: xq holds one s8 code per element ([M, K] bytes) instead of packed nibbles.
 pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
                               void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg,
-                              cudaStream_t st) {
+                              cudaStream_t st, bool a8) {
   CUtensorMap ta, tb, to;
-  if (!make_packed_map(ctx, &ta, xq, M, K / 2, BM_CTA) || !make_packed_map(ctx, &tb, wq, N, K / 2, BN_CTA))
+  if (!(a8 ? make_s8_map(ctx, &ta, xq, M, K) : make_packed_map(ctx, &ta, xq, M, K / 2, BM_CTA)) ||
+      !make_packed_map(ctx, &tb, wq, N, K / 2, BN_CTA))
     return PQ_ERR_CUDA;
   GemmParams p;
   p.tma_store = (ldo % 8 == 0) && ((reinterpret_cast<uintptr_t>(out) & 15) == 0);
@@ -523,7 +592,9 @@ pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq,
   p.tiles_n = static_cast<int>((N + BN - 1) / BN);
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_w4a4_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(gemm_w4a4_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(SMEM_BYTES)) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w4a4_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(SMEM_BYTES)) != cudaSuccess)
       return PQ_ERR_CUDA;
     attr_set = true;
@@ -547,6 +618,8 @@ pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq,
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  if (cudaLaunchKernelEx(&cfg, gemm_w4a4_pair_kernel, ta, tb, to, p) != cudaSuccess) return PQ_ERR_CUDA;
+  if ((a8 ? cudaLaunchKernelEx(&cfg, gemm_w4a4_pair_kernel<true>, ta, tb, to, p)
+          : cudaLaunchKernelEx(&cfg, gemm_w4a4_pair_kernel<false>, ta, tb, to, p)) != cudaSuccess)
+    return PQ_ERR_CUDA;
   return pq_launch_status();
 }

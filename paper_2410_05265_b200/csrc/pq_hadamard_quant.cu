@@ -1,6 +1,7 @@
 // Online Walsh-Hadamard rotation of a linear layer's input (App. B, "Online Rotation") fused with
 // the static per-tensor INT4 quantizer (Table 1, O2; Eq. 1) and the nibble pack; the same
-// butterfly also serves the calibration helper that produces the static scale.
+// butterfly also serves the calibration helper that produces the static scale, and the 8-bit
+// quantizer of the W4A8 precision (Sec. 5.1), which stores one signed byte per element.
 //
 // A B-wide block (B = 2^LOGB) is transformed by B/64 threads, 64 values per thread, in two
 // register passes joined by one trip through shared memory:
@@ -21,10 +22,12 @@ constexpr int HQ_CTAS_PER_SM = 5;         // 33 KB of shared memory and about 11
 constexpr int HQ_ELEMS = HQ_THREADS * 64;             // elements handled per CTA iteration
 constexpr int HQ_SMEM_FLOATS = HQ_ELEMS + HQ_ELEMS / 64;  // + 2 floats of padding per 128
 
-template <int LOGB, bool ROTATE, bool CALIB>
+template <int LOGB, bool ROTATE, bool CALIB, int BITS>
 __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
     hadamard_quant_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int64_t n_rows, int64_t K,
                           const float* __restrict__ s_a_in, uint8_t* __restrict__ xq, float* __restrict__ s_a_out) {
+  static_assert(BITS == 4 || BITS == 8, "code width");
+  constexpr int QMAX = BITS == 4 ? 7 : 127;  // codes lie in [-QMAX - 1, QMAX]
   constexpr int B = 1 << LOGB;
   constexpr int TPB = B / 64;                  // threads per block of the transform
   constexpr int G = HQ_THREADS / TPB;          // blocks per CTA iteration
@@ -151,37 +154,57 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
           const float2 tq = __ffma2_rn(W[4 * wd + b], inv2, magic2);
-          lo[b] = max(min(__float_as_int(tq.x), 0x4B400007), 0x4B3FFFF8);
-          hi[b] = max(min(__float_as_int(tq.y), 0x4B400007), 0x4B3FFFF8);
+          lo[b] = max(min(__float_as_int(tq.x), 0x4B400000 + QMAX), 0x4B400000 - QMAX - 1);
+          hi[b] = max(min(__float_as_int(tq.y), 0x4B400000 + QMAX), 0x4B400000 - QMAX - 1);
         }
-        pw[wd] = __byte_perm(__byte_perm(lo[0], lo[1], 0x0040), __byte_perm(lo[2], lo[3], 0x0040), 0x5410) & 0x0F0F0F0Fu;
-        pw[wd + 8] = __byte_perm(__byte_perm(hi[0], hi[1], 0x0040), __byte_perm(hi[2], hi[3], 0x0040), 0x5410) & 0x0F0F0F0Fu;
+        pw[wd] = __byte_perm(__byte_perm(lo[0], lo[1], 0x0040), __byte_perm(lo[2], lo[3], 0x0040), 0x5410);
+        pw[wd + 8] = __byte_perm(__byte_perm(hi[0], hi[1], 0x0040), __byte_perm(hi[2], hi[3], 0x0040), 0x5410);
       }
-      uint32_t fin[8];
+      // This thread holds the elements of one parity of its 128-wide segment (pw[0..7]: first half,
+      // pw[8..15]: second half); its neighbour holds the other parity. Each sends the half the other
+      // is going to store, so that both write contiguous bytes.
+      if (BITS == 4) {
+        uint32_t fin[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        uint32_t send = par ? pw[j] : pw[8 + j];
-        uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
-        fin[j] = par ? (recv | (pw[8 + j] << 4)) : (pw[j] | (recv << 4));
-      }
-      if (active) {
-        uint4* dst = reinterpret_cast<uint4*>(xq + row * (K / 2) + (col0 + seg * 128) / 2 + par * 32);
-        dst[0] = make_uint4(fin[0], fin[1], fin[2], fin[3]);
-        dst[1] = make_uint4(fin[4], fin[5], fin[6], fin[7]);
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t mine = (par ? pw[8 + j] : pw[j]) & 0x0F0F0F0Fu;
+          const uint32_t recv = __shfl_xor_sync(0xffffffffu, (par ? pw[j] : pw[8 + j]) & 0x0F0F0F0Fu, 1);
+          fin[j] = par ? (recv | (mine << 4)) : (mine | (recv << 4));
+        }
+        if (active) {
+          uint4* dst = reinterpret_cast<uint4*>(xq + row * (K / 2) + (col0 + seg * 128) / 2 + par * 32);
+          dst[0] = make_uint4(fin[0], fin[1], fin[2], fin[3]);
+          dst[1] = make_uint4(fin[4], fin[5], fin[6], fin[7]);
+        }
+      } else {
+        uint32_t fin[16];  // 64 consecutive codes: the first half of the segment for parity 0, the second for parity 1
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t mine = par ? pw[8 + j] : pw[j];
+          const uint32_t recv = __shfl_xor_sync(0xffffffffu, par ? pw[j] : pw[8 + j], 1);
+          const uint32_t even = par ? recv : mine, odd = par ? mine : recv;
+          fin[2 * j] = __byte_perm(even, odd, 0x5140);
+          fin[2 * j + 1] = __byte_perm(even, odd, 0x7362);
+        }
+        if (active) {
+          uint4* dst = reinterpret_cast<uint4*>(xq + row * K + col0 + seg * 128 + par * 64);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) dst[j] = make_uint4(fin[4 * j], fin[4 * j + 1], fin[4 * j + 2], fin[4 * j + 3]);
+        }
       }
     }
   }
   if (CALIB) {
     for (int o = 16; o > 0; o >>= 1) cal_max = fmaxf(cal_max, __shfl_xor_sync(0xffffffffu, cal_max, o));
     if ((tid & 31) == 0 && cal_max > 0.0f)
-      atomicMax(reinterpret_cast<int*>(s_a_out), __float_as_int(__fdiv_rn(cal_max, 7.0f)));
+      atomicMax(reinterpret_cast<int*>(s_a_out), __float_as_int(__fdiv_rn(cal_max, static_cast<float>(QMAX))));
   }
 }
 
-template <int LOGB, bool ROTATE, bool CALIB>
+template <int LOGB, bool ROTATE, bool CALIB, int BITS>
 pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_t K, const float* s_a_in, uint8_t* xq,
                  float* s_a_out, cudaStream_t st) {
-  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB>;
+  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS>;
   constexpr size_t smem = HQ_SMEM_FLOATS * sizeof(float);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
     return PQ_ERR_CUDA;
@@ -206,7 +229,7 @@ pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_
   return pq_launch_status();
 }
 
-template <bool CALIB>
+template <bool CALIB, int BITS>
 pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block, int64_t row_begin,
                    const float* s_a_in, uint8_t* xq, float* s_a_out, void* stream) {
   if (!ctx || !x || (!CALIB && (!s_a_in || !xq)) || (CALIB && !s_a_out)) return PQ_ERR_INVALID_ARG;
@@ -221,17 +244,17 @@ pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx
   if (row_begin >= M) return PQ_OK;
   const int64_t n_rows = M - row_begin;
   const void* x0 = static_cast<const __nv_bfloat16*>(x) + row_begin * ldx;
-  uint8_t* xq0 = CALIB ? nullptr : xq + row_begin * (K / 2);
+  uint8_t* xq0 = CALIB ? nullptr : xq + row_begin * (BITS == 4 ? K / 2 : K);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   switch (had_block) {
-    case 0: return launch<7, false, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 128: return launch<7, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 256: return launch<8, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 512: return launch<9, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 1024: return launch<10, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 2048: return launch<11, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 4096: return launch<12, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 8192: return launch<13, true, CALIB>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 0: return launch<7, false, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 128: return launch<7, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 256: return launch<8, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 512: return launch<9, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 1024: return launch<10, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 2048: return launch<11, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 4096: return launch<12, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 8192: return launch<13, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
     default: return PQ_ERR_SHAPE;
   }
 }
@@ -241,10 +264,21 @@ pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx
 extern "C" pq_status pq_hadamard_quant_act(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx,
                                            int had_block, int64_t row_begin, const float* s_a, uint8_t* xq,
                                            void* stream) {
-  return dispatch<false>(ctx, x, M, K, ldx, had_block, row_begin, s_a, xq, nullptr, stream);
+  return dispatch<false, 4>(ctx, x, M, K, ldx, had_block, row_begin, s_a, xq, nullptr, stream);
 }
 
 extern "C" pq_status pq_calib_act_scale(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
                                         int64_t row_begin, float* s_a, void* stream) {
-  return dispatch<true>(ctx, x, M, K, ldx, had_block, row_begin, nullptr, nullptr, s_a, stream);
+  return dispatch<true, 4>(ctx, x, M, K, ldx, had_block, row_begin, nullptr, nullptr, s_a, stream);
+}
+
+extern "C" pq_status pq_hadamard_quant_act8(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx,
+                                            int had_block, int64_t row_begin, const float* s_a, int8_t* xq8,
+                                            void* stream) {
+  return dispatch<false, 8>(ctx, x, M, K, ldx, had_block, row_begin, s_a, reinterpret_cast<uint8_t*>(xq8), nullptr, stream);
+}
+
+extern "C" pq_status pq_calib_act_scale8(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                         int64_t row_begin, float* s_a, void* stream) {
+  return dispatch<true, 8>(ctx, x, M, K, ldx, had_block, row_begin, nullptr, nullptr, s_a, stream);
 }
