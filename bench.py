@@ -262,6 +262,7 @@ def run_gpu(args):
     if rank == 0 and world == 1 and not args.no_sections:
         sections = {}
         try:
+            sections["w4a8_prefill_linear_set"] = section_w4a8(ctx, device, peaks, acts, wqs, sws)
             sections["decode_gemm"] = section_decode_gemm(ctx, device, peaks)
             sections["decode_attention"] = section_decode_attention(ctx, device, peaks)
             sections["block_llama3_70b_prefill4096"] = section_block(ctx, device, peaks)
@@ -404,6 +405,55 @@ def section_decode_attention(ctx, device, peaks):
             "bytes_per_step": by}
 
 
+def section_w4a8(ctx, device, peaks, acts, wqs, sws):
+    """The linear set of configs[1] at the W4A8 precision (Sec. 5.1): 8-bit static per-tensor activation
+    codes, the same packed 4-bit weights; timed like the main step (events around a loop of steps, GEMM
+    launches timed on their own as well)."""
+    import torch
+
+    L = linear_launches()
+    m_rows = M_TOKENS - N_PREFIX
+    scales = [ctx.calib_act_scale8(acts[i], had, N_PREFIX) for i, (_, _, _, had, _) in enumerate(L)]
+    xqs = [torch.zeros((M_TOKENS, K), dtype=torch.int8, device=device) for _, _, K, _, _ in L]
+    outs = [torch.zeros((M_TOKENS, N), dtype=torch.bfloat16, device=device) for _, N, _, _, _ in L]
+    ev = []
+
+    def step(timed):
+        for i, (name, N, K, had, inp) in enumerate(L):
+            ctx.hadamard_quant_act8(acts[i], had, scales[i], N_PREFIX, out=xqs[i])
+            if timed:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            ctx.w4a8_gemm(xqs[i], wqs[i], scales[i], sws[i], N_PREFIX, out=outs[i])
+            if timed:
+                e1.record()
+                ev.append((name, e0, e1))
+
+    steps = 50
+    for _ in range(5):
+        step(False)
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        step(True)
+    t1.record()
+    torch.cuda.synchronize()
+    ctx.check()
+    ms = t0.elapsed_time(t1) / steps
+    per = {}
+    for name, e0, e1 in ev:
+        per.setdefault(name, []).append(e0.elapsed_time(e1))
+    gemm_ms = sum(statistics.mean(v) for v in per.values())
+    int8_peak = 2.0 * peaks["bf16_sus"]
+    gemm_tops = step_ops(m_rows) / (gemm_ms * 1e-3) / 1e12
+    return {"ms_per_step": round(ms, 4), "TOPS": round(step_ops(m_rows) / (ms * 1e-3) / 1e12, 1), "gemm_TOPS": round(gemm_tops, 1),
+            "gemm_frac_of_2x_bf16_sustained": round(gemm_tops / int8_peak, 4), "gemm_frac_of_nominal_4500": round(gemm_tops / NOMINAL_INT8_TOPS, 4),
+            "per_launch": {k: {"ms": round(statistics.mean(v), 4),
+                               "tops": round(2.0 * m_rows * next(n * kk for nm, n, kk, _, _ in L if nm == k) / (statistics.mean(v) * 1e-3) / 1e12, 1)}
+                           for k, v in per.items()}}
+
+
 def section_block(ctx, device, peaks):
     """configs[4]: one Llama-3-70B-shaped W4A4KV4 block at prefill, 4096 ordinary tokens after 4 prefixed
     tokens whose K/V sit in the cache in fp16; static scales from a seed-1 calibration pass."""
@@ -537,6 +587,21 @@ def run_case(args):
         out = torch.zeros((M, N), dtype=torch.bfloat16, device=dev)
         fn = lambda: ctx.w4a4_gemm(xq, wq, s_a, s_w, out=out)
         work = 2.0 * M * N * K
+    elif name == "gemm8":
+        M, N, K = dims or [2048, 28672, 4096]
+        xq8 = torch.randint(-128, 128, (M, K), dtype=torch.int8, device=dev)
+        wq = torch.randint(0, 256, (N, K // 2), dtype=torch.uint8, device=dev)
+        s_a, s_w = torch.full((1,), 0.003, device=dev), torch.full((N,), 0.003, device=dev)
+        out = torch.zeros((M, N), dtype=torch.bfloat16, device=dev)
+        fn = lambda: ctx.w4a8_gemm(xq8, wq, s_a, s_w, out=out)
+        work = 2.0 * M * N * K
+    elif name == "hadamard8":
+        M, K, B = dims or [8192, 14336, 2048]
+        x = inputs.activations(M, K, seed=0, device=dev)
+        s_a = ctx.calib_act_scale8(x, B)
+        out = torch.zeros((M, K), dtype=torch.int8, device=dev)
+        fn = lambda: ctx.hadamard_quant_act8(x, B, s_a, out=out)
+        work = 3.0 * M * K
     elif name == "hadamard":
         M, K, B = dims or [8192, 14336, 2048]
         x = inputs.activations(M, K, seed=0, device=dev)
