@@ -478,6 +478,28 @@ void orc_rope(const uint16_t* x, int64_t T, int64_t H, int64_t D, int64_t pos0, 
   });
 }
 
+// Rotary embedding followed by the online head-wise rotation R3 (App. B, "Online Rotation": the outputs
+// of q_proj and k_proj after RoPE are multiplied by the Hadamard matrix of the head dimension):
+// y = RoPE(x) H_D / sqrt(D) per head, everything in double, one rounding to bf16.
+void orc_rope_rotate(const uint16_t* x, int64_t T, int64_t H, int64_t D, int64_t pos0, double theta, uint16_t* y) {
+  parallel_rows(T, [&](int64_t t) {
+    double pos = static_cast<double>(pos0 + t);
+    std::vector<double> r(D), z(D);
+    for (int64_t h = 0; h < H; ++h) {
+      for (int64_t i = 0; i < D / 2; ++i) {
+        double ang = pos * std::pow(theta, -2.0 * static_cast<double>(i) / static_cast<double>(D));
+        double c = std::cos(ang), s = std::sin(ang);
+        double a = bf16_to_double(x[(t * H + h) * D + i]);
+        double b = bf16_to_double(x[(t * H + h) * D + i + D / 2]);
+        r[i] = a * c - b * s;
+        r[i + D / 2] = b * c + a * s;
+      }
+      rotate_row(r.data(), z.data(), D, static_cast<int>(D));
+      for (int64_t i = 0; i < D; ++i) y[(t * H + h) * D + i] = double_to_bf16(z[i]);
+    }
+  });
+}
+
 // SwiGLU gate: y = silu(gate) * up = gate / (1 + exp(-gate)) * up, rounded once to bf16.
 void orc_silu_mul(const uint16_t* gate, const uint16_t* up, int64_t n, uint16_t* y) {
   for (int64_t i = 0; i < n; ++i) {

@@ -300,6 +300,15 @@ def rope(x_bits, pos0: int, theta: float):
     return y
 
 
+def rope_rotate(x_bits, pos0: int, theta: float):
+    """RoPE, then the head-wise Hadamard rotation R3 (x H_D / sqrt(D)), one rounding to bf16. x [T,H,D]."""
+    x_bits = _u16(x_bits)
+    T, H, D = x_bits.shape
+    y = np.empty_like(x_bits)
+    lib().orc_rope_rotate(_p(x_bits, c_uint16), c_int64(T), c_int64(H), c_int64(D), c_int64(pos0), c_double(theta), _p(y, c_uint16))
+    return y
+
+
 def silu_mul(gate_bits, up_bits):
     gate_bits, up_bits = _u16(gate_bits), _u16(up_bits)
     y = np.empty(gate_bits.shape, np.uint16)

@@ -465,6 +465,35 @@ def test_rope_matches_complex_rotation_and_relative_property():
     assert abs(d1 - d2) < 1e-10
 
 
+def test_rope_rotate_is_complex_rotation_times_library_hadamard():
+    """R3 (App. B): after the rotary embedding every head is multiplied by H_D / sqrt(D)."""
+    T, H, D, theta = 5, 3, 128, 500000.0
+    x = inputs.normal(11, inputs.STREAM_Q, (T, H, D), dtype=torch.bfloat16)
+    y = orc.bf16_to_f64(orc.rope_rotate(inputs.bits(x), 4, theta))
+    xd = x.to(torch.float64).numpy()
+    z = xd[..., :D // 2] + 1j * xd[..., D // 2:]
+    freq = theta ** (-np.arange(D // 2) * 2.0 / D)
+    zr = z * np.exp(1j * (4 + np.arange(T))[:, None, None] * freq[None, None, :])
+    roped = np.concatenate([zr.real, zr.imag], -1)
+    ref = roped @ hadamard(D).astype(np.float64) / math.sqrt(D)
+    assert np.all(np.abs(y - ref) <= np.abs(ref) * 2.0**-8 + 1e-30), "one rounding to bf16 of the exact product"
+    # at position 0 the rotary part is the identity: what is left is the plain rotation of the input
+    y0 = orc.bf16_to_f64(orc.rope_rotate(inputs.bits(x[:1]), 0, theta))
+    r0 = orc.rotate_bf16(inputs.bits(x[:1]).reshape(H, D), D)
+    assert np.all(np.abs(y0.reshape(H, D) - r0) <= np.abs(r0) * 2.0**-8 + 1e-30)
+    # computational invariance: scores between rotated q and k equal the scores without R3 (up to the bf16 store)
+    plain = orc.bf16_to_f64(orc.rope(inputs.bits(x), 4, theta))
+    s_rot = np.einsum("thd,shd->hts", y, y)
+    s_plain = np.einsum("thd,shd->hts", plain, plain)
+    assert np.allclose(s_rot, s_plain, rtol=0, atol=2.0**-7 * np.abs(s_plain).max())
+    # a unit vector in dim j at position 0 becomes column j of H / sqrt(D): every entry +-1/sqrt(128), sign by popcount
+    e = np.zeros((1, 1, D))
+    e[0, 0, 5] = 1.0
+    ye = orc.bf16_to_f64(orc.rope_rotate(bf16_bits(e), 0, theta))[0, 0]
+    sign = np.array([(-1.0) ** bin(5 & j).count("1") for j in range(D)])
+    assert np.array_equal(ye, orc.bf16_to_f64(bf16_bits(sign / math.sqrt(D))))
+
+
 def test_rmsnorm_silu_add_closed_forms():
     x = inputs.activations(5, 64, seed=0)
     g = torch.ones(64, dtype=torch.bfloat16)
