@@ -504,12 +504,37 @@ def section_block(ctx, device, peaks):
             continue
         stages[name] = round(prev.elapsed_time(ev), 4)
         prev = ev
+    # the same block with the online head-wise rotation R3 of q and k fused into the rotary step
+    shape.r3 = True
+    blk.forward(inputs.activations(T, shape.hidden, seed=1, device=device), calibrate=True)
+    for _ in range(2):
+        blk.forward(x)
+    marks.clear()
+    r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    r0.record()
+    for _ in range(reps):
+        blk.forward(x)
+    r1.record()
+    torch.cuda.synchronize()
+    ms_r3 = r0.elapsed_time(r1) / reps
+    start3 = torch.cuda.Event(enable_timing=True)
+    start3.record()
+    blk.forward(x, tap=tap)
+    torch.cuda.synchronize()
+    prev3, rope_r3 = start3, None
+    for name, ev in marks:
+        if name == "qkv_rope":
+            rope_r3 = round(prev3.elapsed_time(ev), 4)
+        prev3 = ev
+    shape.r3 = False
+    ctx.check()
     gemm_ops = 2.0 * T * shape.hidden * (qd + 2 * kvd + qd + 2 * shape.ffn + shape.ffn)
     attn_flops = 4.0 * D * c["n_q_heads"] * (T * (T + 1) / 2 + T * P)
     gemm_ms = sum(stages[k] for k in ("qkv", "o", "gu", "d"))
     return {"tokens_per_s": round(T / (ms * 1e-3), 1), "ms": round(ms, 4), "tokens": T, "n_prefix": P,
             "gemm_TOPS": round(gemm_ops / (gemm_ms * 1e-3) / 1e12, 1), "gemm_share": round(gemm_ms / sum(stages.values()), 3),
             "attention_TFLOPS": round(attn_flops / (stages["attn"] * 1e-3) / 1e12, 1), "stage_ms": stages,
+            "with_r3": {"ms": round(ms_r3, 4), "rope_rotate_ms": rope_r3},
             "launches": block.Block.LAUNCHES_PER_FORWARD}
 
 

@@ -190,12 +190,17 @@ pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, int
  *                    y[i+64] = x[i+64] cos + x[i] sin       x, y [T,H,D] with ld elements between tokens
  *                    (ld >= H*D, so the q and k heads of a concatenated q|k|v output are rotated in one
  *                    call); y may alias x
+ *   pq_rope_rotate   the same followed by the online head-wise rotation R3 (App. B, "Online Rotation": the
+ *                    outputs of q_proj and k_proj after RoPE): y = RoPE(x) H_D / sqrt(D) per head, H in
+ *                    Sylvester order; scores q . k are unchanged, K is quantized in the rotated basis
  *   pq_silu_mul      y = gate / (1 + exp(-gate)) * up        gate, up [M,F] with row stride ld_in (the two
  *                    halves of a concatenated gate|up GEMM output), y [M,F] with row stride ldy; F % 8 == 0
  *   pq_residual_add  y = a + b over n elements, n % 8 == 0; y may alias a or b */
 pq_status pq_rmsnorm(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, const void* g, float eps, void* y,
                      int64_t ldy, void* stream);
 pq_status pq_rope(pq_ctx* ctx, const void* x, int64_t T, int32_t H, int32_t D, int64_t ld, int64_t pos0, double theta,
+                  void* y, void* stream);
+pq_status pq_rope_rotate(pq_ctx* ctx, const void* x, int64_t T, int32_t H, int32_t D, int64_t ld, int64_t pos0, double theta,
                   void* y, void* stream);
 pq_status pq_silu_mul(pq_ctx* ctx, const void* gate, const void* up, int64_t M, int64_t F, int64_t ld_in, void* y,
                       int64_t ldy, void* stream);

@@ -25,7 +25,7 @@ EXPORTS = [
     "pq_calib_act_scale", "pq_w4a4_gemm_workspace_bytes", "pq_w4a4_gemm", "pq_kv4_append",
     "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix", "pq_decode_attn_kv4_prefix_noalloc",
     "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add", "pq_prefill_attn_kv4_prefix", "pq_kv4_append_strided", "pq_calib_kv_scale",
-    "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm",
+    "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
 ]
 
 
@@ -80,6 +80,7 @@ def load_library() -> ctypes.CDLL:
                                                c_void_p]
     lib.pq_rmsnorm.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_float, c_void_p, c_int64, c_void_p]
     lib.pq_rope.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_int32, c_int64, c_int64, c_double, c_void_p, c_void_p]
+    lib.pq_rope_rotate.argtypes = lib.pq_rope.argtypes
     lib.pq_silu_mul.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p]
     lib.pq_residual_add.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p]
     lib.pq_hadamard_quant_act8.argtypes = lib.pq_hadamard_quant_act.argtypes
@@ -311,14 +312,16 @@ class Context:
                                 _stream()), "pq_rmsnorm")
         return out
 
-    def rope(self, x: torch.Tensor, pos0: int, theta: float, out: torch.Tensor | None = None):
+    def rope(self, x: torch.Tensor, pos0: int, theta: float, out: torch.Tensor | None = None, rotate: bool = False):
+        """Rotary embedding of x [T, H, D]; with rotate=True followed by the head-wise Hadamard rotation R3."""
         _dev(x, torch.bfloat16, "x")
         T, H, D = x.shape
         assert x.stride(2) == 1 and x.stride(1) == D
         if out is None:
             out = torch.empty((T, H, D), dtype=x.dtype, device=x.device)
         assert out.stride() == x.stride() or (out.is_contiguous() and x.is_contiguous())
-        _ok(self.lib.pq_rope(self.h, _ptr(x), T, H, D, x.stride(0), int(pos0), float(theta), _ptr(out), _stream()), "pq_rope")
+        fn, name = (self.lib.pq_rope_rotate, "pq_rope_rotate") if rotate else (self.lib.pq_rope, "pq_rope")
+        _ok(fn(self.h, _ptr(x), T, H, D, x.stride(0), int(pos0), float(theta), _ptr(out), _stream()), name)
         return out
 
     def silu_mul(self, gate: torch.Tensor, up: torch.Tensor, out: torch.Tensor | None = None):

@@ -2,7 +2,8 @@
 
 Nothing is computed here: the class owns the device buffers of one block (packed weights, static
 scales, the KV cache with its full-precision prefix) and issues the C-ABI calls in the order of the
-block in App. B of the paper: RMSNorm -> [rotate + quantize] -> q|k|v GEMM -> rotary embedding ->
+block in App. B of the paper: RMSNorm -> [rotate + quantize] -> q|k|v GEMM -> rotary embedding (optionally
+followed by the head-wise rotation R3 of q and k) ->
 KV4 append -> causal attention over [prefix || INT4 cache] -> [rotate + quantize] -> o GEMM ->
 residual -> RMSNorm -> [rotate + quantize] -> gate|up GEMM -> SwiGLU -> [block rotate + quantize] ->
 down GEMM -> residual. The tokens that enter are ordinary tokens: the prefixed outlier tokens are
@@ -27,6 +28,7 @@ class BlockShape:
     head_dim: int = 128
     rope_theta: float = 500000.0
     eps: float = 1e-5
+    r3: bool = False  # online head-wise Hadamard rotation of q and k after RoPE (App. B, R3)
 
     @property
     def q_dim(self):
@@ -103,7 +105,7 @@ class Block:
         ctx.w4a4_gemm(b["xq_h"], self.wq_qkv, self.s_a[0], self.sw_qkv, out=b["qkv"])
         tap("qkv", b["qkv"])
         qk = b["qkv"][:, : s.q_dim + s.kv_dim].unflatten(1, (s.n_q_heads + s.n_kv_heads, s.head_dim))
-        ctx.rope(qk, self.n_prefix, s.rope_theta, out=qk)
+        ctx.rope(qk, self.n_prefix, s.rope_theta, out=qk, rotate=s.r3)
         tap("qkv_rope", b["qkv"])
         q = b["qkv"][:, : s.q_dim].unflatten(1, (s.n_q_heads, s.head_dim))
         k = b["qkv"][:, s.q_dim: s.q_dim + s.kv_dim].unflatten(1, (s.n_kv_heads, s.head_dim))

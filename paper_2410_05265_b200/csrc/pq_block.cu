@@ -105,6 +105,53 @@ __global__ void __launch_bounds__(RP_THREADS)
   }
 }
 
+// Rotary embedding followed by the online head-wise rotation R3 (App. B): y = RoPE(x) H_128 / sqrt(128)
+// per head, H in Sylvester order. One warp per head: lane l holds the elements 2l, 2l+1, 64+2l, 65+2l
+// (both rotate-half pairs are inside the lane); the butterflies on index bits 0 and 6 run inside
+// the lane, those on bits 1..5 across lanes. fp32 throughout, one rounding to bf16.
+__global__ void __launch_bounds__(RP_THREADS)
+    rope_rotate_kernel(const __nv_bfloat16* x, __nv_bfloat16* y, int64_t T, int H, int64_t ld, int64_t pos0,
+                       double log2_theta) {
+  __shared__ float cs[64], sn[64];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int64_t t = blockIdx.x; t < T; t += gridDim.x) {
+    if (threadIdx.x < 64) {
+      const double inv_freq = exp2(-2.0 * static_cast<double>(threadIdx.x) / 128.0 * log2_theta);
+      double s, c;
+      sincos(static_cast<double>(pos0 + t) * inv_freq, &s, &c);
+      cs[threadIdx.x] = static_cast<float>(c), sn[threadIdx.x] = static_cast<float>(s);
+    }
+    __syncthreads();
+    const float c0 = cs[2 * lane], s0 = sn[2 * lane], c1 = cs[2 * lane + 1], s1 = sn[2 * lane + 1];
+    for (int hd = warp; hd < H; hd += RP_THREADS / 32) {
+      const __nv_bfloat16* px = x + t * ld + hd * 128;
+      __nv_bfloat16* py = y + t * ld + hd * 128;
+      const uint32_t wa = *reinterpret_cast<const uint32_t*>(px + 2 * lane);  // y may alias x: the warp reads its head first
+      const uint32_t wb = *reinterpret_cast<const uint32_t*>(px + 64 + 2 * lane);
+      const float a0 = bf16_lo(wa), a1 = bf16_hi(wa), b0 = bf16_lo(wb), b1 = bf16_hi(wb);
+      float v0 = a0 * c0 - b0 * s0, v1 = a1 * c1 - b1 * s1, v2 = b0 * c0 + a0 * s0, v3 = b1 * c1 + a1 * s1;
+      float u;
+      u = v0, v0 = u + v1, v1 = u - v1;  // index bit 0
+      u = v2, v2 = u + v3, v3 = u - v3;
+      u = v0, v0 = u + v2, v2 = u - v2;  // index bit 6
+      u = v1, v1 = u + v3, v3 = u - v3;
+#pragma unroll
+      for (int m = 1; m < 32; m <<= 1) {  // index bits 1..5: the upper partner holds the difference
+        const bool up = lane & m;
+        const float o0 = __shfl_xor_sync(0xffffffffu, v0, m), o1 = __shfl_xor_sync(0xffffffffu, v1, m);
+        const float o2 = __shfl_xor_sync(0xffffffffu, v2, m), o3 = __shfl_xor_sync(0xffffffffu, v3, m);
+        v0 = up ? o0 - v0 : v0 + o0, v1 = up ? o1 - v1 : v1 + o1;
+        v2 = up ? o2 - v2 : v2 + o2, v3 = up ? o3 - v3 : v3 + o3;
+      }
+      const float norm = 0.08838834764831845f;  // 1 / sqrt(128)
+      __syncwarp();
+      *reinterpret_cast<uint32_t*>(py + 2 * lane) = pack_bf16(v0 * norm, v1 * norm);
+      *reinterpret_cast<uint32_t*>(py + 64 + 2 * lane) = pack_bf16(v2 * norm, v3 * norm);
+    }
+    __syncthreads();
+  }
+}
+
 // ---- SwiGLU gate: y = gate / (1 + exp(-gate)) * up ------------------------------------------------
 constexpr int EW_THREADS = 256;
 
@@ -192,6 +239,18 @@ extern "C" pq_status pq_rope(pq_ctx* ctx, const void* x, int64_t T, int32_t H, i
   if (!aligned16(x) || !aligned16(y) || ld % 8 != 0) return PQ_ERR_ALIGN;
   if (T == 0) return PQ_OK;
   rope_kernel<<<grid_for(ctx, T, 1), RP_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(y), T, H, ld, pos0, log2(theta));
+  return pq_launch_status();
+}
+
+extern "C" pq_status pq_rope_rotate(pq_ctx* ctx, const void* x, int64_t T, int32_t H, int32_t D, int64_t ld,
+                                    int64_t pos0, double theta, void* y, void* stream) {
+  if (!ctx || !x || !y) return PQ_ERR_INVALID_ARG;
+  if (T < 0 || H <= 0 || pos0 < 0 || !(theta > 1.0) || ld < static_cast<int64_t>(H) * 128) return PQ_ERR_INVALID_ARG;
+  if (D != 128) return PQ_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(y) || ld % 8 != 0) return PQ_ERR_ALIGN;
+  if (T == 0) return PQ_OK;
+  rope_rotate_kernel<<<grid_for(ctx, T, 1), RP_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(y), T, H, ld, pos0, log2(theta));
   return pq_launch_status();
 }

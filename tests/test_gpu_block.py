@@ -19,13 +19,14 @@ def _bits(t):
     return inputs.bits(t.detach().cpu().contiguous())
 
 
-@pytest.mark.parametrize("T,hidden,Hq,Hkv,ffn,P", [(40, 512, 4, 2, 6144, 4), (19, 256, 8, 1, 1024, 0)])
-def test_block_stages_match_oracle(T, hidden, Hq, Hkv, ffn, P):
+@pytest.mark.parametrize("T,hidden,Hq,Hkv,ffn,P,r3", [(40, 512, 4, 2, 6144, 4, False), (19, 256, 8, 1, 1024, 0, False),
+                                                      (40, 512, 4, 2, 6144, 4, True)])
+def test_block_stages_match_oracle(T, hidden, Hq, Hkv, ffn, P, r3):
     from paper_2410_05265_b200 import binding, block
 
     ctx = binding.Context()
     D = 128
-    shape = block.BlockShape(hidden=hidden, n_q_heads=Hq, n_kv_heads=Hkv, ffn=ffn)
+    shape = block.BlockShape(hidden=hidden, n_q_heads=Hq, n_kv_heads=Hkv, ffn=ffn, r3=r3)
     qd, kvd = Hq * D, Hkv * D
     w_qkv = inputs.weights(qd + 2 * kvd, hidden, seed=2, std=0.05)
     w_o = inputs.weights(hidden, qd, seed=3, std=0.05)
@@ -64,7 +65,7 @@ def test_block_stages_match_oracle(T, hidden, Hq, Hkv, ffn, P):
     check_gemm("qkv", "xq1", inputs.bits(w_qkv), s_a[0])
     qkv = taps["qkv"]
     qk = qkv[:, : qd + kvd].reshape(T, Hq + Hkv, D).contiguous()
-    ref_rope = orc.rope(inputs.bits(qk), P, 500000.0)
+    ref_rope = (orc.rope_rotate if r3 else orc.rope)(inputs.bits(qk), P, 500000.0)
     got_rope = taps["qkv_rope"][:, : qd + kvd].reshape(T, Hq + Hkv, D).contiguous()
     assert_bf16_close(inputs.bits(got_rope), ref_rope, "rope")
     assert torch.equal(taps["qkv_rope"][:, qd + kvd:], qkv[:, qd + kvd:]), "v must pass through the rotary step untouched"

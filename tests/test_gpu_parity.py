@@ -290,6 +290,27 @@ def test_rope_matches_oracle(ctx, T, H, pos0):
     assert torch.equal(xin, got)
 
 
+@pytest.mark.parametrize("T,H,pos0", [(3, 2, 0), (33, 9, 4), (5, 72, 4090)])
+def test_rope_rotate_matches_oracle(ctx, T, H, pos0):
+    """Rotary embedding + head-wise rotation R3 in one call; strided (q|k of a q|k|v row) and in place."""
+    x = inputs.kv_tensor(1, T, H, 128, 0, "k")[0]
+    ref = orc.rope_rotate(inputs.bits(x), pos0, 500000.0)
+    got = ctx.rope(x.cuda().contiguous(), pos0, 500000.0, rotate=True)
+    ctx.check()
+    assert_bf16_close(inputs.bits(got), ref, "rope + R3")
+    wide = torch.zeros((T, H * 128 + 256), dtype=torch.bfloat16, device="cuda")
+    wide[:, : H * 128] = x.cuda().reshape(T, H * 128)
+    wide[:, H * 128:] = 7.0
+    view = wide[:, : H * 128].unflatten(1, (H, 128))
+    ctx.rope(view, pos0, 500000.0, out=view, rotate=True)
+    ctx.check()
+    assert torch.equal(view, got) and bool((wide[:, H * 128:] == 7.0).all())
+    # the rotation keeps the scores: q' . k' == q . k up to the bf16 store
+    plain = ctx.rope(x.cuda().contiguous(), pos0, 500000.0).double()
+    s_plain, s_rot = torch.einsum("thd,shd->hts", plain, plain), torch.einsum("thd,shd->hts", got.double(), got.double())
+    assert float((s_plain - s_rot).abs().max()) <= 2.0**-6 * float(s_plain.abs().max())
+
+
 def test_silu_mul_and_residual_match_oracle(ctx):
     M, F = 19, 1024
     gu = (inputs.activations(M, 2 * F, seed=3) * 2).to(torch.bfloat16)
