@@ -332,6 +332,50 @@ int orc_gemm_i8i4(const int8_t* xq, const uint8_t* wq, int64_t M, int64_t N, int
   return overflow.load();
 }
 
+// ---- per-token dynamic activation quantization (Table 1, O1; Sec. 3 "Dynamic and Static") ---------
+// One step per token, computed online from the rotated row itself: s[t] = fp32(clip * max |fp32(y_t)| / 7),
+// clip being the layer's clipping factor shared by all tokens (gamma of Eq. 1, symmetric form); 1 for an
+// all-zero row. Rows below row_begin keep whatever s holds.
+void orc_dyn_act_scale(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin, float clip,
+                       float* s) {
+  parallel_rows(M, [&](int64_t m) {
+    if (m < row_begin) return;
+    std::vector<double> xr(K), yr(K);
+    for (int64_t j = 0; j < K; ++j) xr[j] = bf16_to_double(x[m * ldx + j]);
+    rotate_row(xr.data(), yr.data(), K, B);
+    double mx = 0.0;
+    for (int64_t j = 0; j < K; ++j) mx = std::max(mx, std::fabs(static_cast<double>(static_cast<float>(yr[j]))));
+    s[m] = mx == 0.0 ? 1.0f : static_cast<float>(static_cast<double>(clip) * mx / 7.0);
+  });
+}
+
+// code[t,k] = clamp(round_half_even(y[t,k] / s[t]), -8, 7) with one step per row; otherwise as orc_quant_act.
+void orc_quant_act_rows(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin, const float* s_tok,
+                        uint8_t* xq, float* tie_dist) {
+  parallel_rows(M, [&](int64_t m) {
+    if (m < row_begin) return;
+    const double s = static_cast<double>(s_tok[m]);
+    std::vector<double> xr(K), yr(K);
+    for (int64_t j = 0; j < K; ++j) xr[j] = bf16_to_double(x[m * ldx + j]);
+    rotate_row(xr.data(), yr.data(), K, B);
+    uint8_t* out = xq + m * (K / 2);
+    for (int64_t j = 0; j < K; ++j) {
+      double r = yr[j] / s;
+      nib_set(out, j, clampi(std::lrint(std::nearbyint(r)), -8, 7));
+      if (tie_dist) tie_dist[m * K + j] = static_cast<float>(std::fabs(r - std::floor(r) - 0.5));
+    }
+  });
+}
+
+// out[t,n] = bf16( acc[t,n] * s_tok[t] * s_w[n] ), product in double, one rounding.
+void orc_dequant_bf16_rows(const int32_t* acc, int64_t M, int64_t N, const float* s_tok, const float* s_w, uint16_t* out) {
+  parallel_rows(M, [&](int64_t t) {
+    for (int64_t n = 0; n < N; ++n)
+      out[t * N + n] = double_to_bf16(static_cast<double>(acc[t * N + n]) * static_cast<double>(s_tok[t]) *
+                                      static_cast<double>(s_w[n]));
+  });
+}
+
 // ---- per-head static KV scale and KV4 append (Table 1, O2: per-head static KV cache) ----------
 // kv bf16 [B,T,H,D]; s[h] = fp32(max |kv[:,:,h,:]|) / 7 in double then fp32 (1 if all zero).
 void orc_calib_kv_scale(const uint16_t* kv, int64_t B, int64_t T, int64_t H, int64_t D, float* s) {

@@ -183,6 +183,39 @@ def gemm_i8i4(xq8: np.ndarray, wq: np.ndarray) -> np.ndarray:
     return acc
 
 
+def dyn_act_scale(x_bits: np.ndarray, block: int, clip: float = 1.0, row_begin: int = 0) -> np.ndarray:
+    """Per-token dynamic steps s[t] = clip * max |rotated x_t| / 7 (rows < row_begin: 0)."""
+    x_bits = _u16(x_bits)
+    M, K = x_bits.shape
+    s = np.zeros(M, np.float32)
+    lib().orc_dyn_act_scale(_p(x_bits, c_uint16), c_int64(K), c_int64(M), c_int64(K), c_int(block), c_int64(row_begin),
+                            c_float(float(clip)), _p(s, c_float))
+    return s
+
+
+def quant_act_rows(x_bits: np.ndarray, block: int, s_tok: np.ndarray, row_begin: int = 0, want_tie_dist: bool = False):
+    """Packed codes [M,K/2] with one step per row (rows < row_begin zero) and, optionally, the tie distances."""
+    x_bits = _u16(x_bits)
+    M, K = x_bits.shape
+    s_tok = np.ascontiguousarray(s_tok, np.float32)
+    assert s_tok.shape == (M,)
+    xq = np.zeros((M, K // 2), np.uint8)
+    tie = np.full((M, K), 0.5, np.float32) if want_tie_dist else None
+    lib().orc_quant_act_rows(_p(x_bits, c_uint16), c_int64(K), c_int64(M), c_int64(K), c_int(block), c_int64(row_begin),
+                             _p(s_tok, c_float), _p(xq, c_uint8), _p(tie, c_float) if want_tie_dist else None)
+    return (xq, tie) if want_tie_dist else xq
+
+
+def dequant_bf16_rows(acc: np.ndarray, s_tok: np.ndarray, s_w: np.ndarray) -> np.ndarray:
+    acc = np.ascontiguousarray(acc, np.int32)
+    M, N = acc.shape
+    s_tok, s_w = np.ascontiguousarray(s_tok, np.float32), np.ascontiguousarray(s_w, np.float32)
+    assert s_tok.shape == (M,) and s_w.shape == (N,)
+    out = np.empty((M, N), np.uint16)
+    lib().orc_dequant_bf16_rows(_p(acc, c_int32), c_int64(M), c_int64(N), _p(s_tok, c_float), _p(s_w, c_float), _p(out, c_uint16))
+    return out
+
+
 # ---- weights ---------------------------------------------------------------------------------------
 def quant_weights(w_bits: np.ndarray):
     w_bits = _u16(w_bits)

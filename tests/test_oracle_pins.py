@@ -298,6 +298,42 @@ def test_gemm_i8i4_brute_force_and_library_matmul():
     assert np.array_equal(orc.gemm_i8i4(x4, pk), orc.gemm_i4(orc.pack_int4(x4), pk))
 
 
+# ---------------------------------------------------------------- per-token dynamic activations (O1)
+def test_dynamic_per_token_quantizer_reduces_to_the_static_one_row_by_row():
+    M, K, P = 7, 256, 2
+    x = inputs.activations(M, K, seed=4, n_prefix=P)
+    x[4] = 0
+    xb = inputs.bits(x)
+    s = orc.dyn_act_scale(xb, K, 1.0, row_begin=P)
+    assert np.all(s[:P] == 0) and s[4] == 1.0
+    codes, tie = orc.quant_act_rows(xb, K, np.where(s == 0, 1, s).astype(np.float32), row_begin=P, want_tie_dist=True)
+    for m in range(P, M):
+        # a single row is a one-row tensor: the per-tensor routines (pinned above) give its step and its codes
+        assert s[m] == orc.calib_act_scale(xb[m:m + 1], K)
+        ref, t1 = orc.quant_act(xb[m:m + 1], K, s[m], want_tie_dist=True)
+        assert np.array_equal(codes[m:m + 1], ref) and np.array_equal(tie[m:m + 1], t1)
+        if m != 4:
+            assert np.abs(orc.unpack_int4(codes[m:m + 1])).max() == 7, "every token uses its full range"
+    assert np.all(codes[:P] == 0) and np.all(codes[4] == 0)
+    # the clipping factor is shared by the tokens of a layer and scales every step
+    s_half = orc.dyn_act_scale(xb, K, 0.5, row_begin=P)
+    live = np.arange(M) != 4
+    assert np.allclose(s_half[P:][live[P:]], 0.5 * s[P:][live[P:]], rtol=2e-7)
+    # dynamic means scale-free: a token multiplied by 2^k keeps its codes, its step takes the factor
+    x2 = x.clone()
+    x2[3] *= 8
+    s2 = orc.dyn_act_scale(inputs.bits(x2), K, 1.0, row_begin=P)
+    c2 = orc.quant_act_rows(inputs.bits(x2), K, np.where(s2 == 0, 1, s2).astype(np.float32), row_begin=P)
+    assert s2[3] == 8 * s[3] and np.array_equal(c2, codes)
+    # epilogue: a constant per-token step is the static epilogue
+    acc = rng.integers(-(1 << 20), 1 << 20, (M, 9)).astype(np.int32)
+    s_w = (rng.random(9) * 0.01 + 0.001).astype(np.float32)
+    assert np.array_equal(orc.dequant_bf16_rows(acc, np.full(M, 0.37, np.float32), s_w), orc.dequant_bf16(acc, np.float32(0.37), s_w))
+    got = orc.bf16_to_f64(orc.dequant_bf16_rows(acc, s.clip(1e-3), s_w))
+    want = acc.astype(np.float64) * s.clip(1e-3).astype(np.float64)[:, None] * s_w.astype(np.float64)[None, :]
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0**-8 + 1e-30)
+
+
 def test_dequant_epilogue_closed_form_and_one_rounding():
     acc = np.array([[3, -5, 0, 1 << 20]], np.int32)
     s_w = np.array([0.25, 0.5, 7.0, 2.0**-10], np.float32)
