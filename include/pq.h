@@ -122,6 +122,24 @@ pq_status pq_w4a8_gemm(pq_ctx* ctx, const int8_t* xq8, const uint8_t* wq, const 
                        int64_t ldo, int64_t M, int64_t N, int64_t K, int64_t row_begin, int32_t* acc_dbg, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Per-token dynamic activations (Table 1, O1; Sec. 3 "Dynamic and Static": the step is computed online
+ * from every token instead of offline per tensor). Symmetric form of Eq. 1 with one clipping factor per
+ * layer shared by all tokens:
+ *     s_tok[t] = clip * max_k |y[t, k]| / 7          pq_dyn_act_scale   (first pass; 0 < clip <= 1)
+ *     xq[t, :] = pack(clamp(rne(y[t, :] / s_tok[t]), -8, 7))   pq_hadamard_quant_act_rows (second pass)
+ *     out[t, n] = bf16(acc[t, n] * s_tok[t] * s_w[n])          pq_w4a4_gemm_rows
+ *   s_tok  f32 [M] on the device; rows below row_begin are neither read nor written; an all-zero row
+ *   gets step 0 and codes 0. Every other argument as in the static calls. The GEMM uses the
+ *   tensor-core kernel with the token operand in shared memory for every K (M - row_begin > 16). */
+pq_status pq_dyn_act_scale(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                           int64_t row_begin, float clip, float* s_tok, void* stream);
+pq_status pq_hadamard_quant_act_rows(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                     int64_t row_begin, const float* s_tok, uint8_t* xq, void* stream);
+pq_status pq_w4a4_gemm_rows(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_tok, const float* s_w,
+                            void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int64_t row_begin,
+                            int32_t* acc_dbg, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * KV cache with a full-precision prefix region and a 4-bit region (Sec. 4.2, Eq. 3; Table 1, O2:
  * per-head static KV scales). All buffers are the caller's.
  *   prefix_k, prefix_v  fp16 [Hkv, n_prefix, D]  K/V of the prefixed tokens, computed once by the

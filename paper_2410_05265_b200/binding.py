@@ -26,6 +26,7 @@ EXPORTS = [
     "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix", "pq_decode_attn_kv4_prefix_noalloc",
     "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add", "pq_prefill_attn_kv4_prefix", "pq_kv4_append_strided", "pq_calib_kv_scale",
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
+    "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows",
 ]
 
 
@@ -87,6 +88,9 @@ def load_library() -> ctypes.CDLL:
     lib.pq_calib_act_scale8.argtypes = lib.pq_calib_act_scale.argtypes
     lib.pq_w4a8_gemm.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int64,
                                  c_int64, c_void_p, c_void_p]
+    lib.pq_dyn_act_scale.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_float, c_void_p, c_void_p]
+    lib.pq_hadamard_quant_act_rows.argtypes = lib.pq_hadamard_quant_act.argtypes
+    lib.pq_w4a4_gemm_rows.argtypes = lib.pq_w4a8_gemm.argtypes
     for name in EXPORTS:
         getattr(lib, name)
         if name not in ("pq_status_string", "pq_w4a4_gemm_workspace_bytes", "pq_decode_attn_workspace_bytes"):
@@ -211,6 +215,44 @@ class Context:
             assert acc_dbg.shape == (M, N) and acc_dbg.is_contiguous()
         _ok(self.lib.pq_w4a4_gemm(self.h, _ptr(xq), _ptr(wq), _ptr(s_a), _ptr(s_w), _ptr(out), out.stride(0), M, N, K2 * 2,
                                   row_begin, _ptr(acc_dbg), c_void_p(0), 0, _stream()), "pq_w4a4_gemm")
+        return out
+
+    # ---- per-token dynamic activations (Table 1, O1) ---------------------------------------------------
+    def dyn_act_scale(self, x: torch.Tensor, had_block: int, clip: float = 1.0, row_begin: int = 0, out: torch.Tensor | None = None):
+        _dev(x, torch.bfloat16, "x")
+        M, K = x.shape
+        if out is None:
+            out = torch.zeros((M,), dtype=torch.float32, device=x.device)
+        _dev(out, torch.float32, "out")
+        _ok(self.lib.pq_dyn_act_scale(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, float(clip), _ptr(out), _stream()),
+            "pq_dyn_act_scale")
+        return out
+
+    def hadamard_quant_act_rows(self, x: torch.Tensor, had_block: int, s_tok: torch.Tensor, row_begin: int = 0,
+                                out: torch.Tensor | None = None):
+        _dev(x, torch.bfloat16, "x"), _dev(s_tok, torch.float32, "s_tok")
+        M, K = x.shape
+        assert x.stride(1) == 1 and s_tok.shape == (M,) and s_tok.is_contiguous()
+        if out is None:
+            out = torch.zeros((M, K // 2), dtype=torch.uint8, device=x.device)
+        _ok(self.lib.pq_hadamard_quant_act_rows(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, _ptr(s_tok), _ptr(out),
+                                                _stream()), "pq_hadamard_quant_act_rows")
+        return out
+
+    def w4a4_gemm_rows(self, xq: torch.Tensor, wq: torch.Tensor, s_tok: torch.Tensor, s_w: torch.Tensor, row_begin: int = 0,
+                       out: torch.Tensor | None = None, acc_dbg: torch.Tensor | None = None):
+        _dev(xq, torch.uint8, "xq"), _dev(wq, torch.uint8, "wq")
+        _dev(s_tok, torch.float32, "s_tok"), _dev(s_w, torch.float32, "s_w")
+        M, K2 = xq.shape
+        N = wq.shape[0]
+        assert wq.shape[1] == K2 and xq.is_contiguous() and wq.is_contiguous() and s_tok.shape == (M,) and s_tok.is_contiguous()
+        if out is None:
+            out = torch.zeros((M, N), dtype=torch.bfloat16, device=xq.device)
+        if acc_dbg is not None:
+            _dev(acc_dbg, torch.int32, "acc_dbg")
+            assert acc_dbg.shape == (M, N) and acc_dbg.is_contiguous()
+        _ok(self.lib.pq_w4a4_gemm_rows(self.h, _ptr(xq), _ptr(wq), _ptr(s_tok), _ptr(s_w), _ptr(out), out.stride(0), M, N, K2 * 2,
+                                       row_begin, _ptr(acc_dbg), _stream()), "pq_w4a4_gemm_rows")
         return out
 
     # ---- W4A8: 8-bit activation codes, one signed byte per element (Sec. 5.1) -------------------------

@@ -99,6 +99,7 @@ constexpr size_t SMEM_BYTES =
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 struct GemmParams {
+  const float* s_row;  // per-token steps [M] (dynamic setting) or null: the scalar s_a applies
   const float* s_a;
   const float* s_w;
   __nv_bfloat16* out;
@@ -418,7 +419,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
     // ------------------------------------------------------------------ epilogue warps
     constexpr int SHIFT = A8 ? 4 : 8;  // the factors 16 the expanded codes carry
     const int q = warp & 3;  // TMEM lane quarter this warp may access
-    const float s_a = __ldg(p.s_a);
+    const float s_a = p.s_row ? 1.0f : __ldg(p.s_a);
     uint8_t* my_buf = epi_buf + q * EPI_BUFS * EPI_BUF;
     float* my_scale = scale_buf + q * BN;
     uint32_t tcount = 0, n_store = 0;
@@ -441,6 +442,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
       }
       pq::tc_fence_after();
       const int row = m0 + lane;
+      const float rs = p.s_row ? (row < p.M ? __ldg(p.s_row + row) : 0.0f) : 1.0f;  // this lane's token step
       const uint32_t taddr = tmem_base + ab * BN + (static_cast<uint32_t>(q * 32) << 16);
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
@@ -464,14 +466,14 @@ __global__ void __launch_bounds__(N_THREADS, 1)
             const float4 sa = *reinterpret_cast<const float4*>(my_scale + c * 32 + g * 8);
             const float4 sb = *reinterpret_cast<const float4*>(my_scale + c * 32 + g * 8 + 4);
             const int b = g * 8;
-            const __nv_bfloat162 p0 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 0]) >> SHIFT) * sa.x,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 1]) >> SHIFT) * sa.y);
-            const __nv_bfloat162 p1 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 2]) >> SHIFT) * sa.z,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 3]) >> SHIFT) * sa.w);
-            const __nv_bfloat162 p2 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 4]) >> SHIFT) * sb.x,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 5]) >> SHIFT) * sb.y);
-            const __nv_bfloat162 p3 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 6]) >> SHIFT) * sb.z,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 7]) >> SHIFT) * sb.w);
+            const __nv_bfloat162 p0 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 0]) >> SHIFT) * sa.x * rs,
+                                                            static_cast<float>(static_cast<int32_t>(r[b + 1]) >> SHIFT) * sa.y * rs);
+            const __nv_bfloat162 p1 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 2]) >> SHIFT) * sa.z * rs,
+                                                            static_cast<float>(static_cast<int32_t>(r[b + 3]) >> SHIFT) * sa.w * rs);
+            const __nv_bfloat162 p2 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 4]) >> SHIFT) * sb.x * rs,
+                                                            static_cast<float>(static_cast<int32_t>(r[b + 5]) >> SHIFT) * sb.y * rs);
+            const __nv_bfloat162 p3 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 6]) >> SHIFT) * sb.z * rs,
+                                                            static_cast<float>(static_cast<int32_t>(r[b + 7]) >> SHIFT) * sb.w * rs);
             const int chunk = (c & 1) * 4 + g;  // 16-byte chunk inside the 128-byte staging row
             *reinterpret_cast<uint4*>(buf + lane * 128 + ((chunk ^ (lane & 7)) << 4)) =
                 make_uint4(*reinterpret_cast<const uint32_t*>(&p0), *reinterpret_cast<const uint32_t*>(&p1),
@@ -492,7 +494,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
             const int col = col0 + i;
             if (col < p.N)
               p.out[static_cast<int64_t>(row) * p.ldo + col] =
-                  __float2bfloat16_rn(static_cast<float>(static_cast<int32_t>(r[i]) >> SHIFT) * my_scale[c * 32 + i]);
+                  __float2bfloat16_rn(static_cast<float>(static_cast<int32_t>(r[i]) >> SHIFT) * my_scale[c * 32 + i] * rs);
           }
         }
         if (p.acc_dbg && row < p.M) {
@@ -565,9 +567,10 @@ bool make_out_map(pq_ctx* ctx, CUtensorMap* map, void* out, int64_t M, int64_t N
 
 // Launches the CTA-pair kernel on rows [0, M) of xq/out (the caller has already applied row_begin).
 // a8: xq holds one s8 code per element ([M, K] bytes) instead of packed nibbles.
+// s_row: per-token steps (then s_a is ignored), or null.
 pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
                               void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg,
-                              cudaStream_t st, bool a8) {
+                              cudaStream_t st, bool a8, const float* s_row) {
   CUtensorMap ta, tb, to;
   if (!(a8 ? make_s8_map(ctx, &ta, xq, M, K) : make_packed_map(ctx, &ta, xq, M, K / 2, BM_CTA)) ||
       !make_packed_map(ctx, &tb, wq, N, K / 2, BN_CTA))
@@ -579,6 +582,7 @@ pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq,
   } else {
     to = ta;  // never dereferenced
   }
+  p.s_row = s_row;
   p.s_a = s_a;
   p.s_w = s_w;
   p.out = static_cast<__nv_bfloat16*>(out);

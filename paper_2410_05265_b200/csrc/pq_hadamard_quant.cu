@@ -22,10 +22,13 @@ constexpr int HQ_CTAS_PER_SM = 5;         // 33 KB of shared memory and about 11
 constexpr int HQ_ELEMS = HQ_THREADS * 64;             // elements handled per CTA iteration
 constexpr int HQ_SMEM_FLOATS = HQ_ELEMS + HQ_ELEMS / 64;  // + 2 floats of padding per 128
 
-template <int LOGB, bool ROTATE, bool CALIB, int BITS>
+// PER_TOKEN (the dynamic setting, Table 1, O1): one step per row instead of one per tensor; s_a_in / s_a_out
+// are then arrays indexed by row, and the calibration pass is the online first pass of every call.
+template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN>
 __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
     hadamard_quant_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int64_t n_rows, int64_t K,
-                          const float* __restrict__ s_a_in, uint8_t* __restrict__ xq, float* __restrict__ s_a_out) {
+                          const float* __restrict__ s_a_in, uint8_t* __restrict__ xq, float* __restrict__ s_a_out,
+                          float clip) {
   static_assert(BITS == 4 || BITS == 8, "code width");
   constexpr int QMAX = BITS == 4 ? 7 : 127;  // codes lie in [-QMAX - 1, QMAX]
   constexpr int B = 1 << LOGB;
@@ -54,7 +57,7 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
 
   const float norm = ROTATE ? __fdiv_rn(1.0f, __fsqrt_rn(static_cast<float>(B))) : 1.0f;
   float inv = norm;
-  if (!CALIB) inv = __fdiv_rn(norm, __ldg(s_a_in));
+  if (!CALIB && !PER_TOKEN) inv = __fdiv_rn(norm, __ldg(s_a_in));
   float cal_max = 0.0f;
 
   for (int64_t sb = blockIdx.x; sb < n_super; sb += gridDim.x) {
@@ -62,6 +65,10 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
     const bool active = gb < total_blocks;
     const int64_t row = active ? gb / blocks_per_row : 0;
     const int64_t col0 = active ? (gb % blocks_per_row) * B : 0;
+    if (!CALIB && PER_TOKEN) {
+      const float s_row = __ldg(s_a_in + row);
+      inv = __fdiv_rn(norm, s_row == 0.0f ? 1.0f : s_row);  // an all-zero row has no step: any will do
+    }
 
     // ---- pass 1 --------------------------------------------------------------------------
     // V[r] = (x[2u + r*RSTRIDE], x[2u+1 + r*RSTRIDE]) after the stage on index bit 0; the other five
@@ -138,9 +145,21 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
       }
     }
     if (CALIB) {
+      float it_max = 0.0f;
       if (active) {
 #pragma unroll
-        for (int q = 0; q < 32; ++q) cal_max = fmaxf(cal_max, fmaxf(fabsf(W[q].x * norm), fabsf(W[q].y * norm)));
+        for (int q = 0; q < 32; ++q) it_max = fmaxf(it_max, fmaxf(fabsf(W[q].x * norm), fabsf(W[q].y * norm)));
+      }
+      if (PER_TOKEN) {
+        // the maximum of this row's block, over the TPB threads that hold it (a warp or a part of one; blocks
+        // wider than a warp's 2048 elements, and rows of several blocks, meet in the atomic)
+        constexpr int SPAN = TPB < 32 ? TPB : 32;
+#pragma unroll
+        for (int o = SPAN / 2; o > 0; o >>= 1) it_max = fmaxf(it_max, __shfl_xor_sync(0xffffffffu, it_max, o));
+        if ((tid % SPAN) == 0 && active && it_max > 0.0f)
+          atomicMax(reinterpret_cast<int*>(s_a_out + row), __float_as_int(__fdiv_rn(it_max * clip, static_cast<float>(QMAX))));
+      } else {
+        cal_max = fmaxf(cal_max, it_max);
       }
     } else {
       // ---- quantize and pack -----------------------------------------------------------------
@@ -194,17 +213,17 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
       }
     }
   }
-  if (CALIB) {
+  if (CALIB && !PER_TOKEN) {
     for (int o = 16; o > 0; o >>= 1) cal_max = fmaxf(cal_max, __shfl_xor_sync(0xffffffffu, cal_max, o));
     if ((tid & 31) == 0 && cal_max > 0.0f)
       atomicMax(reinterpret_cast<int*>(s_a_out), __float_as_int(__fdiv_rn(cal_max, static_cast<float>(QMAX))));
   }
 }
 
-template <int LOGB, bool ROTATE, bool CALIB, int BITS>
+template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN>
 pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_t K, const float* s_a_in, uint8_t* xq,
-                 float* s_a_out, cudaStream_t st) {
-  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS>;
+                 float* s_a_out, float clip, cudaStream_t st) {
+  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN>;
   constexpr size_t smem = HQ_SMEM_FLOATS * sizeof(float);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
     return PQ_ERR_CUDA;
@@ -224,14 +243,15 @@ pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x), ldx, n_rows, K, s_a_in, xq, s_a_out) != cudaSuccess)
+  if (cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x), ldx, n_rows, K, s_a_in, xq, s_a_out, clip) !=
+      cudaSuccess)
     return PQ_ERR_CUDA;
   return pq_launch_status();
 }
 
-template <bool CALIB, int BITS>
+template <bool CALIB, int BITS, bool PER_TOKEN = false>
 pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block, int64_t row_begin,
-                   const float* s_a_in, uint8_t* xq, float* s_a_out, void* stream) {
+                   const float* s_a_in, uint8_t* xq, float* s_a_out, void* stream, float clip = 1.0f) {
   if (!ctx || !x || (!CALIB && (!s_a_in || !xq)) || (CALIB && !s_a_out)) return PQ_ERR_INVALID_ARG;
   if (M < 0 || K <= 0 || ldx < K || row_begin < 0 || had_block < 0) return PQ_ERR_INVALID_ARG;
   if (K % 128 != 0) return PQ_ERR_SHAPE;
@@ -246,15 +266,20 @@ pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx
   const void* x0 = static_cast<const __nv_bfloat16*>(x) + row_begin * ldx;
   uint8_t* xq0 = CALIB ? nullptr : xq + row_begin * (BITS == 4 ? K / 2 : K);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (PER_TOKEN) {  // the arrays are indexed by row
+    if (s_a_in) s_a_in += row_begin;
+    if (s_a_out) s_a_out += row_begin;
+    if (CALIB && cudaMemsetAsync(s_a_out, 0, static_cast<size_t>(n_rows) * sizeof(float), st) != cudaSuccess) return PQ_ERR_CUDA;
+  }
   switch (had_block) {
-    case 0: return launch<7, false, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 128: return launch<7, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 256: return launch<8, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 512: return launch<9, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 1024: return launch<10, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 2048: return launch<11, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 4096: return launch<12, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
-    case 8192: return launch<13, true, CALIB, BITS>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, st);
+    case 0: return launch<7, false, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
+    case 128: return launch<7, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
+    case 256: return launch<8, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
+    case 512: return launch<9, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
+    case 1024: return launch<10, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
+    case 2048: return launch<11, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
+    case 4096: return launch<12, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
+    case 8192: return launch<13, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
     default: return PQ_ERR_SHAPE;
   }
 }
@@ -281,4 +306,17 @@ extern "C" pq_status pq_hadamard_quant_act8(pq_ctx* ctx, const void* x, int64_t 
 extern "C" pq_status pq_calib_act_scale8(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
                                          int64_t row_begin, float* s_a, void* stream) {
   return dispatch<true, 8>(ctx, x, M, K, ldx, had_block, row_begin, nullptr, nullptr, s_a, stream);
+}
+
+// ---- per-token dynamic activations (Table 1, O1): the step of a row is computed online from the row ----
+extern "C" pq_status pq_dyn_act_scale(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                      int64_t row_begin, float clip, float* s_tok, void* stream) {
+  if (!(clip > 0.0f) || !(clip <= 1.0f)) return PQ_ERR_INVALID_ARG;
+  return dispatch<true, 4, true>(ctx, x, M, K, ldx, had_block, row_begin, nullptr, nullptr, s_tok, stream, clip);
+}
+
+extern "C" pq_status pq_hadamard_quant_act_rows(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx,
+                                                int had_block, int64_t row_begin, const float* s_tok, uint8_t* xq,
+                                                void* stream) {
+  return dispatch<false, 4, true>(ctx, x, M, K, ldx, had_block, row_begin, s_tok, xq, nullptr, stream);
 }
