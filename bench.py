@@ -263,6 +263,7 @@ def run_gpu(args):
         sections = {}
         try:
             sections["w4a8_prefill_linear_set"] = section_w4a8(ctx, device, peaks, acts, wqs, sws)
+            sections["w4a4_dynamic_per_token_linear_set"] = section_dynamic(ctx, device, peaks, acts, wqs, sws)
             sections["decode_gemm"] = section_decode_gemm(ctx, device, peaks)
             sections["decode_attention"] = section_decode_attention(ctx, device, peaks)
             sections["block_llama3_70b_prefill4096"] = section_block(ctx, device, peaks)
@@ -452,6 +453,40 @@ def section_w4a8(ctx, device, peaks, acts, wqs, sws):
             "per_launch": {k: {"ms": round(statistics.mean(v), 4),
                                "tops": round(2.0 * m_rows * next(n * kk for nm, n, kk, _, _ in L if nm == k) / (statistics.mean(v) * 1e-3) / 1e12, 1)}
                            for k, v in per.items()}}
+
+
+def section_dynamic(ctx, device, peaks, acts, wqs, sws):
+    """The linear set of configs[1] in the per-token dynamic setting (Table 1, O1): per linear one pass for the
+    token steps, one for the codes, then the GEMM with the per-token epilogue. The paper's comparison
+    setting: it reports the static path as the faster one."""
+    import torch
+
+    L = linear_launches()
+    m_rows = M_TOKENS - N_PREFIX
+    s_tok = [torch.zeros((M_TOKENS,), dtype=torch.float32, device=device) for _ in L]
+    xqs = [torch.zeros((M_TOKENS, K // 2), dtype=torch.uint8, device=device) for _, _, K, _, _ in L]
+    outs = [torch.zeros((M_TOKENS, N), dtype=torch.bfloat16, device=device) for _, N, _, _, _ in L]
+
+    def step():
+        for i, (name, N, K, had, inp) in enumerate(L):
+            ctx.dyn_act_scale(acts[i], had, 1.0, N_PREFIX, out=s_tok[i])
+            ctx.hadamard_quant_act_rows(acts[i], had, s_tok[i], N_PREFIX, out=xqs[i])
+            ctx.w4a4_gemm_rows(xqs[i], wqs[i], s_tok[i], sws[i], N_PREFIX, out=outs[i])
+
+    steps = 50
+    for _ in range(5):
+        step()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        step()
+    t1.record()
+    torch.cuda.synchronize()
+    ctx.check()
+    ms = t0.elapsed_time(t1) / steps
+    return {"ms_per_step": round(ms, 4), "TOPS": round(step_ops(m_rows) / (ms * 1e-3) / 1e12, 1),
+            "launches_per_step": "4 x (dyn_act_scale + memset + hadamard_quant_act_rows + w4a4_gemm_rows)"}
 
 
 def section_block(ctx, device, peaks):
