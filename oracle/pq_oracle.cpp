@@ -376,6 +376,33 @@ void orc_dequant_bf16_rows(const int32_t* acc, int64_t M, int64_t N, const float
   });
 }
 
+// ---- outlier tokens (Sec. 4.1, "Definition of Outlier Token", Eq. 2) ------------------------------------
+// M[i] = max_c |X[i,c]|; R[i] = M[i] / median(M); token i is an upper outlier when R[i] > eta1 and a lower
+// outlier when 1 / R[i] > eta2 (flags 1 and 2, else 0). The median of an even number of tokens is the mean
+// of the two middle values. M is exact (bf16 inputs); the median and the two ratios M / median and
+// median / M are rounded to fp32, the precision in which the thresholds are compared.
+void orc_outlier_tokens(const uint16_t* x, int64_t ldx, int64_t T, int64_t C, float eta1, float eta2, float* M, float* R,
+                        int32_t* flags, float* median_out) {
+  std::vector<float> m(T);
+  for (int64_t i = 0; i < T; ++i) {
+    double mx = 0.0;
+    for (int64_t c = 0; c < C; ++c) mx = std::max(mx, std::fabs(bf16_to_double(x[i * ldx + c])));
+    m[i] = static_cast<float>(mx);
+    M[i] = m[i];
+  }
+  std::vector<float> sorted(m);
+  std::sort(sorted.begin(), sorted.end());
+  const float med = T == 0 ? 0.0f
+                           : static_cast<float>(0.5 * (static_cast<double>(sorted[(T - 1) / 2]) + static_cast<double>(sorted[T / 2])));
+  *median_out = med;
+  for (int64_t i = 0; i < T; ++i) {
+    const float r = static_cast<float>(static_cast<double>(m[i]) / static_cast<double>(med));
+    const float inv = static_cast<float>(static_cast<double>(med) / static_cast<double>(m[i]));
+    R[i] = r;
+    flags[i] = r > eta1 ? 1 : (inv > eta2 ? 2 : 0);
+  }
+}
+
 // ---- per-head static KV scale and KV4 append (Table 1, O2: per-head static KV cache) ----------
 // kv bf16 [B,T,H,D]; s[h] = fp32(max |kv[:,:,h,:]|) / 7 in double then fp32 (1 if all zero).
 void orc_calib_kv_scale(const uint16_t* kv, int64_t B, int64_t T, int64_t H, int64_t D, float* s) {

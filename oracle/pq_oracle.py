@@ -216,6 +216,17 @@ def dequant_bf16_rows(acc: np.ndarray, s_tok: np.ndarray, s_w: np.ndarray) -> np
     return out
 
 
+def outlier_tokens(x_bits: np.ndarray, eta1: float = 64.0, eta2: float = 8.0):
+    """Token-wise maxima M, outlier degrees R = M / median(M), flags (1 upper, 2 lower, 0 neither) and the median."""
+    x_bits = _u16(x_bits)
+    T, C = x_bits.shape
+    M, R = np.empty(T, np.float32), np.empty(T, np.float32)
+    flags, med = np.empty(T, np.int32), np.zeros(1, np.float32)
+    lib().orc_outlier_tokens(_p(x_bits, c_uint16), c_int64(C), c_int64(T), c_int64(C), c_float(eta1), c_float(eta2),
+                             _p(M, c_float), _p(R, c_float), _p(flags, c_int32), _p(med, c_float))
+    return M, R, flags, float(med[0])
+
+
 # ---- weights ---------------------------------------------------------------------------------------
 def quant_weights(w_bits: np.ndarray):
     w_bits = _u16(w_bits)

@@ -334,6 +334,41 @@ def test_dynamic_per_token_quantizer_reduces_to_the_static_one_row_by_row():
     assert np.all(np.abs(got - want) <= np.abs(want) * 2.0**-8 + 1e-30)
 
 
+# ---------------------------------------------------------------- outlier tokens (Sec. 4.1, Eq. 2)
+def test_outlier_tokens_hand_example_library_median_and_invariances():
+    # six tokens with maxima 1, 2, 3, 4, 200, 0.25: median 2.5; R = 0.4, 0.8, 1.2, 1.6, 80, 0.1
+    rows = np.zeros((6, 8))
+    for i, m in enumerate([1, 2, 3, 4, 200, 0.25]):
+        rows[i, i] = -m if i % 2 else m  # the maximum is of absolute values
+        rows[i, 7] = 0.125 * (1 if i % 2 else -1)
+    M, R, flags, med = orc.outlier_tokens(bf16_bits(rows))
+    assert M.tolist() == [1, 2, 3, 4, 200, 0.25] and med == 2.5
+    assert np.allclose(R, [0.4, 0.8, 1.2, 1.6, 80, 0.1], rtol=1e-6)
+    assert flags.tolist() == [0, 0, 0, 0, 1, 2]  # 80 > 64 is an upper outlier, 1 / 0.1 = 10 > 8 a lower one
+    # thresholds are strict and can be moved
+    assert orc.outlier_tokens(bf16_bits(rows), eta1=80.0, eta2=10.0)[2].tolist() == [0, 0, 0, 0, 0, 0]
+    assert orc.outlier_tokens(bf16_bits(rows), eta1=1.5, eta2=2.4)[2].tolist() == [2, 0, 0, 1, 1, 2]
+    # against numpy on a random batch: odd and even token counts
+    for T in (33, 64):
+        x = inputs.activations(T, 256, seed=6)
+        xb = inputs.bits(x)
+        M, R, flags, med = orc.outlier_tokens(xb)
+        Mref = np.abs(x.to(torch.float64).numpy()).max(1)
+        assert np.array_equal(M, Mref.astype(np.float32)) and med == np.float32(np.median(Mref))
+        assert np.allclose(R, Mref / np.median(Mref), rtol=2e-7)
+        # token order does not matter, a common factor does not matter
+        perm = rng.permutation(T)
+        M2, R2, f2, med2 = orc.outlier_tokens(xb[perm])
+        assert np.array_equal(R2, R[perm]) and np.array_equal(f2, flags[perm]) and med2 == med
+        _, R3, f3, med3 = orc.outlier_tokens(inputs.bits(x * 4))
+        assert np.array_equal(R3, R) and np.array_equal(f3, flags) and med3 == 4 * med
+    # the synthetic prefix rows (1000 times larger) are exactly the upper outliers; a silent token is a lower one
+    x = inputs.activations(40, 512, seed=1, n_prefix=4)
+    x[17] *= 0.01
+    flags = orc.outlier_tokens(inputs.bits(x))[2]
+    assert flags[:4].tolist() == [1, 1, 1, 1] and flags[17] == 2 and int((flags != 0).sum()) == 5
+
+
 def test_dequant_epilogue_closed_form_and_one_rounding():
     acc = np.array([[3, -5, 0, 1 << 20]], np.int32)
     s_w = np.array([0.25, 0.5, 7.0, 2.0**-10], np.float32)
