@@ -251,6 +251,18 @@ pq_status pq_residual_add(pq_ctx* ctx, const void* a, const void* b, void* y, in
 pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache, const void* q, void* out, float sm_scale,
                                             void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Outlier tokens (Sec. 4.1, "Definition of Outlier Token", Eq. 2), the cheap part of the offline analysis
+ * that decides which tokens are prefixed:
+ *     M[i] = max_c |x[i, c]|,  R[i] = M[i] / median(M),
+ *     flags[i] = 1 (upper outlier) when R[i] > eta1, 2 (lower outlier) when 1 / R[i] > eta2, else 0
+ *   x bf16 [T, C], row stride ldx (16-byte aligned, C and ldx multiples of 8), T <= 8192;
+ *   M, R f32 [T], flags int32 [T], median f32 scalar, all on the device. The median of an even number of
+ *   tokens is the mean of the two middle values; ratios and comparisons are fp32. The paper uses
+ *   eta1 = 64, eta2 = 8. */
+pq_status pq_outlier_tokens(pq_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ldx, float eta1, float eta2, float* M,
+                            float* R, int32_t* flags, float* median, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -26,7 +26,7 @@ EXPORTS = [
     "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix", "pq_decode_attn_kv4_prefix_noalloc",
     "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add", "pq_prefill_attn_kv4_prefix", "pq_kv4_append_strided", "pq_calib_kv_scale",
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
-    "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows",
+    "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
 ]
 
 
@@ -91,6 +91,8 @@ def load_library() -> ctypes.CDLL:
     lib.pq_dyn_act_scale.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_float, c_void_p, c_void_p]
     lib.pq_hadamard_quant_act_rows.argtypes = lib.pq_hadamard_quant_act.argtypes
     lib.pq_w4a4_gemm_rows.argtypes = lib.pq_w4a8_gemm.argtypes
+    lib.pq_outlier_tokens.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_float, c_float, c_void_p, c_void_p, c_void_p,
+                                      c_void_p, c_void_p]
     for name in EXPORTS:
         getattr(lib, name)
         if name not in ("pq_status_string", "pq_w4a4_gemm_workspace_bytes", "pq_decode_attn_workspace_bytes"):
@@ -216,6 +218,20 @@ class Context:
         _ok(self.lib.pq_w4a4_gemm(self.h, _ptr(xq), _ptr(wq), _ptr(s_a), _ptr(s_w), _ptr(out), out.stride(0), M, N, K2 * 2,
                                   row_begin, _ptr(acc_dbg), c_void_p(0), 0, _stream()), "pq_w4a4_gemm")
         return out
+
+    # ---- offline analysis: outlier tokens (Sec. 4.1, Eq. 2) -------------------------------------------
+    def outlier_tokens(self, x: torch.Tensor, eta1: float = 64.0, eta2: float = 8.0):
+        """Returns (M, R, flags, median) for x bf16 [T, C]: token maxima, outlier degrees, 1/2/0 flags."""
+        _dev(x, torch.bfloat16, "x")
+        T, C = x.shape
+        assert x.stride(1) == 1
+        M = torch.empty((T,), dtype=torch.float32, device=x.device)
+        R = torch.empty_like(M)
+        flags = torch.empty((T,), dtype=torch.int32, device=x.device)
+        med = torch.empty((1,), dtype=torch.float32, device=x.device)
+        _ok(self.lib.pq_outlier_tokens(self.h, _ptr(x), T, C, x.stride(0), float(eta1), float(eta2), _ptr(M), _ptr(R), _ptr(flags),
+                                       _ptr(med), _stream()), "pq_outlier_tokens")
+        return M, R, flags, med
 
     # ---- per-token dynamic activations (Table 1, O1) ---------------------------------------------------
     def dyn_act_scale(self, x: torch.Tensor, had_block: int, clip: float = 1.0, row_begin: int = 0, out: torch.Tensor | None = None):

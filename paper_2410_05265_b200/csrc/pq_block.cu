@@ -289,3 +289,72 @@ extern "C" pq_status pq_calib_kv_scale(pq_ctx* ctx, const void* x, int64_t n_tok
       static_cast<const __nv_bfloat16*>(x), n_tok, Hkv, ld_tok, s);
   return pq_launch_status();
 }
+
+// ================================================================================= outlier tokens
+// Sec. 4.1, Eq. 2: M[i] = max_c |X[i,c]|, R[i] = M[i] / median(M); an upper outlier has R > eta1, a lower one
+// 1 / R > eta2. Two launches: a warp per token takes the maximum of the absolute values (the bf16 pattern
+// without its sign is monotone: integer maximum), then one CTA sorts the maxima in shared memory (bitonic, on
+// the fp32 bit patterns, all non-negative), takes the median (mean of the two middle values) and classifies.
+namespace {
+constexpr int OT_MAX_TOKENS = 8192;
+constexpr int OT_THREADS = 1024;
+
+__global__ void __launch_bounds__(256) token_absmax_kernel(const __nv_bfloat16* x, int64_t ldx, int64_t T, int64_t C, float* M) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= T) return;
+  const uint4* src = reinterpret_cast<const uint4*>(x + row * ldx);
+  uint32_t mx = 0;
+  for (int64_t i = lane; i < C / 8; i += 32) {
+    const uint4 v = __ldg(src + i);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) mx = max(mx, max(w[e] & 0x7FFFu, (w[e] >> 16) & 0x7FFFu));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if (lane == 0) M[row] = __uint_as_float(mx << 16);
+}
+
+__global__ void __launch_bounds__(OT_THREADS) outlier_classify_kernel(const float* M, int T, float eta1, float eta2, float* R,
+                                                                       int32_t* flags, float* median_out) {
+  __shared__ uint32_t key[OT_MAX_TOKENS];
+  int n = 1;
+  while (n < T) n <<= 1;
+  for (int i = threadIdx.x; i < n; i += OT_THREADS) key[i] = i < T ? __float_as_uint(M[i]) : 0xFFFFFFFFu;
+  __syncthreads();
+  for (int k = 2; k <= n; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = threadIdx.x; i < n; i += OT_THREADS) {
+        const int partner = i ^ j;
+        if (partner > i) {
+          const uint32_t a = key[i], b = key[partner];
+          const bool up = (i & k) == 0;
+          if ((a > b) == up) key[i] = b, key[partner] = a;
+        }
+      }
+      __syncthreads();
+    }
+  }
+  const float med = __fmul_rn(0.5f, __fadd_rn(__uint_as_float(key[(T - 1) / 2]), __uint_as_float(key[T / 2])));
+  if (threadIdx.x == 0) *median_out = med;
+  for (int i = threadIdx.x; i < T; i += OT_THREADS) {
+    const float m = M[i];
+    const float r = __fdiv_rn(m, med), inv = __fdiv_rn(med, m);
+    R[i] = r;
+    flags[i] = r > eta1 ? 1 : (inv > eta2 ? 2 : 0);
+  }
+}
+}  // namespace
+
+extern "C" pq_status pq_outlier_tokens(pq_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ldx, float eta1, float eta2,
+                                       float* M, float* R, int32_t* flags, float* median, void* stream) {
+  if (!ctx || !x || !M || !R || !flags || !median) return PQ_ERR_INVALID_ARG;
+  if (T <= 0 || C <= 0 || ldx < C || !(eta1 > 0.0f) || !(eta2 > 0.0f)) return PQ_ERR_INVALID_ARG;
+  if (T > OT_MAX_TOKENS || C % 8 != 0) return PQ_ERR_SHAPE;
+  if (!aligned16(x) || ldx % 8 != 0) return PQ_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  token_absmax_kernel<<<static_cast<unsigned>((T + 7) / 8), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), ldx, T, C, M);
+  outlier_classify_kernel<<<1, OT_THREADS, 0, st>>>(M, static_cast<int>(T), eta1, eta2, R, flags, median);
+  return pq_launch_status();
+}

@@ -358,3 +358,25 @@ def test_prefill_attention_matches_oracle(ctx, T, Hq, Hkv, P, mag):
     tol = 2e-3 * vmax + bf16_ulp(r) + 1e-30
     bad = np.abs(got - r) > tol
     assert not bad.any(), f"{bad.sum()} of {bad.size} outside tolerance; worst {np.max(np.abs(got - r) / np.maximum(vmax, 1e-30))}"
+
+
+# ------------------------------------------------------------------------------- outlier tokens (Sec. 4.1, Eq. 2)
+@pytest.mark.parametrize("T,C", [(1, 128), (33, 256), (64, 4096), (2048, 4096), (8192, 128)])
+def test_outlier_tokens_match_oracle_bit_for_bit(ctx, T, C):
+    x = inputs.activations(T, C, seed=3, n_prefix=min(4, T - 1))
+    if T > 20:
+        x[17] *= 0.01   # a lower outlier
+        x[9] = 0        # a silent token: 1 / R is infinite
+    M_ref, R_ref, f_ref, med_ref = orc.outlier_tokens(inputs.bits(x))
+    M, R, flags, med = ctx.outlier_tokens(x.cuda())
+    ctx.check()
+    assert np.array_equal(to_np(M), M_ref) and float(med) == med_ref
+    assert np.array_equal(to_np(R), R_ref, equal_nan=True) and np.array_equal(to_np(flags), f_ref)
+    if T > 20:
+        assert to_np(flags)[:4].tolist() == [1, 1, 1, 1] and int(flags[17]) == 2 and int(flags[9]) == 2
+    # a strided view (the first C columns of a wider matrix) gives the same answer
+    wide = torch.zeros((T, C + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, :C] = x.cuda()
+    wide[:, C:] = 1e6
+    _, R2, f2, _ = ctx.outlier_tokens(wide[:, :C])
+    assert torch.equal(f2, flags) and np.array_equal(to_np(R2), R_ref, equal_nan=True)
