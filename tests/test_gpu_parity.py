@@ -236,6 +236,15 @@ def test_decode_attention_ragged_lengths_and_empty_cache(ctx):
     _run_attention(ctx, 2, 8, 2, 0, 3, 64, 1.0, start=[0, 40])
 
 
+def test_decode_attention_short_sequences_in_long_caches(ctx):
+    """Most splits have nothing to do: their first round is requested before the length is known and must be
+    waited for and ignored (32 splits through the workspace; 8 splits merged inside a cluster)."""
+    _run_attention(ctx, 1, 8, 1, 2, 1, 8192, 1.0, start=[129])
+    _run_attention(ctx, 1, 8, 1, 0, 1, 8192, 1.0, start=[0])
+    _run_attention(ctx, 1, 4, 1, 3, 1, 8000, 1.0, start=[7935])   # the last rounds do not fit the allocation as a whole
+    _run_attention(ctx, 8, 32, 8, 4, 1, 4096, 1.0, start=[0, 10, 200, 1000, 127, 128, 129, 4000])
+
+
 def test_kv4_append_refuses_overflow(ctx):
     from paper_2410_05265_b200 import binding
 
