@@ -112,8 +112,9 @@ pq_status pq_w4a4_gemm(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const 
  *     *s_a = max(*s_a, max |y| / 127)                      calibration helper
  *     acc[t, n] = sum_k xq8[t, k] * wq[n, k]   exact, int32;   out[t, n] = bf16(acc * s_a * s_w[n])
  *   xq8  s8 [M, K] dense rows, base 16-byte aligned; every other argument as in the 4-bit calls.
- * The GEMM runs on the tensor-core kernel for every M (the token bytes go to the MMA operand
- * buffer untouched, only the weights are expanded); K % 32 == 0, K <= 65536. */
+ * Above 16 tokens the GEMM runs on the tensor-core kernel (the token bytes go to the MMA operand
+ * buffer untouched, only the weights are expanded), else on the weight-streaming kernel;
+ * K % 32 == 0, K <= 65536. */
 pq_status pq_hadamard_quant_act8(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
                                  int64_t row_begin, const float* s_a, int8_t* xq8, void* stream);
 pq_status pq_calib_act_scale8(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,

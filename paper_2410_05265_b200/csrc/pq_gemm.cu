@@ -9,7 +9,7 @@ pq_status pq_gemm_pair_ts_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* 
                                  void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st);
 pq_status pq_gemm_stream_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a,
                                 const float* s_w, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K,
-                                int32_t* acc_dbg, cudaStream_t st, bool per_token);
+                                int32_t* acc_dbg, cudaStream_t st, bool per_token, bool a8);
 
 extern "C" size_t pq_w4a4_gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
 
@@ -31,7 +31,7 @@ extern "C" pq_status pq_w4a4_gemm(pq_ctx* ctx, const uint8_t* xq, const uint8_t*
   int32_t* dbg0 = acc_dbg ? acc_dbg + row_begin * N : nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (K == 0) return PQ_ERR_SHAPE;
-  if (m <= 16) return pq_gemm_stream_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st, false);
+  if (m <= 16) return pq_gemm_stream_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st, false, false);
   // Two CTA-pair kernels: with the token operand in shared memory the accumulator is double-buffered
   // and the epilogue is free, which wins for short K; with the token operand in tensor memory the
   // expansion costs a third less shared-memory traffic, which wins once a tile's K loop is long enough
@@ -40,8 +40,8 @@ extern "C" pq_status pq_w4a4_gemm(pq_ctx* ctx, const uint8_t* xq, const uint8_t*
   return pq_gemm_pair_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st, false, nullptr);
 }
 
-// W4A8 (Sec. 5.1): the token operand is one s8 code per element. Every shape goes through the
-// CTA-pair tensor-core kernel (a tile of 256 token rows; short batches waste most of it).
+// W4A8 (Sec. 5.1): the token operand is one s8 code per element: the weight-streaming kernel for up to 16
+// tokens, the CTA-pair tensor-core kernel above that.
 extern "C" pq_status pq_w4a8_gemm(pq_ctx* ctx, const int8_t* xq8, const uint8_t* wq, const float* s_a,
                                   const float* s_w, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K,
                                   int64_t row_begin, int32_t* acc_dbg, void* stream) {
@@ -57,7 +57,9 @@ extern "C" pq_status pq_w4a8_gemm(pq_ctx* ctx, const int8_t* xq8, const uint8_t*
   const uint8_t* xq0 = reinterpret_cast<const uint8_t*>(xq8) + row_begin * K;
   void* out0 = static_cast<__nv_bfloat16*>(out) + row_begin * ldo;
   int32_t* dbg0 = acc_dbg ? acc_dbg + row_begin * N : nullptr;
-  return pq_gemm_pair_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, static_cast<cudaStream_t>(stream), true, nullptr);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (m <= 16) return pq_gemm_stream_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st, false, true);
+  return pq_gemm_pair_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st, true, nullptr);
 }
 
 // W4A4 with per-token dynamic activation steps (Table 1, O1): out[t,n] = bf16(acc * s_tok[t] * s_w[n]).
@@ -77,6 +79,6 @@ extern "C" pq_status pq_w4a4_gemm_rows(pq_ctx* ctx, const uint8_t* xq, const uin
   void* out0 = static_cast<__nv_bfloat16*>(out) + row_begin * ldo;
   int32_t* dbg0 = acc_dbg ? acc_dbg + row_begin * N : nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (m <= 16) return pq_gemm_stream_launch(ctx, xq0, wq, s0, s_w, out0, ldo, m, N, K, dbg0, st, true);
+  if (m <= 16) return pq_gemm_stream_launch(ctx, xq0, wq, s0, s_w, out0, ldo, m, N, K, dbg0, st, true, false);
   return pq_gemm_pair_launch(ctx, xq0, wq, nullptr, s_w, out0, ldo, m, N, K, dbg0, st, false, s0);
 }

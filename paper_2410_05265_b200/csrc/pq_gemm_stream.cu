@@ -40,9 +40,20 @@ __device__ __forceinline__ uint4 ld_stream(const uint8_t* p) {
   return v;
 }
 
+// 32 s8 activation codes of a K step (two 16-byte loads) in the order the expanded weights have: the
+// even-position codes of every eight in one word, the odd-position codes in the next. The value fed to the
+// MMA is the code itself (the weights carry their factor 16 alone: the sum is shifted by 4, not 8).
+__device__ __forceinline__ void permute_s8(const uint4& lo, const uint4& hi, uint32_t (&o)[8]) {
+  o[0] = __byte_perm(lo.x, lo.y, 0x6420), o[1] = __byte_perm(lo.x, lo.y, 0x7531);
+  o[2] = __byte_perm(lo.z, lo.w, 0x6420), o[3] = __byte_perm(lo.z, lo.w, 0x7531);
+  o[4] = __byte_perm(hi.x, hi.y, 0x6420), o[5] = __byte_perm(hi.x, hi.y, 0x7531);
+  o[6] = __byte_perm(hi.z, hi.w, 0x6420), o[7] = __byte_perm(hi.z, hi.w, 0x7531);
+}
+
 // HALF_ROWS: the CTA owns 8 output channels instead of 16 (rows 8..15 of the MMA tile stay zero), which
 // doubles the CTA count of narrow layers.
-template <bool TWO_GROUPS, bool HALF_ROWS>
+// A8: the token operand is one s8 code per element ([M, K] bytes) instead of packed nibbles (W4A8).
+template <bool TWO_GROUPS, bool HALF_ROWS, bool A8>
 __global__ void __launch_bounds__(GS_THREADS)
     gemm_w4a4_stream_kernel(const uint8_t* __restrict__ xq, const uint8_t* __restrict__ wq,
                             const float* __restrict__ s_a, const float* __restrict__ s_w,
@@ -60,8 +71,9 @@ __global__ void __launch_bounds__(GS_THREADS)
   const bool x0_ok = g < M, x1_ok = TWO_GROUPS && (g + 8 < M);
   const uint8_t* w0p = wq + static_cast<int64_t>(n0 + g) * kbytes + t * 16;
   const uint8_t* w1p = wq + static_cast<int64_t>(n0 + g + 8) * kbytes + t * 16;
-  const uint8_t* x0p = xq + static_cast<int64_t>(g) * kbytes + t * 16;
-  const uint8_t* x1p = xq + static_cast<int64_t>(g + 8) * kbytes + t * 16;
+  constexpr int XS = A8 ? 2 : 1;  // activation bytes per packed weight byte
+  const uint8_t* x0p = xq + (static_cast<int64_t>(g) * kbytes + t * 16) * XS;
+  const uint8_t* x1p = xq + (static_cast<int64_t>(g + 8) * kbytes + t * 16) * XS;
 
   int c0[4] = {0, 0, 0, 0}, c1[4] = {0, 0, 0, 0};
   const uint4 zero = make_uint4(0, 0, 0, 0);
@@ -73,6 +85,7 @@ __global__ void __launch_bounds__(GS_THREADS)
   bool first = true;
   for (int base = warp; base < n_steps; base += GS_WARPS * GS_UNROLL) {
     uint4 wa[GS_UNROLL], wb[GS_UNROLL], xa[GS_UNROLL], xb[GS_UNROLL];
+    uint4 xa2[A8 ? GS_UNROLL : 1], xb2[A8 ? GS_UNROLL : 1];  // second half of a lane's 32 s8 codes
 #pragma unroll
     for (int u = 0; u < GS_UNROLL; ++u) {
       const int ks = base + u * GS_WARPS;
@@ -90,19 +103,25 @@ __global__ void __launch_bounds__(GS_THREADS)
       const int ks = base + u * GS_WARPS;
       const int off = ks * 64;
       const bool in_k = ks < n_steps && off + t * 16 < kbytes;
-      xa[u] = (in_k && x0_ok) ? __ldg(reinterpret_cast<const uint4*>(x0p + off)) : zero;
-      if (TWO_GROUPS) xb[u] = (in_k && x1_ok) ? __ldg(reinterpret_cast<const uint4*>(x1p + off)) : zero;
+      xa[u] = (in_k && x0_ok) ? __ldg(reinterpret_cast<const uint4*>(x0p + off * XS)) : zero;
+      if (TWO_GROUPS) xb[u] = (in_k && x1_ok) ? __ldg(reinterpret_cast<const uint4*>(x1p + off * XS)) : zero;
+      if (A8) {
+        xa2[u] = (in_k && x0_ok) ? __ldg(reinterpret_cast<const uint4*>(x0p + off * XS) + 1) : zero;
+        if (TWO_GROUPS) xb2[u] = (in_k && x1_ok) ? __ldg(reinterpret_cast<const uint4*>(x1p + off * XS) + 1) : zero;
+      }
     }
 #pragma unroll
     for (int u = 0; u < GS_UNROLL; ++u) {
       uint32_t ea[8], eb[8], ex[8];
       expand(wa[u], ea);
       expand(wb[u], eb);
-      expand(xa[u], ex);
+      if (A8) permute_s8(xa[u], xa2[u], ex);
+      else expand(xa[u], ex);
 #pragma unroll
       for (int j = 0; j < 4; ++j) mma_s8_16832(c0, ea[2 * j], eb[2 * j], ea[2 * j + 1], eb[2 * j + 1], ex[2 * j], ex[2 * j + 1]);
       if (TWO_GROUPS) {
-        expand(xb[u], ex);
+        if (A8) permute_s8(xb[u], xb2[u], ex);
+        else expand(xb[u], ex);
 #pragma unroll
         for (int j = 0; j < 4; ++j)
           mma_s8_16832(c1, ea[2 * j], eb[2 * j], ea[2 * j + 1], eb[2 * j + 1], ex[2 * j], ex[2 * j + 1]);
@@ -129,7 +148,7 @@ __global__ void __launch_bounds__(GS_THREADS)
       int s = 0;
 #pragma unroll
       for (int w = 0; w < GS_WARPS; ++w) s += red[w][ch][tok];
-      s >>= 8;  // exact: every product carries the factor 16*16
+      s >>= A8 ? 4 : 8;  // exact: every product carries the factor 16 once per 4-bit operand
       const float f = static_cast<float>(s) * (__ldg(s_a + tok * sa_stride) * __ldg(s_w + n));  // stride 1: one step per token
       out[static_cast<int64_t>(tok) * ldo + n] = __float2bfloat16_rn(f);
       if (acc_dbg) acc_dbg[static_cast<int64_t>(tok) * N + n] = s;
@@ -140,7 +159,7 @@ __global__ void __launch_bounds__(GS_THREADS)
 }  // namespace
 
 // Rows [0, M) of xq/out, M <= 16 (the caller has already applied row_begin).
-template <bool TWO, bool HALF>
+template <bool TWO, bool HALF, bool A8>
 static pq_status launch_stream(const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w, void* out,
                                int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st,
                                int sa_stride) {
@@ -157,7 +176,7 @@ static pq_status launch_stream(const uint8_t* xq, const uint8_t* wq, const float
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, gemm_w4a4_stream_kernel<TWO, HALF>, xq, wq, s_a, s_w, static_cast<__nv_bfloat16*>(out), ldo,
+  if (cudaLaunchKernelEx(&cfg, gemm_w4a4_stream_kernel<TWO, HALF, A8>, xq, wq, s_a, s_w, static_cast<__nv_bfloat16*>(out), ldo,
                          static_cast<int>(M), static_cast<int>(N), static_cast<int>(K), acc_dbg, sa_stride) != cudaSuccess)
     return PQ_ERR_CUDA;
   return pq_launch_status();
@@ -165,13 +184,19 @@ static pq_status launch_stream(const uint8_t* xq, const uint8_t* wq, const float
 
 pq_status pq_gemm_stream_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
                                 void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg,
-                                cudaStream_t st, bool per_token) {
+                                cudaStream_t st, bool per_token, bool a8) {
   const int sa_stride = per_token ? 1 : 0;  // s_a is then an array of M per-token steps
   // 16 channels per CTA when that still gives every SM several CTAs, else 8 (only for up to 8 tokens:
   // with two token groups the narrower CTA repeats too much of the activation expansion)
   const bool half = M <= 8 && (N + GS_CH - 1) / GS_CH < 4LL * ctx->sm_count;
+  if (a8) {
+    if (M <= 8)
+      return half ? launch_stream<false, true, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride)
+                  : launch_stream<false, false, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride);
+    return launch_stream<true, false, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride);
+  }
   if (M <= 8)
-    return half ? launch_stream<false, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride)
-                : launch_stream<false, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride);
-  return launch_stream<true, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride);
+    return half ? launch_stream<false, true, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride)
+                : launch_stream<false, false, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride);
+  return launch_stream<true, false, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride);
 }

@@ -95,6 +95,17 @@ def test_w4a8_gemm_bit_exact(ctx, M, N, K):
     _gemm8_case(ctx, M, N, K, seed=M + N + K)
 
 
+@pytest.mark.parametrize("M", [1, 4, 8, 9, 16])
+@pytest.mark.parametrize("N,K", [(48, 4096), (1024, 4096), (40, 160), (4096, 14336)])
+def test_w4a8_gemm_decode_shapes_bit_exact(ctx, M, N, K):
+    """Up to 16 tokens: the weight-streaming kernel with s8 activation codes."""
+    if N * K > 1 << 24 and M not in (1, 16):
+        pytest.skip("large shape covered at M=1 and M=16")
+    _gemm8_case(ctx, M, N, K, seed=M * 7 + N)
+    if M == 9:
+        _gemm8_case(ctx, M + 4, N, K, seed=N, row_begin=4)
+
+
 def test_w4a8_gemm_many_tiles_and_row_begin(ctx):
     _gemm8_case(ctx, 1024, 5120, 256, seed=5)       # 80 tiles on 74 CTA pairs: some pairs take a second tile
     _gemm8_case(ctx, 260, 256, 256, seed=11, row_begin=4)
