@@ -403,6 +403,73 @@ void orc_outlier_tokens(const uint16_t* x, int64_t ldx, int64_t T, int64_t C, fl
   }
 }
 
+// ---- Eq. 1 as printed: asymmetric, with a zero point (static per-tensor activations, N = 4) ------------
+// Range of the rotated calibration rows >= row_begin: mn = min fp32(y), mx = max fp32(y).
+void orc_calib_act_minmax(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin, float* mn_out,
+                          float* mx_out) {
+  double mn = INFINITY, mx = -INFINITY;
+  std::vector<double> xr(K), yr(K);
+  for (int64_t m = row_begin; m < M; ++m) {
+    for (int64_t j = 0; j < K; ++j) xr[j] = bf16_to_double(x[m * ldx + j]);
+    rotate_row(xr.data(), yr.data(), K, B);
+    for (int64_t j = 0; j < K; ++j) {
+      const double v = static_cast<double>(static_cast<float>(yr[j]));
+      mn = std::min(mn, v), mx = std::max(mx, v);
+    }
+  }
+  *mn_out = static_cast<float>(mn), *mx_out = static_cast<float>(mx);
+}
+
+// Max-min initialisation (gamma = beta = 1): s = (mx - mn) / (2^N - 1), z = -round(mn / s), every step an
+// IEEE fp32 operation (the precision the GPU takes them in); a constant tensor gets s = 1, z = 0. z is
+// kept inside the code range.
+void orc_asym_params(float mn, float mx, int bits, float* s_out, int32_t* z_out) {
+  const int qmax = (1 << bits) - 1;
+  if (!(mx > mn)) {
+    *s_out = 1.0f, *z_out = 0;
+    return;
+  }
+  const float d = static_cast<float>(static_cast<double>(mx) - static_cast<double>(mn));
+  const float s = static_cast<float>(static_cast<double>(d) / static_cast<double>(qmax));
+  const float q = static_cast<float>(static_cast<double>(mn) / static_cast<double>(s));
+  *s_out = s;
+  *z_out = clampi(-std::lrint(std::nearbyint(static_cast<double>(q))), 0, qmax);
+}
+
+// X_INT = clamp(round_half_even(y / s) + z, 0, 15), one byte per element, y the rotated row; rows < row_begin
+// are left untouched; tie_dist as in orc_quant_act.
+void orc_quant_act_asym(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin, float s_a, int32_t z,
+                        uint8_t* u, float* tie_dist) {
+  const double s = static_cast<double>(s_a);
+  parallel_rows(M, [&](int64_t m) {
+    if (m < row_begin) return;
+    std::vector<double> xr(K), yr(K);
+    for (int64_t j = 0; j < K; ++j) xr[j] = bf16_to_double(x[m * ldx + j]);
+    rotate_row(xr.data(), yr.data(), K, B);
+    for (int64_t j = 0; j < K; ++j) {
+      double r = yr[j] / s;
+      u[m * K + j] = static_cast<uint8_t>(clampi(std::lrint(std::nearbyint(r)) + z, 0, 15));
+      if (tie_dist) tie_dist[m * K + j] = static_cast<float>(std::fabs(r - std::floor(r) - 0.5));
+    }
+  });
+}
+
+// acc[t,n] = sum_k (u[t,k] - z) * wq[n,k]: the dequantized activation (up to its step) times the weight codes,
+// written out as such (no correction-term algebra). Returns 1 if an accumulator does not fit int32.
+int orc_gemm_asym(const uint8_t* u, int32_t z, const uint8_t* wq, int64_t M, int64_t N, int64_t K, int32_t* acc) {
+  std::atomic<int> overflow{0};
+  parallel_rows(M, [&](int64_t t) {
+    for (int64_t n = 0; n < N; ++n) {
+      int64_t s = 0;
+      for (int64_t k = 0; k < K; ++k)
+        s += (static_cast<int64_t>(u[t * K + k]) - z) * static_cast<int64_t>(nib_get(wq + n * (K / 2), k));
+      if (s > INT32_MAX || s < INT32_MIN) overflow = 1;
+      acc[t * N + n] = static_cast<int32_t>(s);
+    }
+  });
+  return overflow.load();
+}
+
 // ---- per-head static KV scale and KV4 append (Table 1, O2: per-head static KV cache) ----------
 // kv bf16 [B,T,H,D]; s[h] = fp32(max |kv[:,:,h,:]|) / 7 in double then fp32 (1 if all zero).
 void orc_calib_kv_scale(const uint16_t* kv, int64_t B, int64_t T, int64_t H, int64_t D, float* s) {

@@ -227,6 +227,47 @@ def outlier_tokens(x_bits: np.ndarray, eta1: float = 64.0, eta2: float = 8.0):
     return M, R, flags, float(med[0])
 
 
+def calib_act_minmax(x_bits: np.ndarray, block: int, row_begin: int = 0):
+    """(min, max) of the rotated rows >= row_begin, as fp32."""
+    x_bits = _u16(x_bits)
+    M, K = x_bits.shape
+    mn, mx = np.zeros(1, np.float32), np.zeros(1, np.float32)
+    lib().orc_calib_act_minmax(_p(x_bits, c_uint16), c_int64(K), c_int64(M), c_int64(K), c_int(block), c_int64(row_begin),
+                               _p(mn, c_float), _p(mx, c_float))
+    return np.float32(mn[0]), np.float32(mx[0])
+
+
+def asym_params(mn, mx, bits: int = 4):
+    """Eq. 1 with gamma = beta = 1: step s = (mx - mn) / (2^bits - 1) and zero point z = -round(mn / s)."""
+    s, z = np.zeros(1, np.float32), np.zeros(1, np.int32)
+    lib().orc_asym_params(c_float(float(mn)), c_float(float(mx)), c_int(bits), _p(s, c_float), _p(z, c_int32))
+    return np.float32(s[0]), int(z[0])
+
+
+def quant_act_asym(x_bits: np.ndarray, block: int, s_a, z: int, row_begin: int = 0, want_tie_dist: bool = False):
+    """Unsigned codes [M,K] in 0..15 (rows < row_begin zero) and, optionally, the tie distances."""
+    x_bits = _u16(x_bits)
+    M, K = x_bits.shape
+    u = np.zeros((M, K), np.uint8)
+    tie = np.full((M, K), 0.5, np.float32) if want_tie_dist else None
+    lib().orc_quant_act_asym(_p(x_bits, c_uint16), c_int64(K), c_int64(M), c_int64(K), c_int(block), c_int64(row_begin),
+                             c_float(float(s_a)), c_int32(int(z)), _p(u, c_uint8), _p(tie, c_float) if want_tie_dist else None)
+    return (u, tie) if want_tie_dist else u
+
+
+def gemm_asym(u: np.ndarray, z: int, wq: np.ndarray) -> np.ndarray:
+    """sum_k (u[t,k] - z) * w[n,k] with unsigned activation codes and packed signed weight codes -> int32 [M,N]."""
+    u = np.ascontiguousarray(u, np.uint8)
+    wq = np.ascontiguousarray(wq, np.uint8)
+    M, K = u.shape
+    N = wq.shape[0]
+    assert wq.shape[1] * 2 == K
+    acc = np.empty((M, N), np.int32)
+    if lib().orc_gemm_asym(_p(u, c_uint8), c_int32(int(z)), _p(wq, c_uint8), c_int64(M), c_int64(N), c_int64(K), _p(acc, c_int32)):
+        raise OverflowError("accumulator does not fit int32")
+    return acc
+
+
 # ---- weights ---------------------------------------------------------------------------------------
 def quant_weights(w_bits: np.ndarray):
     w_bits = _u16(w_bits)

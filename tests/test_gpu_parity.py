@@ -276,6 +276,30 @@ def test_argument_errors_are_synchronous(ctx):
         ctx.w4a4_gemm(xq, xq, s, torch.ones(4, device="cuda"))   # K = 48 not a multiple of 32
 
 
+def test_argument_errors_of_the_widened_entry_points(ctx):
+    from paper_2410_05265_b200.binding import PQError
+
+    s = torch.ones(1, device="cuda")
+    x = torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(PQError):
+        ctx.hadamard_quant_act8(x, 192, s)                                  # not a power of two
+    with pytest.raises(PQError):
+        ctx.dyn_act_scale(x, 256, clip=1.5)                                 # clip must lie in (0, 1]
+    with pytest.raises(PQError):
+        ctx.dyn_act_scale(x, 256, clip=0.0)
+    xq8 = torch.zeros((4, 48), dtype=torch.int8, device="cuda")
+    wq = torch.zeros((4, 24), dtype=torch.uint8, device="cuda")
+    with pytest.raises(PQError):
+        ctx.w4a8_gemm(xq8, wq, s, torch.ones(4, device="cuda"))            # K = 48 not a multiple of 32
+    with pytest.raises(PQError):
+        ctx.outlier_tokens(torch.zeros((8193, 128), dtype=torch.bfloat16, device="cuda"))   # more than 8192 tokens
+    with pytest.raises(PQError):
+        ctx.outlier_tokens(torch.zeros((8, 100), dtype=torch.bfloat16, device="cuda"))      # C % 8 != 0
+    with pytest.raises(PQError):
+        ctx.rope(torch.zeros((2, 2, 64), dtype=torch.bfloat16, device="cuda"), 0, 500000.0, rotate=True)  # head_dim != 128
+    ctx.check()
+
+
 # ------------------------------------------------------------------------------- a6 block glue
 @pytest.mark.parametrize("M,K", [(5, 128), (37, 4096), (9, 8192), (3, 16384)])
 def test_rmsnorm_matches_oracle(ctx, M, K):

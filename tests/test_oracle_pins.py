@@ -369,6 +369,57 @@ def test_outlier_tokens_hand_example_library_median_and_invariances():
     assert flags[:4].tolist() == [1, 1, 1, 1] and flags[17] == 2 and int((flags != 0).sum()) == 5
 
 
+# ---------------------------------------------------------------- Eq. 1 as printed: asymmetric with a zero point
+def test_asymmetric_quantizer_hand_values_and_reduction_to_the_symmetric_one():
+    # range [-1, 2.75]: s = 3.75 / 15 = 0.25, z = -round(-1 / 0.25) = 4
+    s, z = orc.asym_params(-1.0, 2.75)
+    assert s == 0.25 and z == 4
+    assert orc.asym_params(3.0, 3.0) == (1.0, 0)                       # a constant tensor
+    assert orc.asym_params(0.0, 15.0) == (1.0, 0) and orc.asym_params(-15.0, 0.0) == (1.0, 15)
+    vals = np.array([-1.0, 2.75, 0.125, 0.375, -0.125, -0.375, 5.0, -3.0, 0.0, 1.0, 0.3, -0.3])
+    want = np.array([0, 15, 4, 6, 4, 2, 15, 0, 4, 8, 5, 3])           # round(x / s) + z, ties to even, clamp to [0, 15]
+    pad = np.zeros(128 - len(vals))
+    u = orc.quant_act_asym(bf16_bits(np.concatenate([vals, pad])[None, :]), 0, s, z)
+    assert u.dtype == np.uint8 and u[0, :len(vals)].tolist() == want.tolist() and np.all(u[0, len(vals):] == 4)
+    # dequantization s (u - z) is within half a step inside the range
+    deq = s * (u[0, :len(vals)].astype(np.float64) - z)
+    inside = (vals >= -1.0) & (vals <= 2.75)
+    xb = orc.bf16_to_f64(bf16_bits(vals))
+    assert np.all(np.abs(deq[inside] - xb[inside]) <= 0.125 + 1e-12)
+    # with z = 8 the unsigned code is the signed code of the symmetric quantizer (pinned above) plus 8
+    M, K = 5, 256
+    xr = inputs.bits(inputs.activations(M, K, seed=7))
+    s_sym = orc.calib_act_scale(xr, K)
+    u8, tie = orc.quant_act_asym(xr, K, s_sym, 8, want_tie_dist=True)
+    c_sym, tie_sym = orc.quant_act(xr, K, s_sym, want_tie_dist=True)
+    assert np.array_equal(u8.astype(int) - 8, orc.unpack_int4(c_sym)) and np.array_equal(tie, tie_sym)
+    # range of a rotated batch: prefix rows excluded; the codes of the calibration batch itself use the full range
+    x = inputs.activations(12, K, seed=1, n_prefix=4)
+    xb = inputs.bits(x)
+    mn, mx = orc.calib_act_minmax(xb, K, row_begin=4)
+    y = orc.rotate_bf16(xb, K)[4:].astype(np.float32)
+    assert mn == y.min() and mx == y.max()
+    s2, z2 = orc.asym_params(mn, mx)
+    u2 = orc.quant_act_asym(xb, K, s2, z2, row_begin=4)
+    assert u2[4:].min() == 0 and u2[4:].max() == 15 and np.all(u2[:4] == 0)
+    assert np.all(np.abs(s2 * (u2[4:].astype(np.float64) - z2) - y) <= 0.5 * s2 * (1 + 1e-5) + 1e-6)
+
+
+def test_gemm_asym_is_the_dequantized_product():
+    M, N, K, z = 7, 11, 96, 5
+    u = rng.integers(0, 16, (M, K)).astype(np.uint8)
+    w = rng.integers(-8, 8, (N, K)).astype(np.int8)
+    acc = orc.gemm_asym(u, z, orc.pack_int4(w))
+    assert np.array_equal(acc, (u.astype(np.int64) - z) @ w.astype(np.int64).T)
+    for t, n in itertools.product(range(2), range(3)):
+        assert acc[t, n] == sum((int(u[t, k]) - z) * int(w[n, k]) for k in range(K))
+    # zero point 8: the symmetric GEMM on the codes u - 8
+    assert np.array_equal(orc.gemm_asym(u, 8, orc.pack_int4(w)), orc.gemm_i4(orc.pack_int4((u.astype(int) - 8).astype(np.int8)), orc.pack_int4(w)))
+    # the correction-term identity the GPU epilogue uses: sum (u - z) w = sum (u - 8) w - (z - 8) sum_k w
+    raw = orc.gemm_i4(orc.pack_int4((u.astype(int) - 8).astype(np.int8)), orc.pack_int4(w))
+    assert np.array_equal(acc, raw - (z - 8) * w.astype(np.int64).sum(1)[None, :])
+
+
 def test_dequant_epilogue_closed_form_and_one_rounding():
     acc = np.array([[3, -5, 0, 1 << 20]], np.int32)
     s_w = np.array([0.25, 0.5, 7.0, 2.0**-10], np.float32)
