@@ -253,6 +253,28 @@ pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache, const voi
                                             void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Eq. 1 as printed: asymmetric static per-tensor activation quantizer with a zero point (N = 4),
+ *     s = (max y - min y) / 15,  z = -round(min y / s)        max-min initialisation (gamma = beta = 1)
+ *     u = clamp(round_half_even(y / s) + z, 0, 15),           dequantized value s (u - z)
+ *     out[t, n] = bf16(s_a * s_w[n] * sum_k (u[t,k] - z) * w[n,k])
+ *   pq_calib_act_asym           range of the rotated rows >= row_begin of one calibration batch -> *s_a, *z_a
+ *                               (device scalars, overwritten; a constant batch gives s = 1, z = 0)
+ *   pq_hadamard_quant_act_asym  xq [M, K/2]: the packed signed nibbles hold u - 8 (the operand format of the
+ *                               symmetric path, so the same GEMM kernels read it)
+ *   pq_weight_code_sums         wsum[n] = sum_k w[n,k] over the packed codes of pq_quant_weights (offline), K % 8 == 0
+ *   pq_w4a4_gemm_asym           the GEMM; its epilogue subtracts (z - 8) * wsum[n] from the exact integer sum
+ *                               (acc_dbg, when given, receives sum_k (u - z) w). Other arguments as in pq_w4a4_gemm.
+ * The grid search the paper runs over s and z is offline and not part of this library: any s, z can be passed. */
+pq_status pq_calib_act_asym(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block, int64_t row_begin,
+                            float* s_a, int32_t* z_a, void* stream);
+pq_status pq_hadamard_quant_act_asym(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                     int64_t row_begin, const float* s_a, const int32_t* z_a, uint8_t* xq, void* stream);
+pq_status pq_weight_code_sums(pq_ctx* ctx, const uint8_t* wq, int64_t N, int64_t K, int32_t* wsum, void* stream);
+pq_status pq_w4a4_gemm_asym(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const int32_t* z_a,
+                            const float* s_w, const int32_t* wsum, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                            int64_t row_begin, int32_t* acc_dbg, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Outlier tokens (Sec. 4.1, "Definition of Outlier Token", Eq. 2), the cheap part of the offline analysis
  * that decides which tokens are prefixed:
  *     M[i] = max_c |x[i, c]|,  R[i] = M[i] / median(M),

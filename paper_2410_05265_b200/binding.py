@@ -27,6 +27,7 @@ EXPORTS = [
     "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add", "pq_prefill_attn_kv4_prefix", "pq_kv4_append_strided", "pq_calib_kv_scale",
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
     "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
+    "pq_calib_act_asym", "pq_hadamard_quant_act_asym", "pq_weight_code_sums", "pq_w4a4_gemm_asym",
 ]
 
 
@@ -93,6 +94,12 @@ def load_library() -> ctypes.CDLL:
     lib.pq_w4a4_gemm_rows.argtypes = lib.pq_w4a8_gemm.argtypes
     lib.pq_outlier_tokens.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_float, c_float, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p]
+    lib.pq_calib_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p, c_void_p, c_void_p]
+    lib.pq_hadamard_quant_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p, c_void_p,
+                                               c_void_p, c_void_p]
+    lib.pq_weight_code_sums.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p]
+    lib.pq_w4a4_gemm_asym.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64,
+                                      c_int64, c_int64, c_int64, c_void_p, c_void_p]
     for name in EXPORTS:
         getattr(lib, name)
         if name not in ("pq_status_string", "pq_w4a4_gemm_workspace_bytes", "pq_decode_attn_workspace_bytes"):
@@ -217,6 +224,52 @@ class Context:
             assert acc_dbg.shape == (M, N) and acc_dbg.is_contiguous()
         _ok(self.lib.pq_w4a4_gemm(self.h, _ptr(xq), _ptr(wq), _ptr(s_a), _ptr(s_w), _ptr(out), out.stride(0), M, N, K2 * 2,
                                   row_begin, _ptr(acc_dbg), c_void_p(0), 0, _stream()), "pq_w4a4_gemm")
+        return out
+
+    # ---- Eq. 1 as printed: asymmetric activation quantizer with a zero point ---------------------------
+    def calib_act_asym(self, x: torch.Tensor, had_block: int, row_begin: int = 0):
+        """Returns device scalars (s_a f32, z_a int32) from the range of the rotated rows >= row_begin."""
+        _dev(x, torch.bfloat16, "x")
+        M, K = x.shape
+        s_a = torch.zeros((1,), dtype=torch.float32, device=x.device)
+        z_a = torch.zeros((1,), dtype=torch.int32, device=x.device)
+        _ok(self.lib.pq_calib_act_asym(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, _ptr(s_a), _ptr(z_a), _stream()),
+            "pq_calib_act_asym")
+        return s_a, z_a
+
+    def hadamard_quant_act_asym(self, x: torch.Tensor, had_block: int, s_a: torch.Tensor, z_a: torch.Tensor, row_begin: int = 0,
+                                out: torch.Tensor | None = None):
+        _dev(x, torch.bfloat16, "x"), _dev(s_a, torch.float32, "s_a"), _dev(z_a, torch.int32, "z_a")
+        M, K = x.shape
+        assert x.stride(1) == 1
+        if out is None:
+            out = torch.zeros((M, K // 2), dtype=torch.uint8, device=x.device)
+        _ok(self.lib.pq_hadamard_quant_act_asym(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, _ptr(s_a), _ptr(z_a),
+                                                _ptr(out), _stream()), "pq_hadamard_quant_act_asym")
+        return out
+
+    def weight_code_sums(self, wq: torch.Tensor) -> torch.Tensor:
+        _dev(wq, torch.uint8, "wq")
+        N, K2 = wq.shape
+        assert wq.is_contiguous()
+        wsum = torch.empty((N,), dtype=torch.int32, device=wq.device)
+        _ok(self.lib.pq_weight_code_sums(self.h, _ptr(wq), N, K2 * 2, _ptr(wsum), _stream()), "pq_weight_code_sums")
+        return wsum
+
+    def w4a4_gemm_asym(self, xq: torch.Tensor, wq: torch.Tensor, s_a: torch.Tensor, z_a: torch.Tensor, s_w: torch.Tensor,
+                       wsum: torch.Tensor, row_begin: int = 0, out: torch.Tensor | None = None, acc_dbg: torch.Tensor | None = None):
+        _dev(xq, torch.uint8, "xq"), _dev(wq, torch.uint8, "wq"), _dev(z_a, torch.int32, "z_a"), _dev(wsum, torch.int32, "wsum")
+        _dev(s_a, torch.float32, "s_a"), _dev(s_w, torch.float32, "s_w")
+        M, K2 = xq.shape
+        N = wq.shape[0]
+        assert wq.shape[1] == K2 and xq.is_contiguous() and wq.is_contiguous() and wsum.shape == (N,)
+        if out is None:
+            out = torch.zeros((M, N), dtype=torch.bfloat16, device=xq.device)
+        if acc_dbg is not None:
+            _dev(acc_dbg, torch.int32, "acc_dbg")
+            assert acc_dbg.shape == (M, N) and acc_dbg.is_contiguous()
+        _ok(self.lib.pq_w4a4_gemm_asym(self.h, _ptr(xq), _ptr(wq), _ptr(s_a), _ptr(z_a), _ptr(s_w), _ptr(wsum), _ptr(out),
+                                       out.stride(0), M, N, K2 * 2, row_begin, _ptr(acc_dbg), _stream()), "pq_w4a4_gemm_asym")
         return out
 
     # ---- offline analysis: outlier tokens (Sec. 4.1, Eq. 2) -------------------------------------------

@@ -58,7 +58,8 @@ __global__ void __launch_bounds__(GS_THREADS)
     gemm_w4a4_stream_kernel(const uint8_t* __restrict__ xq, const uint8_t* __restrict__ wq,
                             const float* __restrict__ s_a, const float* __restrict__ s_w,
                             __nv_bfloat16* __restrict__ out, int64_t ldo, int M, int N, int K,
-                            int32_t* __restrict__ acc_dbg, int sa_stride) {
+                            int32_t* __restrict__ acc_dbg, int sa_stride, const int32_t* __restrict__ zp,
+                            const int32_t* __restrict__ wsum) {
   __shared__ int red[GS_WARPS][GS_CH][16];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -149,6 +150,7 @@ __global__ void __launch_bounds__(GS_THREADS)
 #pragma unroll
       for (int w = 0; w < GS_WARPS; ++w) s += red[w][ch][tok];
       s >>= A8 ? 4 : 8;  // exact: every product carries the factor 16 once per 4-bit operand
+      if (zp) s -= (__ldg(zp) - 8) * __ldg(wsum + n);  // zero-point form of Eq. 1: sum (u - z) w from sum (u - 8) w
       const float f = static_cast<float>(s) * (__ldg(s_a + tok * sa_stride) * __ldg(s_w + n));  // stride 1: one step per token
       out[static_cast<int64_t>(tok) * ldo + n] = __float2bfloat16_rn(f);
       if (acc_dbg) acc_dbg[static_cast<int64_t>(tok) * N + n] = s;
@@ -162,7 +164,7 @@ __global__ void __launch_bounds__(GS_THREADS)
 template <bool TWO, bool HALF, bool A8>
 static pq_status launch_stream(const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w, void* out,
                                int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st,
-                               int sa_stride) {
+                               int sa_stride, const int32_t* zp, const int32_t* wsum) {
   const int ch = HALF ? GS_CH / 2 : GS_CH;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>((N + ch - 1) / ch));
@@ -177,26 +179,26 @@ static pq_status launch_stream(const uint8_t* xq, const uint8_t* wq, const float
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (cudaLaunchKernelEx(&cfg, gemm_w4a4_stream_kernel<TWO, HALF, A8>, xq, wq, s_a, s_w, static_cast<__nv_bfloat16*>(out), ldo,
-                         static_cast<int>(M), static_cast<int>(N), static_cast<int>(K), acc_dbg, sa_stride) != cudaSuccess)
+                         static_cast<int>(M), static_cast<int>(N), static_cast<int>(K), acc_dbg, sa_stride, zp, wsum) != cudaSuccess)
     return PQ_ERR_CUDA;
   return pq_launch_status();
 }
 
 pq_status pq_gemm_stream_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
                                 void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg,
-                                cudaStream_t st, bool per_token, bool a8) {
+                                cudaStream_t st, bool per_token, bool a8, const int32_t* zp, const int32_t* wsum) {
   const int sa_stride = per_token ? 1 : 0;  // s_a is then an array of M per-token steps
   // 16 channels per CTA when that still gives every SM several CTAs, else 8 (only for up to 8 tokens:
   // with two token groups the narrower CTA repeats too much of the activation expansion)
   const bool half = M <= 8 && (N + GS_CH - 1) / GS_CH < 4LL * ctx->sm_count;
   if (a8) {
     if (M <= 8)
-      return half ? launch_stream<false, true, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride)
-                  : launch_stream<false, false, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride);
-    return launch_stream<true, false, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride);
+      return half ? launch_stream<false, true, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride, zp, wsum)
+                  : launch_stream<false, false, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride, zp, wsum);
+    return launch_stream<true, false, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride, zp, wsum);
   }
   if (M <= 8)
-    return half ? launch_stream<false, true, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride)
-                : launch_stream<false, false, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride);
-  return launch_stream<true, false, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride);
+    return half ? launch_stream<false, true, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride, zp, wsum)
+                : launch_stream<false, false, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride, zp, wsum);
+  return launch_stream<true, false, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride, zp, wsum);
 }

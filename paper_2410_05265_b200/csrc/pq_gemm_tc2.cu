@@ -81,6 +81,7 @@ constexpr int EPI_COLS = 64;                // columns per TMA store (128 bytes 
 constexpr int EPI_BUF = 32 * EPI_COLS * 2;  // 4 KB: one warp's 32 rows x 64 columns
 constexpr int EPI_BYTES = 4 * EPI_BUFS * EPI_BUF;
 constexpr int SCALE_BYTES = 4 * BN * 4;     // per-warp copy of s_a * s_w[n0 .. n0+255]
+constexpr int ZW_BYTES = 4 * BN * 4;        // per-warp copy of (z - 8) * wsum[n0 .. n0+255] (zero-point correction)
 
 struct __align__(8) Barriers {
   uint64_t pk_full[N_PK], pk_empty[N_PK];
@@ -95,10 +96,12 @@ struct __align__(8) Barriers {
 };
 
 constexpr size_t SMEM_BYTES =
-    1024 /*alignment slack*/ + N_S8 * S8_STAGE + N_PK * PK_STAGE + EPI_BYTES + SCALE_BYTES + sizeof(Barriers);
+    1024 /*alignment slack*/ + N_S8 * S8_STAGE + N_PK * PK_STAGE + EPI_BYTES + SCALE_BYTES + ZW_BYTES + sizeof(Barriers);
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 struct GemmParams {
+  const int32_t* zp;    // ZP kernels: the activation zero point z (device scalar) ...
+  const int32_t* wsum;  // ... and the sum of every output channel's weight codes [N]
   const float* s_row;  // per-token steps [M] (dynamic setting) or null: the scalar s_a applies
   const float* s_a;
   const float* s_w;
@@ -208,7 +211,10 @@ __device__ __forceinline__ void bulk_wait_read() {
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-template <bool A8>
+// ZP (Eq. 1 as printed): the stored token codes are u - 8 for unsigned codes u with zero point z; what the
+// layer needs is sum_k (u - z) w = sum_k (u - 8) w - (z - 8) sum_k w, so the epilogue subtracts (z - 8) * wsum[n]
+// from the exact integer sum before scaling.
+template <bool A8, bool ZP>
 __global__ void __launch_bounds__(N_THREADS, 1)
     gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                           const __grid_constant__ CUtensorMap tmap_out, const GemmParams p) {
@@ -218,7 +224,8 @@ __global__ void __launch_bounds__(N_THREADS, 1)
   uint8_t* pk_buf = s8_buf + N_S8 * S8_STAGE;               // N_PK stages: packed A rows then packed B rows
   uint8_t* epi_buf = pk_buf + N_PK * PK_STAGE;              // 4 warps x 2 buffers, 1024-aligned
   float* scale_buf = reinterpret_cast<float*>(epi_buf + EPI_BYTES);
-  Barriers* bars = reinterpret_cast<Barriers*>(reinterpret_cast<uint8_t*>(scale_buf) + SCALE_BYTES);
+  int32_t* zw_buf = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(scale_buf) + SCALE_BYTES);
+  Barriers* bars = reinterpret_cast<Barriers*>(reinterpret_cast<uint8_t*>(zw_buf) + ZW_BYTES);
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");  // operands and output may belong to the previous kernel
@@ -422,6 +429,8 @@ __global__ void __launch_bounds__(N_THREADS, 1)
     const float s_a = p.s_row ? 1.0f : __ldg(p.s_a);
     uint8_t* my_buf = epi_buf + q * EPI_BUFS * EPI_BUF;
     float* my_scale = scale_buf + q * BN;
+    int32_t* my_zw = zw_buf + q * BN;
+    const int zp8 = ZP ? __ldg(p.zp) - 8 : 0;
     uint32_t tcount = 0, n_store = 0;
     bool ok = true;
     for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++tcount) {
@@ -433,6 +442,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
       for (int i = 0; i < BN / 32; ++i) {
         const int col = n0 + i * 32 + lane;
         my_scale[i * 32 + lane] = col < p.N ? s_a * __ldg(p.s_w + col) : 0.0f;
+        if (ZP) my_zw[i * 32 + lane] = col < p.N ? zp8 * __ldg(p.wsum + col) : 0;
       }
       __syncwarp();
       const bool stuck = !wait_bar(&bars->acc_full[ab], aph, abort_flag);
@@ -466,14 +476,14 @@ __global__ void __launch_bounds__(N_THREADS, 1)
             const float4 sa = *reinterpret_cast<const float4*>(my_scale + c * 32 + g * 8);
             const float4 sb = *reinterpret_cast<const float4*>(my_scale + c * 32 + g * 8 + 4);
             const int b = g * 8;
-            const __nv_bfloat162 p0 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 0]) >> SHIFT) * sa.x * rs,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 1]) >> SHIFT) * sa.y * rs);
-            const __nv_bfloat162 p1 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 2]) >> SHIFT) * sa.z * rs,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 3]) >> SHIFT) * sa.w * rs);
-            const __nv_bfloat162 p2 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 4]) >> SHIFT) * sb.x * rs,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 5]) >> SHIFT) * sb.y * rs);
-            const __nv_bfloat162 p3 = __floats2bfloat162_rn(static_cast<float>(static_cast<int32_t>(r[b + 6]) >> SHIFT) * sb.z * rs,
-                                                            static_cast<float>(static_cast<int32_t>(r[b + 7]) >> SHIFT) * sb.w * rs);
+            const __nv_bfloat162 p0 = __floats2bfloat162_rn(static_cast<float>((static_cast<int32_t>(r[b + 0]) >> SHIFT) - (ZP ? my_zw[c * 32 + b + 0] : 0)) * sa.x * rs,
+                                                            static_cast<float>((static_cast<int32_t>(r[b + 1]) >> SHIFT) - (ZP ? my_zw[c * 32 + b + 1] : 0)) * sa.y * rs);
+            const __nv_bfloat162 p1 = __floats2bfloat162_rn(static_cast<float>((static_cast<int32_t>(r[b + 2]) >> SHIFT) - (ZP ? my_zw[c * 32 + b + 2] : 0)) * sa.z * rs,
+                                                            static_cast<float>((static_cast<int32_t>(r[b + 3]) >> SHIFT) - (ZP ? my_zw[c * 32 + b + 3] : 0)) * sa.w * rs);
+            const __nv_bfloat162 p2 = __floats2bfloat162_rn(static_cast<float>((static_cast<int32_t>(r[b + 4]) >> SHIFT) - (ZP ? my_zw[c * 32 + b + 4] : 0)) * sb.x * rs,
+                                                            static_cast<float>((static_cast<int32_t>(r[b + 5]) >> SHIFT) - (ZP ? my_zw[c * 32 + b + 5] : 0)) * sb.y * rs);
+            const __nv_bfloat162 p3 = __floats2bfloat162_rn(static_cast<float>((static_cast<int32_t>(r[b + 6]) >> SHIFT) - (ZP ? my_zw[c * 32 + b + 6] : 0)) * sb.z * rs,
+                                                            static_cast<float>((static_cast<int32_t>(r[b + 7]) >> SHIFT) - (ZP ? my_zw[c * 32 + b + 7] : 0)) * sb.w * rs);
             const int chunk = (c & 1) * 4 + g;  // 16-byte chunk inside the 128-byte staging row
             *reinterpret_cast<uint4*>(buf + lane * 128 + ((chunk ^ (lane & 7)) << 4)) =
                 make_uint4(*reinterpret_cast<const uint32_t*>(&p0), *reinterpret_cast<const uint32_t*>(&p1),
@@ -494,13 +504,13 @@ __global__ void __launch_bounds__(N_THREADS, 1)
             const int col = col0 + i;
             if (col < p.N)
               p.out[static_cast<int64_t>(row) * p.ldo + col] =
-                  __float2bfloat16_rn(static_cast<float>(static_cast<int32_t>(r[i]) >> SHIFT) * my_scale[c * 32 + i] * rs);
+                  __float2bfloat16_rn(static_cast<float>((static_cast<int32_t>(r[i]) >> SHIFT) - (ZP ? my_zw[c * 32 + i] : 0)) * my_scale[c * 32 + i] * rs);
           }
         }
         if (p.acc_dbg && row < p.M) {
           for (int i = 0; i < 32; ++i) {
             const int col = col0 + i;
-            if (col < p.N) p.acc_dbg[static_cast<int64_t>(row) * p.N + col] = static_cast<int32_t>(r[i]) >> SHIFT;
+            if (col < p.N) p.acc_dbg[static_cast<int64_t>(row) * p.N + col] = (static_cast<int32_t>(r[i]) >> SHIFT) - (ZP ? my_zw[c * 32 + i] : 0);
           }
         }
       }
@@ -570,7 +580,7 @@ bool make_out_map(pq_ctx* ctx, CUtensorMap* map, void* out, int64_t M, int64_t N
 // s_row: per-token steps (then s_a is ignored), or null.
 pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
                               void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg,
-                              cudaStream_t st, bool a8, const float* s_row) {
+                              cudaStream_t st, bool a8, const float* s_row, const int32_t* zp, const int32_t* wsum) {
   CUtensorMap ta, tb, to;
   if (!(a8 ? make_s8_map(ctx, &ta, xq, M, K) : make_packed_map(ctx, &ta, xq, M, K / 2, BM_CTA)) ||
       !make_packed_map(ctx, &tb, wq, N, K / 2, BN_CTA))
@@ -583,6 +593,8 @@ pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq,
     to = ta;  // never dereferenced
   }
   p.s_row = s_row;
+  p.zp = zp;
+  p.wsum = wsum;
   p.s_a = s_a;
   p.s_w = s_w;
   p.out = static_cast<__nv_bfloat16*>(out);
@@ -596,9 +608,11 @@ pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq,
   p.tiles_n = static_cast<int>((N + BN - 1) / BN);
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_w4a4_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(gemm_w4a4_pair_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(SMEM_BYTES)) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_w4a4_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(gemm_w4a4_pair_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(SMEM_BYTES)) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_w4a4_pair_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(SMEM_BYTES)) != cudaSuccess)
       return PQ_ERR_CUDA;
     attr_set = true;
@@ -622,8 +636,10 @@ pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq,
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  if ((a8 ? cudaLaunchKernelEx(&cfg, gemm_w4a4_pair_kernel<true>, ta, tb, to, p)
-          : cudaLaunchKernelEx(&cfg, gemm_w4a4_pair_kernel<false>, ta, tb, to, p)) != cudaSuccess)
+  if (zp && (a8 || !wsum)) return PQ_ERR_INVALID_ARG;
+  if ((zp   ? cudaLaunchKernelEx(&cfg, gemm_w4a4_pair_kernel<false, true>, ta, tb, to, p)
+       : a8 ? cudaLaunchKernelEx(&cfg, gemm_w4a4_pair_kernel<true, false>, ta, tb, to, p)
+            : cudaLaunchKernelEx(&cfg, gemm_w4a4_pair_kernel<false, false>, ta, tb, to, p)) != cudaSuccess)
     return PQ_ERR_CUDA;
   return pq_launch_status();
 }

@@ -24,11 +24,22 @@ constexpr int HQ_SMEM_FLOATS = HQ_ELEMS + HQ_ELEMS / 64;  // + 2 floats of paddi
 
 // PER_TOKEN (the dynamic setting, Table 1, O1): one step per row instead of one per tensor; s_a_in / s_a_out
 // are then arrays indexed by row, and the calibration pass is the online first pass of every call.
-template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN>
+// ZP (Eq. 1 as printed, with a zero point): the quantizer adds z - 8 to the rounded value before the clamp, so
+// that the stored signed nibble is the unsigned code minus 8; the calibration pass collects the minimum and
+// the maximum of the rotated values (as order-preserving integer keys in s_a_out[0] and s_a_out[1]).
+__device__ __forceinline__ uint32_t float_key(float f) {
+  const uint32_t b = __float_as_uint(f);
+  return b ^ ((b >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k) {
+  return __uint_as_float(k ^ ((k >> 31) ? 0x80000000u : 0xFFFFFFFFu));
+}
+
+template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP>
 __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
     hadamard_quant_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int64_t n_rows, int64_t K,
                           const float* __restrict__ s_a_in, uint8_t* __restrict__ xq, float* __restrict__ s_a_out,
-                          float clip) {
+                          float clip, const int32_t* __restrict__ zp_in) {
   static_assert(BITS == 4 || BITS == 8, "code width");
   constexpr int QMAX = BITS == 4 ? 7 : 127;  // codes lie in [-QMAX - 1, QMAX]
   constexpr int B = 1 << LOGB;
@@ -58,7 +69,8 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
   const float norm = ROTATE ? __fdiv_rn(1.0f, __fsqrt_rn(static_cast<float>(B))) : 1.0f;
   float inv = norm;
   if (!CALIB && !PER_TOKEN) inv = __fdiv_rn(norm, __ldg(s_a_in));
-  float cal_max = 0.0f;
+  float cal_max = 0.0f, cal_lo = INFINITY, cal_hi = -INFINITY;
+  const int zp = (ZP && !CALIB) ? __ldg(zp_in) - 8 : 0;
 
   for (int64_t sb = blockIdx.x; sb < n_super; sb += gridDim.x) {
     const int64_t gb = sb * G + blk_local;
@@ -150,7 +162,15 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
 #pragma unroll
         for (int q = 0; q < 32; ++q) it_max = fmaxf(it_max, fmaxf(fabsf(W[q].x * norm), fabsf(W[q].y * norm)));
       }
-      if (PER_TOKEN) {
+      if (ZP) {
+        if (active) {
+#pragma unroll
+          for (int q = 0; q < 32; ++q) {
+            const float a = W[q].x * norm, b = W[q].y * norm;
+            cal_lo = fminf(cal_lo, fminf(a, b)), cal_hi = fmaxf(cal_hi, fmaxf(a, b));
+          }
+        }
+      } else if (PER_TOKEN) {
         // the maximum of this row's block, over the TPB threads that hold it (a warp or a part of one; blocks
         // wider than a warp's 2048 elements, and rows of several blocks, meet in the atomic)
         constexpr int SPAN = TPB < 32 ? TPB : 32;
@@ -173,8 +193,8 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
           const float2 tq = __ffma2_rn(W[4 * wd + b], inv2, magic2);
-          lo[b] = max(min(__float_as_int(tq.x), 0x4B400000 + QMAX), 0x4B400000 - QMAX - 1);
-          hi[b] = max(min(__float_as_int(tq.y), 0x4B400000 + QMAX), 0x4B400000 - QMAX - 1);
+          lo[b] = max(min(__float_as_int(tq.x) + zp, 0x4B400000 + QMAX), 0x4B400000 - QMAX - 1);
+          hi[b] = max(min(__float_as_int(tq.y) + zp, 0x4B400000 + QMAX), 0x4B400000 - QMAX - 1);
         }
         pw[wd] = __byte_perm(__byte_perm(lo[0], lo[1], 0x0040), __byte_perm(lo[2], lo[3], 0x0040), 0x5410);
         pw[wd + 8] = __byte_perm(__byte_perm(hi[0], hi[1], 0x0040), __byte_perm(hi[2], hi[3], 0x0040), 0x5410);
@@ -213,17 +233,26 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
       }
     }
   }
-  if (CALIB && !PER_TOKEN) {
+  if (CALIB && ZP) {
+    for (int o = 16; o > 0; o >>= 1) {
+      cal_lo = fminf(cal_lo, __shfl_xor_sync(0xffffffffu, cal_lo, o));
+      cal_hi = fmaxf(cal_hi, __shfl_xor_sync(0xffffffffu, cal_hi, o));
+    }
+    if ((tid & 31) == 0 && cal_hi >= cal_lo) {
+      atomicMax(reinterpret_cast<uint32_t*>(s_a_out), float_key(cal_hi));
+      atomicMin(reinterpret_cast<uint32_t*>(s_a_out) + 1, float_key(cal_lo));
+    }
+  } else if (CALIB && !PER_TOKEN) {
     for (int o = 16; o > 0; o >>= 1) cal_max = fmaxf(cal_max, __shfl_xor_sync(0xffffffffu, cal_max, o));
     if ((tid & 31) == 0 && cal_max > 0.0f)
       atomicMax(reinterpret_cast<int*>(s_a_out), __float_as_int(__fdiv_rn(cal_max, static_cast<float>(QMAX))));
   }
 }
 
-template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN>
+template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP>
 pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_t K, const float* s_a_in, uint8_t* xq,
-                 float* s_a_out, float clip, cudaStream_t st) {
-  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN>;
+                 float* s_a_out, float clip, const int32_t* zp_in, cudaStream_t st) {
+  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN, ZP>;
   constexpr size_t smem = HQ_SMEM_FLOATS * sizeof(float);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
     return PQ_ERR_CUDA;
@@ -243,15 +272,16 @@ pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x), ldx, n_rows, K, s_a_in, xq, s_a_out, clip) !=
+  if (cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x), ldx, n_rows, K, s_a_in, xq, s_a_out, clip, zp_in) !=
       cudaSuccess)
     return PQ_ERR_CUDA;
   return pq_launch_status();
 }
 
-template <bool CALIB, int BITS, bool PER_TOKEN = false>
+template <bool CALIB, int BITS, bool PER_TOKEN = false, bool ZP = false>
 pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block, int64_t row_begin,
-                   const float* s_a_in, uint8_t* xq, float* s_a_out, void* stream, float clip = 1.0f) {
+                   const float* s_a_in, uint8_t* xq, float* s_a_out, void* stream, float clip = 1.0f,
+                   const int32_t* zp_in = nullptr) {
   if (!ctx || !x || (!CALIB && (!s_a_in || !xq)) || (CALIB && !s_a_out)) return PQ_ERR_INVALID_ARG;
   if (M < 0 || K <= 0 || ldx < K || row_begin < 0 || had_block < 0) return PQ_ERR_INVALID_ARG;
   if (K % 128 != 0) return PQ_ERR_SHAPE;
@@ -272,14 +302,14 @@ pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx
     if (CALIB && cudaMemsetAsync(s_a_out, 0, static_cast<size_t>(n_rows) * sizeof(float), st) != cudaSuccess) return PQ_ERR_CUDA;
   }
   switch (had_block) {
-    case 0: return launch<7, false, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
-    case 128: return launch<7, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
-    case 256: return launch<8, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
-    case 512: return launch<9, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
-    case 1024: return launch<10, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
-    case 2048: return launch<11, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
-    case 4096: return launch<12, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
-    case 8192: return launch<13, true, CALIB, BITS, PER_TOKEN>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, st);
+    case 0: return launch<7, false, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
+    case 128: return launch<7, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
+    case 256: return launch<8, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
+    case 512: return launch<9, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
+    case 1024: return launch<10, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
+    case 2048: return launch<11, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
+    case 4096: return launch<12, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
+    case 8192: return launch<13, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
     default: return PQ_ERR_SHAPE;
   }
 }
@@ -319,4 +349,45 @@ extern "C" pq_status pq_hadamard_quant_act_rows(pq_ctx* ctx, const void* x, int6
                                                 int had_block, int64_t row_begin, const float* s_tok, uint8_t* xq,
                                                 void* stream) {
   return dispatch<false, 4, true>(ctx, x, M, K, ldx, had_block, row_begin, s_tok, xq, nullptr, stream);
+}
+
+// ---- Eq. 1 as printed: asymmetric static per-tensor quantizer with a zero point -------------------------
+namespace {
+// Max-min initialisation (gamma = beta = 1) from the collected range: s = (mx - mn) / 15, z = -round(mn / s),
+// every step one IEEE fp32 operation; a constant (or empty) range gives s = 1, z = 0.
+__global__ void asym_params_kernel(uint32_t* keys, float* s_a, int32_t* z_a) {
+  const float mx = key_float(keys[0]), mn = key_float(keys[1]);
+  float s = 1.0f;
+  int z = 0;
+  if (keys[0] >= keys[1] && mx > mn) {
+    s = __fdiv_rn(__fsub_rn(mx, mn), 15.0f);
+    z = -__float2int_rn(__fdiv_rn(mn, s));
+    z = z < 0 ? 0 : (z > 15 ? 15 : z);
+  }
+  *s_a = s;
+  *z_a = z;
+}
+constexpr int ASYM_KEY0 = 8;  // two words of the context's counter array hold the range keys during a call
+}  // namespace
+
+extern "C" pq_status pq_calib_act_asym(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                       int64_t row_begin, float* s_a, int32_t* z_a, void* stream) {
+  if (!ctx || !s_a || !z_a) return PQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* keys = ctx->d_tickets + ASYM_KEY0;
+  if (cudaMemsetAsync(keys, 0x00, sizeof(uint32_t), st) != cudaSuccess ||
+      cudaMemsetAsync(keys + 1, 0xFF, sizeof(uint32_t), st) != cudaSuccess)
+    return PQ_ERR_CUDA;
+  pq_status rc = dispatch<true, 4, false, true>(ctx, x, M, K, ldx, had_block, row_begin, nullptr, nullptr,
+                                                reinterpret_cast<float*>(keys), stream);
+  if (rc != PQ_OK) return rc;
+  asym_params_kernel<<<1, 1, 0, st>>>(keys, s_a, z_a);
+  return pq_launch_status();
+}
+
+extern "C" pq_status pq_hadamard_quant_act_asym(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx,
+                                                int had_block, int64_t row_begin, const float* s_a, const int32_t* z_a,
+                                                uint8_t* xq, void* stream) {
+  if (!z_a) return PQ_ERR_INVALID_ARG;
+  return dispatch<false, 4, false, true>(ctx, x, M, K, ldx, had_block, row_begin, s_a, xq, nullptr, stream, 1.0f, z_a);
 }

@@ -52,3 +52,33 @@ extern "C" pq_status pq_quant_weights(pq_ctx* ctx, const void* W, int64_t N, int
       static_cast<const __nv_bfloat16*>(W), N, K, ldw, wq, s_w);
   return pq_launch_status();
 }
+
+// Sum of the signed 4-bit codes of every weight row (the zero-point correction of the asymmetric activation
+// quantizer needs it): a warp per row; `(w << 4) & 0xF0F0F0F0` and `w & 0xF0F0F0F0` are the codes times 16
+// as signed bytes, summed four at a time with dp4a.
+namespace {
+__global__ void __launch_bounds__(256) weight_code_sums_kernel(const uint8_t* wq, int64_t N, int64_t kwords, int32_t* wsum) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= N) return;
+  const uint32_t* src = reinterpret_cast<const uint32_t*>(wq) + row * kwords;
+  int acc = 0;
+  for (int64_t i = lane; i < kwords; i += 32) {
+    const uint32_t w = __ldg(src + i);
+    acc = __dp4a(static_cast<int>((w << 4) & 0xF0F0F0F0u), 0x01010101, acc);
+    acc = __dp4a(static_cast<int>(w & 0xF0F0F0F0u), 0x01010101, acc);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) wsum[row] = acc >> 4;  // exact: every term carries the factor 16
+}
+}  // namespace
+
+extern "C" pq_status pq_weight_code_sums(pq_ctx* ctx, const uint8_t* wq, int64_t N, int64_t K, int32_t* wsum, void* stream) {
+  if (!ctx || !wq || !wsum || N < 0 || K <= 0) return PQ_ERR_INVALID_ARG;
+  if (K % 8 != 0) return PQ_ERR_SHAPE;
+  if (reinterpret_cast<uintptr_t>(wq) & 3) return PQ_ERR_ALIGN;
+  if (N == 0) return PQ_OK;
+  weight_code_sums_kernel<<<static_cast<unsigned>((N + 7) / 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(wq, N, K / 8, wsum);
+  return pq_launch_status();
+}
