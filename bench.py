@@ -561,6 +561,15 @@ def section_block(ctx, device, peaks):
             continue
         stages[name] = round(prev.elapsed_time(ev), 4)
         prev = ev
+    # the SwiGLU + rotate + quantize launch of the un-tapped pass, on its own
+    gu_buf = blk.buf["gu"]
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for _ in range(reps):
+        ctx.swiglu_hadamard_quant_act(gu_buf[:, : shape.ffn], gu_buf[:, shape.ffn:], shape.had_block(shape.ffn), blk.s_a[3], out=blk.buf["xq_f"])
+    f1.record()
+    torch.cuda.synchronize()
+    fused_ms = f0.elapsed_time(f1) / reps
     # the same block with the online head-wise rotation R3 of q and k fused into the rotary step
     shape.r3 = True
     blk.forward(inputs.activations(T, shape.hidden, seed=1, device=device), calibrate=True)
@@ -591,6 +600,8 @@ def section_block(ctx, device, peaks):
     return {"tokens_per_s": round(T / (ms * 1e-3), 1), "ms": round(ms, 4), "tokens": T, "n_prefix": P,
             "gemm_TOPS": round(gemm_ops / (gemm_ms * 1e-3) / 1e12, 1), "gemm_share": round(gemm_ms / sum(stages.values()), 3),
             "attention_TFLOPS": round(attn_flops / (stages["attn"] * 1e-3) / 1e12, 1), "stage_ms": stages,
+            "swiglu_rotate_quant_fused_ms": round(fused_ms, 4),
+            "stage_note": "stage_ms comes from a pass that stops after every stage (SwiGLU as its own launch: act + xq4); the timed pass fuses them",
             "with_r3": {"ms": round(ms_r3, 4), "rope_rotate_ms": rope_r3},
             "launches": block.Block.LAUNCHES_PER_FORWARD}
 

@@ -89,6 +89,14 @@ pq_status pq_hadamard_quant_act(pq_ctx* ctx, const void* x, int64_t M, int64_t K
 pq_status pq_calib_act_scale(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
                              int64_t row_begin, float* s_a, void* stream);
 
+/* The same quantizer with the SwiGLU of the MLP in front (App. B: the online rotation R4 sits between the
+ * activation function and down_proj): the transform's input is bf16(SiLU(gate) * up), formed in registers with
+ * the arithmetic and the rounding of pq_silu_mul, so the result equals pq_silu_mul followed by
+ * pq_hadamard_quant_act bit for bit while the [M, K] activation tensor never goes to memory.
+ *   gate, up  bf16 [M, K] with ld_in elements between rows (the two halves of a concatenated gate|up output) */
+pq_status pq_swiglu_hadamard_quant_act(pq_ctx* ctx, const void* gate, const void* up, int64_t M, int64_t K, int64_t ld_in,
+                                       int had_block, int64_t row_begin, const float* s_a, uint8_t* xq, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * W4A4 linear layer (Sec. 3: low-bit matrix multiplication; Table 1, O2):
  *     acc[t, n] = sum_k xq[t, k] * wq[n, k]          exact, int32

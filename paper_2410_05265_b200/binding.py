@@ -28,6 +28,7 @@ EXPORTS = [
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
     "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
     "pq_calib_act_asym", "pq_hadamard_quant_act_asym", "pq_weight_code_sums", "pq_w4a4_gemm_asym",
+    "pq_swiglu_hadamard_quant_act",
 ]
 
 
@@ -100,6 +101,8 @@ def load_library() -> ctypes.CDLL:
     lib.pq_weight_code_sums.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p]
     lib.pq_w4a4_gemm_asym.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64,
                                       c_int64, c_int64, c_int64, c_void_p, c_void_p]
+    lib.pq_swiglu_hadamard_quant_act.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p,
+                                                 c_void_p, c_void_p]
     for name in EXPORTS:
         getattr(lib, name)
         if name not in ("pq_status_string", "pq_w4a4_gemm_workspace_bytes", "pq_decode_attn_workspace_bytes"):
@@ -208,6 +211,18 @@ class Context:
             out = torch.zeros((M, K // 2), dtype=torch.uint8, device=x.device)
         _ok(self.lib.pq_hadamard_quant_act(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, _ptr(s_a), _ptr(out),
                                            _stream()), "pq_hadamard_quant_act")
+        return out
+
+    def swiglu_hadamard_quant_act(self, gate: torch.Tensor, up: torch.Tensor, had_block: int, s_a: torch.Tensor, row_begin: int = 0,
+                                  out: torch.Tensor | None = None):
+        """pq_silu_mul followed by pq_hadamard_quant_act in one launch; gate and up are the halves of a gate|up output."""
+        _dev(gate, torch.bfloat16, "gate"), _dev(up, torch.bfloat16, "up"), _dev(s_a, torch.float32, "s_a")
+        M, K = gate.shape
+        assert up.shape == (M, K) and gate.stride(1) == 1 and up.stride(1) == 1 and gate.stride(0) == up.stride(0)
+        if out is None:
+            out = torch.zeros((M, K // 2), dtype=torch.uint8, device=gate.device)
+        _ok(self.lib.pq_swiglu_hadamard_quant_act(self.h, _ptr(gate), _ptr(up), M, K, gate.stride(0), had_block, row_begin, _ptr(s_a),
+                                                  _ptr(out), _stream()), "pq_swiglu_hadamard_quant_act")
         return out
 
     def w4a4_gemm(self, xq: torch.Tensor, wq: torch.Tensor, s_a: torch.Tensor, s_w: torch.Tensor, row_begin: int = 0,

@@ -5,7 +5,7 @@ scales, the KV cache with its full-precision prefix) and issues the C-ABI calls 
 block in App. B of the paper: RMSNorm -> [rotate + quantize] -> q|k|v GEMM -> rotary embedding (optionally
 followed by the head-wise rotation R3 of q and k) ->
 KV4 append -> causal attention over [prefix || INT4 cache] -> [rotate + quantize] -> o GEMM ->
-residual -> RMSNorm -> [rotate + quantize] -> gate|up GEMM -> SwiGLU -> [block rotate + quantize] ->
+residual -> RMSNorm -> [rotate + quantize] -> gate|up GEMM -> [SwiGLU + block rotate + quantize, one launch] ->
 down GEMM -> residual. The tokens that enter are ordinary tokens: the prefixed outlier tokens are
 never run through the quantized path, their K/V sit in the cache in fp16 (Sec. 4.2).
 """
@@ -92,6 +92,7 @@ class Block:
         before using them (a calibration batch; call it once with seed-1 data before timing anything).
         `tap(name, tensor)`, if given, is called after every stage with its output (buffers are reused
         later in the block, so a test that wants to look at one has to copy it there)."""
+        staged = tap is not None  # a caller that looks at every stage gets the SwiGLU output as a tensor of its own
         tap = tap or (lambda name, t: None)
         ctx, s, T = self.ctx, self.shape, x.shape[0]
         b = self._buffers(T, x.device)
@@ -136,11 +137,14 @@ class Block:
         tap("xq3", b["xq_h"])
         ctx.w4a4_gemm(b["xq_h"], self.wq_gu, self.s_a[2], self.sw_gu, out=b["gu"])
         tap("gu", b["gu"])
-        ctx.silu_mul(b["gu"][:, : s.ffn], b["gu"][:, s.ffn:], out=b["act"])
-        tap("act", b["act"])
-        if calibrate:
-            ctx.calib_act_scale(b["act"], s.had_block(s.ffn), 0, s_a=self.s_a[3])
-        ctx.hadamard_quant_act(b["act"], s.had_block(s.ffn), self.s_a[3], out=b["xq_f"])
+        if calibrate or staged:
+            ctx.silu_mul(b["gu"][:, : s.ffn], b["gu"][:, s.ffn:], out=b["act"])
+            tap("act", b["act"])
+            if calibrate:
+                ctx.calib_act_scale(b["act"], s.had_block(s.ffn), 0, s_a=self.s_a[3])
+            ctx.hadamard_quant_act(b["act"], s.had_block(s.ffn), self.s_a[3], out=b["xq_f"])
+        else:  # the SwiGLU is formed inside the rotation kernel: same bits, the activation tensor stays on chip
+            ctx.swiglu_hadamard_quant_act(b["gu"][:, : s.ffn], b["gu"][:, s.ffn:], s.had_block(s.ffn), self.s_a[3], out=b["xq_f"])
         tap("xq4", b["xq_f"])
         ctx.w4a4_gemm(b["xq_f"], self.wq_down, self.s_a[3], self.sw_down, out=b["d"])
         tap("d", b["d"])
@@ -148,4 +152,4 @@ class Block:
         tap("y", b["y"])
         return b["y"]
 
-    LAUNCHES_PER_FORWARD = 16
+    LAUNCHES_PER_FORWARD = 15  # 16 when every stage is tapped (the SwiGLU then is a launch of its own)

@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(EW_THREADS)
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const float g0 = bf16_lo(gw[e]), g1 = bf16_hi(gw[e]);
-      o[e] = pack_bf16(g0 / (1.0f + expf(-g0)) * bf16_lo(uw[e]), g1 / (1.0f + expf(-g1)) * bf16_hi(uw[e]));
+      o[e] = pack_bf16(pq::silu_mul_f32(g0, bf16_lo(uw[e])), pq::silu_mul_f32(g1, bf16_hi(uw[e])));
     }
     *reinterpret_cast<uint4*>(y + row * ldy + col) = make_uint4(o[0], o[1], o[2], o[3]);
   }

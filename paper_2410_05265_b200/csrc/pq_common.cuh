@@ -33,6 +33,11 @@ namespace pq {
 
 __device__ __forceinline__ void report(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
 
+// SiLU(g) * u in fp32 with the hardware exponential and reciprocal (about 2 ulp of fp32, far below the bf16
+// rounding that follows); the stand-alone kernel and the one fused into the rotation share it, so they agree
+// bit for bit.
+__device__ __forceinline__ float silu_mul_f32(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
 // ---- mbarrier -----------------------------------------------------------------------------

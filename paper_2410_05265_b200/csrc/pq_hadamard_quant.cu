@@ -35,11 +35,18 @@ __device__ __forceinline__ float key_float(uint32_t k) {
   return __uint_as_float(k ^ ((k >> 31) ? 0x80000000u : 0xFFFFFFFFu));
 }
 
-template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP>
+// SWIGLU: the input of the transform is SiLU(x) * x2 (the gate and up halves of the MLP, App. B), computed in fp32
+// and rounded to bf16 exactly as the stand-alone kernel stores it, so that fusing it changes no bit; the
+// activation tensor of the down projection then never goes to memory.
+__device__ __forceinline__ float swiglu_bf16(float g, float u) {
+  return __bfloat162float(__float2bfloat16_rn(pq::silu_mul_f32(g, u)));
+}
+
+template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU>
 __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
     hadamard_quant_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int64_t n_rows, int64_t K,
                           const float* __restrict__ s_a_in, uint8_t* __restrict__ xq, float* __restrict__ s_a_out,
-                          float clip, const int32_t* __restrict__ zp_in) {
+                          float clip, const int32_t* __restrict__ zp_in, const __nv_bfloat16* __restrict__ x2) {
   static_assert(BITS == 4 || BITS == 8, "code width");
   constexpr int QMAX = BITS == 4 ? 7 : 127;  // codes lie in [-QMAX - 1, QMAX]
   constexpr int B = 1 << LOGB;
@@ -91,10 +98,21 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
       uint32_t w[32];
 #pragma unroll
       for (int r = 0; r < 32; ++r) w[r] = active ? __ldg(src + r * (RSTRIDE / 2)) : 0u;
+      if (SWIGLU) {
+        const uint32_t* src2 = reinterpret_cast<const uint32_t*>(x2 + row * ldx + col0) + u;
 #pragma unroll
-      for (int r = 0; r < 32; ++r) {
-        const float a = __uint_as_float(w[r] << 16), b = __uint_as_float(w[r] & 0xFFFF0000u);
-        V[r] = ROTATE ? make_float2(a + b, a - b) : make_float2(a, b);
+        for (int r = 0; r < 32; ++r) {
+          const uint32_t w2 = active ? __ldg(src2 + r * (RSTRIDE / 2)) : 0u;
+          const float a = swiglu_bf16(__uint_as_float(w[r] << 16), __uint_as_float(w2 << 16));
+          const float b = swiglu_bf16(__uint_as_float(w[r] & 0xFFFF0000u), __uint_as_float(w2 & 0xFFFF0000u));
+          V[r] = ROTATE ? make_float2(a + b, a - b) : make_float2(a, b);
+        }
+      } else {
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+          const float a = __uint_as_float(w[r] << 16), b = __uint_as_float(w[r] & 0xFFFF0000u);
+          V[r] = ROTATE ? make_float2(a + b, a - b) : make_float2(a, b);
+        }
       }
     }
     if (ROTATE) {
@@ -249,10 +267,10 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
   }
 }
 
-template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP>
+template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU>
 pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_t K, const float* s_a_in, uint8_t* xq,
-                 float* s_a_out, float clip, const int32_t* zp_in, cudaStream_t st) {
-  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN, ZP>;
+                 float* s_a_out, float clip, const int32_t* zp_in, const void* x2, cudaStream_t st) {
+  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>;
   constexpr size_t smem = HQ_SMEM_FLOATS * sizeof(float);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
     return PQ_ERR_CUDA;
@@ -272,16 +290,17 @@ pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x), ldx, n_rows, K, s_a_in, xq, s_a_out, clip, zp_in) !=
-      cudaSuccess)
+  if (cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x), ldx, n_rows, K, s_a_in, xq, s_a_out, clip, zp_in,
+                         static_cast<const __nv_bfloat16*>(x2)) != cudaSuccess)
     return PQ_ERR_CUDA;
   return pq_launch_status();
 }
 
-template <bool CALIB, int BITS, bool PER_TOKEN = false, bool ZP = false>
+template <bool CALIB, int BITS, bool PER_TOKEN = false, bool ZP = false, bool SWIGLU = false>
 pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block, int64_t row_begin,
                    const float* s_a_in, uint8_t* xq, float* s_a_out, void* stream, float clip = 1.0f,
-                   const int32_t* zp_in = nullptr) {
+                   const int32_t* zp_in = nullptr, const void* x2 = nullptr) {
+  if (SWIGLU && (!x2 || (reinterpret_cast<uintptr_t>(x2) & 3))) return x2 ? PQ_ERR_ALIGN : PQ_ERR_INVALID_ARG;
   if (!ctx || !x || (!CALIB && (!s_a_in || !xq)) || (CALIB && !s_a_out)) return PQ_ERR_INVALID_ARG;
   if (M < 0 || K <= 0 || ldx < K || row_begin < 0 || had_block < 0) return PQ_ERR_INVALID_ARG;
   if (K % 128 != 0) return PQ_ERR_SHAPE;
@@ -294,6 +313,7 @@ pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx
   if (row_begin >= M) return PQ_OK;
   const int64_t n_rows = M - row_begin;
   const void* x0 = static_cast<const __nv_bfloat16*>(x) + row_begin * ldx;
+  const void* x20 = SWIGLU ? static_cast<const __nv_bfloat16*>(x2) + row_begin * ldx : nullptr;
   uint8_t* xq0 = CALIB ? nullptr : xq + row_begin * (BITS == 4 ? K / 2 : K);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (PER_TOKEN) {  // the arrays are indexed by row
@@ -302,14 +322,14 @@ pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx
     if (CALIB && cudaMemsetAsync(s_a_out, 0, static_cast<size_t>(n_rows) * sizeof(float), st) != cudaSuccess) return PQ_ERR_CUDA;
   }
   switch (had_block) {
-    case 0: return launch<7, false, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
-    case 128: return launch<7, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
-    case 256: return launch<8, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
-    case 512: return launch<9, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
-    case 1024: return launch<10, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
-    case 2048: return launch<11, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
-    case 4096: return launch<12, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
-    case 8192: return launch<13, true, CALIB, BITS, PER_TOKEN, ZP>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, st);
+    case 0: return launch<7, false, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
+    case 128: return launch<7, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
+    case 256: return launch<8, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
+    case 512: return launch<9, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
+    case 1024: return launch<10, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
+    case 2048: return launch<11, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
+    case 4096: return launch<12, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
+    case 8192: return launch<13, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
     default: return PQ_ERR_SHAPE;
   }
 }
@@ -390,4 +410,12 @@ extern "C" pq_status pq_hadamard_quant_act_asym(pq_ctx* ctx, const void* x, int6
                                                 uint8_t* xq, void* stream) {
   if (!z_a) return PQ_ERR_INVALID_ARG;
   return dispatch<false, 4, false, true>(ctx, x, M, K, ldx, had_block, row_begin, s_a, xq, nullptr, stream, 1.0f, z_a);
+}
+
+// ---- SwiGLU fused into the rotation of the down projection's input (App. B: R4 sits between the two) ------
+extern "C" pq_status pq_swiglu_hadamard_quant_act(pq_ctx* ctx, const void* gate, const void* up, int64_t M, int64_t K,
+                                                  int64_t ld_in, int had_block, int64_t row_begin, const float* s_a,
+                                                  uint8_t* xq, void* stream) {
+  return dispatch<false, 4, false, false, true>(ctx, gate, M, K, ld_in, had_block, row_begin, s_a, xq, nullptr, stream, 1.0f,
+                                                nullptr, up);
 }

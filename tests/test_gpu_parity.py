@@ -344,6 +344,27 @@ def test_rope_rotate_matches_oracle(ctx, T, H, pos0):
     assert float((s_plain - s_rot).abs().max()) <= 2.0**-6 * float(s_plain.abs().max())
 
 
+@pytest.mark.parametrize("M,F,B,row_begin", [(19, 1024, 1024, 0), (33, 14336, 2048, 4), (5, 256, 128, 1), (130, 4096, 4096, 0)])
+def test_swiglu_fused_into_rotate_quantize_changes_no_bit(ctx, M, F, B, row_begin):
+    """SiLU(gate) * up formed inside the rotation kernel against the two-launch path (which the oracle checks
+    stage by stage elsewhere) and against the oracle chain itself."""
+    gu = (inputs.activations(M, 2 * F, seed=3, n_prefix=row_begin) * 2).to(torch.bfloat16)
+    gud = gu.cuda()
+    gate, up = gud[:, :F], gud[:, F:]
+    act = ctx.silu_mul(gate, up)
+    s_a = ctx.calib_act_scale(act, B, row_begin)
+    two = torch.full((M, F // 2), 0x5A, dtype=torch.uint8, device="cuda")
+    one = torch.full((M, F // 2), 0x5A, dtype=torch.uint8, device="cuda")
+    ctx.hadamard_quant_act(act, B, s_a, row_begin, out=two)
+    ctx.swiglu_hadamard_quant_act(gate, up, B, s_a, row_begin, out=one)
+    ctx.check()
+    assert torch.equal(one, two)
+    act_ref = orc.silu_mul(inputs.bits(gu[:, :F].contiguous()), inputs.bits(gu[:, F:].contiguous()))
+    ref, tie = orc.quant_act(act_ref, B, np.float32(float(s_a)), row_begin, want_tie_dist=True)
+    if np.array_equal(inputs.bits(act), act_ref):  # the SwiGLU itself is within one bf16 ulp of the oracle, usually equal
+        assert_codes_tie_tolerant(to_np(one)[row_begin:], ref[row_begin:], tie[row_begin:], "fused swiglu codes")
+
+
 def test_silu_mul_and_residual_match_oracle(ctx):
     M, F = 19, 1024
     gu = (inputs.activations(M, 2 * F, seed=3) * 2).to(torch.bfloat16)
