@@ -210,7 +210,7 @@ __global__ void __launch_bounds__(32 * G) prefill_attn_kernel(const PrefillParam
     for (int j = 0; j < 8; ++j) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        float v = s[j][e] * scale;
+        float v = s[j][e];  // raw: the (positive) score scale is applied with the subtraction of the maximum below
         if (need_mask) {
           const int key = 8 * j + 2 * t + (e & 1);  // within the block
           const int tok = (e & 2) ? tok_b : tok_a;
@@ -226,19 +226,23 @@ __global__ void __launch_bounds__(32 * G) prefill_attn_kernel(const PrefillParam
     for (int r = 0; r < 2; ++r) {
       mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
       mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-      const float m_new = fmaxf(m_run[r], mx[r]);
+      const float m_new = fmaxf(m_run[r], mx[r] * scale);
       alpha[r] = m_new == -INFINITY ? 1.0f : ex2f(m_run[r] - m_new);
       m_run[r] = m_new;
       l_run[r] *= alpha[r];
     }
+    // after the first blocks the running maximum seldom moves: the rescaling is skipped when no row of the warp needs it
+    if (__any_sync(0xffffffffu, alpha[0] != 1.0f || alpha[1] != 1.0f)) {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) o[i][0] *= alpha[0], o[i][1] *= alpha[0], o[i][2] *= alpha[1], o[i][3] *= alpha[1];
+      for (int i = 0; i < 16; ++i) o[i][0] *= alpha[0], o[i][1] *= alpha[0], o[i][2] *= alpha[1], o[i][3] *= alpha[1];
+    }
     const float pscale = blk < 0 ? inv_sv : 1.0f;  // prefix values are real values, the accumulator is in code units
     uint32_t pa[4][4];  // A fragments of P for the four 16-key steps
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const float ma = m_run[0] == -INFINITY ? 0.0f : m_run[0], mb = m_run[1] == -INFINITY ? 0.0f : m_run[1];
-      const float p0 = ex2f(s[j][0] - ma), p1 = ex2f(s[j][1] - ma), p2 = ex2f(s[j][2] - mb), p3 = ex2f(s[j][3] - mb);
+      const float p0 = ex2f(fmaf(s[j][0], scale, -ma)), p1 = ex2f(fmaf(s[j][1], scale, -ma));
+      const float p2 = ex2f(fmaf(s[j][2], scale, -mb)), p3 = ex2f(fmaf(s[j][3], scale, -mb));
       const uint32_t lo = pack_h2(p0 * pscale, p1 * pscale), hi = pack_h2(p2 * pscale, p3 * pscale);
       // the denominator sums what the MMA multiplies with (rounded to fp16), in probability units
       const float2 fl = __half22float2(*reinterpret_cast<const __half2*>(&lo)), fh = __half22float2(*reinterpret_cast<const __half2*>(&hi));
