@@ -420,10 +420,18 @@ def section_decode_attention(ctx, device, peaks):
     for c in caches:
         c.length.fill_(T - 40)
     ms_both = _graph_time(torch, both, 32, reps=3)
+    for c in caches:
+        c.length.fill_(T - 40)
+
+    def fused(i):
+        ctx.kv4_append_decode_attn(caches[i % layers], k1, v1, q, sm, ws, out=out)
+
+    ms_fused = _graph_time(torch, fused, 32, reps=3)
     ctx.check()
     by = B * Hkv * (T + 1) * (D // 2) * 2 + Hkv * P * D * 2 * 2 + 2 * B * Hq * D * 2 + 2 * Hkv * 4
     gbs = by / (ms_attn * 1e-3) / 1e9
     return {"attention_us": round(ms_attn * 1e3, 3), "append_us": round(ms_app * 1e3, 3), "append+attention_us": round(ms_both * 1e3, 3),
+            "append+attention_one_launch_us": round(ms_fused * 1e3, 3),
             "GB/s": round(gbs, 1), "frac_measured_hbm": round(gbs / peaks["hbm"], 3), "frac_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 3),
             "bytes_per_step": by}
 

@@ -195,6 +195,14 @@ size_t pq_decode_attn_workspace_bytes(const pq_kv4_cache* cache);
 pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, const void* q, void* out, float sm_scale,
                                     void* ws, size_t ws_bytes, void* stream);
 
+/* pq_kv4_append (T_new = 1) and pq_decode_attn_kv4_prefix in one launch: the new token's k, v bf16 [B, 1, Hkv, D]
+ * (dense) are quantized and written at position len[b], the attention sees every prefixed key, the cached keys
+ * 0 .. len[b] - 1 and the new one (as its dequantized codes, exactly what a later call reads back), and
+ * len[b] advances by one. If any sequence is full nothing is appended anywhere, the attention runs over the
+ * cache as it is and PQ_ERR_SHAPE is reported through the status word. Arguments as in the two calls. */
+pq_status pq_kv4_append_decode_attn(pq_ctx* ctx, const pq_kv4_cache* cache, const void* k, const void* v, const void* q,
+                                    void* out, float sm_scale, void* ws, size_t ws_bytes, void* stream);
+
 /* Causal prefill attention of one sequence over [prefix || 4-bit cache] (Sec. 4.2, Eq. 3): query
  * token t sees every prefixed key and the cached keys 0..t of sequence `seq` (the cache rows must
  * already hold the T tokens: call pq_kv4_append first).

@@ -28,7 +28,7 @@ EXPORTS = [
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
     "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
     "pq_calib_act_asym", "pq_hadamard_quant_act_asym", "pq_weight_code_sums", "pq_w4a4_gemm_asym",
-    "pq_swiglu_hadamard_quant_act",
+    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn",
 ]
 
 
@@ -103,6 +103,8 @@ def load_library() -> ctypes.CDLL:
                                       c_int64, c_int64, c_int64, c_void_p, c_void_p]
     lib.pq_swiglu_hadamard_quant_act.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p,
                                                  c_void_p, c_void_p]
+    lib.pq_kv4_append_decode_attn.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_void_p, c_void_p, c_void_p, c_void_p, c_float,
+                                              c_void_p, c_size_t, c_void_p]
     for name in EXPORTS:
         getattr(lib, name)
         if name not in ("pq_status_string", "pq_w4a4_gemm_workspace_bytes", "pq_decode_attn_workspace_bytes"):
@@ -413,6 +415,18 @@ class Context:
             out = torch.empty_like(q)
         _ok(self.lib.pq_decode_attn_kv4_prefix(self.h, ctypes.byref(cache.struct), _ptr(q), _ptr(out), float(sm_scale),
                                                _ptr(ws), ws.numel(), _stream()), "pq_decode_attn_kv4_prefix")
+        return out
+
+    def kv4_append_decode_attn(self, cache: KV4Cache, k: torch.Tensor, v: torch.Tensor, q: torch.Tensor, sm_scale: float,
+                               ws: torch.Tensor, out: torch.Tensor | None = None):
+        """kv4_append of one token per sequence and decode_attn in one launch (k, v bf16 [B, 1, Hkv, D], dense)."""
+        _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v")
+        assert q.shape == (cache.B, cache.Hq, cache.D) and q.is_contiguous()
+        assert k.shape == (cache.B, 1, cache.Hkv, cache.D) and v.shape == k.shape and k.is_contiguous() and v.is_contiguous()
+        if out is None:
+            out = torch.empty_like(q)
+        _ok(self.lib.pq_kv4_append_decode_attn(self.h, ctypes.byref(cache.struct), _ptr(k), _ptr(v), _ptr(q), _ptr(out),
+                                               float(sm_scale), _ptr(ws), ws.numel(), _stream()), "pq_kv4_append_decode_attn")
         return out
 
 

@@ -186,6 +186,12 @@ struct AttnParams {
   int32_t* status;  // device status word; null for the entry point that has no context
   float sm_scale;
   int B, Hq, Hkv, G, n_prefix, Tmax;
+  // fused append (decode_attn_kernel<.., true>): the new token's k, v [B, Hkv, 128], the writable lengths and one
+  // counter per sequence
+  const __nv_bfloat16* k_new;
+  const __nv_bfloat16* v_new;
+  int32_t* len_rw;
+  uint32_t* len_tickets;
 };
 
 // Grid (splits, Hkv, B). The cache of one (sequence, KV head) is cut into rounds of 128 keys; split s
@@ -210,7 +216,12 @@ struct AttnParams {
 // CLUSTER: the splits of a (sequence, head) form one thread-block cluster and merge their partials
 // through distributed shared memory (no workspace, no ticket); otherwise the partials go through the
 // caller's workspace and the last CTA to finish merges them.
-template <bool CLUSTER>
+// FUSED: the call also appends one token per sequence (what pq_kv4_append does for T_new = 1). The attention
+// streams the cache as it was; the CTA of the last split quantizes the new k and v of its head, writes their codes
+// to row len[b] and folds the new key into its partial like one more full-precision key whose key and value are
+// the dequantized codes. The last CTA of a sequence to finish (every CTA of the sequence has read len[b] by then)
+// advances len[b]. As with the two calls, nothing is appended anywhere when any sequence is full.
+template <bool CLUSTER, bool FUSED>
 __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnParams p) {
   extern __shared__ __align__(128) uint8_t da_stage[];  // DA_SLOTS slots of [K rows | V rows] of one round
   // the per-warp partial outputs reuse the staging area once the key loop is over
@@ -221,7 +232,10 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   __shared__ float2 cl_ml[DA_ROWS];
   __shared__ __align__(8) uint64_t full[DA_SLOTS][DA_CHUNKS];
   __shared__ float sm_ml[DA_WARPS][DA_ROWS][2];
-  __shared__ float sm_pre[DA_ROWS][DA_MAX_PREFIX];
+  __shared__ float sm_pre[DA_ROWS][DA_MAX_PREFIX + 1];  // the last column: the key appended by this call
+  __shared__ float sm_newv[FUSED ? 128 : 1];             // its dequantized value
+  __shared__ float sm_red[DA_WARPS][DA_ROWS];
+  __shared__ int sm_full;
   __shared__ int is_last;
 
   const int split = blockIdx.x, S = gridDim.x, h = blockIdx.y, b = blockIdx.z;
@@ -253,6 +267,13 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
                       ? __ldg(reinterpret_cast<const uint2*>(p.prefix_v + (static_cast<int64_t>(h) * p.n_prefix + j) * 128) + lane)
                       : make_uint2(0u, 0u);
 
+  const bool has_extra = FUSED && split == S - 1;
+  float k_new_d = 0.0f, v_new_d = 0.0f;  // this thread's head dim of the token being appended
+  if (has_extra) {
+    const int64_t off = (static_cast<int64_t>(b) * p.Hkv + h) * 128 + threadIdx.x;
+    k_new_d = __bfloat162float(p.k_new[off]), v_new_d = __bfloat162float(p.v_new[off]);
+  }
+  if (FUSED && threadIdx.x == 0) sm_full = 0;
   // the operands of the first 16 (head, prefix key) pairs (all of them for a 4-token prefix under 4 heads)
   uint4 pre_q[2] = {}, pre_k[2] = {};
   if (has_prefix) {
@@ -286,6 +307,30 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
       if (speculated(n / DA_CHUNKS)) issue_chunk(n / DA_CHUNKS, n % DA_CHUNKS, DA_CHUNK);
   }
   __syncthreads();  // every barrier is initialised (all warps are still together here: this costs nothing)
+  if (FUSED) {  // one verdict for the whole batch, as the append call gives it
+    for (int i = threadIdx.x; i < p.B; i += DA_THREADS) {
+      const int l = __ldg(p.len + i);
+      if (l < 0 || l + 1 > p.Tmax) sm_full = 1;
+    }
+    __syncthreads();
+  }
+  const bool append_ok = FUSED && !sm_full;
+  const int len_raw = len_b;
+  // called by every CTA when it is done: the last one of this sequence advances the length
+  auto finish_append = [&]() {
+    if (FUSED && threadIdx.x == 0) {
+      if (!append_ok) {
+        if (p.status && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) pq::report(p.status, PQ_ERR_SHAPE);
+      } else {
+        __threadfence();
+        const uint32_t n_ctas = gridDim.x * gridDim.y;  // splits x KV heads of this sequence
+        if (atomicAdd(p.len_tickets + b, 1u) == n_ctas - 1) {
+          p.len_rw[b] = len_raw + 1;
+          p.len_tickets[b] = 0;
+        }
+      }
+    }
+  };
   len_b = len_b < 0 ? 0 : (len_b > p.Tmax ? p.Tmax : len_b);
   const int t1 = len_b;
   const int n_rounds_all = (len_b + DA_ROUND - 1) / DA_ROUND;
@@ -324,6 +369,34 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
       acc += __shfl_xor_sync(0xffffffffu, acc, 2);
       acc += __shfl_xor_sync(0xffffffffu, acc, 4);
       if (ok && sub == 0) sm_pre[r][j] = acc * p.sm_scale * 1.4426950408889634f;
+    }
+  }
+
+  // ---- the appended token: codes to the cache, score and value of the new key for this CTA's partial ----------
+  if (has_extra && append_ok) {
+    const float sk_h = s_k_h;
+    const int kc = max(-8, min(7, __float2int_rn(__fdiv_rn(k_new_d, sk_h))));
+    const int vc = max(-8, min(7, __float2int_rn(__fdiv_rn(v_new_d, s_v_h))));
+    // two head dims per byte, low nibble first: the even thread of a pair writes
+    const int kc_hi = __shfl_down_sync(0xffffffffu, kc, 1), vc_hi = __shfl_down_sync(0xffffffffu, vc, 1);
+    if ((threadIdx.x & 1) == 0) {
+      const int64_t row = (static_cast<int64_t>(bh) * p.Tmax + len_raw) * 64 + (threadIdx.x >> 1);
+      const_cast<uint8_t*>(p.kq)[row] = static_cast<uint8_t>((kc & 0xF) | ((kc_hi & 0xF) << 4));
+      const_cast<uint8_t*>(p.vq)[row] = static_cast<uint8_t>((vc & 0xF) | ((vc_hi & 0xF) << 4));
+    }
+    sm_newv[FUSED ? threadIdx.x : 0] = static_cast<float>(vc) * s_v_h;
+    for (int r = 0; r < G; ++r) {  // q[r] . k_code over the 128 threads
+      float part = __bfloat162float(p.q[(static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + threadIdx.x]) * static_cast<float>(kc);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+      if (lane == 0) sm_red[warp][r] = part;
+    }
+    __syncthreads();
+    if (threadIdx.x < G) {
+      float dot = 0.0f;
+#pragma unroll
+      for (int w = 0; w < DA_WARPS; ++w) dot += sm_red[w][threadIdx.x];
+      sm_pre[threadIdx.x][p.n_prefix] = dot * sk_h * p.sm_scale * 1.4426950408889634f;
     }
   }
 
@@ -535,6 +608,7 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   {
     // warp w takes the heads w, w + 4; lane c4 of it the head dims 4 c4 .. 4 c4 + 3
     const int n_pre = has_prefix ? p.n_prefix : 0;
+    const bool extra = has_extra && append_ok;  // the appended key sits in column n_prefix of sm_pre
     const int c4 = lane;
     const int qpos = 16 * ((2 * c4) & 7) + 2 * (c4 >> 2);  // dims 4 c4, +1 here, dims 4 c4 + 2, +3 sixteen floats on
     for (int r = warp; r < G; r += DA_WARPS) {
@@ -542,6 +616,7 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
 #pragma unroll
       for (int w = 0; w < DA_WARPS; ++w) m = fmaxf(m, sm_ml[w][r][0]);
       for (int j = 0; j < n_pre; ++j) m = fmaxf(m, sm_pre[r][j]);
+      if (extra) m = fmaxf(m, sm_pre[r][p.n_prefix]);
       float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
       float l = 0.0f;
 #pragma unroll
@@ -565,6 +640,12 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
         const float2 v01 = __half22float2(*reinterpret_cast<const __half2*>(&pv.x));
         const float2 v23 = __half22float2(*reinterpret_cast<const __half2*>(&pv.y));
         acc.x = fmaf(e, v01.x, acc.x), acc.y = fmaf(e, v01.y, acc.y), acc.z = fmaf(e, v23.x, acc.z), acc.w = fmaf(e, v23.y, acc.w);
+        l += e;
+      }
+      if (extra) {
+        const float e = ex2(sm_pre[r][p.n_prefix] - m);
+        const float4 nv = *reinterpret_cast<const float4*>(sm_newv + (FUSED ? 4 * c4 : 0));
+        acc.x = fmaf(e, nv.x, acc.x), acc.y = fmaf(e, nv.y, acc.y), acc.z = fmaf(e, nv.z, acc.z), acc.w = fmaf(e, nv.w, acc.w);
         l += e;
       }
       if (CLUSTER) {
@@ -615,13 +696,17 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
       *reinterpret_cast<uint2*>(p.out + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + 4 * c4) = packed;
     }
     cluster_arrive_wait();  // no CTA leaves while a peer may still read its shared memory
+    finish_append();
     return;
   }
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) is_last = (atomicAdd(p.tickets + DA_TICKET0 + bh, 1u) == static_cast<uint32_t>(S - 1));
   __syncthreads();
-  if (!is_last) return;
+  if (!is_last) {
+    finish_append();
+    return;
+  }
   __threadfence();
 
   // ---- last CTA of this (sequence, KV head): merge the S partials --------------------------------
@@ -681,6 +766,7 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
     *reinterpret_cast<uint2*>(p.out + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + 4 * c4) = packed;
   }
   if (threadIdx.x == 0) p.tickets[DA_TICKET0 + bh] = 0;
+  finish_append();
 }
 
 // The kernel needs the dynamic shared-memory attribute set once per device (this allocates nothing).
@@ -689,9 +775,13 @@ bool set_attn_smem() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
   if (!done[dev]) {
-    if (cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) !=
+    if (cudaFuncSetAttribute(decode_attn_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) !=
             cudaSuccess ||
-        cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) !=
+        cudaFuncSetAttribute(decode_attn_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(decode_attn_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(decode_attn_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) !=
             cudaSuccess)
       return false;
     done[dev] = true;
@@ -752,14 +842,19 @@ extern "C" size_t pq_decode_attn_workspace_bytes(const pq_kv4_cache* cache) {
   return static_cast<size_t>(cache->B) * cache->Hkv * DA_MAX_SPLITS * G * (128 + 2) * sizeof(float);
 }
 
-extern "C" pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, const void* q, void* out,
-                                               float sm_scale, void* ws, size_t ws_bytes, void* stream) {
+namespace {
+constexpr int DA_LEN_TICKET0 = PQ_N_TICKETS / 2;  // one counter per sequence for the fused append
+
+// k_new, v_new: null for the plain attention; else the token appended by the same launch.
+pq_status decode_attn_launch(pq_ctx* ctx, const pq_kv4_cache* cache, const void* q, void* out, float sm_scale, void* ws,
+                             size_t ws_bytes, void* stream, const void* k_new, const void* v_new) {
   if (!ctx || !q || !out) return PQ_ERR_INVALID_ARG;
   pq_status st = check_cache(cache);
   if (st != PQ_OK) return st;
   if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 7)) return PQ_ERR_ALIGN;
   if (cache->B == 0) return PQ_OK;
-  if (static_cast<int64_t>(cache->B) * cache->Hkv > PQ_N_TICKETS - DA_TICKET0 || cache->B > 65535 || cache->Hkv > 65535)
+  if (static_cast<int64_t>(cache->B) * cache->Hkv > DA_LEN_TICKET0 - DA_TICKET0 || cache->B > DA_LEN_TICKET0 ||
+      cache->Hkv > 65535)
     return PQ_ERR_SHAPE;
   if (!ws || ws_bytes < pq_decode_attn_workspace_bytes(cache)) return PQ_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(ws) & 15) return PQ_ERR_ALIGN;
@@ -785,6 +880,11 @@ extern "C" pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* 
   p.status = ctx->d_status;
   p.sm_scale = sm_scale;
   p.B = cache->B, p.Hq = cache->Hq, p.Hkv = cache->Hkv, p.G = G, p.n_prefix = cache->n_prefix, p.Tmax = cache->Tmax;
+  const bool fused = k_new != nullptr;
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.len_rw = cache->len;
+  p.len_tickets = ctx->d_tickets + DA_LEN_TICKET0;
   dim3 grid(S, cache->Hkv, cache->B);
   if (!set_attn_smem()) return PQ_ERR_CUDA;
   if (cluster) {
@@ -800,11 +900,30 @@ extern "C" pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_attn_kernel<true>, p) != cudaSuccess) return PQ_ERR_CUDA;
+    if ((fused ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<true, true>, p)
+               : cudaLaunchKernelEx(&cfg, decode_attn_kernel<true, false>, p)) != cudaSuccess)
+      return PQ_ERR_CUDA;
     return pq_launch_status();
   }
-  decode_attn_kernel<false><<<grid, DA_THREADS, DA_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(p);
+  if (fused)
+    decode_attn_kernel<false, true><<<grid, DA_THREADS, DA_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(p);
+  else
+    decode_attn_kernel<false, false><<<grid, DA_THREADS, DA_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(p);
   return pq_launch_status();
+}
+}  // namespace
+
+extern "C" pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, const void* q, void* out,
+                                               float sm_scale, void* ws, size_t ws_bytes, void* stream) {
+  return decode_attn_launch(ctx, cache, q, out, sm_scale, ws, ws_bytes, stream, nullptr, nullptr);
+}
+
+extern "C" pq_status pq_kv4_append_decode_attn(pq_ctx* ctx, const pq_kv4_cache* cache, const void* k, const void* v,
+                                               const void* q, void* out, float sm_scale, void* ws, size_t ws_bytes,
+                                               void* stream) {
+  if (!k || !v) return PQ_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(k) & 1) || (reinterpret_cast<uintptr_t>(v) & 1)) return PQ_ERR_ALIGN;
+  return decode_attn_launch(ctx, cache, q, out, sm_scale, ws, ws_bytes, stream, k, v);
 }
 
 // ================================================================================= no-allocation variant
@@ -894,6 +1013,6 @@ extern "C" pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache
   p.B = cache->B, p.Hq = cache->Hq, p.Hkv = cache->Hkv, p.G = G, p.n_prefix = cache->n_prefix, p.Tmax = cache->Tmax;
   dim3 grid(S, cache->Hkv, cache->B);
   if (!set_attn_smem()) return PQ_ERR_CUDA;
-  decode_attn_kernel<false><<<grid, DA_THREADS, DA_SMEM_BYTES, cs>>>(p);
+  decode_attn_kernel<false, false><<<grid, DA_THREADS, DA_SMEM_BYTES, cs>>>(p);
   return pq_launch_status();
 }

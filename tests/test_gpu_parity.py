@@ -245,6 +245,70 @@ def test_decode_attention_short_sequences_in_long_caches(ctx):
     _run_attention(ctx, 8, 32, 8, 4, 1, 4096, 1.0, start=[0, 10, 200, 1000, 127, 128, 129, 4000])
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,P,Tmax,start", [
+    (1, 4, 1, 0, 64, [0]),                      # empty cache, no prefix: the new key is the only key
+    (2, 8, 2, 2, 128, [99, 0]),
+    (3, 32, 8, 4, 400, [333, 17, 398]),
+    (8, 32, 8, 4, 4096, [4091, 10, 200, 1000, 127, 128, 129, 4000]),   # cluster merge
+    (1, 8, 1, 3, 8192, [129]),                  # 32 splits through the workspace
+])
+def test_fused_append_and_decode_attention_equals_the_two_calls(ctx, B, Hq, Hkv, P, Tmax, start):
+    from paper_2410_05265_b200 import binding
+
+    D = 128
+    k, v, s_k, s_v, pk, pv, q = _kv_setup(B, Hq, Hkv, D, P, 1, Tmax, 1.0, 0)
+    start = np.asarray(start, np.int32)
+    kq_ref = np.full((B, Hkv, Tmax, D // 2), 0x11, np.uint8)
+    vq_ref = np.full_like(kq_ref, 0x11)
+    len_ref = start.copy()
+    assert orc.kv4_append(inputs.bits(k), inputs.bits(v), s_k, s_v, kq_ref, vq_ref, len_ref) == 0
+    _, out_ref = orc.decode_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq_ref, vq_ref, s_k, s_v, len_ref,
+                                 1 / math.sqrt(D), want_f64=True)
+
+    def fresh():
+        kq = torch.full((B, Hkv, Tmax, D // 2), 0x11, dtype=torch.uint8, device="cuda")
+        vq = torch.full_like(kq, 0x11)
+        return binding.KV4Cache(pk.cuda() if P else None, pv.cuda() if P else None, kq, vq, dev(s_k), dev(s_v), dev(start), Hq)
+
+    cache = fresh()
+    ws = ctx.decode_attn_workspace(cache)
+    out = ctx.kv4_append_decode_attn(cache, k.cuda(), v.cuda(), q.cuda(), 1 / math.sqrt(D), ws)
+    ctx.check()
+    assert np.array_equal(to_np(cache.length), len_ref)
+    assert np.array_equal(to_np(cache.kq), kq_ref) and np.array_equal(to_np(cache.vq), vq_ref), "appended codes must match bit for bit"
+    assert_attn_close(inputs.bits(out), out_ref, "fused append + decode attention")
+    # the two calls on a fresh cache agree with the fused one (same codes, same keys; both round to bf16, whose ulp
+    # alone is 4e-3 of a value)
+    cache2 = fresh()
+    ctx.kv4_append(cache2, k.cuda(), v.cuda())
+    out2 = ctx.decode_attn(cache2, q.cuda(), 1 / math.sqrt(D), ws)
+    ctx.check()
+    assert torch.equal(cache2.kq, cache.kq) and torch.equal(cache2.length, cache.length)
+    assert float((out.float() - out2.float()).abs().max()) <= 8e-3 * float(out2.float().abs().max()) + 1e-6
+    # a second fused call appends the next token
+    out3 = ctx.kv4_append_decode_attn(cache, k.cuda(), v.cuda(), q.cuda(), 1 / math.sqrt(D), ws)
+    ctx.check()
+    assert np.array_equal(to_np(cache.length), len_ref + 1)
+
+
+def test_fused_append_refuses_a_full_sequence(ctx):
+    from paper_2410_05265_b200 import binding
+
+    B, Hq, Hkv, D, Tmax = 2, 4, 2, 128, 64
+    k, v, s_k, s_v, pk, pv, q = _kv_setup(B, Hq, Hkv, D, 0, 1, Tmax, 1.0, 0)
+    kq = torch.full((B, Hkv, Tmax, D // 2), 0x11, dtype=torch.uint8, device="cuda")
+    vq = torch.full_like(kq, 0x11)
+    length = torch.tensor([10, 64], dtype=torch.int32, device="cuda")   # the second sequence is full
+    cache = binding.KV4Cache(None, None, kq, vq, dev(s_k), dev(s_v), length, Hq)
+    ws = ctx.decode_attn_workspace(cache)
+    out = ctx.kv4_append_decode_attn(cache, k.cuda(), v.cuda(), q.cuda(), 1 / math.sqrt(D), ws)
+    assert ctx.check_status() == 2                                      # PQ_ERR_SHAPE through the status word
+    assert length.tolist() == [10, 64] and bool((kq == 0x11).all()), "nothing is appended anywhere"
+    ref = ctx.decode_attn(cache, q.cuda(), 1 / math.sqrt(D), ws)       # the attention ran over the cache as it was
+    assert ctx.check_status() == 0
+    assert float((out.float() - ref.float()).abs().max()) <= 1e-6
+
+
 def test_kv4_append_refuses_overflow(ctx):
     from paper_2410_05265_b200 import binding
 
