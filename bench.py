@@ -428,10 +428,25 @@ def section_decode_attention(ctx, device, peaks):
 
     ms_fused = _graph_time(torch, fused, 32, reps=3)
     ctx.check()
+    # one long sequence (Llama-3-70B heads, 32K context): few (sequence, head) pairs, several clusters of splits each
+    del caches
+    Bl, Hql, Tl, Tmaxl, nl = 1, 64, 32764, 32768, 10
+    long_caches = [binding.KV4Cache(pk, pv, torch.randint(0, 256, (Bl, Hkv, Tmaxl, D // 2), dtype=torch.uint8, device=device),
+                                    torch.randint(0, 256, (Bl, Hkv, Tmaxl, D // 2), dtype=torch.uint8, device=device), s_k, s_v,
+                                    torch.full((Bl,), Tl, dtype=torch.int32, device=device), Hql) for _ in range(nl)]
+    ql = inputs.queries(Bl, Hql, D, 0, device=device)
+    wsl = ctx.decode_attn_workspace(long_caches[0])
+    outl = torch.empty_like(ql)
+    ms_long = _graph_time(torch, lambda i: ctx.decode_attn(long_caches[i % nl], ql, sm, wsl, out=outl), 8 * nl)
+    ctx.check()
+    del long_caches
+    by_long = Bl * Hkv * Tl * D
     by = B * Hkv * (T + 1) * (D // 2) * 2 + Hkv * P * D * 2 * 2 + 2 * B * Hq * D * 2 + 2 * Hkv * 4
     gbs = by / (ms_attn * 1e-3) / 1e9
     return {"attention_us": round(ms_attn * 1e3, 3), "append_us": round(ms_app * 1e3, 3), "append+attention_us": round(ms_both * 1e3, 3),
             "append+attention_one_launch_us": round(ms_fused * 1e3, 3),
+            "long_context_b1_hq64_t32764": {"attention_us": round(ms_long * 1e3, 3),
+                                            "frac_measured_hbm": round(by_long / (ms_long * 1e-3) / 1e9 / peaks["hbm"], 3)},
             "GB/s": round(gbs, 1), "frac_measured_hbm": round(gbs / peaks["hbm"], 3), "frac_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 3),
             "bytes_per_step": by}
 

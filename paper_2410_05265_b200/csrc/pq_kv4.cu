@@ -221,7 +221,8 @@ struct AttnParams {
 // to row len[b] and folds the new key into its partial like one more full-precision key whose key and value are
 // the dequantized codes. The last CTA of a sequence to finish (every CTA of the sequence has read len[b] by then)
 // advances len[b]. As with the two calls, nothing is appended anywhere when any sequence is full.
-template <bool CLUSTER, bool FUSED>
+// MULTI (with CLUSTER): a (sequence, head) has several clusters of eight splits.
+template <bool CLUSTER, bool FUSED, bool MULTI = false>
 __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnParams p) {
   extern __shared__ __align__(128) uint8_t da_stage[];  // DA_SLOTS slots of [K rows | V rows] of one round
   // the per-warp partial outputs reuse the staging area once the key loop is over
@@ -658,11 +659,17 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
       }
     }
   }
+  // Clusters hold up to eight consecutive splits. One cluster per (sequence, head) writes the result itself;
+  // several (few sequences, long caches) each leave one merged partial in the workspace and the last cluster to
+  // finish merges those few.
+  const int csize = S < 8 ? S : 8, n_clusters = MULTI ? S / csize : 1;
+  const int n_parts = CLUSTER ? n_clusters : S;  // partials per (sequence, head) that meet in the workspace
   if (CLUSTER) {
     // every split's partial is in its CTA's shared memory; thread i of the cluster takes (head, four
-    // dims) item i and reads the S partials through distributed shared memory, all loads at once
+    // dims) item i and reads the cluster's partials through distributed shared memory, all loads at once
     cluster_arrive_wait();
-    const int item = split * DA_THREADS + threadIdx.x;  // split == rank in the cluster
+    const int rank = split % csize, ci = split / csize;
+    const int item = rank * DA_THREADS + threadIdx.x;
     if (item < G * 32) {
       const int r = item >> 5, c4 = item & 31;
       const uint32_t o_addr = pq::smem_u32(cl_o + r * 128 + 4 * c4), ml_addr = pq::smem_u32(cl_ml + r);
@@ -670,7 +677,7 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
       float2 ml[8];
 #pragma unroll
       for (int sp = 0; sp < 8; ++sp) {
-        if (sp < S) {
+        if (sp < csize) {
           v[sp] = ld_cluster_f4(map_cta(o_addr, sp));
           ml[sp] = ld_cluster_f2(map_cta(ml_addr, sp));
         } else {
@@ -689,19 +696,28 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
         acc.x = fmaf(v[sp].x, w, acc.x), acc.y = fmaf(v[sp].y, w, acc.y), acc.z = fmaf(v[sp].z, w, acc.z), acc.w = fmaf(v[sp].w, w, acc.w);
         l = fmaf(ml[sp].y, w, l);
       }
-      const float inv = l > 0.0f ? 1.0f / l : 0.0f;
-      const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-      uint2 packed;
-      packed.x = *reinterpret_cast<const uint32_t*>(&lo), packed.y = *reinterpret_cast<const uint32_t*>(&hi);
-      *reinterpret_cast<uint2*>(p.out + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + 4 * c4) = packed;
+      if (n_clusters == 1) {
+        const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+        uint2 packed;
+        packed.x = *reinterpret_cast<const uint32_t*>(&lo), packed.y = *reinterpret_cast<const uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(p.out + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + 4 * c4) = packed;
+      } else {  // this cluster's partial, in the layout of a split's partial
+        const int64_t slot = (static_cast<int64_t>(bh) * n_clusters + ci) * G + r;
+        *reinterpret_cast<float4*>(p.ws_o + slot * 128 + 4 * c4) = acc;
+        if (c4 == 0) *reinterpret_cast<float2*>(p.ws_ml + slot * 2) = make_float2(m, l);
+        __threadfence();
+      }
     }
     cluster_arrive_wait();  // no CTA leaves while a peer may still read its shared memory
-    finish_append();
-    return;
+    if (n_clusters == 1 || rank != 0) {
+      finish_append();
+      return;
+    }
   }
   __threadfence();
   __syncthreads();
-  if (threadIdx.x == 0) is_last = (atomicAdd(p.tickets + DA_TICKET0 + bh, 1u) == static_cast<uint32_t>(S - 1));
+  if (threadIdx.x == 0) is_last = (atomicAdd(p.tickets + DA_TICKET0 + bh, 1u) == static_cast<uint32_t>(n_parts - 1));
   __syncthreads();
   if (!is_last) {
     finish_append();
@@ -709,33 +725,33 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   }
   __threadfence();
 
-  // ---- last CTA of this (sequence, KV head): merge the S partials --------------------------------
+  // ---- last CTA of this (sequence, KV head): merge the partials --------------------------------
   // One L2 round trip: every (m, l) pair and the first eight partial columns of each thread are
   // requested together; the weights are computed while the columns are in flight.
   float* part_m = reinterpret_cast<float*>(da_stage);  // [S][G]; the staging area is free again
   float* part_l = part_m + DA_MAX_SPLITS * DA_ROWS;
   float* part_w = part_l + DA_MAX_SPLITS * DA_ROWS;
   float* head_l = part_w + DA_MAX_SPLITS * DA_ROWS;    // [G]
-  for (int i = threadIdx.x; i < S * G; i += DA_THREADS) {
-    const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.ws_ml) + static_cast<int64_t>(bh) * S * G + i);
+  for (int i = threadIdx.x; i < n_parts * G; i += DA_THREADS) {
+    const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.ws_ml) + static_cast<int64_t>(bh) * n_parts * G + i);
     part_m[i] = ml.x, part_l[i] = ml.y;
   }
-  const float4* wo = reinterpret_cast<const float4*>(p.ws_o) + static_cast<int64_t>(bh) * S * G * 32;
+  const float4* wo = reinterpret_cast<const float4*>(p.ws_o) + static_cast<int64_t>(bh) * n_parts * G * 32;
   const int n_items = G * 32;  // (head, group of four dims)
   float4 pre[8];
   {
     const int item = threadIdx.x, r = item >> 5, c4 = item & 31;
 #pragma unroll
     for (int sp = 0; sp < 8; ++sp)
-      pre[sp] = (item < n_items && sp < S) ? __ldcg(wo + (sp * G + r) * 32 + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      pre[sp] = (item < n_items && sp < n_parts) ? __ldcg(wo + (sp * G + r) * 32 + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   __syncthreads();
   if (threadIdx.x < G) {
     const int r = threadIdx.x;
     float m = -INFINITY;
-    for (int sp = 0; sp < S; ++sp) m = fmaxf(m, part_m[sp * G + r]);
+    for (int sp = 0; sp < n_parts; ++sp) m = fmaxf(m, part_m[sp * G + r]);
     float l = 0.0f;
-    for (int sp = 0; sp < S; ++sp) {
+    for (int sp = 0; sp < n_parts; ++sp) {
       const float ms = part_m[sp * G + r];
       const float e = ms == -INFINITY ? 0.0f : ex2(ms - m);  // also covers m == -inf (nothing cached, no prefix)
       part_w[sp * G + r] = e;
@@ -747,11 +763,11 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   for (int item = threadIdx.x; item < n_items; item += DA_THREADS) {
     const int r = item >> 5, c4 = item & 31;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int sp0 = 0; sp0 < S; sp0 += 8) {
+    for (int sp0 = 0; sp0 < n_parts; sp0 += 8) {
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const int sp = sp0 + u;
-        if (sp < S) {
+        if (sp < n_parts) {
           const float4 v = (sp0 == 0 && item == static_cast<int>(threadIdx.x)) ? pre[u] : __ldcg(wo + (sp * G + r) * 32 + c4);
           const float w = part_w[sp * G + r];
           acc.x = fmaf(v.x, w, acc.x), acc.y = fmaf(v.y, w, acc.y), acc.z = fmaf(v.z, w, acc.z), acc.w = fmaf(v.w, w, acc.w);
@@ -782,7 +798,11 @@ bool set_attn_smem() {
         cudaFuncSetAttribute(decode_attn_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) !=
             cudaSuccess ||
         cudaFuncSetAttribute(decode_attn_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DA_SMEM_BYTES) !=
-            cudaSuccess)
+            cudaSuccess ||
+        cudaFuncSetAttribute(decode_attn_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             DA_SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_attn_kernel<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             DA_SMEM_BYTES) != cudaSuccess)
       return false;
     done[dev] = true;
   }
@@ -861,8 +881,16 @@ pq_status decode_attn_launch(pq_ctx* ctx, const pq_kv4_cache* cache, const void*
   int S = choose_splits(ctx, cache);
   // With enough (sequence, head) pairs, eight splits already fill the GPU: the splits then form one
   // cluster and merge through distributed shared memory (the workspace and the tickets stay unused).
-  const bool cluster = static_cast<int64_t>(cache->B) * cache->Hkv * 8 >= 2LL * ctx->sm_count;
+  bool cluster = static_cast<int64_t>(cache->B) * cache->Hkv * 8 >= 2LL * ctx->sm_count;
   if (cluster && S > 8) S = 8;
+  // Few (sequence, head) pairs with long caches: several clusters of eight splits per pair; each merges its eight
+  // partials on chip, the workspace sees one partial per cluster.
+  if (!cluster && S >= 16) {
+    S = S / 8 * 8;
+    cluster = true;
+  }
+  const int n_parts = cluster ? (S < 8 ? 1 : S / 8) : S;
+  const bool multi = cluster && n_parts > 1;
   const int G = cache->Hq / cache->Hkv;
   AttnParams p;
   p.q = static_cast<const __nv_bfloat16*>(q);
@@ -875,7 +903,7 @@ pq_status decode_attn_launch(pq_ctx* ctx, const pq_kv4_cache* cache, const void*
   p.s_v = cache->s_v;
   p.len = cache->len;
   p.ws_o = static_cast<float*>(ws);
-  p.ws_ml = p.ws_o + static_cast<size_t>(cache->B) * cache->Hkv * S * G * 128;
+  p.ws_ml = p.ws_o + static_cast<size_t>(cache->B) * cache->Hkv * n_parts * G * 128;
   p.tickets = ctx->d_tickets;
   p.status = ctx->d_status;
   p.sm_scale = sm_scale;
@@ -895,14 +923,19 @@ pq_status decode_attn_launch(pq_ctx* ctx, const pq_kv4_cache* cache, const void*
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = S;
+    attr[0].val.clusterDim.x = S < 8 ? S : 8;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if ((fused ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<true, true>, p)
-               : cudaLaunchKernelEx(&cfg, decode_attn_kernel<true, false>, p)) != cudaSuccess)
-      return PQ_ERR_CUDA;
+    cudaError_t e;
+    if (multi)
+      e = fused ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<true, true, true>, p)
+                : cudaLaunchKernelEx(&cfg, decode_attn_kernel<true, false, true>, p);
+    else
+      e = fused ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<true, true, false>, p)
+                : cudaLaunchKernelEx(&cfg, decode_attn_kernel<true, false, false>, p);
+    if (e != cudaSuccess) return PQ_ERR_CUDA;
     return pq_launch_status();
   }
   if (fused)
