@@ -220,8 +220,8 @@ def run_gpu(args):
     int8_peak = 2.0 * peaks["bf16_sus"]  # dense INT8 = 2x dense bf16 (nominal ratio 4.5 / 2.25 PFLOP/s)
     achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
     roofline = {
-        "kernel": "gemm_w4a4_pair_kernel<false>", "bound": "tensor", "achieved": round(achieved, 1), "peak": round(int8_peak, 1),
-        "unit": "TOPS", "frac": round(achieved / int8_peak, 4), "traffic": 132744960,
+        "kernel": "gemm_w4a4_pair_kernel<false, false>", "bound": "tensor", "achieved": round(achieved, 1), "peak": round(int8_peak, 1),
+        "unit": "TOPS", "frac": round(achieved / int8_peak, 4), "traffic": 134375936,
         "traffic_note": "dram bytes read+written by the gate|up launch (ncu, profiles/gemm_w4a4_pair_2048x28672x4096.md); algorithmic 180.4 MB, the output partly still in L2",
         "peak_source": f"2 x bf16 sustained GEMM of {peaks['src']}", "frac_of_nominal_4500": round(achieved / NOMINAL_INT8_TOPS, 4),
         "frac_of_2x_bf16_burst": round(achieved / (2.0 * peaks["bf16"]), 4),
