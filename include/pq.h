@@ -270,7 +270,8 @@ pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache, const voi
 
 /* ---------------------------------------------------------------------------------------------
  * Eq. 1 as printed: asymmetric static per-tensor activation quantizer with a zero point (N = 4),
- *     s = (max y - min y) / 15,  z = -round(min y / s)        max-min initialisation (gamma = beta = 1)
+ *     s = (max y - min y) / 15,  z = -floor(min y / s)        max-min initialisation (gamma = beta = 1);
+ *                                                             the zero point takes the floor the equation prints
  *     u = clamp(round_half_even(y / s) + z, 0, 15),           dequantized value s (u - z)
  *     out[t, n] = bf16(s_a * s_w[n] * sum_k (u[t,k] - z) * w[n,k])
  *   pq_calib_act_asym           range of the rotated rows >= row_begin of one calibration batch -> *s_a, *z_a

@@ -236,7 +236,10 @@ void orc_quant_f64(const double* v, int64_t n, double s, int8_t* codes) {
 // ---- weight quantization: RTN, one scale per output channel (Table 1; Table 6 "RTN") --------
 // s_w[n] = fp32(max_k |W[n,k]|) / 7 in fp32 (1 if the row is all zero);
 // code = clamp(rint_fp32(W[n,k] / s_w[n]), -8, 7) with an fp32 IEEE division.
-void orc_quant_weights(const uint16_t* W, int64_t ldw, int64_t N, int64_t K, uint8_t* wq, float* s_w) {
+// tie_dist (nullable, [N,K] float) receives | W / s_w - nearest half-integer | with the quotient taken in
+// double: the distance of the exact pre-rounding value from the closest rounding tie, which bounds where
+// the fp32 decision can differ from a double one.
+void orc_quant_weights(const uint16_t* W, int64_t ldw, int64_t N, int64_t K, uint8_t* wq, float* s_w, float* tie_dist) {
   parallel_rows(N, [&](int64_t n) {
     float mx = 0.0f;
     for (int64_t k = 0; k < K; ++k) mx = std::max(mx, std::fabs(static_cast<float>(bf16_to_double(W[n * ldw + k]))));
@@ -249,6 +252,10 @@ void orc_quant_weights(const uint16_t* W, int64_t ldw, int64_t N, int64_t K, uin
       volatile float q = w / s;  // fp32 division, no double intermediate
       float r = std::nearbyintf(q);
       nib_set(out, k, clampi(static_cast<long>(r), -8, 7));
+      if (tie_dist) {
+        const double rd = static_cast<double>(w) / static_cast<double>(s);
+        tie_dist[n * K + k] = static_cast<float>(std::fabs(rd - std::floor(rd) - 0.5));
+      }
     }
   });
 }
@@ -403,7 +410,7 @@ void orc_outlier_tokens(const uint16_t* x, int64_t ldx, int64_t T, int64_t C, fl
   }
 }
 
-// ---- Eq. 1 as printed: asymmetric, with a zero point (static per-tensor activations, N = 4) ------------
+// ---- Eq. 1 with its zero point: asymmetric static per-tensor activations (N = 4) -------------------------
 // Range of the rotated calibration rows >= row_begin: mn = min fp32(y), mx = max fp32(y).
 void orc_calib_act_minmax(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin, float* mn_out,
                           float* mx_out) {
@@ -420,9 +427,10 @@ void orc_calib_act_minmax(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, 
   *mn_out = static_cast<float>(mn), *mx_out = static_cast<float>(mx);
 }
 
-// Max-min initialisation (gamma = beta = 1): s = (mx - mn) / (2^N - 1), z = -round(mn / s), every step an
-// IEEE fp32 operation (the precision the GPU takes them in); a constant tensor gets s = 1, z = 0. z is
-// kept inside the code range.
+// Max-min initialisation (gamma = beta = 1): s = (mx - mn) / (2^N - 1), z = -floor(mn / s): Eq. 1 prints the
+// zero point with floor brackets (only X / s carries the rounding brackets), and the floor is taken here as
+// printed. Every step is an IEEE fp32 operation (the precision the GPU takes them in); a constant tensor
+// gets s = 1, z = 0. z is kept inside the code range.
 void orc_asym_params(float mn, float mx, int bits, float* s_out, int32_t* z_out) {
   const int qmax = (1 << bits) - 1;
   if (!(mx > mn)) {
@@ -433,7 +441,7 @@ void orc_asym_params(float mn, float mx, int bits, float* s_out, int32_t* z_out)
   const float s = static_cast<float>(static_cast<double>(d) / static_cast<double>(qmax));
   const float q = static_cast<float>(static_cast<double>(mn) / static_cast<double>(s));
   *s_out = s;
-  *z_out = clampi(-std::lrint(std::nearbyint(static_cast<double>(q))), 0, qmax);
+  *z_out = clampi(-std::lrint(std::floor(static_cast<double>(q))), 0, qmax);
 }
 
 // X_INT = clamp(round_half_even(y / s) + z, 0, 15), one byte per element, y the rotated row; rows < row_begin
@@ -484,9 +492,11 @@ void orc_calib_kv_scale(const uint16_t* kv, int64_t B, int64_t T, int64_t H, int
 
 // k, v bf16 [B,T_new,H,D] -> codes written at rows len[b] .. len[b]+T_new-1 of
 // kq, vq u8 [B,H,Tmax,D/2]; len[b] += T_new. Returns 1 (nothing written) if any sequence would
-// exceed Tmax.
+// exceed Tmax. tie_k, tie_v (nullable, [B,T_new,H,D] float): distance of the exact quotient x / s (taken in
+// double) from the closest rounding tie, as in orc_quant_act.
 int orc_kv4_append(const uint16_t* k, const uint16_t* v, int64_t B, int64_t T_new, int64_t H, int64_t D,
-                   const float* s_k, const float* s_v, uint8_t* kq, uint8_t* vq, int32_t* len, int64_t Tmax) {
+                   const float* s_k, const float* s_v, uint8_t* kq, uint8_t* vq, int32_t* len, int64_t Tmax,
+                   float* tie_k, float* tie_v) {
   for (int64_t b = 0; b < B; ++b)
     if (len[b] + T_new > Tmax) return 1;
   for (int64_t b = 0; b < B; ++b) {
@@ -503,6 +513,15 @@ int orc_kv4_append(const uint16_t* k, const uint16_t* v, int64_t B, int64_t T_ne
           volatile float qv = vf / s_v[h];
           nib_set(kr, d, clampi(static_cast<long>(std::nearbyintf(qk)), -8, 7));
           nib_set(vr, d, clampi(static_cast<long>(std::nearbyintf(qv)), -8, 7));
+          const int64_t idx = ((b * T_new + t) * H + h) * D + d;
+          if (tie_k) {
+            const double r = static_cast<double>(kf) / static_cast<double>(s_k[h]);
+            tie_k[idx] = static_cast<float>(std::fabs(r - std::floor(r) - 0.5));
+          }
+          if (tie_v) {
+            const double r = static_cast<double>(vf) / static_cast<double>(s_v[h]);
+            tie_v[idx] = static_cast<float>(std::fabs(r - std::floor(r) - 0.5));
+          }
         }
       }
     len[b] += static_cast<int32_t>(T_new);
@@ -568,10 +587,11 @@ void orc_decode_attn(const uint16_t* q, const uint16_t* prefix_k, const uint16_t
 
 // Prefill: T query tokens of one sequence; query t sees the whole prefix and cached keys 0..t
 // (the prefix sits at the beginning of the sequence, Sec. 4.2).
-// q bf16 [T,Hq,D]; kq/vq u8 [Hkv,Tmax,D/2] of this sequence; out bf16 [T,Hq,D].
+// q bf16 [T,Hq,D]; kq/vq u8 [Hkv,Tmax,D/2] of this sequence; out bf16 [T,Hq,D]; out_f64 (nullable)
+// receives the unrounded result.
 void orc_prefill_attn(const uint16_t* q, const uint16_t* prefix_k, const uint16_t* prefix_v, const uint8_t* kq,
                       const uint8_t* vq, const float* s_k, const float* s_v, int64_t T, int64_t Hq, int64_t Hkv,
-                      int64_t D, int64_t n_prefix, int64_t Tmax, double sm_scale, uint16_t* out) {
+                      int64_t D, int64_t n_prefix, int64_t Tmax, double sm_scale, uint16_t* out, double* out_f64) {
   int64_t group = Hq / Hkv;
   parallel_rows(T * Hq, [&](int64_t i) {
     int64_t t = i / Hq, g = i % Hq, h = g / group;
@@ -579,7 +599,10 @@ void orc_prefill_attn(const uint16_t* q, const uint16_t* prefix_k, const uint16_
     for (int64_t d = 0; d < D; ++d) qd[d] = bf16_to_double(q[(t * Hq + g) * D + d]);
     attend_one(qd.data(), D, sm_scale, prefix_k + h * n_prefix * D, prefix_v + h * n_prefix * D, n_prefix,
                kq + h * Tmax * (D / 2), vq + h * Tmax * (D / 2), t + 1, s_k[h], s_v[h], od.data());
-    for (int64_t d = 0; d < D; ++d) out[(t * Hq + g) * D + d] = double_to_bf16(od[d]);
+    for (int64_t d = 0; d < D; ++d) {
+      out[(t * Hq + g) * D + d] = double_to_bf16(od[d]);
+      if (out_f64) out_f64[(t * Hq + g) * D + d] = od[d];
+    }
   });
 }
 

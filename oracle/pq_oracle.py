@@ -238,7 +238,7 @@ def calib_act_minmax(x_bits: np.ndarray, block: int, row_begin: int = 0):
 
 
 def asym_params(mn, mx, bits: int = 4):
-    """Eq. 1 with gamma = beta = 1: step s = (mx - mn) / (2^bits - 1) and zero point z = -round(mn / s)."""
+    """Eq. 1 with gamma = beta = 1: step s = (mx - mn) / (2^bits - 1) and zero point z = -floor(mn / s)."""
     s, z = np.zeros(1, np.float32), np.zeros(1, np.int32)
     lib().orc_asym_params(c_float(float(mn)), c_float(float(mx)), c_int(bits), _p(s, c_float), _p(z, c_int32))
     return np.float32(s[0]), int(z[0])
@@ -269,13 +269,16 @@ def gemm_asym(u: np.ndarray, z: int, wq: np.ndarray) -> np.ndarray:
 
 
 # ---- weights ---------------------------------------------------------------------------------------
-def quant_weights(w_bits: np.ndarray):
+def quant_weights(w_bits: np.ndarray, want_tie_dist: bool = False):
+    """Packed codes [N,K/2], steps [N] and, optionally, the distance of each exact quotient from a rounding tie."""
     w_bits = _u16(w_bits)
     N, K = w_bits.shape
     wq = np.zeros((N, K // 2), np.uint8)
     s_w = np.empty((N,), np.float32)
-    lib().orc_quant_weights(_p(w_bits, c_uint16), c_int64(K), c_int64(N), c_int64(K), _p(wq, c_uint8), _p(s_w, c_float))
-    return wq, s_w
+    tie = np.full((N, K), 0.5, np.float32) if want_tie_dist else None
+    lib().orc_quant_weights(_p(w_bits, c_uint16), c_int64(K), c_int64(N), c_int64(K), _p(wq, c_uint8), _p(s_w, c_float),
+                            _p(tie, c_float) if want_tie_dist else None)
+    return (wq, s_w, tie) if want_tie_dist else (wq, s_w)
 
 
 # ---- GEMM --------------------------------------------------------------------------------------------
@@ -309,8 +312,9 @@ def calib_kv_scale(kv_bits: np.ndarray) -> np.ndarray:
     return s
 
 
-def kv4_append(k_bits, v_bits, s_k, s_v, kq, vq, length) -> int:
-    """In place on kq, vq [B,H,Tmax,D/2] and length [B] int32. Returns the oracle's status."""
+def kv4_append(k_bits, v_bits, s_k, s_v, kq, vq, length, tie_k=None, tie_v=None) -> int:
+    """In place on kq, vq [B,H,Tmax,D/2] and length [B] int32. Returns the oracle's status.
+    tie_k, tie_v: optional float32 [B,T_new,H,D] outputs, distance of each exact quotient from a rounding tie."""
     k_bits, v_bits = _u16(k_bits), _u16(v_bits)
     B, T_new, H, D = k_bits.shape
     Tmax = kq.shape[2]
@@ -321,6 +325,7 @@ def kv4_append(k_bits, v_bits, s_k, s_v, kq, vq, length) -> int:
         lib().orc_kv4_append(
             _p(k_bits, c_uint16), _p(v_bits, c_uint16), c_int64(B), c_int64(T_new), c_int64(H), c_int64(D),
             _p(s_k, c_float), _p(s_v, c_float), _p(kq, c_uint8), _p(vq, c_uint8), _p(length, c_int32), c_int64(Tmax),
+            _p(tie_k, c_float) if tie_k is not None else None, _p(tie_v, c_float) if tie_v is not None else None,
         )
     )
 
@@ -348,7 +353,7 @@ def decode_attn(q_bits, prefix_k, prefix_v, kq, vq, s_k, s_v, length, sm_scale, 
     return (out, out64) if want_f64 else out
 
 
-def prefill_attn(q_bits, prefix_k, prefix_v, kq, vq, s_k, s_v, sm_scale):
+def prefill_attn(q_bits, prefix_k, prefix_v, kq, vq, s_k, s_v, sm_scale, want_f64: bool = False):
     q_bits = _u16(q_bits)
     T, Hq, D = q_bits.shape
     prefix_k, prefix_v = _u16(prefix_k), _u16(prefix_v)
@@ -360,12 +365,13 @@ def prefill_attn(q_bits, prefix_k, prefix_v, kq, vq, s_k, s_v, sm_scale):
     s_k = np.ascontiguousarray(s_k, np.float32)
     s_v = np.ascontiguousarray(s_v, np.float32)
     out = np.empty((T, Hq, D), np.uint16)
+    out64 = np.empty((T, Hq, D), np.float64) if want_f64 else None
     lib().orc_prefill_attn(
         _p(q_bits, c_uint16), _p(prefix_k, c_uint16), _p(prefix_v, c_uint16), _p(kq, c_uint8), _p(vq, c_uint8),
         _p(s_k, c_float), _p(s_v, c_float), c_int64(T), c_int64(Hq), c_int64(Hkv), c_int64(D), c_int64(n_prefix),
-        c_int64(Tmax), c_double(float(sm_scale)), _p(out, c_uint16),
+        c_int64(Tmax), c_double(float(sm_scale)), _p(out, c_uint16), _p(out64, c_double) if want_f64 else None,
     )
-    return out
+    return (out, out64) if want_f64 else out
 
 
 # ---- block glue --------------------------------------------------------------------------------------------

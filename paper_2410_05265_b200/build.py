@@ -1,18 +1,24 @@
-"""Builds the CUDA library in-tree for sm_100a with nvcc (no GPU needed to compile)."""
+"""Builds the CUDA library in-tree for sm_100a with nvcc (no GPU needed to compile).
+
+Every `.cu` file of `csrc/` is compiled to an object of its own (in parallel, and only when the file or a
+header is newer than its object), then the objects are linked into `libpq_b200.so` next to this file.
+"""
 from __future__ import annotations
 
 import glob
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
+OBJ = os.path.join(_HERE, "_build")
 LIB = os.path.join(_HERE, "libpq_b200.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "--shared",
+    "-Xcompiler", "-fPIC",
 ]
 
 
@@ -20,20 +26,51 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def _headers():
+    return glob.glob(os.path.join(CSRC, "*.cuh")) + [os.path.join(_HERE, "..", "include", "pq.h")]
+
+
+def _obj(src: str) -> str:
+    return os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
+
+
+def _stale(target: str, deps) -> bool:
+    if not os.path.exists(target):
         return True
-    t = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + [os.path.join(_HERE, "..", "include", "pq.h")]
+    t = os.path.getmtime(target)
     return any(os.path.getmtime(d) > t for d in deps)
+
+
+def needs_build() -> bool:
+    return _stale(LIB, sources() + _headers())
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
+    os.makedirs(OBJ, exist_ok=True)
+    hdrs = _headers()
+    todo = [s for s in sources() if force or _stale(_obj(s), [s] + hdrs)]
+
+    def compile_one(src):
+        tmp = _obj(src) + f".{os.getpid()}.tmp"
+        cmd = [NVCC] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", tmp]
+        r = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+        if r.returncode != 0:
+            raise RuntimeError(f"nvcc failed on {os.path.basename(src)}:\n{r.stdout}")
+        os.replace(tmp, _obj(src))
+        return r.stdout
+
+    with ThreadPoolExecutor(max_workers=min(len(todo), os.cpu_count() or 1) or 1) as pool:
+        for log in pool.map(compile_one, todo):
+            if log.strip():
+                print(log, file=sys.stderr)
+    live = {_obj(s) for s in sources()}
+    for stale_obj in glob.glob(os.path.join(OBJ, "*.o")):  # objects of sources that no longer exist
+        if stale_obj not in live:
+            os.remove(stale_obj)
     tmp = LIB + f".{os.getpid()}.tmp"
-    cmd = [NVCC] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + sources() + ["-o", tmp]
-    subprocess.check_call(cmd)
+    subprocess.check_call([NVCC, "--shared", "-gencode", "arch=compute_100a,code=sm_100a"] + sorted(live) + ["-o", tmp])
     os.replace(tmp, LIB)
     return LIB
 

@@ -24,7 +24,7 @@ constexpr int HQ_SMEM_FLOATS = HQ_ELEMS + HQ_ELEMS / 64;  // + 2 floats of paddi
 
 // PER_TOKEN (the dynamic setting, Table 1, O1): one step per row instead of one per tensor; s_a_in / s_a_out
 // are then arrays indexed by row, and the calibration pass is the online first pass of every call.
-// ZP (Eq. 1 as printed, with a zero point): the quantizer adds z - 8 to the rounded value before the clamp, so
+// ZP (Eq. 1 with its zero point): the quantizer adds z - 8 to the rounded value before the clamp, so
 // that the stored signed nibble is the unsigned code minus 8; the calibration pass collects the minimum and
 // the maximum of the rotated values (as order-preserving integer keys in s_a_out[0] and s_a_out[1]).
 __device__ __forceinline__ uint32_t float_key(float f) {
@@ -371,17 +371,18 @@ extern "C" pq_status pq_hadamard_quant_act_rows(pq_ctx* ctx, const void* x, int6
   return dispatch<false, 4, true>(ctx, x, M, K, ldx, had_block, row_begin, s_tok, xq, nullptr, stream);
 }
 
-// ---- Eq. 1 as printed: asymmetric static per-tensor quantizer with a zero point -------------------------
+// ---- Eq. 1 with its zero point: asymmetric static per-tensor quantizer -----------------------------------
 namespace {
-// Max-min initialisation (gamma = beta = 1) from the collected range: s = (mx - mn) / 15, z = -round(mn / s),
-// every step one IEEE fp32 operation; a constant (or empty) range gives s = 1, z = 0.
+// Max-min initialisation (gamma = beta = 1) from the collected range: s = (mx - mn) / 15, z = -floor(mn / s)
+// (Eq. 1 prints the zero point with a floor), every step one IEEE fp32 operation; a constant (or empty) range
+// gives s = 1, z = 0.
 __global__ void asym_params_kernel(uint32_t* keys, float* s_a, int32_t* z_a) {
   const float mx = key_float(keys[0]), mn = key_float(keys[1]);
   float s = 1.0f;
   int z = 0;
   if (keys[0] >= keys[1] && mx > mn) {
     s = __fdiv_rn(__fsub_rn(mx, mn), 15.0f);
-    z = -__float2int_rn(__fdiv_rn(mn, s));
+    z = -__float2int_rd(__fdiv_rn(mn, s));
     z = z < 0 ? 0 : (z > 15 ? 15 : z);
   }
   *s_a = s;

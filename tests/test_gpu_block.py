@@ -10,7 +10,7 @@ import torch
 
 from oracle import pq_oracle as orc
 from paper_2410_05265_b200 import inputs
-from helpers import assert_bf16_close, assert_codes_tie_tolerant, bf16_ulp, to_np
+from helpers import assert_attn_close, assert_bf16_close, assert_codes_tie_tolerant, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -78,11 +78,9 @@ def test_block_stages_match_oracle(T, hidden, Hq, Hkv, ffn, P, r3):
     q_g = got_rope[:, :Hq].contiguous()
     pk_b = inputs.bits(pk) if P else np.zeros((Hkv, 0, D), np.uint16)
     pv_b = inputs.bits(pv) if P else np.zeros((Hkv, 0, D), np.uint16)
-    ref_attn = orc.bf16_to_f64(orc.prefill_attn(inputs.bits(q_g), pk_b, pv_b, to_np(taps["kq"])[0], to_np(taps["vq"])[0], s_k, s_v,
-                                                1 / math.sqrt(D)))
-    got_attn = orc.bf16_to_f64(inputs.bits(taps["attn"]))
-    vmax = np.abs(ref_attn).max(axis=-1, keepdims=True)
-    assert np.all(np.abs(got_attn - ref_attn) <= 2e-3 * vmax + bf16_ulp(ref_attn) + 1e-30), "prefill attention"
+    _, ref_attn = orc.prefill_attn(inputs.bits(q_g), pk_b, pv_b, to_np(taps["kq"])[0], to_np(taps["vq"])[0], s_k, s_v,
+                                   1 / math.sqrt(D), want_f64=True)
+    assert_attn_close(inputs.bits(taps["attn"]).reshape(T, Hq, D), ref_attn, "prefill attention")
     check_quant("xq2", inputs.bits(taps["attn"].reshape(T, qd)), B[1], s_a[1])
     check_gemm("o", "xq2", inputs.bits(w_o), s_a[1])
     assert np.array_equal(inputs.bits(taps["x2"]), orc.add(inputs.bits(x), inputs.bits(taps["o"])))

@@ -423,10 +423,13 @@ def test_swiglu_fused_into_rotate_quantize_changes_no_bit(ctx, M, F, B, row_begi
     ctx.swiglu_hadamard_quant_act(gate, up, B, s_a, row_begin, out=one)
     ctx.check()
     assert torch.equal(one, two)
+    # the SwiGLU itself against the oracle (within one bf16 ulp), then the oracle's rotation + quantizer on the GPU's
+    # own activation bits, so that an ulp of difference in the SwiGLU never hides the check of the codes
     act_ref = orc.silu_mul(inputs.bits(gu[:, :F].contiguous()), inputs.bits(gu[:, F:].contiguous()))
-    ref, tie = orc.quant_act(act_ref, B, np.float32(float(s_a)), row_begin, want_tie_dist=True)
-    if np.array_equal(inputs.bits(act), act_ref):  # the SwiGLU itself is within one bf16 ulp of the oracle, usually equal
-        assert_codes_tie_tolerant(to_np(one)[row_begin:], ref[row_begin:], tie[row_begin:], "fused swiglu codes")
+    assert_bf16_close(inputs.bits(act), act_ref, "silu_mul feeding the rotation")
+    ref, tie = orc.quant_act(inputs.bits(act), B, np.float32(float(s_a)), row_begin, want_tie_dist=True)
+    n = assert_codes_tie_tolerant(to_np(one)[row_begin:], ref[row_begin:], tie[row_begin:], "fused swiglu codes")
+    assert n <= max(2, int(2e-4 * act.numel()))
 
 
 def test_silu_mul_and_residual_match_oracle(ctx):
@@ -461,21 +464,15 @@ def test_prefill_attention_matches_oracle(ctx, T, Hq, Hkv, P, mag):
     pv = inputs.prefix_kv(Hkv, max(P, 1), D, 0, "v", mag)[:, :P].contiguous()
     seq = 1
     q = inputs.kv_tensor(1, T, Hq, D, 3, "k")[0].contiguous()
-    ref = orc.prefill_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq_ref[seq], vq_ref[seq], s_k, s_v,
-                           1 / math.sqrt(D))
+    _, ref64 = orc.prefill_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq_ref[seq], vq_ref[seq], s_k, s_v,
+                                1 / math.sqrt(D), want_f64=True)
     cache = binding.KV4Cache(pk.cuda() if P else None, pv.cuda() if P else None, dev(kq_ref), dev(vq_ref), dev(s_k), dev(s_v),
                              torch.full((B,), T, dtype=torch.int32, device="cuda"), Hq)
     out = torch.full((T, Hq, D), 7.0, dtype=torch.bfloat16, device="cuda")
     ctx.prefill_attn(cache, seq, q.cuda(), 1 / math.sqrt(D), out=out)
     ctx.check()
-    got = orc.bf16_to_f64(inputs.bits(out))
-    r = orc.bf16_to_f64(ref)
-    vmax = np.abs(r).max(axis=-1, keepdims=True)
-    # the stated attention tolerance on the computed value, plus the bf16 store rounding of both sides
-    # (half an ulp each: the oracle's prefill result is only available rounded)
-    tol = 2e-3 * vmax + bf16_ulp(r) + 1e-30
-    bad = np.abs(got - r) > tol
-    assert not bad.any(), f"{bad.sum()} of {bad.size} outside tolerance; worst {np.max(np.abs(got - r) / np.maximum(vmax, 1e-30))}"
+    # the stated attention tolerance against the oracle's unrounded result (plus the bf16 store's own half ulp)
+    assert_attn_close(inputs.bits(out), ref64, f"prefill attention T{T} Hq{Hq} Hkv{Hkv} P{P}")
 
 
 # ------------------------------------------------------------------------------- outlier tokens (Sec. 4.1, Eq. 2)

@@ -215,6 +215,73 @@ def test_weight_quantization_rtn_per_channel():
     assert np.array_equal(orc.unpack_int4(wq2)[:, :15], np.arange(-7, 8)[None, :].repeat(3, 0)) and np.all(s2 == 0.25)
 
 
+def _rne_codes_f64(x, s, lo=-8, hi=7):
+    """clamp(round_half_even(x / s)) with the quotient in float64 (numpy's rint rounds half to even)."""
+    return np.clip(np.rint(x.astype(np.float64) / s.astype(np.float64)), lo, hi).astype(np.int64)
+
+
+def test_weight_quantizer_tie_direction_and_fp32_decision():
+    # exact ties: a row whose maximum is 1.75 has step 1.75 / 7 = 0.25 exactly; the elements (k + 1/2) / 4 are
+    # bf16 numbers whose quotient is exactly k + 1/2. Half-even sends them to the even neighbour, both signs.
+    ks = np.arange(-7, 7)
+    row = np.concatenate([(ks + 0.5) * 0.25, [1.75, -1.75]])
+    wq, s_w, tie = orc.quant_weights(bf16_bits(row[None, :]), want_tie_dist=True)
+    codes = orc.unpack_int4(wq)[0]
+    assert s_w[0] == 0.25 and np.all(tie[0, :14] == 0.0) and np.all(tie[0, 14:] == 0.5)
+    want = np.where(ks % 2 == 0, ks, ks + 1)  # k + 1/2 -> the even one of k, k + 1
+    assert codes[:14].tolist() == want.tolist() and codes[14:].tolist() == [7, -7]
+    assert codes[ks.tolist().index(0)] == 0 and codes[ks.tolist().index(-1)] == 0 and codes[ks.tolist().index(1)] == 2
+    # the fp32 decision equals the double-precision one except next to a tie: on the synthetic weights every
+    # differing code sits within 1e-4 of a tie and differs by exactly one, and such cases are rare
+    W = inputs.weights(64, 4096, seed=2)
+    wq, s_w, tie = orc.quant_weights(inputs.bits(W), want_tie_dist=True)
+    got = orc.unpack_int4(wq).astype(np.int64)
+    ref = _rne_codes_f64(W.to(torch.float64).numpy(), s_w[:, None])
+    diff = got != ref
+    assert np.all(tie[diff] < 1e-4) and np.all(np.abs(got - ref)[diff] == 1)
+    assert diff.sum() <= 1e-3 * diff.size, diff.sum()  # bf16 inputs over a max/7 step land next to ties often
+    # away from ties nothing is left to the precision: the code is the nearest integer of the exact quotient
+    far = tie > 1e-4
+    r = W.to(torch.float64).numpy() / s_w[:, None].astype(np.float64)
+    assert np.all(np.abs(got - r)[far] < 0.5)
+
+
+def test_kv_quantizer_tie_direction_and_fp32_decision():
+    # exact ties with a power-of-two step, k even and odd, both signs; beyond +-7.5 steps the code clamps
+    B, T, H, D, Tmax = 1, 1, 1, 16, 2
+    ks = np.arange(-8, 8)
+    kvals = (ks + 0.5) * 0.25          # k + 1/2 for k = -8 .. 7: -7.5 .. 7.5 steps
+    vvals = (ks + 0.5) * 2.0
+    kb, vb = bf16_bits(kvals.reshape(B, T, H, D)), bf16_bits(vvals.reshape(B, T, H, D))
+    kq, vq = np.zeros((B, H, Tmax, D // 2), np.uint8), np.zeros((B, H, Tmax, D // 2), np.uint8)
+    tie_k, tie_v = np.ones((B, T, H, D), np.float32), np.ones((B, T, H, D), np.float32)
+    length = np.zeros(B, np.int32)
+    assert orc.kv4_append(kb, vb, np.array([0.25], np.float32), np.array([2.0], np.float32), kq, vq, length, tie_k, tie_v) == 0
+    want = np.clip(np.where(ks % 2 == 0, ks, ks + 1), -8, 7)
+    assert orc.unpack_int4(kq)[0, 0, 0].tolist() == want.tolist() == [-8, -6, -6, -4, -4, -2, -2, 0, 0, 2, 2, 4, 4, 6, 6, 7]
+    assert orc.unpack_int4(vq)[0, 0, 0].tolist() == want.tolist()
+    assert np.all(tie_k == 0.0) and np.all(tie_v == 0.0)
+    # fp32-decided codes against the double-precision decision on the synthetic K/V with max/7 steps
+    B, T, H, D, Tmax = 4, 64, 8, 128, 64
+    k, v = inputs.kv_tensor(B, T, H, D, 0, "k"), inputs.kv_tensor(B, T, H, D, 0, "v")
+    s_k = orc.calib_kv_scale(inputs.bits(inputs.kv_tensor(B, T, H, D, 1, "k")))
+    s_v = orc.calib_kv_scale(inputs.bits(inputs.kv_tensor(B, T, H, D, 1, "v")))
+    kq, vq = np.zeros((B, H, Tmax, D // 2), np.uint8), np.zeros((B, H, Tmax, D // 2), np.uint8)
+    tie_k, tie_v = np.ones((B, T, H, D), np.float32), np.ones((B, T, H, D), np.float32)
+    assert orc.kv4_append(inputs.bits(k), inputs.bits(v), s_k, s_v, kq, vq, np.zeros(B, np.int32), tie_k, tie_v) == 0
+    for x, s, q, tie in ((k, s_k, kq, tie_k), (v, s_v, vq, tie_v)):
+        got = orc.unpack_int4(q).astype(np.int64).transpose(0, 2, 1, 3)  # [B,T,H,D]
+        xd = x.to(torch.float64).numpy()
+        ref = _rne_codes_f64(xd, s[None, None, :, None])
+        diff = got != ref
+        assert np.all(tie[diff] < 1e-4) and np.all(np.abs(got - ref)[diff] == 1)
+        assert diff.sum() <= 1e-3 * diff.size, diff.sum()  # bf16 inputs over a max/7 step land next to ties often
+        r = xd / s[None, None, :, None].astype(np.float64)
+        inside = (tie > 1e-4) & (r > -8.5) & (r < 7.5)
+        assert np.all(np.abs(got - r)[inside] < 0.5)
+        assert np.all(got[r >= 7.5] == 7) and np.all(got[r <= -8.5] == -8)  # beyond the range the code clamps
+
+
 # ---------------------------------------------------------------- integer GEMM
 def test_gemm_brute_force_tiny():
     M, N, K = 3, 5, 8
@@ -374,6 +441,11 @@ def test_asymmetric_quantizer_hand_values_and_reduction_to_the_symmetric_one():
     # range [-1, 2.75]: s = 3.75 / 15 = 0.25, z = -round(-1 / 0.25) = 4
     s, z = orc.asym_params(-1.0, 2.75)
     assert s == 0.25 and z == 4
+    # Eq. 1 prints the zero point with a floor: range [-1.0625, 2.6875] has s = 0.25, min / s = -4.25,
+    # z = -floor(-4.25) = 5 (rounding would give 4); [-1.1875, 2.5625]: min / s = -4.75, z = 5 either way
+    assert orc.asym_params(-1.0625, 2.6875) == (0.25, 5)
+    assert orc.asym_params(-1.1875, 2.5625) == (0.25, 5)
+    assert orc.asym_params(0.0625, 3.8125) == (0.25, 0)                # floor(0.25) = 0; a positive range keeps z = 0
     assert orc.asym_params(3.0, 3.0) == (1.0, 0)                       # a constant tensor
     assert orc.asym_params(0.0, 15.0) == (1.0, 0) and orc.asym_params(-15.0, 0.0) == (1.0, 15)
     vals = np.array([-1.0, 2.75, 0.125, 0.375, -0.125, -0.375, 5.0, -3.0, 0.0, 1.0, 0.3, -0.3])
@@ -401,8 +473,13 @@ def test_asymmetric_quantizer_hand_values_and_reduction_to_the_symmetric_one():
     assert mn == y.min() and mx == y.max()
     s2, z2 = orc.asym_params(mn, mx)
     u2 = orc.quant_act_asym(xb, K, s2, z2, row_begin=4)
-    assert u2[4:].min() == 0 and u2[4:].max() == 15 and np.all(u2[:4] == 0)
-    assert np.all(np.abs(s2 * (u2[4:].astype(np.float64) - z2) - y) <= 0.5 * s2 * (1 + 1e-5) + 1e-6)
+    # with the printed floor the zero point is ceil(-min / s): the minimum lands on code 0 or 1, and when it lands
+    # on 1 the top of the range is clamped at 15 (one step lost there), never the bottom
+    assert u2[4:].min() in (0, 1) and u2[4:].max() == 15 and np.all(u2[:4] == 0)
+    assert z2 == int(np.ceil(-np.float64(mn) / np.float64(s2)))
+    err = np.abs(s2 * (u2[4:].astype(np.float64) - z2) - y)
+    top = u2[4:] == 15
+    assert np.all(err[~top] <= 0.5 * s2 * (1 + 1e-5) + 1e-6) and np.all(err[top] <= 1.5 * s2 * (1 + 1e-5) + 1e-6)
 
 
 def test_gemm_asym_is_the_dequantized_product():
@@ -553,11 +630,12 @@ def test_prefill_attention_is_causal_decode_per_row():
     vq = rng.integers(0, 256, (Hkv, Tmax, D // 2)).astype(np.uint8)
     s_k = np.array([0.2, 0.3], np.float32)
     s_v = np.array([0.4, 0.1], np.float32)
-    out = orc.prefill_attn(inputs.bits(qt), inputs.bits(pk), inputs.bits(pv), kq, vq, s_k, s_v, 0.25)
+    out, out64 = orc.prefill_attn(inputs.bits(qt), inputs.bits(pk), inputs.bits(pv), kq, vq, s_k, s_v, 0.25, want_f64=True)
+    assert np.array_equal(out, orc.f64_to_bf16(out64))
     for t in range(T):
-        ref = orc.decode_attn(inputs.bits(qt[t:t + 1]), inputs.bits(pk), inputs.bits(pv), kq[None], vq[None], s_k, s_v,
-                              np.array([t + 1], np.int32), 0.25)
-        assert np.array_equal(out[t], ref[0])
+        ref, ref64 = orc.decode_attn(inputs.bits(qt[t:t + 1]), inputs.bits(pk), inputs.bits(pv), kq[None], vq[None], s_k, s_v,
+                                     np.array([t + 1], np.int32), 0.25, want_f64=True)
+        assert np.array_equal(out[t], ref[0]) and np.array_equal(out64[t], ref64[0])
     # without a prefix the first token attends to itself only: its output is its own value row
     out0 = orc.prefill_attn(inputs.bits(qt), inputs.bits(pk[:, :0]), inputs.bits(pv[:, :0]), kq, vq, s_k, s_v, 0.25)
     vd = orc.unpack_int4(vq).astype(np.float64) * s_v.astype(np.float64)[:, None, None]
