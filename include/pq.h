@@ -107,7 +107,14 @@ pq_status pq_swiglu_hadamard_quant_act(pq_ctx* ctx, const void* gate, const void
  *   acc_dbg  nullable int32 [M, N] dense: receives the raw accumulators (parity checks)
  *   K % 32 == 0, K <= 65536. Output rows below row_begin are left untouched.
  * Shapes with M - row_begin > 16 run on the tensor-core kernel (TMA + tcgen05, kind::i8);
- * smaller M runs the weight-streaming kernel. No workspace is needed (ws may be NULL). */
+ * smaller M runs the weight-streaming kernel. No workspace is needed (ws may be NULL).
+ * Weights are static (Sec. 3: quantized offline): the weight-streaming kernel starts fetching wq
+ * while the kernel before it in the stream is still draining (programmatic dependent launch), and
+ * only xq, the scales and out are ordered behind that kernel. wq (and wsum of the _asym call)
+ * must therefore be complete before the kernel that precedes this call in the stream starts.
+ * Weights written earlier in the same stream by pq_quant_weights / pq_weight_code_sums or by a copy
+ * always are: those never let a successor start early. This holds for pq_w4a4_gemm, pq_w4a8_gemm,
+ * pq_w4a4_gemm_rows and pq_w4a4_gemm_asym alike. */
 size_t pq_w4a4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
 pq_status pq_w4a4_gemm(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
                        void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int64_t row_begin, int32_t* acc_dbg,
@@ -264,7 +271,10 @@ pq_status pq_residual_add(pq_ctx* ctx, const void* a, const void* b, void* y, in
  *     contents: the counters are cleared in stream order at the start of each call, the partials
  *     are fully rewritten before they are read. Two calls that overlap on the GPU (different
  *     streams, or different host threads without ordering) race on it and give wrong results;
- *     issue them in one stream or order them yourself. */
+ *     issue them in one stream or order them yourself.
+ *   - There is no status word without a context: should a bounded wait inside the kernel run out
+ *     (PQ_ERR_TIMEOUT of the regular entry point), this entry point cannot report it and the output
+ *     is then undefined. */
 pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache, const void* q, void* out, float sm_scale,
                                             void* stream);
 

@@ -185,12 +185,17 @@ class Context:
         return int(self.lib.pq_check(self.h, _stream()))
 
     # ---- offline -----------------------------------------------------------------------------
-    def quant_weights(self, W: torch.Tensor):
+    def quant_weights(self, W: torch.Tensor, out=None):
         _dev(W, torch.bfloat16, "W")
         N, K = W.shape
         assert W.stride(1) == 1
-        wq = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
-        s_w = torch.empty((N,), dtype=torch.float32, device=W.device)
+        if out is None:
+            wq = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
+            s_w = torch.empty((N,), dtype=torch.float32, device=W.device)
+        else:
+            wq, s_w = out
+            _dev(wq, torch.uint8, "wq"), _dev(s_w, torch.float32, "s_w")
+            assert wq.shape == (N, K // 2) and wq.is_contiguous() and s_w.shape == (N,)
         _ok(self.lib.pq_quant_weights(self.h, _ptr(W), N, K, W.stride(0), _ptr(wq), _ptr(s_w), _stream()), "pq_quant_weights")
         return wq, s_w
 

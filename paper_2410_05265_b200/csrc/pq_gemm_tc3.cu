@@ -555,12 +555,13 @@ pq_status pq_gemm_pair_ts_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* 
   p.K = static_cast<int>(K);
   p.tiles_m = static_cast<int>((M + 2 * BM_CTA - 1) / (2 * BM_CTA));
   p.tiles_n = static_cast<int>((N + BN - 1) / BN);
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[64] = {};  // the attribute belongs to the device's copy of the kernel: once per device
+  if (ctx->device < 0 || ctx->device >= 64) return PQ_ERR_UNSUPPORTED;
+  if (!attr_set[ctx->device]) {
     if (cudaFuncSetAttribute(gemm_w4a4_pair_ts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(SMEM_BYTES)) != cudaSuccess)
       return PQ_ERR_CUDA;
-    attr_set = true;
+    attr_set[ctx->device] = true;
   }
   const int n_tiles = p.tiles_m * p.tiles_n;
   const int max_pairs = ctx->sm_count / 2;

@@ -187,7 +187,7 @@ struct AttnParams {
   float sm_scale;
   int B, Hq, Hkv, G, n_prefix, Tmax;
   // fused append (decode_attn_kernel<.., true>): the new token's k, v [B, Hkv, 128], the writable lengths and one
-  // counter per sequence
+  // grid-wide counter
   const __nv_bfloat16* k_new;
   const __nv_bfloat16* v_new;
   int32_t* len_rw;
@@ -219,8 +219,8 @@ struct AttnParams {
 // FUSED: the call also appends one token per sequence (what pq_kv4_append does for T_new = 1). The attention
 // streams the cache as it was; the CTA of the last split quantizes the new k and v of its head, writes their codes
 // to row len[b] and folds the new key into its partial like one more full-precision key whose key and value are
-// the dequantized codes. The last CTA of a sequence to finish (every CTA of the sequence has read len[b] by then)
-// advances len[b]. As with the two calls, nothing is appended anywhere when any sequence is full.
+// the dequantized codes. The last CTA of the grid to finish (every CTA has read the lengths by then) advances
+// every len[b]. As with the two calls, nothing is appended anywhere when any sequence is full.
 // MULTI (with CLUSTER): a (sequence, head) has several clusters of eight splits.
 template <bool CLUSTER, bool FUSED, bool MULTI = false>
 __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnParams p) {
@@ -257,7 +257,8 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
 #pragma unroll
     for (int w = 0; w < 4; ++w) q_raw[w] = row_ok ? __ldg(q4 + w) : make_uint4(0, 0, 0, 0);
   }
-  int len_b = __ldg(p.len + b);
+  // the fused kernel writes the lengths at its end: it reads them past the read-only path
+  int len_b = FUSED ? __ldcg(p.len + b) : __ldg(p.len + b);
   const float s_k_h = __ldg(p.s_k + h), s_v_h = __ldg(p.s_v + h);
   // prefix values of the four head dims this thread merges after the key loop, so that the merge does
   // not wait for them (keys past the fourth are read there)
@@ -310,26 +311,32 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   __syncthreads();  // every barrier is initialised (all warps are still together here: this costs nothing)
   if (FUSED) {  // one verdict for the whole batch, as the append call gives it
     for (int i = threadIdx.x; i < p.B; i += DA_THREADS) {
-      const int l = __ldg(p.len + i);
+      const int l = __ldcg(p.len + i);
       if (l < 0 || l + 1 > p.Tmax) sm_full = 1;
     }
     __syncthreads();
   }
   const bool append_ok = FUSED && !sm_full;
   const int len_raw = len_b;
-  // called by every CTA when it is done: the last one of this sequence advances the length
+  // Called by every thread of every CTA when the CTA is done. The last CTA of the whole grid advances every length:
+  // by then each CTA has read the lengths it needs (its own sequence's, and all of them for the verdict above),
+  // so no CTA can ever see a length this launch has already moved.
   auto finish_append = [&]() {
-    if (FUSED && threadIdx.x == 0) {
-      if (!append_ok) {
-        if (p.status && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) pq::report(p.status, PQ_ERR_SHAPE);
-      } else {
-        __threadfence();
-        const uint32_t n_ctas = gridDim.x * gridDim.y;  // splits x KV heads of this sequence
-        if (atomicAdd(p.len_tickets + b, 1u) == n_ctas - 1) {
-          p.len_rw[b] = len_raw + 1;
-          p.len_tickets[b] = 0;
-        }
-      }
+    if (!FUSED) return;
+    if (!append_ok) {
+      if (threadIdx.x == 0 && p.status && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) pq::report(p.status, PQ_ERR_SHAPE);
+      return;
+    }
+    __syncthreads();  // is_last is free again, and this CTA's cache writes precede the ticket
+    if (threadIdx.x == 0) {
+      __threadfence();
+      const uint32_t n_ctas = gridDim.x * gridDim.y * gridDim.z;
+      is_last = atomicAdd(p.len_tickets, 1u) == n_ctas - 1;
+    }
+    __syncthreads();
+    if (is_last) {
+      for (int i = threadIdx.x; i < p.B; i += DA_THREADS) p.len_rw[i] = __ldcg(p.len_rw + i) + 1;
+      if (threadIdx.x == 0) *p.len_tickets = 0;
     }
   };
   len_b = len_b < 0 ? 0 : (len_b > p.Tmax ? p.Tmax : len_b);
@@ -863,7 +870,7 @@ extern "C" size_t pq_decode_attn_workspace_bytes(const pq_kv4_cache* cache) {
 }
 
 namespace {
-constexpr int DA_LEN_TICKET0 = PQ_N_TICKETS / 2;  // one counter per sequence for the fused append
+constexpr int DA_LEN_TICKET0 = PQ_N_TICKETS / 2;  // the grid-wide counter of the fused append
 
 // k_new, v_new: null for the plain attention; else the token appended by the same launch.
 pq_status decode_attn_launch(pq_ctx* ctx, const pq_kv4_cache* cache, const void* q, void* out, float sm_scale, void* ws,
@@ -892,7 +899,7 @@ pq_status decode_attn_launch(pq_ctx* ctx, const pq_kv4_cache* cache, const void*
   const int n_parts = cluster ? (S < 8 ? 1 : S / 8) : S;
   const bool multi = cluster && n_parts > 1;
   const int G = cache->Hq / cache->Hkv;
-  AttnParams p;
+  AttnParams p{};
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.prefix_k = static_cast<const __half*>(cache->prefix_k);
@@ -1028,7 +1035,7 @@ extern "C" pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache
   // the array keeps whatever the previous call left: the counters must start at zero
   if (cudaMemsetAsync(tickets + DA_TICKET0, 0, static_cast<size_t>(bh) * sizeof(uint32_t), cs) != cudaSuccess)
     return PQ_ERR_CUDA;
-  AttnParams p;
+  AttnParams p{};
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.prefix_k = static_cast<const __half*>(cache->prefix_k);

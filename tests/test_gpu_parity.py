@@ -291,6 +291,63 @@ def test_fused_append_and_decode_attention_equals_the_two_calls(ctx, B, Hq, Hkv,
     assert np.array_equal(to_np(cache.length), len_ref + 1)
 
 
+def test_fused_append_grid_larger_than_resident_with_a_sequence_that_fills_up(ctx):
+    """More CTAs than the GPU holds at once, and one sequence whose append fills it exactly: CTAs that start late
+    must not see a length this launch has already advanced (they would take the batch for full)."""
+    from paper_2410_05265_b200 import binding
+
+    B, Hq, Hkv, D, Tmax = 96, 8, 8, 128, 128          # 768 CTAs of one split each
+    k, v, s_k, s_v, pk, pv, q = _kv_setup(B, Hq, Hkv, D, 0, 1, Tmax, 1.0, 0)
+    start = (np.arange(B, dtype=np.int32) * 5) % (Tmax - 1)
+    start[0] = Tmax - 1
+    start[B - 1] = Tmax - 1
+    kq_ref = np.random.default_rng(3).integers(0, 256, (B, Hkv, Tmax, D // 2)).astype(np.uint8)
+    vq_ref = np.random.default_rng(4).integers(0, 256, (B, Hkv, Tmax, D // 2)).astype(np.uint8)
+    kq, vq = dev(kq_ref), dev(vq_ref)
+    len_ref = start.copy()
+    assert orc.kv4_append(inputs.bits(k), inputs.bits(v), s_k, s_v, kq_ref, vq_ref, len_ref) == 0
+    z = np.zeros((Hkv, 0, D), np.uint16)
+    _, out_ref = orc.decode_attn(inputs.bits(q), z, z, kq_ref, vq_ref, s_k, s_v, len_ref, 1 / math.sqrt(D), want_f64=True)
+    cache = binding.KV4Cache(None, None, kq, vq, dev(s_k), dev(s_v), dev(start), Hq)
+    ws = ctx.decode_attn_workspace(cache)
+    out = ctx.kv4_append_decode_attn(cache, k.cuda(), v.cuda(), q.cuda(), 1 / math.sqrt(D), ws)
+    assert ctx.check_status() == 0
+    assert np.array_equal(to_np(cache.length), len_ref) and int(len_ref[0]) == Tmax
+    assert np.array_equal(to_np(kq), kq_ref) and np.array_equal(to_np(vq), vq_ref)
+    assert_attn_close(inputs.bits(out), out_ref, "fused append, grid above residency")
+    # the next call finds two full sequences: nothing moves, the verdict comes through the status word
+    ctx.kv4_append_decode_attn(cache, k.cuda(), v.cuda(), q.cuda(), 1 / math.sqrt(D), ws)
+    assert ctx.check_status() == 2
+    assert np.array_equal(to_np(cache.length), len_ref) and np.array_equal(to_np(kq), kq_ref)
+    # and after the full ones are emptied the counters are in order: the append goes through again
+    cache.length[0] = 0
+    cache.length[B - 1] = 0
+    ctx.kv4_append_decode_attn(cache, k.cuda(), v.cuda(), q.cuda(), 1 / math.sqrt(D), ws)
+    assert ctx.check_status() == 0
+    len_ref[0] = len_ref[B - 1] = 0
+    assert np.array_equal(to_np(cache.length), len_ref + 1)
+
+
+def test_weights_quantized_in_the_same_stream_reach_the_streaming_gemm(ctx):
+    """quantize weights -> rotate + quantize -> M = 1 GEMM enqueued back to back without a synchronisation: the
+    weight-streaming kernel fetches its weights ahead of its predecessor's end, and they must be the new ones."""
+    N, K = 4096, 4096
+    x = inputs.activations(1, K, seed=0)
+    s_a = torch.tensor([0.3], device="cuda")
+    acc = torch.zeros((1, N), dtype=torch.int32, device="cuda")
+    wq = torch.zeros((N, K // 2), dtype=torch.uint8, device="cuda")
+    s_w = torch.zeros(N, device="cuda")
+    xd = x.cuda()
+    for seed in (2, 3, 4):                               # the same buffers are overwritten: stale weights would show
+        W = inputs.weights(N, K, seed=seed).cuda()
+        torch.cuda.synchronize()
+        ctx.quant_weights(W, out=(wq, s_w))
+        xq = ctx.hadamard_quant_act(xd, K, s_a)
+        ctx.w4a4_gemm(xq, wq, s_a, s_w, acc_dbg=acc)
+        ctx.check()
+        assert np.array_equal(to_np(acc), orc.gemm_i4(to_np(xq), to_np(wq)))
+
+
 def test_fused_append_refuses_a_full_sequence(ctx):
     from paper_2410_05265_b200 import binding
 

@@ -38,7 +38,10 @@ def test_noalloc_entry_point_matches_regular_one_twice_in_a_row():
     from paper_2410_05265_b200 import binding
 
     sm = 1 / math.sqrt(128)
-    cases = [(_cache(binding, 4, 32, 8, 4, 700, 768, seed=3)), (_cache(binding, 2, 16, 2, 2, 333, 512, seed=4))]
+    # the last two cases: one (sequence, head) pair with a long cache = 32 splits merged through the array,
+    # with a long and with a short sequence in it
+    cases = [(_cache(binding, 4, 32, 8, 4, 700, 768, seed=3)), (_cache(binding, 2, 16, 2, 2, 333, 512, seed=4)),
+             (_cache(binding, 1, 8, 1, 3, 8000, 8192, seed=5)), (_cache(binding, 1, 4, 1, 0, 200, 8192, seed=6))]
     # the new entry point first: it must work in a process that never created a context
     outs = []
     for cache, q in cases:
@@ -52,6 +55,10 @@ def test_noalloc_entry_point_matches_regular_one_twice_in_a_row():
         ctx.check()
         ref64 = orc.bf16_to_f64(inputs.bits(ref))
         assert_attn_close(inputs.bits(out), ref64, "noalloc vs regular entry point")
+        # and against the CPU oracle's unrounded result, like every other attention test
+        _, orc64 = orc.decode_attn(inputs.bits(q), inputs.bits(cache.prefix_k), inputs.bits(cache.prefix_v), to_np(cache.kq),
+                                   to_np(cache.vq), to_np(cache.s_k), to_np(cache.s_v), to_np(cache.length), sm, want_f64=True)
+        assert_attn_close(inputs.bits(out), orc64, "noalloc vs oracle")
         # and a repeat of the same call reproduces itself (nothing of the previous call survives)
         again = torch.empty_like(out)
         binding.decode_attn_noalloc(cache, q, sm, again)
