@@ -56,6 +56,14 @@ pq_status pq_destroy(pq_ctx* ctx);
  * and clears it. */
 pq_status pq_check(pq_ctx* ctx, void* stream);
 
+/* Bound of the device-side waits (a consumer waiting for a copy or for a producer, a producer waiting for
+ * a free buffer) of the kernels launched through this context from now on, in SM clocks; 0 restores the
+ * default of 2^31 clocks (about a second). A wait that runs out makes its kernel wind down in an orderly
+ * way (copies in flight are awaited, tensor memory is released) and leaves PQ_ERR_TIMEOUT in the status
+ * word; the kernel's output is then undefined. Failure-detection tests set a bound of a few clocks so that
+ * an ordinary wait runs out. */
+pq_status pq_set_wait_limit(pq_ctx* ctx, int64_t sm_clocks);
+
 /* ---------------------------------------------------------------------------------------------
  * Offline weight quantization: round-to-nearest, one symmetric scale per output channel
  * (Table 1 "per-channel" weights; the "RTN" row of Table 6; Eq. 1).

@@ -28,6 +28,7 @@ pq_status pq_create(pq_ctx** out) {
   c->d_tickets = nullptr;
   c->n_tickets = PQ_N_TICKETS;
   c->encode_tiled = nullptr;
+  c->wait_clocks = PQ_DEFAULT_WAIT_CLOCKS;
   cudaDeviceProp prop;
   if (cudaGetDevice(&c->device) != cudaSuccess || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) {
     delete c;
@@ -65,6 +66,12 @@ pq_status pq_destroy(pq_ctx* ctx) {
   cudaFree(ctx->d_status);
   cudaFree(ctx->d_tickets);
   delete ctx;
+  return PQ_OK;
+}
+
+pq_status pq_set_wait_limit(pq_ctx* ctx, int64_t sm_clocks) {
+  if (!ctx || sm_clocks < 0) return PQ_ERR_INVALID_ARG;
+  ctx->wait_clocks = sm_clocks == 0 ? PQ_DEFAULT_WAIT_CLOCKS : static_cast<long long>(sm_clocks);
   return PQ_OK;
 }
 

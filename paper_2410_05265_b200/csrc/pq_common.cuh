@@ -17,7 +17,10 @@ struct pq_ctx {
   uint32_t* d_tickets;  // zero-initialised, self-resetting "last block done" counters
   int n_tickets;
   void* encode_tiled;   // cuTensorMapEncodeTiled resolved through the runtime
+  long long wait_clocks;  // bound of every device-side wait, in SM clocks (pq_set_wait_limit)
 };
+
+#define PQ_DEFAULT_WAIT_CLOCKS (1ll << 31)  // about a second
 
 #define PQ_N_TICKETS 65536
 
@@ -65,16 +68,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after ~2^31 SM clocks (about a second) and returns false.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// Bounded wait: gives up after `limit` SM clocks and returns false.
+__device__ __forceinline__ bool mbar_wait_for(uint64_t* bar, uint32_t parity, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 4096; ++i)
+    for (int i = 0; i < 32; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (clock64() - t0 > (1ll << 31)) return false;
+    if (clock64() - t0 > limit) return false;
   }
+}
+// The same with the default bound of about a second (used where only memory latency is waited for).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  return mbar_wait_for(bar, parity, PQ_DEFAULT_WAIT_CLOCKS);
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

@@ -7,7 +7,10 @@
 // from two weight rows and from one token row, expands the nibbles to s8 values scaled by 16
 // (even-position codes in one word, odd-position codes in the next) and feeds word pairs to four
 // MMAs. Weights and tokens apply the same permutation of k inside a chunk, so the dot product is
-// unchanged; the factor 16*16 is shifted out exactly in the epilogue.
+// unchanged; the factor 16*16 is shifted out exactly in the epilogue. (Staging the rows through shared
+// memory with bulk copies was measured and is slower here: copies below 2 KB do not reach the memory's
+// rate, and the short layers are bound by the dependent chain wait -> token rows -> MMA -> store, which
+// direct loads keep shortest.)
 #include "pq_common.cuh"
 
 namespace {
@@ -15,7 +18,6 @@ namespace {
 constexpr int GS_WARPS = 8;
 constexpr int GS_THREADS = GS_WARPS * 32;
 constexpr int GS_CH = 16;     // output channels per CTA
-constexpr int GS_UNROLL = 4;  // K steps whose loads are in flight together
 
 __device__ __forceinline__ void mma_s8_16832(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                              uint32_t b0, uint32_t b1) {
@@ -53,7 +55,10 @@ __device__ __forceinline__ void permute_s8(const uint4& lo, const uint4& hi, uin
 // HALF_ROWS: the CTA owns 8 output channels instead of 16 (rows 8..15 of the MMA tile stay zero), which
 // doubles the CTA count of narrow layers.
 // A8: the token operand is one s8 code per element ([M, K] bytes) instead of packed nibbles (W4A8).
-template <bool TWO_GROUPS, bool HALF_ROWS, bool A8>
+// DEEP (long K): batches of two steps in two register buffers, so that the next batch's loads are in flight while
+// this one is multiplied; else one buffer of four steps (a K of 4096 is a single batch per warp, and the lower
+// register count keeps more CTAs on an SM, which is what the short layers need).
+template <bool TWO_GROUPS, bool HALF_ROWS, bool A8, bool DEEP>
 __global__ void __launch_bounds__(GS_THREADS)
     gemm_w4a4_stream_kernel(const uint8_t* __restrict__ xq, const uint8_t* __restrict__ wq,
                             const float* __restrict__ s_a, const float* __restrict__ s_w,
@@ -83,53 +88,94 @@ __global__ void __launch_bounds__(GS_THREADS)
   // in the stream: let the next kernel start early, fetch the first weight chunks, and only then wait
   // for the previous kernel (programmatic dependent launch; both instructions do nothing without it).
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  bool first = true;
-  for (int base = warp; base < n_steps; base += GS_WARPS * GS_UNROLL) {
-    uint4 wa[GS_UNROLL], wb[GS_UNROLL], xa[GS_UNROLL], xb[GS_UNROLL];
-    uint4 xa2[A8 ? GS_UNROLL : 1], xb2[A8 ? GS_UNROLL : 1];  // second half of a lane's 32 s8 codes
+  // One batch = GS_UNROLL K steps of this warp (their loads are in flight together). Two register buffers: the
+  // loads of batch b + 1 are issued before batch b is multiplied, so the memory pipe never drains inside a CTA.
+  constexpr int GS_UNROLL = DEEP ? 2 : 4;  // K steps per batch
+  struct Batch {
+    uint4 wa[GS_UNROLL], wb[HALF_ROWS ? 1 : GS_UNROLL], xa[GS_UNROLL], xb[TWO_GROUPS ? GS_UNROLL : 1];
+    uint4 xa2[A8 ? GS_UNROLL : 1], xb2[(A8 && TWO_GROUPS) ? GS_UNROLL : 1];  // second half of a lane's 32 s8 codes
+  };
+  constexpr int STRIDE = GS_WARPS * GS_UNROLL;
+  auto load_w = [&](Batch& b, int base) {
 #pragma unroll
     for (int u = 0; u < GS_UNROLL; ++u) {
       const int ks = base + u * GS_WARPS;
       const int off = ks * 64;
       const bool in_k = ks < n_steps && off + t * 16 < kbytes;
-      wa[u] = (in_k && w0_ok) ? ld_stream(w0p + off) : zero;
-      wb[u] = (in_k && w1_ok) ? ld_stream(w1p + off) : zero;
+      b.wa[u] = (in_k && w0_ok) ? ld_stream(w0p + off) : zero;
+      if (!HALF_ROWS) b.wb[u] = (in_k && w1_ok) ? ld_stream(w1p + off) : zero;
     }
-    if (first) {
-      asm volatile("griddepcontrol.wait;" ::: "memory");
-      first = false;
-    }
+  };
+  auto load_x = [&](Batch& b, int base) {
 #pragma unroll
     for (int u = 0; u < GS_UNROLL; ++u) {
       const int ks = base + u * GS_WARPS;
       const int off = ks * 64;
       const bool in_k = ks < n_steps && off + t * 16 < kbytes;
-      xa[u] = (in_k && x0_ok) ? __ldg(reinterpret_cast<const uint4*>(x0p + off * XS)) : zero;
-      if (TWO_GROUPS) xb[u] = (in_k && x1_ok) ? __ldg(reinterpret_cast<const uint4*>(x1p + off * XS)) : zero;
+      b.xa[u] = (in_k && x0_ok) ? __ldg(reinterpret_cast<const uint4*>(x0p + off * XS)) : zero;
+      if (TWO_GROUPS) b.xb[u] = (in_k && x1_ok) ? __ldg(reinterpret_cast<const uint4*>(x1p + off * XS)) : zero;
       if (A8) {
-        xa2[u] = (in_k && x0_ok) ? __ldg(reinterpret_cast<const uint4*>(x0p + off * XS) + 1) : zero;
-        if (TWO_GROUPS) xb2[u] = (in_k && x1_ok) ? __ldg(reinterpret_cast<const uint4*>(x1p + off * XS) + 1) : zero;
+        b.xa2[u] = (in_k && x0_ok) ? __ldg(reinterpret_cast<const uint4*>(x0p + off * XS) + 1) : zero;
+        if (TWO_GROUPS) b.xb2[u] = (in_k && x1_ok) ? __ldg(reinterpret_cast<const uint4*>(x1p + off * XS) + 1) : zero;
       }
     }
+  };
+  auto multiply = [&](const Batch& b) {
 #pragma unroll
     for (int u = 0; u < GS_UNROLL; ++u) {
       uint32_t ea[8], eb[8], ex[8];
-      expand(wa[u], ea);
-      expand(wb[u], eb);
-      if (A8) permute_s8(xa[u], xa2[u], ex);
-      else expand(xa[u], ex);
+      expand(b.wa[u], ea);
+      if (HALF_ROWS) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) eb[i] = 0u;
+      } else {
+        expand(b.wb[u], eb);
+      }
+      if (A8) permute_s8(b.xa[u], b.xa2[u], ex);
+      else expand(b.xa[u], ex);
 #pragma unroll
       for (int j = 0; j < 4; ++j) mma_s8_16832(c0, ea[2 * j], eb[2 * j], ea[2 * j + 1], eb[2 * j + 1], ex[2 * j], ex[2 * j + 1]);
       if (TWO_GROUPS) {
-        if (A8) permute_s8(xb[u], xb2[u], ex);
-        else expand(xb[u], ex);
+        if (A8) permute_s8(b.xb[u], b.xb2[u], ex);
+        else expand(b.xb[u], ex);
 #pragma unroll
         for (int j = 0; j < 4; ++j)
           mma_s8_16832(c1, ea[2 * j], eb[2 * j], ea[2 * j + 1], eb[2 * j + 1], ex[2 * j], ex[2 * j + 1]);
       }
     }
+  };
+  // what the epilogue needs is requested now, not after the reduction: the output channel's step (static, like the
+  // weights) ahead of the wait, the token's step and the zero point right after it
+  const int e_tok = threadIdx.x & 15, e_ch = threadIdx.x >> 4;  // 16 channels x 16 tokens: consecutive threads read consecutive words
+  const int e_n = n0 + e_ch;
+  const bool e_ok = e_tok < M && e_n < N && e_ch < CH && (TWO_GROUPS || e_tok < 8);
+  const float e_sw = e_ok ? __ldg(s_w + e_n) : 0.0f;
+  const int e_wsum = (e_ok && zp) ? __ldg(wsum + e_n) : 0;
+  Batch b0;
+  int base = warp;
+  if (base < n_steps) load_w(b0, base);               // static weights: requested ahead of the wait
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the token rows may come from the previous kernel
+  const float e_sa = e_ok ? __ldg(s_a + e_tok * sa_stride) : 0.0f;  // stride 1: one step per token
+  const int e_zp8 = (e_ok && zp) ? __ldg(zp) - 8 : 0;
+  if (base < n_steps) load_x(b0, base);
+  if (DEEP) {
+    Batch b1;
+    while (base < n_steps) {
+      if (base + STRIDE < n_steps) load_w(b1, base + STRIDE), load_x(b1, base + STRIDE);
+      multiply(b0);
+      base += STRIDE;
+      if (base >= n_steps) break;
+      if (base + STRIDE < n_steps) load_w(b0, base + STRIDE), load_x(b0, base + STRIDE);
+      multiply(b1);
+      base += STRIDE;
+    }
+  } else {
+    while (base < n_steps) {
+      multiply(b0);
+      base += STRIDE;
+      if (base < n_steps) load_w(b0, base), load_x(b0, base);
+    }
   }
-  if (first) asm volatile("griddepcontrol.wait;" ::: "memory");  // a warp without any K step
   // accumulator layout: c[0], c[1] -> channel g, tokens 2t, 2t+1; c[2], c[3] -> channel g+8
   red[warp][g][2 * t] = c0[0];
   red[warp][g][2 * t + 1] = c0[1];
@@ -142,27 +188,23 @@ __global__ void __launch_bounds__(GS_THREADS)
     red[warp][g + 8][8 + 2 * t + 1] = c1[3];
   }
   __syncthreads();
-  {
-    const int ch = threadIdx.x & 15, tok = threadIdx.x >> 4;  // 16 tokens x 16 channels = 256 threads
-    const int n = n0 + ch;
-    if (tok < M && n < N && ch < CH && (TWO_GROUPS || tok < 8)) {
-      int s = 0;
+  if (e_ok) {
+    int s = 0;
 #pragma unroll
-      for (int w = 0; w < GS_WARPS; ++w) s += red[w][ch][tok];
-      s >>= A8 ? 4 : 8;  // exact: every product carries the factor 16 once per 4-bit operand
-      if (zp) s -= (__ldg(zp) - 8) * __ldg(wsum + n);  // zero-point form of Eq. 1: sum (u - z) w from sum (u - 8) w
-      const float f = static_cast<float>(s) * (__ldg(s_a + tok * sa_stride) * __ldg(s_w + n));  // stride 1: one step per token
-      out[static_cast<int64_t>(tok) * ldo + n] = __float2bfloat16_rn(f);
-      if (acc_dbg) acc_dbg[static_cast<int64_t>(tok) * N + n] = s;
-    }
+    for (int w = 0; w < GS_WARPS; ++w) s += red[w][e_ch][e_tok];
+    s >>= A8 ? 4 : 8;            // exact: every product carries the factor 16 once per 4-bit operand
+    if (zp) s -= e_zp8 * e_wsum;  // zero-point form of Eq. 1: sum (u - z) w from sum (u - 8) w
+    const float f = static_cast<float>(s) * (e_sa * e_sw);
+    out[static_cast<int64_t>(e_tok) * ldo + e_n] = __float2bfloat16_rn(f);
+    if (acc_dbg) acc_dbg[static_cast<int64_t>(e_tok) * N + e_n] = s;
   }
 }
 
 }  // namespace
 
 // Rows [0, M) of xq/out, M <= 16 (the caller has already applied row_begin).
-template <bool TWO, bool HALF, bool A8>
-static pq_status launch_stream(const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w, void* out,
+template <bool TWO, bool HALF, bool A8, bool DEEP>
+static pq_status launch_stream_k(const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w, void* out,
                                int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st,
                                int sa_stride, const int32_t* zp, const int32_t* wsum) {
   const int ch = HALF ? GS_CH / 2 : GS_CH;
@@ -178,10 +220,19 @@ static pq_status launch_stream(const uint8_t* xq, const uint8_t* wq, const float
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, gemm_w4a4_stream_kernel<TWO, HALF, A8>, xq, wq, s_a, s_w, static_cast<__nv_bfloat16*>(out), ldo,
+  if (cudaLaunchKernelEx(&cfg, gemm_w4a4_stream_kernel<TWO, HALF, A8, DEEP>, xq, wq, s_a, s_w, static_cast<__nv_bfloat16*>(out), ldo,
                          static_cast<int>(M), static_cast<int>(N), static_cast<int>(K), acc_dbg, sa_stride, zp, wsum) != cudaSuccess)
     return PQ_ERR_CUDA;
   return pq_launch_status();
+}
+
+template <bool TWO, bool HALF, bool A8>
+static pq_status launch_stream(const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w, void* out,
+                               int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st,
+                               int sa_stride, const int32_t* zp, const int32_t* wsum) {
+  // more than one four-step batch per warp: pipeline the batches
+  if (K > GS_WARPS * 4 * 128) return launch_stream_k<TWO, HALF, A8, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride, zp, wsum);
+  return launch_stream_k<TWO, HALF, A8, false>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride, zp, wsum);
 }
 
 pq_status pq_gemm_stream_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
