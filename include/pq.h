@@ -222,9 +222,9 @@ pq_status pq_kv4_append_decode_attn(pq_ctx* ctx, const pq_kv4_cache* cache, cons
  * token t sees every prefixed key and the cached keys 0..t of sequence `seq` (the cache rows must
  * already hold the T tokens: call pq_kv4_append first).
  *     out[t, g, :] = softmax_j(q[t, g, :] . K_j * sm_scale) . V   over j in prefix and j <= t
- *   q  bf16 [T, Hq, D] with ldq elements between tokens (the q part of a concatenated q|k|v output),
- *   out bf16 [T, Hq, D] dense, both 4-byte aligned; D = 128; Hq / Hkv in {1, 2, 4, 8}; T <= Tmax;
- *   n_prefix <= 64; prefix_k, prefix_v, kq, vq 16-byte aligned. No workspace. */
+ *   q  bf16 [T, Hq, D] with ldq elements between tokens (the q part of a concatenated q|k|v output; ldq a
+ *   multiple of 8), out bf16 [T, Hq, D] dense, both 16-byte aligned; D = 128; Hq / Hkv in {1, 2, 4, 8};
+ *   T <= Tmax; n_prefix <= 64; sm_scale > 0; prefix_k, prefix_v, kq, vq 16-byte aligned. No workspace. */
 pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, int32_t seq, const void* q, int64_t ldq,
                                      int32_t T, void* out, float sm_scale, void* stream);
 
