@@ -321,6 +321,14 @@ pq_status pq_w4a4_gemm_asym(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, c
 pq_status pq_outlier_tokens(pq_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ldx, float eta1, float eta2, float* M,
                             float* R, int32_t* flags, float* median, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Measurement aid (the paper has no counterpart): n_ctas CTAs (at most one per SM) each issue `iters`
+ * tcgen05.mma kind::i8 instructions of 128 x 256 x 32 multiply-accumulates on operands that stay in shared
+ * memory, and write the SM clocks from the first issue to the completion of the last into cycles[cta]
+ * (device, int64; -1 if the wait ran out). iters * 128 * 256 * 32 / cycles is the integer tensor-core rate
+ * per SM and clock that a GEMM reaches when nothing else has to happen: the benchmark's attainable INT8 peak. */
+pq_status pq_probe_i8_mma(pq_ctx* ctx, int32_t iters, int64_t* cycles, int32_t n_ctas, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

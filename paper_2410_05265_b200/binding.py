@@ -28,7 +28,7 @@ EXPORTS = [
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
     "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
     "pq_calib_act_asym", "pq_hadamard_quant_act_asym", "pq_weight_code_sums", "pq_w4a4_gemm_asym",
-    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit",
+    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma",
 ]
 
 
@@ -63,6 +63,7 @@ def load_library() -> ctypes.CDLL:
     lib.pq_destroy.argtypes = [c_void_p]
     lib.pq_check.argtypes = [c_void_p, c_void_p]
     lib.pq_set_wait_limit.argtypes = [c_void_p, c_int64]
+    lib.pq_probe_i8_mma.argtypes = [c_void_p, c_int32, c_void_p, c_int32, c_void_p]
     lib.pq_quant_weights.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p]
     lib.pq_hadamard_quant_act.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p,
                                           c_void_p, c_void_p]
@@ -188,6 +189,13 @@ class Context:
     def set_wait_limit(self, sm_clocks: int) -> None:
         """Bound of the device-side waits of later launches, in SM clocks (0: the default of about a second)."""
         _ok(self.lib.pq_set_wait_limit(self.h, int(sm_clocks)), "pq_set_wait_limit")
+
+    def probe_i8_mma(self, iters: int = 4096, n_ctas: int | None = None) -> torch.Tensor:
+        """SM clocks each of n_ctas CTAs needed for `iters` resident-operand 128x256x32 kind::i8 MMAs (int64 [n_ctas])."""
+        n = n_ctas or torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+        cycles = torch.zeros(n, dtype=torch.int64, device="cuda")
+        _ok(self.lib.pq_probe_i8_mma(self.h, int(iters), _ptr(cycles), n, _stream()), "pq_probe_i8_mma")
+        return cycles
 
     # ---- offline -----------------------------------------------------------------------------
     def quant_weights(self, W: torch.Tensor, out=None):

@@ -50,3 +50,34 @@ def test_job_throughput_single_rank_needs_no_process_group():
 
     ms_per_step, units_per_s = bench.job_throughput(8.0, steps=4, units_per_step_per_rank=50.0, world=1)
     assert ms_per_step == 2.0 and units_per_s == pytest.approx(50.0 / 2e-3)
+
+
+def test_gpus_n_starts_n_ranks_and_rank0_prints_one_line(capfd):
+    """`bench.py --gpus N` started as a plain program re-launches itself as N ranks: the launcher is run here with a
+    CPU stand-in for the timed step (two gloo ranks)."""
+    import json
+
+    import bench
+
+    stub = os.path.join(os.path.dirname(os.path.abspath(__file__)), "rank_stub.py")
+    rc = bench.spawn_ranks(2, stub, ["--gpus", "2", "--steps", "5"])
+    assert rc == 0
+    lines = [ln for ln in capfd.readouterr().out.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, "exactly one result line, from rank 0"
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["argv"] == ["--gpus", "2", "--steps", "5"]
+    assert line["ms_per_step"] == pytest.approx(25.0 / 5) and line["value"] == pytest.approx(2 * 1000.0 / 5e-3)
+
+
+def test_recorded_traffic_is_dropped_when_the_kernel_source_changed(tmp_path, monkeypatch):
+    import bench
+
+    (tmp_path / "profiles").mkdir()
+    src = tmp_path / "k.cu"
+    src.write_text("kernel v1")
+    (tmp_path / "profiles" / "roofline_traffic.txt").write_text(
+        f"launch: gate|up\nsource: k.cu\nsource_sha256: {bench.sha256_of(str(src))}\ndram_bytes_per_launch: 12345\n")
+    monkeypatch.setattr(bench, "ROOT", str(tmp_path))
+    assert bench.recorded_traffic()[0] == 12345
+    src.write_text("kernel v2")
+    assert bench.recorded_traffic()[0] is None
