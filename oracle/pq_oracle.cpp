@@ -462,6 +462,77 @@ void orc_quant_act_asym(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, in
   });
 }
 
+// ---- grid search for the static s and z (Sec. 3, "Initialization of Quantization Parameters") --------------
+// Candidates of Eq. 1 over a grid of clipping factors: gamma_i = 1 - i * step, beta_j = 1 - j * step with
+// step = (1 - lo) / (n - 1) (i, j = 0 .. n-1; n = 1: the max-min pair alone), candidate i * n + j being
+//   s = (gamma_i * mx - beta_j * mn) / (2^N - 1),   z = -floor(beta_j * mn / s)   clamped to the code range,
+// every step one IEEE fp32 operation (the precision the GPU forms them in); a range that is not positive gives
+// s = 1, z = 0.
+void orc_grid_candidates(float mn, float mx, int bits, int n, float lo, float* s_out, int32_t* z_out) {
+  const int qmax = (1 << bits) - 1;
+  volatile float step = n > 1 ? (1.0f - lo) / static_cast<float>(n - 1) : 0.0f;
+  for (int i = 0; i < n; ++i)
+    for (int j = 0; j < n; ++j) {
+      volatile float fi = static_cast<float>(i) * step, fj = static_cast<float>(j) * step;
+      volatile float gamma = 1.0f - fi, beta = 1.0f - fj;
+      volatile float gm = gamma * mx, bm = beta * mn;
+      volatile float d = gm - bm;
+      float s = 1.0f;
+      int32_t z = 0;
+      if (d > 0.0f) {
+        volatile float sv = d / static_cast<float>(qmax);
+        s = sv;
+        volatile float q = bm / sv;
+        z = clampi(-std::lrint(std::floor(static_cast<double>(q))), 0, qmax);
+      }
+      s_out[i * n + j] = s, z_out[i * n + j] = z;
+    }
+}
+
+// Sum over the rotated rows >= row_begin of (y - s (u - z))^2 with u = clamp(round_half_even(y / s) + z, 0, 2^N - 1):
+// the squared error of quantizing and dequantizing the tensor with one candidate, in double.
+double orc_quant_sse_asym(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin, int bits, float s_a,
+                          int32_t z) {
+  const int qmax = (1 << bits) - 1;
+  const double s = static_cast<double>(s_a);
+  std::vector<double> row_sse(M, 0.0);
+  parallel_rows(M, [&](int64_t m) {
+    if (m < row_begin) return;
+    std::vector<double> xr(K), yr(K);
+    for (int64_t j = 0; j < K; ++j) xr[j] = bf16_to_double(x[m * ldx + j]);
+    rotate_row(xr.data(), yr.data(), K, B);
+    double acc = 0.0;
+    for (int64_t j = 0; j < K; ++j) {
+      const long u = clampi(std::lrint(std::nearbyint(yr[j] / s)) + z, 0, qmax);
+      const double e = yr[j] - s * static_cast<double>(u - z);
+      acc += e * e;
+    }
+    row_sse[m] = acc;
+  });
+  double total = 0.0;
+  for (int64_t m = row_begin; m < M; ++m) total += row_sse[m];
+  return total;
+}
+
+// The search itself: range of the rotated calibration rows, the n x n candidates, the squared error of each, and
+// the candidate with the smallest error (the first one in index order among equals). sse_out (nullable) [n*n].
+void orc_grid_search_act(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin, int bits, int n, float lo,
+                         float* s_out, int32_t* z_out, double* sse_out) {
+  float mn, mx;
+  orc_calib_act_minmax(x, ldx, M, K, B, row_begin, &mn, &mx);
+  std::vector<float> cs(n * n);
+  std::vector<int32_t> cz(n * n);
+  orc_grid_candidates(mn, mx, bits, n, lo, cs.data(), cz.data());
+  int best = 0;
+  double best_sse = INFINITY;
+  for (int c = 0; c < n * n; ++c) {
+    const double sse = orc_quant_sse_asym(x, ldx, M, K, B, row_begin, bits, cs[c], cz[c]);
+    if (sse_out) sse_out[c] = sse;
+    if (sse < best_sse) best_sse = sse, best = c;
+  }
+  *s_out = cs[best], *z_out = cz[best];
+}
+
 // acc[t,n] = sum_k (u[t,k] - z) * wq[n,k]: the dequantized activation (up to its step) times the weight codes,
 // written out as such (no correction-term algebra). Returns 1 if an accumulator does not fit int32.
 int orc_gemm_asym(const uint8_t* u, int32_t z, const uint8_t* wq, int64_t M, int64_t N, int64_t K, int32_t* acc) {

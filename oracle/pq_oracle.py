@@ -255,6 +255,33 @@ def quant_act_asym(x_bits: np.ndarray, block: int, s_a, z: int, row_begin: int =
     return (u, tie) if want_tie_dist else u
 
 
+def grid_candidates(mn, mx, n: int, lo: float, bits: int = 4):
+    """The n x n candidates (s, z) of the clipping-factor grid gamma, beta in [lo, 1] (candidate i * n + j)."""
+    s, z = np.zeros(n * n, np.float32), np.zeros(n * n, np.int32)
+    lib().orc_grid_candidates(c_float(float(mn)), c_float(float(mx)), c_int(bits), c_int(n), c_float(float(lo)), _p(s, c_float), _p(z, c_int32))
+    return s, z
+
+
+def quant_sse_asym(x_bits: np.ndarray, block: int, s_a, z: int, row_begin: int = 0, bits: int = 4) -> float:
+    """Squared error of quantizing and dequantizing the rotated rows >= row_begin with step s_a and zero point z."""
+    x_bits = _u16(x_bits)
+    M, K = x_bits.shape
+    f = lib().orc_quant_sse_asym
+    f.restype = c_double
+    return float(f(_p(x_bits, c_uint16), c_int64(K), c_int64(M), c_int64(K), c_int(block), c_int64(row_begin), c_int(bits),
+                   c_float(float(s_a)), c_int32(int(z))))
+
+
+def grid_search_act(x_bits: np.ndarray, block: int, n: int, lo: float, row_begin: int = 0, bits: int = 4):
+    """MSE grid search for the static (s, z): returns s, z and the squared errors of all n * n candidates."""
+    x_bits = _u16(x_bits)
+    M, K = x_bits.shape
+    s, z, sse = np.zeros(1, np.float32), np.zeros(1, np.int32), np.zeros(n * n, np.float64)
+    lib().orc_grid_search_act(_p(x_bits, c_uint16), c_int64(K), c_int64(M), c_int64(K), c_int(block), c_int64(row_begin), c_int(bits),
+                              c_int(n), c_float(float(lo)), _p(s, c_float), _p(z, c_int32), _p(sse, c_double))
+    return np.float32(s[0]), int(z[0]), sse
+
+
 def gemm_asym(u: np.ndarray, z: int, wq: np.ndarray) -> np.ndarray:
     """sum_k (u[t,k] - z) * w[n,k] with unsigned activation codes and packed signed weight codes -> int32 [M,N]."""
     u = np.ascontiguousarray(u, np.uint8)

@@ -482,6 +482,47 @@ def test_asymmetric_quantizer_hand_values_and_reduction_to_the_symmetric_one():
     assert np.all(err[~top] <= 0.5 * s2 * (1 + 1e-5) + 1e-6) and np.all(err[top] <= 1.5 * s2 * (1 + 1e-5) + 1e-6)
 
 
+def test_grid_search_for_s_and_z_brute_force_and_never_worse_than_max_min():
+    # candidates: the first one is the max-min pair (pinned above), the factors step down to lo
+    mn, mx = np.float32(-1.0), np.float32(2.75)
+    cs, cz = orc.grid_candidates(mn, mx, 3, 0.5)
+    assert (cs[0], cz[0]) == orc.asym_params(mn, mx)
+    # gamma, beta in {1, 0.75, 0.5}: s = (gamma * 2.75 + beta) / 15, z = -floor(-beta / s), by hand for two of them
+    assert cs[4] == np.float32((np.float32(0.75 * 2.75) + np.float32(0.75)) / np.float32(15))        # i = j = 1
+    assert cz[4] == int(-np.floor(np.float32(-0.75) / cs[4])) and cs[8] == np.float32(0.5) * cs[0] and cz[8] == cz[0]
+    assert orc.grid_candidates(np.float32(0.0), np.float32(0.0), 2, 0.5)[0].tolist() == [1.0] * 4    # empty range
+    # the squared error against an independent numpy evaluation on a tiny tensor without rotation
+    x = rng.standard_normal((3, 128)) * 2.0 + 0.7
+    x[1, 5] = 40.0                                   # one far value: clipping it pays
+    xb = bf16_bits(x)
+    y = orc.bf16_to_f64(xb)
+    lo_, hi_ = np.float32(y.min()), np.float32(y.max())
+    n, lo = 6, 0.1
+    s_best, z_best, sse = orc.grid_search_act(xb, 0, n, lo)
+    cs, cz = orc.grid_candidates(lo_, hi_, n, lo)
+    ref = np.empty(n * n)
+    for c in range(n * n):
+        sd = np.float64(cs[c])
+        u = np.clip(np.rint(y / sd) + cz[c], 0, 15)
+        ref[c] = ((y - sd * (u - cz[c])) ** 2).sum()
+        assert orc.quant_sse_asym(xb, 0, cs[c], cz[c]) == pytest.approx(ref[c], rel=1e-12)
+    assert np.allclose(sse, ref, rtol=1e-12) and (s_best, z_best) == (cs[ref.argmin()], int(cz[ref.argmin()]))
+    assert ref.min() <= ref[0] and ref.argmin() != 0, "with an outlier in the tensor the max-min pair is not the best one"
+    # a tensor that lies on a candidate's grid is reproduced without error by that candidate
+    s0, z0 = np.float32(0.25), 5
+    grid_vals = (np.arange(16) - z0) * 0.25
+    xg = bf16_bits(np.tile(grid_vals, (2, 8)))
+    assert orc.quant_sse_asym(xg, 0, s0, z0) == 0.0
+    sg, zg, sse_g = orc.grid_search_act(xg, 0, 4, 0.5)
+    assert sse_g[0] == 0.0 and (sg, zg) == (s0, z0), "max-min already is exact here and comes first"
+    # rotation and prefix rows: the error is taken over the rotated rows at and after row_begin only
+    xr = inputs.bits(inputs.activations(10, 256, seed=1, n_prefix=4))
+    yr = orc.rotate_bf16(xr, 256)[4:]
+    s1, z1 = orc.asym_params(np.float32(yr.astype(np.float32).min()), np.float32(yr.astype(np.float32).max()))
+    u = np.clip(np.rint(yr / np.float64(s1)) + z1, 0, 15)
+    assert orc.quant_sse_asym(xr, 256, s1, z1, row_begin=4) == pytest.approx(((yr - np.float64(s1) * (u - z1)) ** 2).sum(), rel=1e-12)
+
+
 def test_gemm_asym_is_the_dequantized_product():
     M, N, K, z = 7, 11, 96, 5
     u = rng.integers(0, 16, (M, K)).astype(np.uint8)
