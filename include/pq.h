@@ -299,7 +299,7 @@ pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache, const voi
  *   pq_weight_code_sums         wsum[n] = sum_k w[n,k] over the packed codes of pq_quant_weights (offline), K % 8 == 0
  *   pq_w4a4_gemm_asym           the GEMM; its epilogue subtracts (z - 8) * wsum[n] from the exact integer sum
  *                               (acc_dbg, when given, receives sum_k (u - z) w). Other arguments as in pq_w4a4_gemm.
- * The grid search the paper runs over s and z is offline and not part of this library: any s, z can be passed. */
+ * Any s, z can be passed to the quantizer and the GEMM; pq_grid_search_act_asym below searches them. */
 pq_status pq_calib_act_asym(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block, int64_t row_begin,
                             float* s_a, int32_t* z_a, void* stream);
 pq_status pq_hadamard_quant_act_asym(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
@@ -308,6 +308,22 @@ pq_status pq_weight_code_sums(pq_ctx* ctx, const uint8_t* wq, int64_t N, int64_t
 pq_status pq_w4a4_gemm_asym(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const int32_t* z_a,
                             const float* s_w, const int32_t* wsum, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K,
                             int64_t row_begin, int32_t* acc_dbg, void* stream);
+
+/* Grid search for the static s and z (Sec. 3, "Initialization of Quantization Parameters": for per-tensor
+ * static quantization the parameters are searched directly, by mean squared error). Offline. Over one calibration
+ * batch, with mn / mx the range of its rotated rows >= row_begin, the n_grid x n_grid candidates
+ *     gamma_i = 1 - i * step,  beta_j = 1 - j * step,  step = (1 - lo) / (n_grid - 1)      (candidate i * n_grid + j)
+ *     s = (gamma_i * mx - beta_j * mn) / 15,  z = -floor(beta_j * mn / s) clamped to [0, 15]      (Eq. 1)
+ * are formed, sse[c] = sum (y - s (u - z))^2 with u = clamp(round_half_even(y / s) + z, 0, 15) is taken over those
+ * rows for each, and the candidate with the smallest error (the first among equals) is written to *s_a, *z_a.
+ * Candidate 0 is the max-min pair of pq_calib_act_asym, so the result is never worse than that one. The paper
+ * measures the error on block outputs; this entry point measures it on the quantized tensor itself.
+ *   n_grid in [1, 16], lo in (0, 1]; cand_s f32 [n_grid^2], cand_z int32 [n_grid^2], sse f64 [n_grid^2] (8-byte
+ *   aligned): device buffers of the caller that receive the candidates and their errors. Other arguments as in
+ *   pq_calib_act_asym. */
+pq_status pq_grid_search_act_asym(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block, int64_t row_begin,
+                                  int32_t n_grid, float lo, float* s_a, int32_t* z_a, float* cand_s, int32_t* cand_z, double* sse,
+                                  void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Outlier tokens (Sec. 4.1, "Definition of Outlier Token", Eq. 2), the cheap part of the offline analysis

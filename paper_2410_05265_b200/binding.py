@@ -28,7 +28,7 @@ EXPORTS = [
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
     "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
     "pq_calib_act_asym", "pq_hadamard_quant_act_asym", "pq_weight_code_sums", "pq_w4a4_gemm_asym",
-    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma",
+    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma", "pq_grid_search_act_asym",
 ]
 
 
@@ -98,6 +98,8 @@ def load_library() -> ctypes.CDLL:
     lib.pq_outlier_tokens.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_float, c_float, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p]
     lib.pq_calib_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p, c_void_p, c_void_p]
+    lib.pq_grid_search_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_int32, c_float, c_void_p,
+                                            c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.pq_hadamard_quant_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p, c_void_p,
                                                c_void_p, c_void_p]
     lib.pq_weight_code_sums.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p]
@@ -271,6 +273,20 @@ class Context:
         _ok(self.lib.pq_calib_act_asym(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, _ptr(s_a), _ptr(z_a), _stream()),
             "pq_calib_act_asym")
         return s_a, z_a
+
+    def grid_search_act_asym(self, x: torch.Tensor, had_block: int, n_grid: int, lo: float, row_begin: int = 0):
+        """MSE grid search for the static (s, z). Returns device tensors s_a [1], z_a [1], cand_s [n^2], cand_z [n^2], sse [n^2]."""
+        _dev(x, torch.bfloat16, "x")
+        M, K = x.shape
+        n2 = max(1, n_grid * n_grid)
+        s_a = torch.zeros((1,), dtype=torch.float32, device=x.device)
+        z_a = torch.zeros((1,), dtype=torch.int32, device=x.device)
+        cand_s = torch.zeros((n2,), dtype=torch.float32, device=x.device)
+        cand_z = torch.zeros((n2,), dtype=torch.int32, device=x.device)
+        sse = torch.zeros((n2,), dtype=torch.float64, device=x.device)
+        _ok(self.lib.pq_grid_search_act_asym(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, int(n_grid), float(lo), _ptr(s_a),
+                                             _ptr(z_a), _ptr(cand_s), _ptr(cand_z), _ptr(sse), _stream()), "pq_grid_search_act_asym")
+        return s_a, z_a, cand_s, cand_z, sse
 
     def hadamard_quant_act_asym(self, x: torch.Tensor, had_block: int, s_a: torch.Tensor, z_a: torch.Tensor, row_begin: int = 0,
                                 out: torch.Tensor | None = None):

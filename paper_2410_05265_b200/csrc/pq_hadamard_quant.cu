@@ -42,11 +42,14 @@ __device__ __forceinline__ float swiglu_bf16(float g, float u) {
   return __bfloat162float(__float2bfloat16_rn(pq::silu_mul_f32(g, u)));
 }
 
-template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU>
+// GRID (with CALIB and ZP; the grid search of Sec. 3 for the static s and z): s_a_in / zp_in hold n_cand candidate
+// (s, z) pairs, and the pass adds to s_a_out (n_cand doubles) the squared error of quantizing and dequantizing the
+// rotated values with each of them.
+template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU, bool GRID = false>
 __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
     hadamard_quant_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int64_t n_rows, int64_t K,
                           const float* __restrict__ s_a_in, uint8_t* __restrict__ xq, float* __restrict__ s_a_out,
-                          float clip, const int32_t* __restrict__ zp_in, const __nv_bfloat16* __restrict__ x2) {
+                          float clip, const int32_t* __restrict__ zp_in, const __nv_bfloat16* __restrict__ x2, int n_cand) {
   static_assert(BITS == 4 || BITS == 8, "code width");
   constexpr int QMAX = BITS == 4 ? 7 : 127;  // codes lie in [-QMAX - 1, QMAX]
   constexpr int B = 1 << LOGB;
@@ -180,7 +183,28 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
 #pragma unroll
         for (int q = 0; q < 32; ++q) it_max = fmaxf(it_max, fmaxf(fabsf(W[q].x * norm), fabsf(W[q].y * norm)));
       }
-      if (ZP) {
+      if (GRID) {
+        double* sse = reinterpret_cast<double*>(s_a_out);
+#pragma unroll 1
+        for (int c = 0; c < n_cand; ++c) {
+          const float s = __ldg(s_a_in + c), z = static_cast<float>(__ldg(zp_in + c));
+          const float inv_s = __fdiv_rn(1.0f, s);
+          float acc = 0.0f;
+          if (active) {
+#pragma unroll
+            for (int q = 0; q < 32; ++q) {
+              const float a = W[q].x * norm, b = W[q].y * norm;
+              const float ua = fminf(fmaxf(rintf(a * inv_s) + z, 0.0f), 15.0f), ub = fminf(fmaxf(rintf(b * inv_s) + z, 0.0f), 15.0f);
+              const float ea = a - s * (ua - z), eb = b - s * (ub - z);
+              acc = fmaf(ea, ea, acc);
+              acc = fmaf(eb, eb, acc);
+            }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+          if ((tid & 31) == 0 && acc != 0.0f) atomicAdd(sse + c, static_cast<double>(acc));
+        }
+      } else if (ZP) {
         if (active) {
 #pragma unroll
           for (int q = 0; q < 32; ++q) {
@@ -251,7 +275,9 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
       }
     }
   }
-  if (CALIB && ZP) {
+  if (CALIB && GRID) {
+    // nothing left to fold: every candidate's error went out with the blocks
+  } else if (CALIB && ZP) {
     for (int o = 16; o > 0; o >>= 1) {
       cal_lo = fminf(cal_lo, __shfl_xor_sync(0xffffffffu, cal_lo, o));
       cal_hi = fmaxf(cal_hi, __shfl_xor_sync(0xffffffffu, cal_hi, o));
@@ -267,10 +293,10 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
   }
 }
 
-template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU>
+template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU, bool GRID>
 pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_t K, const float* s_a_in, uint8_t* xq,
-                 float* s_a_out, float clip, const int32_t* zp_in, const void* x2, cudaStream_t st) {
-  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>;
+                 float* s_a_out, float clip, const int32_t* zp_in, const void* x2, cudaStream_t st, int n_cand) {
+  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID>;
   constexpr size_t smem = HQ_SMEM_FLOATS * sizeof(float);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
     return PQ_ERR_CUDA;
@@ -291,15 +317,15 @@ pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x), ldx, n_rows, K, s_a_in, xq, s_a_out, clip, zp_in,
-                         static_cast<const __nv_bfloat16*>(x2)) != cudaSuccess)
+                         static_cast<const __nv_bfloat16*>(x2), n_cand) != cudaSuccess)
     return PQ_ERR_CUDA;
   return pq_launch_status();
 }
 
-template <bool CALIB, int BITS, bool PER_TOKEN = false, bool ZP = false, bool SWIGLU = false>
+template <bool CALIB, int BITS, bool PER_TOKEN = false, bool ZP = false, bool SWIGLU = false, bool GRID = false>
 pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block, int64_t row_begin,
                    const float* s_a_in, uint8_t* xq, float* s_a_out, void* stream, float clip = 1.0f,
-                   const int32_t* zp_in = nullptr, const void* x2 = nullptr) {
+                   const int32_t* zp_in = nullptr, const void* x2 = nullptr, int n_cand = 0) {
   if (SWIGLU && (!x2 || (reinterpret_cast<uintptr_t>(x2) & 3))) return x2 ? PQ_ERR_ALIGN : PQ_ERR_INVALID_ARG;
   if (!ctx || !x || (!CALIB && (!s_a_in || !xq)) || (CALIB && !s_a_out)) return PQ_ERR_INVALID_ARG;
   if (M < 0 || K <= 0 || ldx < K || row_begin < 0 || had_block < 0) return PQ_ERR_INVALID_ARG;
@@ -322,14 +348,14 @@ pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx
     if (CALIB && cudaMemsetAsync(s_a_out, 0, static_cast<size_t>(n_rows) * sizeof(float), st) != cudaSuccess) return PQ_ERR_CUDA;
   }
   switch (had_block) {
-    case 0: return launch<7, false, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
-    case 128: return launch<7, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
-    case 256: return launch<8, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
-    case 512: return launch<9, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
-    case 1024: return launch<10, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
-    case 2048: return launch<11, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
-    case 4096: return launch<12, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
-    case 8192: return launch<13, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st);
+    case 0: return launch<7, false, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st, n_cand);
+    case 128: return launch<7, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st, n_cand);
+    case 256: return launch<8, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st, n_cand);
+    case 512: return launch<9, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st, n_cand);
+    case 1024: return launch<10, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st, n_cand);
+    case 2048: return launch<11, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st, n_cand);
+    case 4096: return launch<12, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st, n_cand);
+    case 8192: return launch<13, true, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st, n_cand);
     default: return PQ_ERR_SHAPE;
   }
 }
@@ -403,6 +429,59 @@ extern "C" pq_status pq_calib_act_asym(pq_ctx* ctx, const void* x, int64_t M, in
                                                 reinterpret_cast<float*>(keys), stream);
   if (rc != PQ_OK) return rc;
   asym_params_kernel<<<1, 1, 0, st>>>(keys, s_a, z_a);
+  return pq_launch_status();
+}
+
+namespace {
+// The n x n candidates of the clipping-factor grid from the collected range, every step one IEEE fp32 operation:
+// gamma_i = 1 - i * step, beta_j = 1 - j * step, s = (gamma mx - beta mn) / 15, z = -floor(beta mn / s) in [0, 15].
+__global__ void grid_candidates_kernel(const uint32_t* keys, int n, float lo, float* cand_s, int32_t* cand_z) {
+  const int c = threadIdx.x;
+  if (c >= n * n) return;
+  const float mx = key_float(keys[0]), mn = key_float(keys[1]);
+  const bool have = keys[0] >= keys[1];
+  const float step = n > 1 ? __fdiv_rn(__fsub_rn(1.0f, lo), static_cast<float>(n - 1)) : 0.0f;
+  const float gamma = __fsub_rn(1.0f, __fmul_rn(static_cast<float>(c / n), step));
+  const float beta = __fsub_rn(1.0f, __fmul_rn(static_cast<float>(c % n), step));
+  const float bm = __fmul_rn(beta, mn), d = __fsub_rn(__fmul_rn(gamma, mx), bm);
+  float s = 1.0f;
+  int z = 0;
+  if (have && d > 0.0f) {
+    s = __fdiv_rn(d, 15.0f);
+    z = -__float2int_rd(__fdiv_rn(bm, s));
+    z = z < 0 ? 0 : (z > 15 ? 15 : z);
+  }
+  cand_s[c] = s, cand_z[c] = z;
+}
+// The candidate with the smallest error, the first one among equals.
+__global__ void grid_argmin_kernel(const double* sse, const float* cand_s, const int32_t* cand_z, int n_cand, float* s_a, int32_t* z_a) {
+  int best = 0;
+  for (int c = 1; c < n_cand; ++c)
+    if (sse[c] < sse[best]) best = c;
+  *s_a = cand_s[best], *z_a = cand_z[best];
+}
+}  // namespace
+
+extern "C" pq_status pq_grid_search_act_asym(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                             int64_t row_begin, int32_t n_grid, float lo, float* s_a, int32_t* z_a, float* cand_s,
+                                             int32_t* cand_z, double* sse, void* stream) {
+  if (!ctx || !s_a || !z_a || !cand_s || !cand_z || !sse) return PQ_ERR_INVALID_ARG;
+  if (n_grid < 1 || n_grid > 16 || !(lo > 0.0f) || !(lo <= 1.0f)) return PQ_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(sse) & 7) return PQ_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_cand = n_grid * n_grid;
+  uint32_t* keys = ctx->d_tickets + ASYM_KEY0;
+  if (cudaMemsetAsync(keys, 0x00, sizeof(uint32_t), st) != cudaSuccess || cudaMemsetAsync(keys + 1, 0xFF, sizeof(uint32_t), st) != cudaSuccess ||
+      cudaMemsetAsync(sse, 0, sizeof(double) * n_cand, st) != cudaSuccess)
+    return PQ_ERR_CUDA;
+  pq_status rc = dispatch<true, 4, false, true>(ctx, x, M, K, ldx, had_block, row_begin, nullptr, nullptr, reinterpret_cast<float*>(keys), stream);
+  if (rc != PQ_OK) return rc;
+  grid_candidates_kernel<<<1, 256, 0, st>>>(keys, n_grid, lo, cand_s, cand_z);
+  if (pq_launch_status() != PQ_OK) return PQ_ERR_CUDA;
+  rc = dispatch<true, 4, false, true, false, true>(ctx, x, M, K, ldx, had_block, row_begin, cand_s, nullptr, reinterpret_cast<float*>(sse), stream,
+                                                   1.0f, cand_z, nullptr, n_cand);
+  if (rc != PQ_OK) return rc;
+  grid_argmin_kernel<<<1, 1, 0, st>>>(sse, cand_s, cand_z, n_cand, s_a, z_a);
   return pq_launch_status();
 }
 

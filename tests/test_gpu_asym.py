@@ -164,3 +164,31 @@ def test_asym_linear_end_to_end_beats_symmetric_on_offset_activations(ctx):
     err_asym = float((out.double().cpu() - ref).pow(2).mean())
     err_sym = float((out_sym.double().cpu() - ref).pow(2).mean())
     assert err_asym < 0.6 * err_sym
+
+
+@pytest.mark.parametrize("M,K,B,row_begin,n_grid,lo,outlier", [(40, 1024, 1024, 4, 6, 0.3, 0.0), (33, 6144, 2048, 0, 4, 0.5, 0.0),
+                                                              (64, 256, 0, 2, 8, 0.2, 60.0), (5, 4096, 4096, 0, 1, 1.0, 0.0),
+                                                              (17, 128, 128, 0, 16, 0.1, 0.0)])
+def test_grid_search_for_s_and_z_matches_oracle(ctx, M, K, B, row_begin, n_grid, lo, outlier):
+    """The n x n candidates against the oracle's (from the oracle's own range), the squared error of every candidate
+    against the oracle's error of the same (s, z), and the chosen pair: one whose oracle error is the minimum up to
+    the tolerance of the comparison (near-equal candidates may swap places in fp32)."""
+    x = inputs.activations(M, K, seed=1, n_prefix=row_begin)
+    if outlier:
+        x[row_begin + 1, 7] = outlier          # a far value in an ordinary row: clipping it pays
+    xb = inputs.bits(x)
+    s_a, z_a, cand_s, cand_z, sse = ctx.grid_search_act_asym(x.cuda(), B, n_grid, lo, row_begin)
+    ctx.check()
+    cs, cz, got = to_np(cand_s), to_np(cand_z), to_np(sse)
+    mn, mx = orc.calib_act_minmax(xb, B, row_begin)
+    cs_ref, cz_ref = orc.grid_candidates(mn, mx, n_grid, lo)
+    assert np.allclose(cs, cs_ref, rtol=4e-6) and np.all(np.abs(cz - cz_ref) <= 1)
+    assert (cs[0], cz[0]) == tuple(float(v) if i == 0 else int(v) for i, v in enumerate(ctx.calib_act_asym(x.cuda(), B, row_begin)))
+    ref = np.array([orc.quant_sse_asym(xb, B, cs[c], int(cz[c]), row_begin) for c in range(n_grid * n_grid)])
+    assert np.allclose(got, ref, rtol=2e-4, atol=1e-9), f"worst {np.max(np.abs(got - ref) / np.maximum(ref, 1e-30))}"
+    pick = [c for c in range(len(cs)) if cs[c] == float(s_a) and cz[c] == int(z_a)]
+    assert pick, "the result is one of the candidates"
+    assert ref[pick[0]] <= ref.min() * (1 + 4e-4) and got[pick[0]] == got.min()
+    assert ref[pick[0]] <= ref[0], "never worse than the max-min pair"
+    if outlier:
+        assert pick[0] != 0 and ref[pick[0]] < 0.7 * ref[0]
