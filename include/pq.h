@@ -105,6 +105,14 @@ pq_status pq_calib_act_scale(pq_ctx* ctx, const void* x, int64_t M, int64_t K, i
 pq_status pq_swiglu_hadamard_quant_act(pq_ctx* ctx, const void* gate, const void* up, int64_t M, int64_t K, int64_t ld_in,
                                        int had_block, int64_t row_begin, const float* s_a, uint8_t* xq, void* stream);
 
+/* The same quantizer with the RMSNorm of the block in front (App. B figure: RMSNorm feeds the q/k/v and the gate/up
+ * linears): the transform's input is bf16(x * r * g), r = 1 / sqrt(mean(x^2) + eps), formed in registers with the
+ * arithmetic and the rounding of pq_rmsnorm, so the result equals pq_rmsnorm followed by pq_hadamard_quant_act with
+ * had_block = K bit for bit while the normalised tensor never goes to memory.
+ *   K a power of two in [128, 8192] (the row is one transform block); g bf16 [K], 4-byte aligned. */
+pq_status pq_rmsnorm_hadamard_quant_act(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, const void* g, float eps,
+                                        int64_t row_begin, const float* s_a, uint8_t* xq, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * W4A4 linear layer (Sec. 3: low-bit matrix multiplication; Table 1, O2):
  *     acc[t, n] = sum_k xq[t, k] * wq[n, k]          exact, int32

@@ -28,7 +28,7 @@ EXPORTS = [
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
     "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
     "pq_calib_act_asym", "pq_hadamard_quant_act_asym", "pq_weight_code_sums", "pq_w4a4_gemm_asym",
-    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma", "pq_grid_search_act_asym",
+    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma", "pq_grid_search_act_asym", "pq_rmsnorm_hadamard_quant_act",
 ]
 
 
@@ -98,6 +98,8 @@ def load_library() -> ctypes.CDLL:
     lib.pq_outlier_tokens.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_float, c_float, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p]
     lib.pq_calib_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p, c_void_p, c_void_p]
+    lib.pq_rmsnorm_hadamard_quant_act.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_float, c_int64, c_void_p,
+                                                  c_void_p, c_void_p]
     lib.pq_grid_search_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_int32, c_float, c_void_p,
                                             c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.pq_hadamard_quant_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p, c_void_p,
@@ -261,6 +263,18 @@ class Context:
             assert acc_dbg.shape == (M, N) and acc_dbg.is_contiguous()
         _ok(self.lib.pq_w4a4_gemm(self.h, _ptr(xq), _ptr(wq), _ptr(s_a), _ptr(s_w), _ptr(out), out.stride(0), M, N, K2 * 2,
                                   row_begin, _ptr(acc_dbg), c_void_p(0), 0, _stream()), "pq_w4a4_gemm")
+        return out
+
+    def rmsnorm_hadamard_quant_act(self, x: torch.Tensor, g: torch.Tensor, eps: float, s_a: torch.Tensor, row_begin: int = 0,
+                                   out: torch.Tensor | None = None):
+        """RMSNorm, rotation over the whole row and static quantizer in one launch (K a power of two up to 8192)."""
+        _dev(x, torch.bfloat16, "x"), _dev(g, torch.bfloat16, "g"), _dev(s_a, torch.float32, "s_a")
+        M, K = x.shape
+        assert x.stride(1) == 1 and g.numel() == K
+        if out is None:
+            out = torch.zeros((M, K // 2), dtype=torch.uint8, device=x.device)
+        _ok(self.lib.pq_rmsnorm_hadamard_quant_act(self.h, _ptr(x), M, K, x.stride(0), _ptr(g), float(eps), row_begin, _ptr(s_a),
+                                                   _ptr(out), _stream()), "pq_rmsnorm_hadamard_quant_act")
         return out
 
     # ---- Eq. 1 as printed: asymmetric activation quantizer with a zero point ---------------------------

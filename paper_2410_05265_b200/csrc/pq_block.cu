@@ -218,6 +218,9 @@ int grid_for(pq_ctx* ctx, int64_t work_items, int per_cta) {
 
 }  // namespace
 
+pq_status pq_rmsnorm_pow2_launch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, const void* g, float eps, void* y,
+                                 int64_t ldy, void* stream);
+
 extern "C" pq_status pq_rmsnorm(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, const void* g, float eps,
                                 void* y, int64_t ldy, void* stream) {
   if (!ctx || !x || !g || !y) return PQ_ERR_INVALID_ARG;
@@ -225,6 +228,9 @@ extern "C" pq_status pq_rmsnorm(pq_ctx* ctx, const void* x, int64_t M, int64_t K
   if (K % 8 != 0 || K > RN_THREADS * RN_MAX_VEC * 8) return PQ_ERR_SHAPE;
   if (!aligned16(x) || !aligned16(g) || !aligned16(y) || ldx % 8 != 0 || ldy % 8 != 0) return PQ_ERR_ALIGN;
   if (M == 0) return PQ_OK;
+  // a row that is one transform block of the online rotation takes the first pass of that kernel, so that
+  // pq_rmsnorm_hadamard_quant_act equals this call followed by pq_hadamard_quant_act bit for bit
+  if ((K & (K - 1)) == 0 && K >= 128 && K <= 8192) return pq_rmsnorm_pow2_launch(ctx, x, M, K, ldx, g, eps, y, ldy, stream);
   rmsnorm_kernel<<<grid_for(ctx, M, 1), RN_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const __nv_bfloat16*>(x), ldx, static_cast<const __nv_bfloat16*>(g), eps,
       static_cast<__nv_bfloat16*>(y), ldy, M, static_cast<int>(K));

@@ -45,7 +45,12 @@ __device__ __forceinline__ float swiglu_bf16(float g, float u) {
 // GRID (with CALIB and ZP; the grid search of Sec. 3 for the static s and z): s_a_in / zp_in hold n_cand candidate
 // (s, z) pairs, and the pass adds to s_a_out (n_cand doubles) the squared error of quantizing and dequantizing the
 // rotated values with each of them.
-template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU, bool GRID = false>
+// NORM (the RMSNorm in front of a block's first linears, App. B figure): the row is one transform block; its values
+// become bf16(x * r * g) with r = 1 / sqrt(mean(x^2) + eps) before the transform, in the arithmetic and with the
+// rounding of the stand-alone call, so that fusing changes no bit. x2 is then the gain g [K], clip carries eps.
+// NORM == 2 stops there and writes the normalised row (bf16, to xq with row pitch n_cand elements): the stand-alone
+// RMSNorm of such widths, which thereby shares every operation that decides r with the fused form.
+template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU, bool GRID = false, int NORM = 0>
 __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
     hadamard_quant_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int64_t n_rows, int64_t K,
                           const float* __restrict__ s_a_in, uint8_t* __restrict__ xq, float* __restrict__ s_a_out,
@@ -58,6 +63,7 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
   constexpr int BLK_FLOATS = B + B / 64;       // padded block footprint in shared memory
   constexpr int RSTRIDE = 1 << (LOGB - 5);     // element distance between consecutive r
   extern __shared__ __align__(16) float sm[];
+  __shared__ float norm_red[HQ_THREADS / 32];
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");  // input, scale and output may belong to the previous kernel
 
@@ -110,6 +116,41 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
           const float b = swiglu_bf16(__uint_as_float(w[r] & 0xFFFF0000u), __uint_as_float(w2 & 0xFFFF0000u));
           V[r] = ROTATE ? make_float2(a + b, a - b) : make_float2(a, b);
         }
+      } else if (NORM) {
+        // sum of squares of the row: this thread's 64 values in a fixed order, then the block's threads (lanes of a
+        // warp by shuffles, warps through shared memory in warp order): the same sequence in both forms
+        float ss = 0.0f;
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+          const float a = __uint_as_float(w[r] << 16), b = __uint_as_float(w[r] & 0xFFFF0000u);
+          ss = __fmaf_rn(a, a, __fmaf_rn(b, b, ss));
+        }
+        constexpr int SPAN = TPB < 32 ? TPB : 32;
+#pragma unroll
+        for (int o = SPAN / 2; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (TPB > 32) {
+          if ((tid & 31) == 0) norm_red[tid >> 5] = ss;
+          __syncthreads();
+          ss = 0.0f;
+#pragma unroll
+          for (int i = 0; i < TPB / 32; ++i) ss += norm_red[blk_local * (TPB / 32) + i];
+          __syncthreads();
+        }
+        const float rr = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(B)), clip)));
+        const uint32_t* gsrc = reinterpret_cast<const uint32_t*>(x2 + col0) + u;
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+          const uint32_t gw = __ldg(gsrc + r * (RSTRIDE / 2));
+          const float a = __bfloat162float(__float2bfloat16_rn(__fmul_rn(__fmul_rn(__uint_as_float(w[r] << 16), rr), __uint_as_float(gw << 16))));
+          const float b = __bfloat162float(__float2bfloat16_rn(__fmul_rn(__fmul_rn(__uint_as_float(w[r] & 0xFFFF0000u), rr), __uint_as_float(gw & 0xFFFF0000u))));
+          if (NORM == 2) {
+            if (active)
+              reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(xq) + row * n_cand + col0)[u + r * (RSTRIDE / 2)] =
+                  (__float_as_uint(a) >> 16) | (__float_as_uint(b) & 0xFFFF0000u);
+          }
+          V[r] = ROTATE ? make_float2(a + b, a - b) : make_float2(a, b);
+        }
+        if (NORM == 2) continue;
       } else {
 #pragma unroll
         for (int r = 0; r < 32; ++r) {
@@ -293,10 +334,10 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
   }
 }
 
-template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU, bool GRID>
+template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU, bool GRID, int NORM = 0>
 pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_t K, const float* s_a_in, uint8_t* xq,
                  float* s_a_out, float clip, const int32_t* zp_in, const void* x2, cudaStream_t st, int n_cand) {
-  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID>;
+  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID, NORM>;
   constexpr size_t smem = HQ_SMEM_FLOATS * sizeof(float);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
     return PQ_ERR_CUDA;
@@ -490,6 +531,49 @@ extern "C" pq_status pq_hadamard_quant_act_asym(pq_ctx* ctx, const void* x, int6
                                                 uint8_t* xq, void* stream) {
   if (!z_a) return PQ_ERR_INVALID_ARG;
   return dispatch<false, 4, false, true>(ctx, x, M, K, ldx, had_block, row_begin, s_a, xq, nullptr, stream, 1.0f, z_a);
+}
+
+// ---- RMSNorm in front of the rotation (the block's first linears): the row is one transform block ----------
+namespace {
+template <int NORM>
+pq_status dispatch_norm(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, const void* g, float eps, int64_t row_begin,
+                        const float* s_a, void* dst, int64_t ld_dst, void* stream) {
+  if (!ctx || !x || !g || !dst || (NORM == 1 && !s_a)) return PQ_ERR_INVALID_ARG;
+  if (M < 0 || K <= 0 || ldx < K || row_begin < 0 || (NORM == 2 && ld_dst < K)) return PQ_ERR_INVALID_ARG;
+  if ((K & (K - 1)) != 0 || K < 128 || K > 8192) return PQ_ERR_SHAPE;
+  if ((ldx & 1) || (reinterpret_cast<uintptr_t>(x) & 3) || (reinterpret_cast<uintptr_t>(g) & 3)) return PQ_ERR_ALIGN;
+  if (NORM == 1 && (reinterpret_cast<uintptr_t>(dst) & 15)) return PQ_ERR_ALIGN;
+  if (NORM == 2 && ((ld_dst & 1) || (reinterpret_cast<uintptr_t>(dst) & 3))) return PQ_ERR_ALIGN;
+  if (row_begin >= M) return PQ_OK;
+  const int64_t n_rows = M - row_begin;
+  const void* x0 = static_cast<const __nv_bfloat16*>(x) + row_begin * ldx;
+  uint8_t* d0 = NORM == 1 ? static_cast<uint8_t*>(dst) + row_begin * (K / 2)
+                          : reinterpret_cast<uint8_t*>(static_cast<__nv_bfloat16*>(dst) + row_begin * ld_dst);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int ld = static_cast<int>(ld_dst);
+  constexpr bool R = NORM == 1;
+  switch (K) {
+    case 128: return launch<7, R, false, 4, false, false, false, false, NORM>(ctx, x0, ldx, n_rows, K, s_a, d0, nullptr, eps, nullptr, g, st, ld);
+    case 256: return launch<8, R, false, 4, false, false, false, false, NORM>(ctx, x0, ldx, n_rows, K, s_a, d0, nullptr, eps, nullptr, g, st, ld);
+    case 512: return launch<9, R, false, 4, false, false, false, false, NORM>(ctx, x0, ldx, n_rows, K, s_a, d0, nullptr, eps, nullptr, g, st, ld);
+    case 1024: return launch<10, R, false, 4, false, false, false, false, NORM>(ctx, x0, ldx, n_rows, K, s_a, d0, nullptr, eps, nullptr, g, st, ld);
+    case 2048: return launch<11, R, false, 4, false, false, false, false, NORM>(ctx, x0, ldx, n_rows, K, s_a, d0, nullptr, eps, nullptr, g, st, ld);
+    case 4096: return launch<12, R, false, 4, false, false, false, false, NORM>(ctx, x0, ldx, n_rows, K, s_a, d0, nullptr, eps, nullptr, g, st, ld);
+    case 8192: return launch<13, R, false, 4, false, false, false, false, NORM>(ctx, x0, ldx, n_rows, K, s_a, d0, nullptr, eps, nullptr, g, st, ld);
+    default: return PQ_ERR_SHAPE;
+  }
+}
+}  // namespace
+
+extern "C" pq_status pq_rmsnorm_hadamard_quant_act(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, const void* g, float eps,
+                                                   int64_t row_begin, const float* s_a, uint8_t* xq, void* stream) {
+  return dispatch_norm<1>(ctx, x, M, K, ldx, g, eps, row_begin, s_a, xq, 0, stream);
+}
+
+// The stand-alone RMSNorm of a row that is one transform block (K a power of two up to 8192): the same first pass.
+pq_status pq_rmsnorm_pow2_launch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, const void* g, float eps, void* y,
+                                 int64_t ldy, void* stream) {
+  return dispatch_norm<2>(ctx, x, M, K, ldx, g, eps, 0, nullptr, y, ldy, stream);
 }
 
 // ---- SwiGLU fused into the rotation of the down projection's input (App. B: R4 sits between the two) ------

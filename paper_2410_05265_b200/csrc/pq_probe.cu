@@ -5,7 +5,7 @@
 
 namespace {
 
-constexpr int PR_M = 128, PR_N = 256, PR_K = 32;  // one instruction: 128 x 256 x 32 multiply-accumulates
+constexpr int PR_M = 128, PR_N = 256;  // one instruction: 128 x 256 x 32 multiply-accumulates
 constexpr int PR_SMEM = 1024 + PR_M * 128 + PR_N * 128;  // 128-byte swizzled rows (only the first 32 bytes are read)
 
 __global__ void __launch_bounds__(128, 1) probe_i8_mma_kernel(int iters, long long* cycles, int32_t* status, long long wait_clocks) {

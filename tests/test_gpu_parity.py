@@ -432,6 +432,28 @@ def test_rmsnorm_matches_oracle(ctx, M, K):
     assert_bf16_close(inputs.bits(got), ref, "rmsnorm")
 
 
+@pytest.mark.parametrize("M,K,row_begin", [(5, 128, 0), (37, 1024, 3), (70, 4096, 4), (19, 8192, 0), (300, 2048, 0)])
+def test_rmsnorm_fused_into_rotate_quantize_changes_no_bit(ctx, M, K, row_begin):
+    """RMSNorm formed inside the rotation kernel against the two-launch path bit for bit (each of whose stages the
+    oracle checks on its own), and the fused codes against the oracle's rotation + quantizer on the GPU's own
+    normalised rows."""
+    x = inputs.activations(M, K, seed=0, n_prefix=row_begin)
+    g = (1.0 + 0.1 * inputs.weights(1, K, seed=7)[0] / 0.02 * 0.1).to(torch.bfloat16)
+    xd, gd = x.cuda(), g.cuda()
+    h = ctx.rmsnorm(xd, gd, 1e-5)
+    assert_bf16_close(inputs.bits(h), orc.rmsnorm(inputs.bits(x), inputs.bits(g), 1e-5), "rmsnorm feeding the rotation")
+    s_a = ctx.calib_act_scale(h, K, row_begin)
+    two = torch.full((M, K // 2), 0x5A, dtype=torch.uint8, device="cuda")
+    one = torch.full((M, K // 2), 0x5A, dtype=torch.uint8, device="cuda")
+    ctx.hadamard_quant_act(h, K, s_a, row_begin, out=two)
+    ctx.rmsnorm_hadamard_quant_act(xd, gd, 1e-5, s_a, row_begin, out=one)
+    ctx.check()
+    assert torch.equal(one, two)
+    ref, tie = orc.quant_act(inputs.bits(h), K, np.float32(float(s_a)), row_begin, want_tie_dist=True)
+    n = assert_codes_tie_tolerant(to_np(one)[row_begin:], ref[row_begin:], tie[row_begin:], "fused rmsnorm codes")
+    assert n <= max(2, int(2e-4 * x.numel()))
+
+
 @pytest.mark.parametrize("T,H,pos0", [(3, 2, 0), (33, 9, 4), (5, 72, 4090)])
 def test_rope_matches_oracle(ctx, T, H, pos0):
     x = inputs.kv_tensor(1, T, H, 128, 0, "k")[0]
