@@ -264,6 +264,17 @@ pq_status pq_silu_mul(pq_ctx* ctx, const void* gate, const void* up, int64_t M, 
                       int64_t ldy, void* stream);
 pq_status pq_residual_add(pq_ctx* ctx, const void* a, const void* b, void* y, int64_t n, void* stream);
 
+/* Rotary embedding and KV4 quantize-on-write of a prefill in one launch (App. B block order: q|k|v projection ->
+ * rotary embedding (-> R3) -> cache): qkv bf16 [T, (Hq + 2 Hkv) * D] with ld elements between tokens is the
+ * concatenated projection output of T tokens of sequence `seq` at positions pos0 .. pos0 + T - 1. The q and k heads
+ * are rotated in place (pq_rope, or pq_rope_rotate when rotate != 0), the rotated k heads and the v heads are
+ * quantized with s_k[h], s_v[h] and written at positions len[seq] .. len[seq] + T - 1, and len[seq] += T: the result
+ * of pq_rope / pq_rope_rotate followed by pq_kv4_append_strided, bit for bit. If the sequence would exceed Tmax the
+ * rotation still happens, nothing is appended and PQ_ERR_SHAPE is left in the status word.
+ *   qkv, kq, vq 16-byte aligned, ld a multiple of 8, D = 128. */
+pq_status pq_rope_kv4_append(pq_ctx* ctx, const pq_kv4_cache* cache, int32_t seq, void* qkv, int64_t T, int64_t ld, int64_t pos0,
+                             double theta, int32_t rotate, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Decode attention for callers that may not allocate. (The paper has no counterpart: this is a
  * packaging variant of pq_decode_attn_kv4_prefix, same kernel, same arguments and result.)

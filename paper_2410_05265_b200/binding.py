@@ -28,7 +28,7 @@ EXPORTS = [
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
     "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
     "pq_calib_act_asym", "pq_hadamard_quant_act_asym", "pq_weight_code_sums", "pq_w4a4_gemm_asym",
-    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma", "pq_grid_search_act_asym", "pq_rmsnorm_hadamard_quant_act",
+    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma", "pq_grid_search_act_asym", "pq_rmsnorm_hadamard_quant_act", "pq_rope_kv4_append",
 ]
 
 
@@ -100,6 +100,8 @@ def load_library() -> ctypes.CDLL:
     lib.pq_calib_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p, c_void_p, c_void_p]
     lib.pq_rmsnorm_hadamard_quant_act.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_float, c_int64, c_void_p,
                                                   c_void_p, c_void_p]
+    lib.pq_rope_kv4_append.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_int32, c_void_p, c_int64, c_int64, c_int64, c_double, c_int32,
+                                       c_void_p]
     lib.pq_grid_search_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_int32, c_float, c_void_p,
                                             c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.pq_hadamard_quant_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p, c_void_p,
@@ -488,6 +490,14 @@ class Context:
         _ok(self.lib.pq_prefill_attn_kv4_prefix(self.h, ctypes.byref(cache.struct), int(seq), _ptr(q), q.stride(0), T, _ptr(out),
                                                 float(sm_scale), _stream()), "pq_prefill_attn_kv4_prefix")
         return out
+
+    def rope_kv4_append(self, cache: KV4Cache, seq: int, qkv: torch.Tensor, pos0: int, theta: float, rotate: bool = False):
+        """Rotary embedding (+ R3) of the q and k heads of qkv [T, (Hq + 2 Hkv) * D] in place and KV4 append of k, v."""
+        _dev(qkv, torch.bfloat16, "qkv")
+        T = qkv.shape[0]
+        assert qkv.dim() == 2 and qkv.stride(1) == 1 and qkv.shape[1] == (cache.Hq + 2 * cache.Hkv) * cache.D
+        _ok(self.lib.pq_rope_kv4_append(self.h, ctypes.byref(cache.struct), int(seq), _ptr(qkv), T, qkv.stride(0), int(pos0), float(theta),
+                                        1 if rotate else 0, _stream()), "pq_rope_kv4_append")
 
     # ---- transformer-block glue -----------------------------------------------------------------
     def rmsnorm(self, x: torch.Tensor, g: torch.Tensor, eps: float = 1e-5, out: torch.Tensor | None = None):

@@ -2,11 +2,11 @@
 
 Nothing is computed here: the class owns the device buffers of one block (packed weights, static
 scales, the KV cache with its full-precision prefix) and issues the C-ABI calls in the order of the
-block in App. B of the paper: RMSNorm -> [rotate + quantize] -> q|k|v GEMM -> rotary embedding (optionally
-followed by the head-wise rotation R3 of q and k) ->
-KV4 append -> causal attention over [prefix || INT4 cache] -> [rotate + quantize] -> o GEMM ->
-residual -> RMSNorm -> [rotate + quantize] -> gate|up GEMM -> [SwiGLU + block rotate + quantize, one launch] ->
-down GEMM -> residual. The tokens that enter are ordinary tokens: the prefixed outlier tokens are
+block in App. B of the paper: [RMSNorm + rotate + quantize, one launch] -> q|k|v GEMM -> [rotary embedding
+(optionally followed by the head-wise rotation R3 of q and k) + KV4 append, one launch] -> causal attention over
+[prefix || INT4 cache] -> [rotate + quantize] -> o GEMM -> residual -> [RMSNorm + rotate + quantize] -> gate|up
+GEMM -> [SwiGLU + block rotate + quantize, one launch] -> down GEMM -> residual. When every stage is looked at
+(tap) or calibrated, the fused launches are replaced by the calls they stand for, which give the same bits. The tokens that enter are ordinary tokens: the prefixed outlier tokens are
 never run through the quantized path, their K/V sit in the cache in fp16 (Sec. 4.2).
 """
 from __future__ import annotations
@@ -97,25 +97,32 @@ class Block:
         ctx, s, T = self.ctx, self.shape, x.shape[0]
         b = self._buffers(T, x.device)
         self.length.zero_()
-        ctx.rmsnorm(x, self.g_attn, s.eps, out=b["h"])
-        tap("h1", b["h"])
-        if calibrate:
-            ctx.calib_act_scale(b["h"], s.had_block(s.hidden), 0, s_a=self.s_a[0])
-        ctx.hadamard_quant_act(b["h"], s.had_block(s.hidden), self.s_a[0], out=b["xq_h"])
+        fused_norm = not (calibrate or staged) and s.hidden & (s.hidden - 1) == 0 and 128 <= s.hidden <= 8192
+        if fused_norm:  # RMSNorm inside the rotate+quantize launch: same bits, the normalised tensor stays on chip
+            ctx.rmsnorm_hadamard_quant_act(x, self.g_attn, s.eps, self.s_a[0], out=b["xq_h"])
+        else:
+            ctx.rmsnorm(x, self.g_attn, s.eps, out=b["h"])
+            tap("h1", b["h"])
+            if calibrate:
+                ctx.calib_act_scale(b["h"], s.had_block(s.hidden), 0, s_a=self.s_a[0])
+            ctx.hadamard_quant_act(b["h"], s.had_block(s.hidden), self.s_a[0], out=b["xq_h"])
         tap("xq1", b["xq_h"])
         ctx.w4a4_gemm(b["xq_h"], self.wq_qkv, self.s_a[0], self.sw_qkv, out=b["qkv"])
         tap("qkv", b["qkv"])
-        qk = b["qkv"][:, : s.q_dim + s.kv_dim].unflatten(1, (s.n_q_heads + s.n_kv_heads, s.head_dim))
-        ctx.rope(qk, self.n_prefix, s.rope_theta, out=qk, rotate=s.r3)
-        tap("qkv_rope", b["qkv"])
         q = b["qkv"][:, : s.q_dim].unflatten(1, (s.n_q_heads, s.head_dim))
         k = b["qkv"][:, s.q_dim: s.q_dim + s.kv_dim].unflatten(1, (s.n_kv_heads, s.head_dim))
         v = b["qkv"][:, s.q_dim + s.kv_dim:].unflatten(1, (s.n_kv_heads, s.head_dim))
-        if calibrate:
-            ctx.calib_kv_scale(k, self.s_k)
-            ctx.calib_kv_scale(v, self.s_v)
         cache = self._cache()
-        ctx.kv4_append(cache, k.unsqueeze(0), v.unsqueeze(0))
+        if calibrate or staged:
+            qk = b["qkv"][:, : s.q_dim + s.kv_dim].unflatten(1, (s.n_q_heads + s.n_kv_heads, s.head_dim))
+            ctx.rope(qk, self.n_prefix, s.rope_theta, out=qk, rotate=s.r3)
+            tap("qkv_rope", b["qkv"])
+            if calibrate:
+                ctx.calib_kv_scale(k, self.s_k)
+                ctx.calib_kv_scale(v, self.s_v)
+            ctx.kv4_append(cache, k.unsqueeze(0), v.unsqueeze(0))
+        else:  # rotary embedding (+ R3) and the KV4 append in one launch: same bits
+            ctx.rope_kv4_append(cache, 0, b["qkv"], self.n_prefix, s.rope_theta, rotate=s.r3)
         tap("kq", self.kq)
         tap("vq", self.vq)
         ctx.prefill_attn(cache, 0, q, 1.0 / math.sqrt(s.head_dim), out=b["attn"])
@@ -129,11 +136,14 @@ class Block:
         tap("o", b["o"])
         ctx.residual_add(x, b["o"], out=b["x2"])
         tap("x2", b["x2"])
-        ctx.rmsnorm(b["x2"], self.g_mlp, s.eps, out=b["h"])
-        tap("h2", b["h"])
-        if calibrate:
-            ctx.calib_act_scale(b["h"], s.had_block(s.hidden), 0, s_a=self.s_a[2])
-        ctx.hadamard_quant_act(b["h"], s.had_block(s.hidden), self.s_a[2], out=b["xq_h"])
+        if fused_norm:
+            ctx.rmsnorm_hadamard_quant_act(b["x2"], self.g_mlp, s.eps, self.s_a[2], out=b["xq_h"])
+        else:
+            ctx.rmsnorm(b["x2"], self.g_mlp, s.eps, out=b["h"])
+            tap("h2", b["h"])
+            if calibrate:
+                ctx.calib_act_scale(b["h"], s.had_block(s.hidden), 0, s_a=self.s_a[2])
+            ctx.hadamard_quant_act(b["h"], s.had_block(s.hidden), self.s_a[2], out=b["xq_h"])
         tap("xq3", b["xq_h"])
         ctx.w4a4_gemm(b["xq_h"], self.wq_gu, self.s_a[2], self.sw_gu, out=b["gu"])
         tap("gu", b["gu"])
@@ -152,4 +162,4 @@ class Block:
         tap("y", b["y"])
         return b["y"]
 
-    LAUNCHES_PER_FORWARD = 15  # 16 when every stage is tapped (the SwiGLU then is a launch of its own)
+    LAUNCHES_PER_FORWARD = 12  # 16 when every stage is tapped (RMSNorm, rotary embedding and SwiGLU then are launches of their own)

@@ -15,6 +15,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// One rotate-half pair: (a, b) -> (a cos - b sin, b cos + a sin), spelled out in single operations so that every
+// kernel that rotates (stand-alone, with R3, fused with the KV4 append) produces the same bits.
+__device__ __forceinline__ void rope_pair(float a, float b, float c, float s, float& lo, float& hi) {
+  lo = __fmaf_rn(a, c, -__fmul_rn(b, s));
+  hi = __fmaf_rn(b, c, __fmul_rn(a, s));
+}
+
 // ---- RMSNorm: y = x * rsqrt(mean(x^2) + eps) * g; one CTA per row, the row is read once ---------
 constexpr int RN_THREADS = 256;
 constexpr int RN_MAX_VEC = 8;  // 8-element vectors per thread kept in registers: K <= 256 * 8 * 8 = 16384
@@ -95,14 +102,42 @@ __global__ void __launch_bounds__(RP_THREADS)
       for (int e = 0; e < 4; ++e) {
         const float c0 = cs[i0 + 2 * e], s0 = sn[i0 + 2 * e], c1 = cs[i0 + 2 * e + 1], s1 = sn[i0 + 2 * e + 1];
         const float a0 = bf16_lo(aw[e]), a1 = bf16_hi(aw[e]), b0 = bf16_lo(bw[e]), b1 = bf16_hi(bw[e]);
-        oa[e] = pack_bf16(a0 * c0 - b0 * s0, a1 * c1 - b1 * s1);
-        ob[e] = pack_bf16(b0 * c0 + a0 * s0, b1 * c1 + a1 * s1);
+        float l0, h0, l1, h1;
+        rope_pair(a0, b0, c0, s0, l0, h0);
+        rope_pair(a1, b1, c1, s1, l1, h1);
+        oa[e] = pack_bf16(l0, l1);
+        ob[e] = pack_bf16(h0, h1);
       }
       *reinterpret_cast<uint4*>(py + i0) = make_uint4(oa[0], oa[1], oa[2], oa[3]);
       *reinterpret_cast<uint4*>(py + 64 + i0) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
     }
     __syncthreads();
   }
+}
+
+// One head of RoPE + R3 in the warp layout (lane l holds elements 2l, 2l+1, 64+2l, 65+2l): returns the two packed
+// bf16 words (elements 2l, 2l+1 and 64+2l, 65+2l).
+__device__ __forceinline__ void rope_rotate_head(float a0, float a1, float b0, float b1, float c0, float s0, float c1, float s1,
+                                                 int lane, uint32_t& pa, uint32_t& pb) {
+  float v0, v1, v2, v3;
+  rope_pair(a0, b0, c0, s0, v0, v2);
+  rope_pair(a1, b1, c1, s1, v1, v3);
+  float u;
+  u = v0, v0 = u + v1, v1 = u - v1;  // index bit 0
+  u = v2, v2 = u + v3, v3 = u - v3;
+  u = v0, v0 = u + v2, v2 = u - v2;  // index bit 6
+  u = v1, v1 = u + v3, v3 = u - v3;
+#pragma unroll
+  for (int m = 1; m < 32; m <<= 1) {  // index bits 1..5: the upper partner holds the difference
+    const bool up = lane & m;
+    const float o0 = __shfl_xor_sync(0xffffffffu, v0, m), o1 = __shfl_xor_sync(0xffffffffu, v1, m);
+    const float o2 = __shfl_xor_sync(0xffffffffu, v2, m), o3 = __shfl_xor_sync(0xffffffffu, v3, m);
+    v0 = up ? o0 - v0 : v0 + o0, v1 = up ? o1 - v1 : v1 + o1;
+    v2 = up ? o2 - v2 : v2 + o2, v3 = up ? o3 - v3 : v3 + o3;
+  }
+  const float norm = 0.08838834764831845f;  // 1 / sqrt(128)
+  pa = pack_bf16(v0 * norm, v1 * norm);
+  pb = pack_bf16(v2 * norm, v3 * norm);
 }
 
 // Rotary embedding followed by the online head-wise rotation R3 (App. B): y = RoPE(x) H_128 / sqrt(128)
@@ -129,26 +164,80 @@ __global__ void __launch_bounds__(RP_THREADS)
       const uint32_t wa = *reinterpret_cast<const uint32_t*>(px + 2 * lane);  // y may alias x: the warp reads its head first
       const uint32_t wb = *reinterpret_cast<const uint32_t*>(px + 64 + 2 * lane);
       const float a0 = bf16_lo(wa), a1 = bf16_hi(wa), b0 = bf16_lo(wb), b1 = bf16_hi(wb);
-      float v0 = a0 * c0 - b0 * s0, v1 = a1 * c1 - b1 * s1, v2 = b0 * c0 + a0 * s0, v3 = b1 * c1 + a1 * s1;
-      float u;
-      u = v0, v0 = u + v1, v1 = u - v1;  // index bit 0
-      u = v2, v2 = u + v3, v3 = u - v3;
-      u = v0, v0 = u + v2, v2 = u - v2;  // index bit 6
-      u = v1, v1 = u + v3, v3 = u - v3;
-#pragma unroll
-      for (int m = 1; m < 32; m <<= 1) {  // index bits 1..5: the upper partner holds the difference
-        const bool up = lane & m;
-        const float o0 = __shfl_xor_sync(0xffffffffu, v0, m), o1 = __shfl_xor_sync(0xffffffffu, v1, m);
-        const float o2 = __shfl_xor_sync(0xffffffffu, v2, m), o3 = __shfl_xor_sync(0xffffffffu, v3, m);
-        v0 = up ? o0 - v0 : v0 + o0, v1 = up ? o1 - v1 : v1 + o1;
-        v2 = up ? o2 - v2 : v2 + o2, v3 = up ? o3 - v3 : v3 + o3;
-      }
-      const float norm = 0.08838834764831845f;  // 1 / sqrt(128)
+      uint32_t pa, pb;
+      rope_rotate_head(a0, a1, b0, b1, c0, s0, c1, s1, lane, pa, pb);
       __syncwarp();
-      *reinterpret_cast<uint32_t*>(py + 2 * lane) = pack_bf16(v0 * norm, v1 * norm);
-      *reinterpret_cast<uint32_t*>(py + 64 + 2 * lane) = pack_bf16(v2 * norm, v3 * norm);
+      *reinterpret_cast<uint32_t*>(py + 2 * lane) = pa;
+      *reinterpret_cast<uint32_t*>(py + 64 + 2 * lane) = pb;
     }
     __syncthreads();
+  }
+}
+
+// Rotary embedding (optionally + R3) of the q and k heads of a concatenated q|k|v row, in place, and the KV4
+// quantize-on-write of the rotated k heads and of the v heads in the same launch (what pq_rope / pq_rope_rotate followed
+// by pq_kv4_append_strided do, bit for bit). One CTA per token, one warp per head in the layout above; a lane's four
+// elements are two bytes of the head's packed row. The last CTA to finish advances the sequence's length.
+__device__ __forceinline__ int kv_code(float x, float s) { return max(-8, min(7, __float2int_rn(__fdiv_rn(x, s)))); }
+
+__global__ void __launch_bounds__(RP_THREADS)
+    rope_kv4_append_kernel(__nv_bfloat16* qkv, int64_t T, int Hq, int Hkv, int64_t ld, int64_t pos0, double log2_theta, int rotate,
+                           uint8_t* __restrict__ kq, uint8_t* __restrict__ vq, const float* __restrict__ s_k,
+                           const float* __restrict__ s_v, int32_t* len, int Tmax, int32_t* status, uint32_t* ticket) {
+  __shared__ float cs[64], sn[64];
+  __shared__ int last;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int len0 = __ldcg(len);
+  const bool bad = len0 < 0 || len0 + T > Tmax;  // every CTA reaches the same verdict: then nothing is appended
+  const int n_heads = Hq + 2 * Hkv;
+  for (int64_t t = blockIdx.x; t < T; t += gridDim.x) {
+    if (threadIdx.x < 64) {
+      const double inv_freq = exp2(-2.0 * static_cast<double>(threadIdx.x) / 128.0 * log2_theta);
+      double s, c;
+      sincos(static_cast<double>(pos0 + t) * inv_freq, &s, &c);
+      cs[threadIdx.x] = static_cast<float>(c), sn[threadIdx.x] = static_cast<float>(s);
+    }
+    __syncthreads();
+    const float c0 = cs[2 * lane], s0 = sn[2 * lane], c1 = cs[2 * lane + 1], s1 = sn[2 * lane + 1];
+    for (int hd = warp; hd < n_heads; hd += RP_THREADS / 32) {
+      __nv_bfloat16* px = qkv + t * ld + hd * 128;
+      uint32_t pa = *reinterpret_cast<const uint32_t*>(px + 2 * lane), pb = *reinterpret_cast<const uint32_t*>(px + 64 + 2 * lane);
+      if (hd < Hq + Hkv) {  // q and k heads are rotated; v passes through
+        const float a0 = bf16_lo(pa), a1 = bf16_hi(pa), b0 = bf16_lo(pb), b1 = bf16_hi(pb);
+        if (rotate) {
+          rope_rotate_head(a0, a1, b0, b1, c0, s0, c1, s1, lane, pa, pb);
+        } else {
+          float l0, h0, l1, h1;
+          rope_pair(a0, b0, c0, s0, l0, h0);
+          rope_pair(a1, b1, c1, s1, l1, h1);
+          pa = pack_bf16(l0, l1), pb = pack_bf16(h0, h1);
+        }
+        *reinterpret_cast<uint32_t*>(px + 2 * lane) = pa;
+        *reinterpret_cast<uint32_t*>(px + 64 + 2 * lane) = pb;
+      }
+      if (hd >= Hq && !bad) {
+        const bool is_v = hd >= Hq + Hkv;
+        const int kvh = is_v ? hd - Hq - Hkv : hd - Hq;
+        const float s = __ldg((is_v ? s_v : s_k) + kvh);
+        uint8_t* row = (is_v ? vq : kq) + (static_cast<int64_t>(kvh) * Tmax + len0 + t) * 64;
+        row[lane] = static_cast<uint8_t>((kv_code(bf16_lo(pa), s) & 0xF) | ((kv_code(bf16_hi(pa), s) & 0xF) << 4));
+        row[32 + lane] = static_cast<uint8_t>((kv_code(bf16_lo(pb), s) & 0xF) | ((kv_code(bf16_hi(pb), s) & 0xF) << 4));
+      }
+    }
+    __syncthreads();
+  }
+  if (bad) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) pq::report(status, PQ_ERR_SHAPE);
+    return;
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+    if (last) {
+      *len = len0 + static_cast<int>(T);
+      *ticket = 0;
+    }
   }
 }
 
@@ -258,6 +347,21 @@ extern "C" pq_status pq_rope_rotate(pq_ctx* ctx, const void* x, int64_t T, int32
   if (T == 0) return PQ_OK;
   rope_rotate_kernel<<<grid_for(ctx, T, 1), RP_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(y), T, H, ld, pos0, log2(theta));
+  return pq_launch_status();
+}
+
+extern "C" pq_status pq_rope_kv4_append(pq_ctx* ctx, const pq_kv4_cache* c, int32_t seq, void* qkv, int64_t T, int64_t ld, int64_t pos0,
+                                        double theta, int32_t rotate, void* stream) {
+  if (!ctx || !c || !qkv || !c->kq || !c->vq || !c->s_k || !c->s_v || !c->len) return PQ_ERR_INVALID_ARG;
+  if (T < 0 || seq < 0 || seq >= c->B || c->Hkv <= 0 || c->Hq <= 0 || pos0 < 0 || !(theta > 1.0)) return PQ_ERR_INVALID_ARG;
+  if (ld < static_cast<int64_t>(c->Hq + 2 * c->Hkv) * 128) return PQ_ERR_INVALID_ARG;
+  if (c->D != 128) return PQ_ERR_SHAPE;
+  if (!aligned16(qkv) || ld % 8 != 0 || !aligned16(c->kq) || !aligned16(c->vq)) return PQ_ERR_ALIGN;
+  if (T == 0) return PQ_OK;
+  const int64_t seq_off = static_cast<int64_t>(seq) * c->Hkv * c->Tmax * 64;
+  rope_kv4_append_kernel<<<grid_for(ctx, T, 1), RP_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<__nv_bfloat16*>(qkv), T, c->Hq, c->Hkv, ld, pos0, log2(theta), rotate, c->kq + seq_off, c->vq + seq_off, c->s_k, c->s_v,
+      c->len + seq, c->Tmax, ctx->d_status, ctx->d_tickets + 1);
   return pq_launch_status();
 }
 

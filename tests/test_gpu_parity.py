@@ -487,6 +487,51 @@ def test_rope_rotate_matches_oracle(ctx, T, H, pos0):
     assert float((s_plain - s_rot).abs().max()) <= 2.0**-6 * float(s_plain.abs().max())
 
 
+@pytest.mark.parametrize("T,Hq,Hkv,rotate,start", [(1, 4, 1, False, 0), (37, 8, 2, False, 5), (300, 8, 2, True, 11), (64, 64, 8, True, 0)])
+def test_rope_fused_with_kv4_append_equals_the_two_calls(ctx, T, Hq, Hkv, rotate, start):
+    """pq_rope_kv4_append against pq_rope (or pq_rope_rotate) followed by pq_kv4_append_strided: the q|k|v buffer, the
+    appended codes and the length bit for bit (each of those calls is checked against the oracle on its own)."""
+    from paper_2410_05265_b200 import binding
+
+    D, Tmax, P = 128, T + start + 3, 4
+    width = (Hq + 2 * Hkv) * D
+    qkv = inputs.kv_tensor(1, T, Hq + 2 * Hkv, D, 5, "k")[0].reshape(T, width).contiguous()
+    s_k = orc.calib_kv_scale(inputs.bits(inputs.kv_tensor(2, 64, Hkv, D, 1, "k")))
+    s_v = orc.calib_kv_scale(inputs.bits(inputs.kv_tensor(2, 64, Hkv, D, 1, "v")))
+
+    def cache(B):
+        kq = torch.full((B, Hkv, Tmax, D // 2), 0x11, dtype=torch.uint8, device="cuda")
+        return binding.KV4Cache(None, None, kq, torch.full_like(kq, 0x11), dev(s_k), dev(s_v),
+                                torch.full((B,), start, dtype=torch.int32, device="cuda"), Hq)
+
+    # the two calls
+    a, ca = qkv.cuda(), cache(1)
+    qk = a[:, : (Hq + Hkv) * D].unflatten(1, (Hq + Hkv, D))
+    ctx.rope(qk, P, 500000.0, out=qk, rotate=rotate)
+    k = a[:, Hq * D: (Hq + Hkv) * D].unflatten(1, (Hkv, D)).unsqueeze(0)
+    v = a[:, (Hq + Hkv) * D:].unflatten(1, (Hkv, D)).unsqueeze(0)
+    ctx.kv4_append(ca, k, v)
+    # one call, on the second sequence of a two-sequence cache
+    b, cb = qkv.cuda(), cache(2)
+    ctx.rope_kv4_append(cb, 1, b, P, 500000.0, rotate=rotate)
+    ctx.check()
+    assert torch.equal(a, b), "rotated q and k (and the untouched v) must be the same bits"
+    assert torch.equal(cb.kq[1], ca.kq[0]) and torch.equal(cb.vq[1], ca.vq[0])
+    assert cb.length.tolist() == [start, start + T] and ca.length.tolist() == [start + T]
+    assert bool((cb.kq[0] == 0x11).all()) and bool((cb.vq[0] == 0x11).all()), "the other sequence is not touched"
+    # past the capacity: the rotation still happens, nothing is appended, the verdict comes through the status word
+    c2 = cache(1)
+    c2.length.fill_(Tmax - T + 1)
+    b2 = qkv.cuda()
+    ctx.rope_kv4_append(c2, 0, b2, P, 500000.0, rotate=rotate)
+    assert ctx.check_status() == 2
+    assert torch.equal(b2, a) and bool((c2.kq == 0x11).all()) and c2.length.tolist() == [Tmax - T + 1]
+    # and the counters are in order afterwards
+    c3 = cache(1)
+    ctx.rope_kv4_append(c3, 0, qkv.cuda(), P, 500000.0, rotate=rotate)
+    assert ctx.check_status() == 0 and torch.equal(c3.kq, ca.kq)
+
+
 @pytest.mark.parametrize("M,F,B,row_begin", [(19, 1024, 1024, 0), (33, 14336, 2048, 4), (5, 256, 128, 1), (130, 4096, 4096, 0)])
 def test_swiglu_fused_into_rotate_quantize_changes_no_bit(ctx, M, F, B, row_begin):
     """SiLU(gate) * up formed inside the rotation kernel against the two-launch path (which the oracle checks
