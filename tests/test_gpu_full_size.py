@@ -147,3 +147,92 @@ def test_gemm_llama70b_prefill_4096_sampled_rows(ctx):
     acc_ref = orc.gemm_i4(to_np(xq[rows]), to_np(wq))
     assert np.array_equal(to_np(acc[rows]), acc_ref)
     assert_bf16_close(inputs.bits(out[rows]), orc.dequant_bf16(acc_ref, np.float32(0.01), to_np(s_w)), "gemm 70B down")
+
+
+def test_block_llama70b_4096_staged_sampled_rows():
+    """configs[4] at full width (hidden 8192, 64 / 8 heads, FFN 28672, 4096 tokens after 4 prefixed ones): every stage
+    of the block against the oracle applied to the GPU's own input of that stage, on sampled token rows; then the
+    untapped pass (fused RMSNorm, rotary + append and SwiGLU launches) must reproduce the tapped one bit for bit."""
+    from paper_2410_05265_b200 import binding, block
+
+    ctx = binding.Context()
+    c = inputs.LLAMA3_70B
+    T, P, D = 4096, N_PREFIX, c["head_dim"]
+    Hq, Hkv = c["n_q_heads"], c["n_kv_heads"]
+    shape = block.BlockShape(hidden=c["hidden"], n_q_heads=Hq, n_kv_heads=Hkv, ffn=c["ffn"])
+    qd, kvd, hidden, ffn = shape.q_dim, shape.kv_dim, shape.hidden, shape.ffn
+    dev = "cuda"
+    W = dict(qkv=inputs.weights(qd + 2 * kvd, hidden, seed=2, device=dev), o=inputs.weights(hidden, qd, seed=3, device=dev),
+             gu=inputs.weights(2 * ffn, hidden, seed=4, device=dev), d=inputs.weights(hidden, ffn, seed=5, device=dev))
+    g1 = torch.ones(hidden, dtype=torch.bfloat16, device=dev)
+    pk, pv = inputs.prefix_kv(Hkv, P, D, 0, "k", 50.0), inputs.prefix_kv(Hkv, P, D, 0, "v", 50.0)
+    blk = block.Block(ctx, shape, W["qkv"], W["o"], W["gu"], W["d"], g1, g1, pk.cuda(), pv.cuda(), t_max=T)
+    blk.forward(inputs.activations(T, hidden, seed=1, device=dev), calibrate=True)
+    x = inputs.activations(T, hidden, seed=0, device=dev)
+    taps = {}
+    y = blk.forward(x, tap=lambda name, t: taps.__setitem__(name, t.detach().clone()))
+    ctx.check()
+    s_a = [float(s.item()) for s in blk.s_a]
+    s_k, s_v = to_np(blk.s_k), to_np(blk.s_v)
+    rows = np.array([0, 1, 127, 128, 255, 256, 2047, 2048, 4095])
+    ridx = torch.from_numpy(rows).cuda()
+    rb = lambda t: inputs.bits(t[ridx].contiguous())           # sampled rows of a device tensor as bf16 bit patterns
+    had = [shape.had_block(hidden), shape.had_block(qd), shape.had_block(hidden), shape.had_block(ffn)]
+
+    def check_quant(name, src, blockw, s):
+        ref, tie = orc.quant_act(rb(src), blockw, np.float32(s), 0, want_tie_dist=True)
+        n = assert_codes_tie_tolerant(to_np(taps[name][ridx]), ref, tie, name)
+        assert n <= max(2, int(2e-4 * ref.size * 2))
+
+    def check_gemm(name, xq_name, wname, wq, sw, s):
+        # weights: sampled output channels of the offline quantizer bit for bit, then the GEMM on the GPU's own codes
+        ch = torch.tensor([0, 1, 255, 256, wq.shape[0] - 1], device=dev)
+        wq_ref, sw_ref = orc.quant_weights(inputs.bits(W[wname][ch].contiguous()))
+        assert np.array_equal(to_np(wq[ch]), wq_ref) and np.array_equal(to_np(sw[ch]), sw_ref)
+        acc = orc.gemm_i4(to_np(taps[xq_name][ridx]), to_np(wq))
+        assert_bf16_close(rb(taps[name]), orc.dequant_bf16(acc, np.float32(s), to_np(sw)), name)
+
+    assert_bf16_close(rb(taps["h1"]), orc.rmsnorm(rb(x), inputs.bits(g1)), "rmsnorm 1")
+    check_quant("xq1", taps["h1"], had[0], s_a[0])
+    check_gemm("qkv", "xq1", "qkv", blk.wq_qkv, blk.sw_qkv, s_a[0])
+    # rotary embedding at positions P + t, one sampled token at a time (the oracle takes a start position)
+    for t in rows[[0, 3, 8]]:
+        qk = taps["qkv"][t: t + 1, : qd + kvd].reshape(1, Hq + Hkv, D).contiguous()
+        got = taps["qkv_rope"][t: t + 1, : qd + kvd].reshape(1, Hq + Hkv, D).contiguous()
+        assert_bf16_close(inputs.bits(got), orc.rope(inputs.bits(qk), P + int(t), 500000.0), "rope")
+    assert torch.equal(taps["qkv_rope"][:, qd + kvd:], taps["qkv"][:, qd + kvd:])
+    # KV4 append of all 4096 tokens (the multi-CTA path): sampled tokens as a batch of one-token sequences
+    n = len(rows)
+    k_s = taps["qkv_rope"][ridx, qd: qd + kvd].reshape(n, 1, Hkv, D).contiguous()
+    v_s = taps["qkv_rope"][ridx, qd + kvd:].reshape(n, 1, Hkv, D).contiguous()
+    kq_ref, vq_ref = np.zeros((n, Hkv, 1, D // 2), np.uint8), np.zeros((n, Hkv, 1, D // 2), np.uint8)
+    assert orc.kv4_append(inputs.bits(k_s), inputs.bits(v_s), s_k, s_v, kq_ref, vq_ref, np.zeros(n, np.int32)) == 0
+    assert np.array_equal(to_np(taps["kq"][0][:, ridx]).transpose(1, 0, 2), kq_ref[:, :, 0])
+    assert np.array_equal(to_np(taps["vq"][0][:, ridx]).transpose(1, 0, 2), vq_ref[:, :, 0])
+    assert int(blk.length[0]) == T
+    # causal attention of sampled tokens over the GPU's own cache
+    toks = rows[[0, 2, 3, 6, 8]]
+    q_s = taps["qkv_rope"][torch.from_numpy(toks).cuda(), :qd].reshape(len(toks), Hq, D).contiguous()
+    kq_b = np.ascontiguousarray(np.broadcast_to(to_np(taps["kq"]), (len(toks), Hkv, T, D // 2)))
+    vq_b = np.ascontiguousarray(np.broadcast_to(to_np(taps["vq"]), (len(toks), Hkv, T, D // 2)))
+    _, ref = orc.decode_attn(inputs.bits(q_s), inputs.bits(pk), inputs.bits(pv), kq_b, vq_b, s_k, s_v, (toks + 1).astype(np.int32),
+                             1 / math.sqrt(D), want_f64=True)
+    assert_attn_close(inputs.bits(taps["attn"][torch.from_numpy(toks).cuda()].contiguous()), ref, "prefill attention in the block")
+    check_quant("xq2", taps["attn"].reshape(T, qd), had[1], s_a[1])
+    check_gemm("o", "xq2", "o", blk.wq_o, blk.sw_o, s_a[1])
+    assert np.array_equal(rb(taps["x2"]), orc.add(rb(x), rb(taps["o"])))
+    assert_bf16_close(rb(taps["h2"]), orc.rmsnorm(rb(taps["x2"]), inputs.bits(g1)), "rmsnorm 2")
+    check_quant("xq3", taps["h2"], had[2], s_a[2])
+    check_gemm("gu", "xq3", "gu", blk.wq_gu, blk.sw_gu, s_a[2])
+    gu = taps["gu"][ridx]
+    assert_bf16_close(rb(taps["act"]), orc.silu_mul(inputs.bits(gu[:, :ffn].contiguous()), inputs.bits(gu[:, ffn:].contiguous())), "silu_mul")
+    check_quant("xq4", taps["act"], had[3], s_a[3])           # the 14-block rotation of the 28672-wide input
+    check_gemm("d", "xq4", "d", blk.wq_down, blk.sw_down, s_a[3])
+    assert np.array_equal(rb(taps["y"]), orc.add(rb(taps["x2"]), rb(taps["d"])))
+    # the pass bench.py times (no taps: fused launches) gives the same bits, twice
+    want = taps["y"]
+    taps.clear()
+    for _ in range(2):
+        assert torch.equal(blk.forward(x), want)
+    ctx.check()
+    ctx.close()
