@@ -604,9 +604,10 @@ int orc_kv4_append(const uint16_t* k, const uint16_t* v, int64_t B, int64_t T_ne
 // One (query row, head) of softmax attention in double over the union of
 //   n_prefix prefix keys/values (fp16, [Hkv, n_prefix, D], one copy shared by every sequence) and
 //   n_ctx quantized keys/values (codes * per-head scale).
+// sk_tok, sv_tok (nullable): one step per cached key (group-wise dynamic KV, Table 1 O1); they replace sk, sv.
 static void attend_one(const double* q, int64_t D, double sm_scale, const uint16_t* pk, const uint16_t* pv,
                        int64_t n_prefix, const uint8_t* kq, const uint8_t* vq, int64_t n_ctx, double sk, double sv,
-                       double* out) {
+                       double* out, const float* sk_tok = nullptr, const float* sv_tok = nullptr) {
   int64_t n = n_prefix + n_ctx;
   std::vector<double> sc(n);
   for (int64_t j = 0; j < n; ++j) {
@@ -614,7 +615,8 @@ static void attend_one(const double* q, int64_t D, double sm_scale, const uint16
     if (j < n_prefix)
       for (int64_t d = 0; d < D; ++d) s += q[d] * fp16_to_double(pk[j * D + d]);
     else
-      for (int64_t d = 0; d < D; ++d) s += q[d] * (nib_get(kq + (j - n_prefix) * (D / 2), d) * sk);
+      for (int64_t d = 0; d < D; ++d)
+        s += q[d] * (nib_get(kq + (j - n_prefix) * (D / 2), d) * (sk_tok ? static_cast<double>(sk_tok[j - n_prefix]) : sk));
     sc[j] = s * sm_scale;
   }
   double mx = -INFINITY;
@@ -630,7 +632,8 @@ static void attend_one(const double* q, int64_t D, double sm_scale, const uint16
     if (j < n_prefix)
       for (int64_t d = 0; d < D; ++d) out[d] += p * fp16_to_double(pv[j * D + d]);
     else
-      for (int64_t d = 0; d < D; ++d) out[d] += p * (nib_get(vq + (j - n_prefix) * (D / 2), d) * sv);
+      for (int64_t d = 0; d < D; ++d)
+        out[d] += p * (nib_get(vq + (j - n_prefix) * (D / 2), d) * (sv_tok ? static_cast<double>(sv_tok[j - n_prefix]) : sv));
   }
 }
 
@@ -670,6 +673,74 @@ void orc_prefill_attn(const uint16_t* q, const uint16_t* prefix_k, const uint16_
     for (int64_t d = 0; d < D; ++d) qd[d] = bf16_to_double(q[(t * Hq + g) * D + d]);
     attend_one(qd.data(), D, sm_scale, prefix_k + h * n_prefix * D, prefix_v + h * n_prefix * D, n_prefix,
                kq + h * Tmax * (D / 2), vq + h * Tmax * (D / 2), t + 1, s_k[h], s_v[h], od.data());
+    for (int64_t d = 0; d < D; ++d) {
+      out[(t * Hq + g) * D + d] = double_to_bf16(od[d]);
+      if (out_f64) out_f64[(t * Hq + g) * D + d] = od[d];
+    }
+  });
+}
+
+// ---- group-wise dynamic KV4 (Table 1, O1: "group-wise dynamic" KV cache, group size 128 = the head dimension) --
+// Every (token, head) vector of 128 values is one group with its own step, computed online when the token is
+// written: s = fp32(max |x|) / 7 in fp32 (1 for an all-zero vector), code = clamp(rint_fp32(x / s), -8, 7) with the
+// fp32 decision of the static path. Steps go to sk_tok, sv_tok f32 [B,H,Tmax] at the token's position.
+int orc_kv4_append_dyn(const uint16_t* k, const uint16_t* v, int64_t B, int64_t T_new, int64_t H, int64_t D, uint8_t* kq,
+                       uint8_t* vq, float* sk_tok, float* sv_tok, int32_t* len, int64_t Tmax) {
+  for (int64_t b = 0; b < B; ++b)
+    if (len[b] + T_new > Tmax) return 1;
+  for (int64_t b = 0; b < B; ++b) {
+    for (int64_t t = 0; t < T_new; ++t)
+      for (int64_t h = 0; h < H; ++h) {
+        const int64_t pos = len[b] + t;
+        for (int which = 0; which < 2; ++which) {
+          const uint16_t* src = (which ? v : k) + ((b * T_new + t) * H + h) * D;
+          uint8_t* row = (which ? vq : kq) + ((b * H + h) * Tmax + pos) * (D / 2);
+          float mx = 0.0f;
+          for (int64_t d = 0; d < D; ++d) mx = std::max(mx, std::fabs(static_cast<float>(bf16_to_double(src[d]))));
+          volatile float sv_ = mx == 0.0f ? 1.0f : mx / 7.0f;
+          const float s = sv_;
+          (which ? sv_tok : sk_tok)[(b * H + h) * Tmax + pos] = s;
+          for (int64_t d = 0; d < D; ++d) {
+            volatile float q = static_cast<float>(bf16_to_double(src[d])) / s;
+            nib_set(row, d, clampi(static_cast<long>(std::nearbyintf(q)), -8, 7));
+          }
+        }
+      }
+    len[b] += static_cast<int32_t>(T_new);
+  }
+  return 0;
+}
+
+// Decode attention (Eq. 3) over [prefix || INT4 cache] with one step per cached key and value vector.
+void orc_decode_attn_dyn(const uint16_t* q, const uint16_t* prefix_k, const uint16_t* prefix_v, const uint8_t* kq,
+                         const uint8_t* vq, const float* sk_tok, const float* sv_tok, const int32_t* len, int64_t B, int64_t Hq,
+                         int64_t Hkv, int64_t D, int64_t n_prefix, int64_t Tmax, double sm_scale, uint16_t* out, double* out_f64) {
+  int64_t group = Hq / Hkv;
+  parallel_rows(B * Hq, [&](int64_t i) {
+    int64_t b = i / Hq, g = i % Hq, h = g / group;
+    std::vector<double> qd(D), od(D);
+    for (int64_t d = 0; d < D; ++d) qd[d] = bf16_to_double(q[(b * Hq + g) * D + d]);
+    attend_one(qd.data(), D, sm_scale, prefix_k + h * n_prefix * D, prefix_v + h * n_prefix * D, n_prefix,
+               kq + (b * Hkv + h) * Tmax * (D / 2), vq + (b * Hkv + h) * Tmax * (D / 2), len[b], 0.0, 0.0, od.data(),
+               sk_tok + (b * Hkv + h) * Tmax, sv_tok + (b * Hkv + h) * Tmax);
+    for (int64_t d = 0; d < D; ++d) {
+      out[(b * Hq + g) * D + d] = double_to_bf16(od[d]);
+      if (out_f64) out_f64[(b * Hq + g) * D + d] = od[d];
+    }
+  });
+}
+
+// Causal prefill attention of one sequence with per-key steps (sk_tok, sv_tok [Hkv,Tmax] of this sequence).
+void orc_prefill_attn_dyn(const uint16_t* q, const uint16_t* prefix_k, const uint16_t* prefix_v, const uint8_t* kq,
+                          const uint8_t* vq, const float* sk_tok, const float* sv_tok, int64_t T, int64_t Hq, int64_t Hkv,
+                          int64_t D, int64_t n_prefix, int64_t Tmax, double sm_scale, uint16_t* out, double* out_f64) {
+  int64_t group = Hq / Hkv;
+  parallel_rows(T * Hq, [&](int64_t i) {
+    int64_t t = i / Hq, g = i % Hq, h = g / group;
+    std::vector<double> qd(D), od(D);
+    for (int64_t d = 0; d < D; ++d) qd[d] = bf16_to_double(q[(t * Hq + g) * D + d]);
+    attend_one(qd.data(), D, sm_scale, prefix_k + h * n_prefix * D, prefix_v + h * n_prefix * D, n_prefix,
+               kq + h * Tmax * (D / 2), vq + h * Tmax * (D / 2), t + 1, 0.0, 0.0, od.data(), sk_tok + h * Tmax, sv_tok + h * Tmax);
     for (int64_t d = 0; d < D; ++d) {
       out[(t * Hq + g) * D + d] = double_to_bf16(od[d]);
       if (out_f64) out_f64[(t * Hq + g) * D + d] = od[d];

@@ -380,6 +380,55 @@ def decode_attn(q_bits, prefix_k, prefix_v, kq, vq, s_k, s_v, length, sm_scale, 
     return (out, out64) if want_f64 else out
 
 
+def kv4_append_dyn(k_bits, v_bits, kq, vq, sk_tok, sv_tok, length) -> int:
+    """Group-wise dynamic KV4 (group = one 128-wide (token, head) vector): in place on kq, vq [B,H,Tmax,D/2], the
+    per-vector steps sk_tok, sv_tok f32 [B,H,Tmax] and length [B]. Returns the oracle's status."""
+    k_bits, v_bits = _u16(k_bits), _u16(v_bits)
+    B, T_new, H, D = k_bits.shape
+    Tmax = kq.shape[2]
+    assert kq.dtype == np.uint8 and vq.dtype == np.uint8 and length.dtype == np.int32
+    assert sk_tok.dtype == np.float32 and sv_tok.dtype == np.float32 and sk_tok.shape == (B, H, Tmax) == sv_tok.shape
+    f = lib().orc_kv4_append_dyn
+    f.restype = c_int
+    return int(f(_p(k_bits, c_uint16), _p(v_bits, c_uint16), c_int64(B), c_int64(T_new), c_int64(H), c_int64(D), _p(kq, c_uint8),
+                 _p(vq, c_uint8), _p(sk_tok, c_float), _p(sv_tok, c_float), _p(length, c_int32), c_int64(Tmax)))
+
+
+def decode_attn_dyn(q_bits, prefix_k, prefix_v, kq, vq, sk_tok, sv_tok, length, sm_scale):
+    """Decode attention with per-key steps; returns (bf16 bits, float64)."""
+    q_bits = _u16(q_bits)
+    B, Hq, D = q_bits.shape
+    prefix_k, prefix_v = _u16(prefix_k), _u16(prefix_v)
+    Hkv, n_prefix = prefix_k.shape[0], prefix_k.shape[1]
+    Tmax = kq.shape[2]
+    kq, vq = np.ascontiguousarray(kq, np.uint8), np.ascontiguousarray(vq, np.uint8)
+    sk_tok, sv_tok = np.ascontiguousarray(sk_tok, np.float32), np.ascontiguousarray(sv_tok, np.float32)
+    assert kq.shape == (B, Hkv, Tmax, D // 2) and sk_tok.shape == (B, Hkv, Tmax)
+    length = np.ascontiguousarray(length, np.int32)
+    out, out64 = np.empty((B, Hq, D), np.uint16), np.empty((B, Hq, D), np.float64)
+    lib().orc_decode_attn_dyn(_p(q_bits, c_uint16), _p(prefix_k, c_uint16), _p(prefix_v, c_uint16), _p(kq, c_uint8), _p(vq, c_uint8),
+                              _p(sk_tok, c_float), _p(sv_tok, c_float), _p(length, c_int32), c_int64(B), c_int64(Hq), c_int64(Hkv),
+                              c_int64(D), c_int64(n_prefix), c_int64(Tmax), c_double(float(sm_scale)), _p(out, c_uint16), _p(out64, c_double))
+    return out, out64
+
+
+def prefill_attn_dyn(q_bits, prefix_k, prefix_v, kq, vq, sk_tok, sv_tok, sm_scale):
+    """Causal prefill attention of one sequence with per-key steps [Hkv,Tmax]; returns (bf16 bits, float64)."""
+    q_bits = _u16(q_bits)
+    T, Hq, D = q_bits.shape
+    prefix_k, prefix_v = _u16(prefix_k), _u16(prefix_v)
+    Hkv, n_prefix = prefix_k.shape[0], prefix_k.shape[1]
+    Tmax = kq.shape[1]
+    kq, vq = np.ascontiguousarray(kq, np.uint8), np.ascontiguousarray(vq, np.uint8)
+    sk_tok, sv_tok = np.ascontiguousarray(sk_tok, np.float32), np.ascontiguousarray(sv_tok, np.float32)
+    assert kq.shape == (Hkv, Tmax, D // 2) and sk_tok.shape == (Hkv, Tmax) and T <= Tmax
+    out, out64 = np.empty((T, Hq, D), np.uint16), np.empty((T, Hq, D), np.float64)
+    lib().orc_prefill_attn_dyn(_p(q_bits, c_uint16), _p(prefix_k, c_uint16), _p(prefix_v, c_uint16), _p(kq, c_uint8), _p(vq, c_uint8),
+                               _p(sk_tok, c_float), _p(sv_tok, c_float), c_int64(T), c_int64(Hq), c_int64(Hkv), c_int64(D),
+                               c_int64(n_prefix), c_int64(Tmax), c_double(float(sm_scale)), _p(out, c_uint16), _p(out64, c_double))
+    return out, out64
+
+
 def prefill_attn(q_bits, prefix_k, prefix_v, kq, vq, s_k, s_v, sm_scale, want_f64: bool = False):
     q_bits = _u16(q_bits)
     T, Hq, D = q_bits.shape

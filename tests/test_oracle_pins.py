@@ -684,6 +684,71 @@ def test_prefill_attention_is_causal_decode_per_row():
         assert np.array_equal(out0[0, g], orc.f64_to_bf16(vd[g // 2, 0]))
 
 
+# ---------------------------------------------------------------- group-wise dynamic KV4 (Table 1, O1)
+def test_groupwise_dynamic_kv_steps_codes_and_attention():
+    B, T, H, D, Tmax, Hq, P = 2, 5, 2, 128, 8, 4, 2
+    k, v = inputs.kv_tensor(B, T, H, D, 0, "k"), inputs.kv_tensor(B, T, H, D, 0, "v")
+    k[1, 2, 0] = 0                                        # an all-zero vector: step 1, codes 0
+    kq, vq = np.full((B, H, Tmax, D // 2), 0xEE, np.uint8), np.full((B, H, Tmax, D // 2), 0xEE, np.uint8)
+    sk, sv = np.full((B, H, Tmax), -1, np.float32), np.full((B, H, Tmax), -1, np.float32)
+    length = np.array([1, 3], np.int32)
+    assert orc.kv4_append_dyn(inputs.bits(k), inputs.bits(v), kq, vq, sk, sv, length) == 0 and length.tolist() == [6, 8]
+    kf, vf = k.to(torch.float32).numpy(), v.to(torch.float32).numpy()
+    for b, l0 in enumerate([1, 3]):
+        # one step per (token, head) vector = its own max / 7 (fp32); positions outside the append untouched
+        mk = np.abs(kf[b]).max(-1).T                      # [H, T]
+        assert np.array_equal(sk[b, :, l0:l0 + T], np.where(mk == 0, np.float32(1), mk / np.float32(7)).astype(np.float32))
+        assert np.array_equal(sv[b, :, l0:l0 + T], (np.abs(vf[b]).max(-1).T / np.float32(7)).astype(np.float32))
+        assert np.all(sk[b, :, :l0] == -1) and np.all(kq[b, :, :l0] == 0xEE) and np.all(sk[b, :, l0 + T:] == -1)
+        codes = orc.unpack_int4(kq[b, :, l0:l0 + T]).astype(np.float64)           # [H, T, D]
+        r = kf[b].transpose(1, 0, 2).astype(np.float64) / sk[b, :, l0:l0 + T, None].astype(np.float64)
+        assert np.all(np.abs(codes - r) <= 0.5 + 1e-6)
+        nz = mk > 0
+        assert np.all(np.abs(codes).max(-1)[nz] == 7), "every vector uses its full range: that is what dynamic means"
+    assert np.all(orc.unpack_int4(kq[1, 0, 3 + 2]) == 0) and sk[1, 0, 3 + 2] == 1.0
+    assert orc.kv4_append_dyn(inputs.bits(k), inputs.bits(v), kq, vq, sk, sv, length) == 1                       # would pass Tmax
+    # scale-free per vector: a vector multiplied by 2^p keeps its codes, its step takes the factor
+    k2 = k.clone()
+    k2[0, 1, 1] *= 8
+    kq2, sk2 = np.zeros_like(kq), np.zeros_like(sk)
+    orc.kv4_append_dyn(inputs.bits(k2), inputs.bits(v), kq2, np.zeros_like(vq), sk2, np.zeros_like(sv), np.array([1, 3], np.int32))
+    assert np.array_equal(kq2[0, 1, 2], kq[0, 1, 2]) and sk2[0, 1, 2] == 8 * sk[0, 1, 2] and np.array_equal(kq2[1], kq[1])
+    # with equal maxima in every vector the steps are all equal and the path is the static one, bit for bit
+    ke = k.clone()
+    ke[..., 0] = 9.0
+    s_stat = np.full(H, np.float32(9.0) / np.float32(7), np.float32)
+    kq_d, vq_d, sk_d, sv_d = np.zeros_like(kq), np.zeros_like(vq), np.zeros_like(sk), np.zeros_like(sv)
+    orc.kv4_append_dyn(inputs.bits(ke), inputs.bits(ke), kq_d, vq_d, sk_d, sv_d, np.zeros(B, np.int32))
+    kq_s, vq_s = np.zeros_like(kq), np.zeros_like(vq)
+    orc.kv4_append(inputs.bits(ke), inputs.bits(ke), s_stat, s_stat, kq_s, vq_s, np.zeros(B, np.int32))
+    assert np.array_equal(kq_d, kq_s) and np.array_equal(vq_d, vq_s) and np.all(sk_d[:, :, :T] == s_stat[0])
+    q = inputs.queries(B, Hq, D, 0)
+    pk, pv = inputs.prefix_kv(H, P, D, 0, "k", 1.0), inputs.prefix_kv(H, P, D, 0, "v", 1.0)
+    lens = np.full(B, T, np.int32)
+    o_d, o64_d = orc.decode_attn_dyn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq_d, vq_d, sk_d, sv_d, lens, 0.1)
+    o_s, o64_s = orc.decode_attn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq_s, vq_s, s_stat, s_stat, lens, 0.1, want_f64=True)
+    assert np.array_equal(o_d, o_s) and np.array_equal(o64_d, o64_s)
+    # general steps: a library softmax attention over the tensors dequantized with their own per-key steps
+    lens = np.array([6, 8], np.int32)
+    _, o64 = orc.decode_attn_dyn(inputs.bits(q), inputs.bits(pk), inputs.bits(pv), kq, vq, sk, sv, lens, 0.1)
+    kd = orc.unpack_int4(kq).astype(np.float64) * sk.astype(np.float64)[..., None]
+    vd = orc.unpack_int4(vq).astype(np.float64) * sv.astype(np.float64)[..., None]
+    for b in range(B):
+        for g in range(Hq):
+            h = g // (Hq // H)
+            K = torch.cat([pk[h].double(), torch.from_numpy(kd[b, h, :lens[b]])])
+            V = torch.cat([pv[h].double(), torch.from_numpy(vd[b, h, :lens[b]])])
+            p = torch.softmax(K @ q[b, g].double() * 0.1, dim=0)
+            assert np.allclose(o64[b, g], (p @ V).numpy(), rtol=1e-12, atol=1e-13)
+    # prefill = the causal rows of the decode form
+    qt = inputs.normal(5, inputs.STREAM_Q, (6, Hq, D), dtype=torch.bfloat16)
+    op, op64 = orc.prefill_attn_dyn(inputs.bits(qt), inputs.bits(pk), inputs.bits(pv), kq[0], vq[0], sk[0], sv[0], 0.1)
+    for t in range(6):
+        od, od64 = orc.decode_attn_dyn(inputs.bits(qt[t:t + 1]), inputs.bits(pk), inputs.bits(pv), kq[:1], vq[:1], sk[:1], sv[:1],
+                                       np.array([t + 1], np.int32), 0.1)
+        assert np.array_equal(op[t], od[0]) and np.array_equal(op64[t], od64[0])
+
+
 # ---------------------------------------------------------------- block glue
 def test_rope_matches_complex_rotation_and_relative_property():
     T, H, D, theta = 6, 2, 16, 500000.0
