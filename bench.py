@@ -531,6 +531,15 @@ def section_decode_attention(ctx, device, peaks):
 
     ms_fused = _graph_time(torch, fused, 32, reps=3)
     ctx.check()
+    # the comparison setting (Table 1, O1): group-wise dynamic KV, one step per cached vector, on the same codes
+    dyn = [binding.KV4Cache(pk, pv, c.kq, c.vq, None, None, c.length, Hq, sk_tok=torch.rand((B, Hkv, Tmax), device=device) * 0.6 + 0.3,
+                            sv_tok=torch.rand((B, Hkv, Tmax), device=device) * 0.6 + 0.3) for c in caches]
+    for c in caches:
+        c.length.fill_(T - 40)
+    ms_dyn_attn = _graph_time(torch, lambda i: ctx.decode_attn(dyn[i % layers], q, sm, ws, out=out), 64, reps=3)
+    ms_dyn_app = _graph_time(torch, lambda i: ctx.kv4_append(dyn[i % layers], k1, v1), 32, reps=3)
+    ctx.check()
+    del dyn
     # one long sequence (Llama-3-70B heads, 32K context): few (sequence, head) pairs, several clusters of splits each
     del caches
     Bl, Hql, Tl, Tmaxl, nl = 1, 64, 32764, 32768, 10
@@ -548,6 +557,8 @@ def section_decode_attention(ctx, device, peaks):
     gbs = by / (ms_attn * 1e-3) / 1e9
     return {"attention_us": round(ms_attn * 1e3, 3), "append_us": round(ms_app * 1e3, 3), "append+attention_us": round(ms_both * 1e3, 3),
             "append+attention_one_launch_us": round(ms_fused * 1e3, 3),
+            "groupwise_dynamic_kv (Table 1 O1)": {"attention_us": round(ms_dyn_attn * 1e3, 3), "append_us": round(ms_dyn_app * 1e3, 3),
+                                                  "note": "per-vector steps (+2 MB of step reads), plain fp32 kernel: the setting the static path is compared with"},
             "append+attention_one_launch_frac_measured_hbm": round(by / (ms_fused * 1e-3) / 1e9 / peaks["hbm"], 3),
             "long_context_b1_hq64_t32764": {"attention_us": round(ms_long * 1e3, 3),
                                             "frac_measured_hbm": round(by_long / (ms_long * 1e-3) / 1e9 / peaks["hbm"], 3)},

@@ -179,7 +179,15 @@ pq_status pq_w4a4_gemm_rows(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, c
  *   kq, vq              u8 [B, Hkv, Tmax, D/2]   packed codes of the ordinary tokens
  *   s_k, s_v            f32 [Hkv]                static per-head steps
  *   len                 int32 [B] on the device  number of 4-bit entries of each sequence
- * D must be 128; Hq a multiple of Hkv with Hq / Hkv <= 8; kq, vq, prefix_k and prefix_v 16-byte aligned. */
+ * D must be 128; Hq a multiple of Hkv with Hq / Hkv <= 8; kq, vq, prefix_k and prefix_v 16-byte aligned.
+ *
+ * Group-wise dynamic KV (Table 1, O1: the comparison setting; group size 128 = one (token, head) vector): when
+ * sk_tok and sv_tok are both non-null, every cached vector carries its own step max |x| / 7, computed when the
+ * token is written, in
+ *   sk_tok, sv_tok      f32 [B, Hkv, Tmax]       (s_k, s_v are then not used and may be null)
+ * pq_kv4_append(_strided) writes codes and steps, pq_decode_attn_kv4_prefix and pq_prefill_attn_kv4_prefix scale
+ * every key's score and every value row by the key's own step. The one-launch forms (pq_kv4_append_decode_attn,
+ * pq_rope_kv4_append) and the allocation-free entry point serve the static setting only (PQ_ERR_UNSUPPORTED). */
 typedef struct pq_kv4_cache {
   const void* prefix_k;
   const void* prefix_v;
@@ -189,6 +197,8 @@ typedef struct pq_kv4_cache {
   const float* s_v;
   int32_t* len;
   int32_t B, Hq, Hkv, D, n_prefix, Tmax;
+  float* sk_tok; /* null in the static setting */
+  float* sv_tok;
 } pq_kv4_cache;
 
 /* Calibration helper for the static per-head KV steps (Table 1, O2): over a calibration batch

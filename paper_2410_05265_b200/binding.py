@@ -43,6 +43,7 @@ class KV4CacheStruct(Structure):
         ("prefix_k", c_void_p), ("prefix_v", c_void_p), ("kq", c_void_p), ("vq", c_void_p),
         ("s_k", c_void_p), ("s_v", c_void_p), ("len", c_void_p),
         ("B", c_int32), ("Hq", c_int32), ("Hkv", c_int32), ("D", c_int32), ("n_prefix", c_int32), ("Tmax", c_int32),
+        ("sk_tok", c_void_p), ("sv_tok", c_void_p),
     ]
 
 
@@ -143,12 +144,17 @@ def _dev(t: torch.Tensor, dtype, name: str):
 class KV4Cache:
     """Caller-owned buffers of one layer's KV cache: fp16 prefix region + packed INT4 region."""
 
-    def __init__(self, prefix_k, prefix_v, kq, vq, s_k, s_v, length, Hq: int):
+    def __init__(self, prefix_k, prefix_v, kq, vq, s_k, s_v, length, Hq: int, sk_tok=None, sv_tok=None):
+        """Static setting: s_k, s_v [Hkv]. Group-wise dynamic setting: sk_tok, sv_tok f32 [B, Hkv, Tmax] (s_k, s_v may be None)."""
         B, Hkv, Tmax, D2 = kq.shape
         self.prefix_k, self.prefix_v, self.kq, self.vq = prefix_k, prefix_v, kq, vq
-        self.s_k, self.s_v, self.length = s_k, s_v, length
-        _dev(kq, torch.uint8, "kq"), _dev(vq, torch.uint8, "vq")
-        _dev(s_k, torch.float32, "s_k"), _dev(s_v, torch.float32, "s_v"), _dev(length, torch.int32, "length")
+        self.s_k, self.s_v, self.length, self.sk_tok, self.sv_tok = s_k, s_v, length, sk_tok, sv_tok
+        _dev(kq, torch.uint8, "kq"), _dev(vq, torch.uint8, "vq"), _dev(length, torch.int32, "length")
+        if sk_tok is not None:
+            _dev(sk_tok, torch.float32, "sk_tok"), _dev(sv_tok, torch.float32, "sv_tok")
+            assert sk_tok.shape == (B, Hkv, Tmax) == sv_tok.shape and sk_tok.is_contiguous() and sv_tok.is_contiguous()
+        else:
+            _dev(s_k, torch.float32, "s_k"), _dev(s_v, torch.float32, "s_v")
         n_prefix = 0 if prefix_k is None else prefix_k.shape[1]
         if n_prefix:
             _dev(prefix_k, torch.float16, "prefix_k"), _dev(prefix_v, torch.float16, "prefix_v")
@@ -157,7 +163,8 @@ class KV4Cache:
         self.B, self.Hq, self.Hkv, self.D, self.n_prefix, self.Tmax = B, Hq, Hkv, D2 * 2, n_prefix, Tmax
         self.struct = KV4CacheStruct(
             prefix_k.data_ptr() if n_prefix else 0, prefix_v.data_ptr() if n_prefix else 0, kq.data_ptr(), vq.data_ptr(),
-            s_k.data_ptr(), s_v.data_ptr(), length.data_ptr(), B, Hq, Hkv, D2 * 2, n_prefix, Tmax,
+            s_k.data_ptr() if s_k is not None else 0, s_v.data_ptr() if s_v is not None else 0, length.data_ptr(), B, Hq, Hkv, D2 * 2,
+            n_prefix, Tmax, sk_tok.data_ptr() if sk_tok is not None else 0, sv_tok.data_ptr() if sv_tok is not None else 0,
         )
 
 

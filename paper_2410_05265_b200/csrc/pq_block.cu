@@ -352,7 +352,9 @@ extern "C" pq_status pq_rope_rotate(pq_ctx* ctx, const void* x, int64_t T, int32
 
 extern "C" pq_status pq_rope_kv4_append(pq_ctx* ctx, const pq_kv4_cache* c, int32_t seq, void* qkv, int64_t T, int64_t ld, int64_t pos0,
                                         double theta, int32_t rotate, void* stream) {
-  if (!ctx || !c || !qkv || !c->kq || !c->vq || !c->s_k || !c->s_v || !c->len) return PQ_ERR_INVALID_ARG;
+  if (!ctx || !c || !qkv || !c->kq || !c->vq || !c->len) return PQ_ERR_INVALID_ARG;
+  if (c->sk_tok || c->sv_tok) return PQ_ERR_UNSUPPORTED;  // the static setting only
+  if (!c->s_k || !c->s_v) return PQ_ERR_INVALID_ARG;
   if (T < 0 || seq < 0 || seq >= c->B || c->Hkv <= 0 || c->Hq <= 0 || pos0 < 0 || !(theta > 1.0)) return PQ_ERR_INVALID_ARG;
   if (ld < static_cast<int64_t>(c->Hq + 2 * c->Hkv) * 128) return PQ_ERR_INVALID_ARG;
   if (c->D != 128) return PQ_ERR_SHAPE;

@@ -826,8 +826,12 @@ int choose_splits(const pq_ctx* ctx, const pq_kv4_cache* c) {
   return static_cast<int>(s);
 }
 
+bool is_dynamic(const pq_kv4_cache* c) { return c->sk_tok != nullptr && c->sv_tok != nullptr; }
+
 pq_status check_cache(const pq_kv4_cache* c) {
-  if (!c || !c->kq || !c->vq || !c->s_k || !c->s_v || !c->len) return PQ_ERR_INVALID_ARG;
+  if (!c || !c->kq || !c->vq || !c->len) return PQ_ERR_INVALID_ARG;
+  if ((c->sk_tok != nullptr) != (c->sv_tok != nullptr)) return PQ_ERR_INVALID_ARG;
+  if (!is_dynamic(c) && (!c->s_k || !c->s_v)) return PQ_ERR_INVALID_ARG;
   if (c->B < 0 || c->Hkv <= 0 || c->Hq <= 0 || c->n_prefix < 0 || c->Tmax < 0) return PQ_ERR_INVALID_ARG;
   if (c->n_prefix > 0 && (!c->prefix_k || !c->prefix_v)) return PQ_ERR_INVALID_ARG;
   if (c->D != 128 || c->Hq % c->Hkv != 0 || c->Hq / c->Hkv > DA_ROWS || c->n_prefix > DA_MAX_PREFIX)
@@ -840,6 +844,11 @@ pq_status check_cache(const pq_kv4_cache* c) {
 
 }  // namespace
 
+pq_status pq_kv4_append_dyn_launch(pq_ctx* ctx, const pq_kv4_cache* c, const void* k, const void* v, int32_t T_new, int64_t ld_tok,
+                                   cudaStream_t st);
+pq_status pq_decode_attn_dyn_launch(pq_ctx* ctx, const pq_kv4_cache* c, const void* q, void* out, float sm_scale, void* ws,
+                                    cudaStream_t st, int ticket0);
+
 extern "C" pq_status pq_kv4_append_strided(pq_ctx* ctx, const pq_kv4_cache* cache, const void* k, const void* v,
                                            int32_t T_new, int64_t ld_tok, void* stream) {
   if (!ctx || !k || !v || T_new < 0) return PQ_ERR_INVALID_ARG;
@@ -848,6 +857,7 @@ extern "C" pq_status pq_kv4_append_strided(pq_ctx* ctx, const pq_kv4_cache* cach
   if (ld_tok < static_cast<int64_t>(cache->Hkv) * 128) return PQ_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(k) & 15) || (reinterpret_cast<uintptr_t>(v) & 15) || ld_tok % 8 != 0) return PQ_ERR_ALIGN;
   if (T_new == 0 || cache->B == 0) return PQ_OK;
+  if (is_dynamic(cache)) return pq_kv4_append_dyn_launch(ctx, cache, k, v, T_new, ld_tok, static_cast<cudaStream_t>(stream));
   const int64_t n_units = static_cast<int64_t>(cache->B) * T_new * cache->Hkv * 4;
   int64_t grid = (n_units + AP_THREADS - 1) / AP_THREADS;
   if (grid > 8LL * ctx->sm_count) grid = 8LL * ctx->sm_count;
@@ -885,6 +895,10 @@ pq_status decode_attn_launch(pq_ctx* ctx, const pq_kv4_cache* cache, const void*
     return PQ_ERR_SHAPE;
   if (!ws || ws_bytes < pq_decode_attn_workspace_bytes(cache)) return PQ_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(ws) & 15) return PQ_ERR_ALIGN;
+  if (is_dynamic(cache)) {
+    if (k_new) return PQ_ERR_UNSUPPORTED;  // the one-launch decode step serves the static setting
+    return pq_decode_attn_dyn_launch(ctx, cache, q, out, sm_scale, ws, static_cast<cudaStream_t>(stream), DA_TICKET0);
+  }
   int S = choose_splits(ctx, cache);
   // With enough (sequence, head) pairs, eight splits already fill the GPU: the splits then form one
   // cluster and merge through distributed shared memory (the workspace and the tickets stay unused).
@@ -1002,6 +1016,7 @@ extern "C" pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache
   pq_status st = check_cache(cache);
   if (st != PQ_OK) return st;
   if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 7)) return PQ_ERR_ALIGN;
+  if (is_dynamic(cache)) return PQ_ERR_UNSUPPORTED;
   if (cache->B == 0) return PQ_OK;
   if (cache->B > 65535 || cache->Hkv > 65535) return PQ_ERR_SHAPE;
   const int64_t bh = static_cast<int64_t>(cache->B) * cache->Hkv;

@@ -60,6 +60,8 @@ struct PrefillParams {
   const uint8_t* vq;
   const float* s_k;
   const float* s_v;
+  const float* sk_tok;      // group-wise dynamic setting: this sequence's per-key steps [Hkv, Tmax]
+  const float* sv_tok;
   int32_t* status;
   long long wait_clocks;
   float sm_scale;
@@ -183,6 +185,10 @@ __device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&r
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// DYN (group-wise dynamic KV, Table 1 O1): every key's score and value row take the key's own step, read by the
+// softmax warps (all lanes the same address); the reference exponent is then the exact running maximum, so that
+// P * step stays inside fp16 for any step, and O is accumulated in value units.
+template <bool DYN>
 __global__ void __launch_bounds__(PA_THREADS, 1) prefill_attn_kernel(const PrefillParams p) {
   extern __shared__ uint8_t pa_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(pa_raw) + 1023) & ~uintptr_t(1023));
@@ -269,8 +275,11 @@ __global__ void __launch_bounds__(PA_THREADS, 1) prefill_attn_kernel(const Prefi
       __syncwarp();
       if (lane == 0) pq::mbar_arrive(&bars->q_ready);
     }
-    const float sk = __ldg(p.s_k + h), sv = __ldg(p.s_v + h);
+    const float sk = DYN ? 1.0f : __ldg(p.s_k + h), sv = DYN ? 1.0f : __ldg(p.s_v + h);
     const float scale_ctx = sk * p.sm_scale * l2e, scale_pre = p.sm_scale * l2e, inv_sv = 1.0f / sv;
+    const float* skb = DYN ? p.sk_tok + static_cast<int64_t>(h) * p.Tmax : nullptr;
+    const float* svb = DYN ? p.sv_tok + static_cast<int64_t>(h) * p.Tmax : nullptr;
+    constexpr float LAZY = DYN ? 0.0f : PA_LAZY;
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t s_addr = tmem_base + lane_base + i * 128, o_addr = tmem_base + lane_base + 256 + i * 128;
     const int tile_min_tok = t0 + (i * PA_ROWS) / G;
@@ -294,7 +303,14 @@ __global__ void __launch_bounds__(PA_THREADS, 1) prefill_attn_kernel(const Prefi
         uint32_t r[32];
         pq::tmem_ld_32x32(s_addr + c * 32, r);
         pq::tmem_ld_wait();
-        if (need_mask) {
+        if (DYN && !is_pre) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const int col = c * 32 + e;
+            const float v = __uint_as_float(r[e]) * __ldg(skb + min(key0 + col, p.Tmax - 1));
+            mx = fmaxf(mx, col < limit ? v : -INFINITY);
+          }
+        } else if (need_mask) {
 #pragma unroll
           for (int e = 0; e < 32; ++e) mx = fmaxf(mx, c * 32 + e < limit ? __uint_as_float(r[e]) : -INFINITY);
         } else {
@@ -303,7 +319,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) prefill_attn_kernel(const Prefi
         }
       }
       const float mx_s = mx * scale;
-      const bool grow = mx_s > m_ref + PA_LAZY;  // also the first visible key of a row (m_ref = -inf)
+      const bool grow = mx_s > m_ref + LAZY;  // also the first visible key of a row (m_ref = -inf)
       if (__any_sync(0xffffffffu, grow)) {
         const float m_new = grow ? mx_s : m_ref;
         const float alpha = grow ? ex2f(m_ref - m_new) : 1.0f;  // 2^(-inf) = 0 for a row that had seen nothing
@@ -329,13 +345,19 @@ __global__ void __launch_bounds__(PA_THREADS, 1) prefill_attn_kernel(const Prefi
         pq::tmem_ld_wait();
 #pragma unroll
         for (int e = 0; e < 32; e += 2) {
-          float p0 = ex2f(fmaf(__uint_as_float(r[e]), scale, -m_use)), p1 = ex2f(fmaf(__uint_as_float(r[e + 1]), scale, -m_use));
-          if (need_mask) {
+          float s0 = __uint_as_float(r[e]), s1 = __uint_as_float(r[e + 1]), w0 = pscale, w1 = pscale;
+          if (DYN && !is_pre) {
+            const int j0 = min(key0 + c * 32 + e, p.Tmax - 1), j1 = min(key0 + c * 32 + e + 1, p.Tmax - 1);
+            s0 *= __ldg(skb + j0), s1 *= __ldg(skb + j1);
+            w0 = __ldg(svb + j0), w1 = __ldg(svb + j1);
+          }
+          float p0 = ex2f(fmaf(s0, scale, -m_use)), p1 = ex2f(fmaf(s1, scale, -m_use));
+          if (need_mask || DYN) {
             p0 = c * 32 + e < limit ? p0 : 0.0f;
             p1 = c * 32 + e + 1 < limit ? p1 : 0.0f;
           }
           l += p0 + p1;
-          pk[e >> 1] = pack_h2(p0 * pscale, p1 * pscale);
+          pk[e >> 1] = pack_h2(p0 * w0, p1 * w1);
         }
         tmem_st_32x16(s_addr + c * 16, pk);
       }
@@ -516,7 +538,10 @@ __global__ void __launch_bounds__(PA_THREADS, 1) prefill_attn_kernel(const Prefi
 
 extern "C" pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* c, int32_t seq, const void* q, int64_t ldq,
                                                 int32_t T, void* out, float sm_scale, void* stream) {
-  if (!ctx || !c || !q || !out || !c->kq || !c->vq || !c->s_k || !c->s_v) return PQ_ERR_INVALID_ARG;
+  if (!ctx || !c || !q || !out || !c->kq || !c->vq) return PQ_ERR_INVALID_ARG;
+  if ((c->sk_tok != nullptr) != (c->sv_tok != nullptr)) return PQ_ERR_INVALID_ARG;
+  const bool dyn = c->sk_tok != nullptr;
+  if (!dyn && (!c->s_k || !c->s_v)) return PQ_ERR_INVALID_ARG;
   if (ldq < static_cast<int64_t>(c->Hq) * 128) return PQ_ERR_INVALID_ARG;
   if (T < 0 || seq < 0 || seq >= c->B || c->Hkv <= 0 || c->Hq <= 0 || c->n_prefix < 0 || !(sm_scale > 0.0f)) return PQ_ERR_INVALID_ARG;
   if (c->n_prefix > 0 && (!c->prefix_k || !c->prefix_v)) return PQ_ERR_INVALID_ARG;
@@ -539,6 +564,8 @@ extern "C" pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache*
   p.vq = c->vq + seq_off;
   p.s_k = c->s_k;
   p.s_v = c->s_v;
+  p.sk_tok = dyn ? c->sk_tok + static_cast<int64_t>(seq) * c->Hkv * c->Tmax : nullptr;
+  p.sv_tok = dyn ? c->sv_tok + static_cast<int64_t>(seq) * c->Hkv * c->Tmax : nullptr;
   p.status = ctx->d_status;
   p.wait_clocks = ctx->wait_clocks;
   p.sm_scale = sm_scale;
@@ -546,12 +573,16 @@ extern "C" pq_status pq_prefill_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache*
   static bool attr_set[64] = {};
   if (ctx->device < 0 || ctx->device >= 64) return PQ_ERR_UNSUPPORTED;
   if (!attr_set[ctx->device]) {
-    if (cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(PA_SMEM_BYTES)) != cudaSuccess)
+    if (cudaFuncSetAttribute(prefill_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(PA_SMEM_BYTES)) != cudaSuccess ||
+        cudaFuncSetAttribute(prefill_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(PA_SMEM_BYTES)) != cudaSuccess)
       return PQ_ERR_CUDA;
     attr_set[ctx->device] = true;
   }
   const int R = 256 / G;
   dim3 grid((T + R - 1) / R, c->Hkv);
-  prefill_attn_kernel<<<grid, PA_THREADS, PA_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(p);
+  if (dyn)
+    prefill_attn_kernel<true><<<grid, PA_THREADS, PA_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(p);
+  else
+    prefill_attn_kernel<false><<<grid, PA_THREADS, PA_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(p);
   return pq_launch_status();
 }
