@@ -232,7 +232,12 @@ pq_status pq_decode_attn_kv4_prefix(pq_ctx* ctx, const pq_kv4_cache* cache, cons
  * (dense) are quantized and written at position len[b], the attention sees every prefixed key, the cached keys
  * 0 .. len[b] - 1 and the new one (as its dequantized codes, exactly what a later call reads back), and
  * len[b] advances by one. If any sequence is full nothing is appended anywhere, the attention runs over the
- * cache as it is and PQ_ERR_SHAPE is reported through the status word. Arguments as in the two calls. */
+ * cache as it is and PQ_ERR_SHAPE is reported through the status word. Arguments as in the two calls.
+ * The kernel may be placed while its predecessor in the stream still runs (programmatic dependent launch) and
+ * requests its first cache rows before it waits for that predecessor; only q, k and v are read after the wait.
+ * The cache rows below len[b], the lengths and the steps must therefore not be written by the two kernels that
+ * precede this call in the stream (in a decode loop their last writer is the same layer's call of the step
+ * before, many kernels back). pq_decode_attn_kv4_prefix has no such condition: it waits before it reads anything. */
 pq_status pq_kv4_append_decode_attn(pq_ctx* ctx, const pq_kv4_cache* cache, const void* k, const void* v, const void* q,
                                     void* out, float sm_scale, void* ws, size_t ws_bytes, void* stream);
 

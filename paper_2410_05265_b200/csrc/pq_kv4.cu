@@ -247,16 +247,24 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   const uint8_t* vbase = p.vq + static_cast<int64_t>(bh) * p.Tmax * 64;
   const uint32_t stage_addr = pq::smem_u32(da_stage);
 
+  // Programmatic dependent launch: the next kernel of the stream may be placed as this one's CTAs retire. What this
+  // kernel reads that its predecessor may have written (everything for the plain call; the query and the new token
+  // for the one-launch decode step, whose cache rows and lengths are older than that by its contract) is read after
+  // griddepcontrol.wait; the one-launch form requests its first cache rows ahead of the wait.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (!FUSED) asm volatile("griddepcontrol.wait;" ::: "memory");
+
   // ---- every small load of the set-up goes out before the first bulk copy: behind the copies of all
   // the CTAs it would wait for megabytes of cache to be served first
   const bool row_ok = g < G;
   const bool has_prefix = split == S - 1 && p.n_prefix > 0;
   uint4 q_raw[4];  // 32 bf16 of query head g: dims 32t .. 32t+31
-  {
+  auto load_q = [&]() {
     const uint4* q4 = reinterpret_cast<const uint4*>(p.q + (static_cast<int64_t>(b) * p.Hq + h * G + (row_ok ? g : 0)) * 128 + 32 * t);
 #pragma unroll
     for (int w = 0; w < 4; ++w) q_raw[w] = row_ok ? __ldg(q4 + w) : make_uint4(0, 0, 0, 0);
-  }
+  };
+  if (!FUSED) load_q();
   // the fused kernel writes the lengths at its end: it reads them past the read-only path
   int len_b = FUSED ? __ldcg(p.len + b) : __ldg(p.len + b);
   const float s_k_h = __ldg(p.s_k + h), s_v_h = __ldg(p.s_v + h);
@@ -271,21 +279,20 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
 
   const bool has_extra = FUSED && split == S - 1;
   float k_new_d = 0.0f, v_new_d = 0.0f;  // this thread's head dim of the token being appended
-  if (has_extra) {
-    const int64_t off = (static_cast<int64_t>(b) * p.Hkv + h) * 128 + threadIdx.x;
-    k_new_d = __bfloat162float(p.k_new[off]), v_new_d = __bfloat162float(p.v_new[off]);
-  }
   if (FUSED && threadIdx.x == 0) sm_full = 0;
   // the operands of the first 16 (head, prefix key) pairs (all of them for a 4-token prefix under 4 heads)
   uint4 pre_q[2] = {}, pre_k[2] = {};
-  if (has_prefix) {
+  auto load_pre = [&](bool want_q, bool want_k) {
+    if (!has_prefix) return;
     const int pair = threadIdx.x >> 3, sub = threadIdx.x & 7;
     const bool ok = pair < G * p.n_prefix;
     const int r = ok ? pair / p.n_prefix : 0, j = ok ? pair % p.n_prefix : 0;
     const uint4* qr = reinterpret_cast<const uint4*>(p.q + (static_cast<int64_t>(b) * p.Hq + h * G + r) * 128 + 16 * sub);
     const uint4* kr = reinterpret_cast<const uint4*>(p.prefix_k + (static_cast<int64_t>(h) * p.n_prefix + j) * 128 + 16 * sub);
-    pre_q[0] = __ldg(qr), pre_q[1] = __ldg(qr + 1), pre_k[0] = __ldg(kr), pre_k[1] = __ldg(kr + 1);
-  }
+    if (want_q) pre_q[0] = __ldg(qr), pre_q[1] = __ldg(qr + 1);
+    if (want_k) pre_k[0] = __ldg(kr), pre_k[1] = __ldg(kr + 1);
+  };
+  load_pre(!FUSED, true);
 
   // ---- staging. Barrier n = 2 * slot + chunk belongs to warp n % 4: its lane 0 initialises it and
   // issues every copy that completes on it. Local round i of this split is the global round
@@ -307,6 +314,16 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
     pq::mbar_fence_init();
     for (int n = warp; n < DA_EARLY * DA_CHUNKS; n += DA_WARPS)
       if (speculated(n / DA_CHUNKS)) issue_chunk(n / DA_CHUNKS, n % DA_CHUNKS, DA_CHUNK);
+  }
+  if (FUSED) {
+    // the first cache rows are on their way: now the predecessor's results (query, new token) may be read
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    load_q();
+    load_pre(true, false);
+    if (has_extra) {
+      const int64_t off = (static_cast<int64_t>(b) * p.Hkv + h) * 128 + threadIdx.x;
+      k_new_d = __bfloat162float(p.k_new[off]), v_new_d = __bfloat162float(p.v_new[off]);
+    }
   }
   __syncthreads();  // every barrier is initialised (all warps are still together here: this costs nothing)
   if (FUSED) {  // one verdict for the whole batch, as the append call gives it
@@ -942,13 +959,15 @@ pq_status decode_attn_launch(pq_ctx* ctx, const pq_kv4_cache* cache, const void*
     cfg.blockDim = dim3(DA_THREADS);
     cfg.dynamicSmemBytes = DA_SMEM_BYTES;
     cfg.stream = static_cast<cudaStream_t>(stream);
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = S < 8 ? S : 8;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = fused ? 2 : 1;  // the plain call gains nothing from an early placement (measured), the one-launch step does
     cudaError_t e;
     if (multi)
       e = fused ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<true, true, true>, p)
@@ -959,10 +978,19 @@ pq_status decode_attn_launch(pq_ctx* ctx, const pq_kv4_cache* cache, const void*
     if (e != cudaSuccess) return PQ_ERR_CUDA;
     return pq_launch_status();
   }
-  if (fused)
-    decode_attn_kernel<false, true><<<grid, DA_THREADS, DA_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(p);
-  else
-    decode_attn_kernel<false, false><<<grid, DA_THREADS, DA_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(DA_THREADS);
+  cfg.dynamicSmemBytes = DA_SMEM_BYTES;
+  cfg.stream = static_cast<cudaStream_t>(stream);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = fused ? 1 : 0;
+  if ((fused ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<false, true, false>, p)
+             : cudaLaunchKernelEx(&cfg, decode_attn_kernel<false, false, false>, p)) != cudaSuccess)
+    return PQ_ERR_CUDA;
   return pq_launch_status();
 }
 }  // namespace

@@ -122,7 +122,7 @@ __device__ __forceinline__ float ex2(float x) {
 // the warp's shared memory and read with four head dims per lane. Split 0 also scores the full-precision prefix.
 // Warps, then splits (workspace + ticket), are merged with the usual (maximum, denominator, weighted sum) rule.
 __global__ void __launch_bounds__(DY_THREADS) decode_attn_dyn_kernel(const DynAttnParams p) {
-  __shared__ float q_s[DY_ROWS][128];
+  __shared__ __align__(16) float q_s[DY_ROWS][128];
   __shared__ __align__(16) float o_s[DY_WARPS][DY_ROWS][128];  // a warp's partial output at the end ...
   uint8_t(*v_s)[DY_ROWS * 128 * 4] = reinterpret_cast<uint8_t(*)[DY_ROWS * 128 * 4]>(o_s);  // ... and its 32 staged value rows before
   __shared__ float ml_s[DY_WARPS][DY_ROWS][2];
@@ -226,13 +226,16 @@ __global__ void __launch_bounds__(DY_THREADS) decode_attn_dyn_kernel(const DynAt
       const uint32_t kw[4] = {kv.x, kv.y, kv.z, kv.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
+        float code[8];
 #pragma unroll
-        for (int n = 0; n < 8; ++n) {
-          const float code = static_cast<float>(static_cast<int>(((kw[e] >> (4 * n)) & 0xF) ^ 8) - 8);
-          const int d = 32 * i + 8 * e + n;
+        for (int n = 0; n < 8; ++n) code[n] = static_cast<float>(static_cast<int>(((kw[e] >> (4 * n)) & 0xF) ^ 8) - 8);
 #pragma unroll
-          for (int g = 0; g < DY_ROWS; ++g)
-            if (g < G) s[g] = fmaf(q_s[g][d], code, s[g]);
+        for (int g = 0; g < DY_ROWS; ++g) {
+          if (g < G) {  // the query row's eight dims in two 16-byte reads (every lane the same address)
+            const float4 qa = *reinterpret_cast<const float4*>(&q_s[g][32 * i + 8 * e]), qb = *reinterpret_cast<const float4*>(&q_s[g][32 * i + 8 * e + 4]);
+            s[g] = fmaf(qa.x, code[0], fmaf(qa.y, code[1], fmaf(qa.z, code[2], fmaf(qa.w, code[3], s[g]))));
+            s[g] = fmaf(qb.x, code[4], fmaf(qb.y, code[5], fmaf(qb.z, code[6], fmaf(qb.w, code[7], s[g]))));
+          }
         }
       }
     }
@@ -315,7 +318,7 @@ pq_status pq_kv4_append_dyn_launch(pq_ctx* ctx, const pq_kv4_cache* c, const voi
 pq_status pq_decode_attn_dyn_launch(pq_ctx* ctx, const pq_kv4_cache* c, const void* q, void* out, float sm_scale, void* ws,
                                     cudaStream_t st, int ticket0) {
   const int64_t bh = static_cast<int64_t>(c->B) * c->Hkv;
-  int64_t S = (2LL * ctx->sm_count) / (bh > 0 ? bh : 1);
+  int64_t S = (4LL * ctx->sm_count) / (bh > 0 ? bh : 1);
   const int64_t by_len = c->Tmax / 256;  // a split's eight warps want a chunk of 32 keys each
   if (S > by_len) S = by_len;
   if (S > DY_MAX_SPLITS) S = DY_MAX_SPLITS;
