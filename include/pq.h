@@ -379,6 +379,12 @@ pq_status pq_outlier_tokens(pq_ctx* ctx, const void* x, int64_t T, int64_t C, in
  * per SM and clock that a GEMM reaches when nothing else has to happen: the benchmark's attainable INT8 peak. */
 pq_status pq_probe_i8_mma(pq_ctx* ctx, int32_t iters, int64_t* cycles, int32_t n_ctas, void* stream);
 
+/* Failure-detection self-test (the paper has no counterpart): launches one thread that waits on a barrier nothing
+ * ever completes. The bounded wait runs out after the context's limit (pq_set_wait_limit; keep it short for this
+ * call), PQ_ERR_TIMEOUT is left in the status word, the kernel returns and the context stays usable.
+ * waited_clocks (device int64, nullable) receives the SM clocks the wait took. */
+pq_status pq_selftest_wait(pq_ctx* ctx, int64_t* waited_clocks, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -28,7 +28,7 @@ EXPORTS = [
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
     "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
     "pq_calib_act_asym", "pq_hadamard_quant_act_asym", "pq_weight_code_sums", "pq_w4a4_gemm_asym",
-    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma", "pq_grid_search_act_asym", "pq_rmsnorm_hadamard_quant_act", "pq_rope_kv4_append",
+    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma", "pq_grid_search_act_asym", "pq_rmsnorm_hadamard_quant_act", "pq_rope_kv4_append", "pq_selftest_wait",
 ]
 
 
@@ -64,6 +64,7 @@ def load_library() -> ctypes.CDLL:
     lib.pq_destroy.argtypes = [c_void_p]
     lib.pq_check.argtypes = [c_void_p, c_void_p]
     lib.pq_set_wait_limit.argtypes = [c_void_p, c_int64]
+    lib.pq_selftest_wait.argtypes = [c_void_p, c_void_p, c_void_p]
     lib.pq_probe_i8_mma.argtypes = [c_void_p, c_int32, c_void_p, c_int32, c_void_p]
     lib.pq_quant_weights.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p]
     lib.pq_hadamard_quant_act.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p,
@@ -202,6 +203,12 @@ class Context:
     def set_wait_limit(self, sm_clocks: int) -> None:
         """Bound of the device-side waits of later launches, in SM clocks (0: the default of about a second)."""
         _ok(self.lib.pq_set_wait_limit(self.h, int(sm_clocks)), "pq_set_wait_limit")
+
+    def selftest_wait(self) -> torch.Tensor:
+        """Launches a wait that nothing satisfies (bounded by the context's limit); returns the clocks it took (int64 [1])."""
+        waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+        _ok(self.lib.pq_selftest_wait(self.h, _ptr(waited), _stream()), "pq_selftest_wait")
+        return waited
 
     def probe_i8_mma(self, iters: int = 4096, n_ctas: int | None = None) -> torch.Tensor:
         """SM clocks each of n_ctas CTAs needed for `iters` resident-operand 128x256x32 kind::i8 MMAs (int64 [n_ctas])."""

@@ -68,14 +68,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after `limit` SM clocks and returns false.
+// Bounded wait: gives up after `limit` SM clocks and returns false (a single try_wait may itself suspend the
+// thread for a short, implementation-defined time, so the bound is checked after every one of them).
 __device__ __forceinline__ bool mbar_wait_for(uint64_t* bar, uint32_t parity, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 32; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     if (clock64() - t0 > limit) return false;
   }
 }

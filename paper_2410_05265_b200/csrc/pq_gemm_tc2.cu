@@ -112,6 +112,7 @@ struct GemmParams {
   int M, N, K;
   int tiles_m, tiles_n;
   int tma_store;  // out can be written with TMA stores (16-byte aligned base and row pitch)
+  long long wait_clocks;  // bound of every device-side wait, in SM clocks
 };
 
 // ---- cluster-scope helpers ---------------------------------------------------------------------
@@ -149,16 +150,14 @@ __device__ __forceinline__ bool mbar_try_wait_local(uint64_t* bar, uint32_t pari
       : "memory");
   return ok != 0;
 }
-// Bounded wait (about a second of SM clocks); also gives up when the CTA's abort flag is raised.
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait (`limit` SM clocks); also gives up when the CTA's abort flag is raised.
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag, long long limit) {
   if (mbar_try_wait_local(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 1024; ++i)
-      if (mbar_try_wait_local(bar, parity)) return true;
+    if (mbar_try_wait_local(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > (1ll << 31)) return false;
+    if (clock64() - t0 > limit) return false;
   }
 }
 
@@ -268,6 +267,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
   cluster_sync_all();  // the peer's barriers exist before anything arrives on them
   pq::tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
+  uint32_t loads_issued = 0;  // producer lanes: stages whose copies were started
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
         const int n_row = (tile / p.tiles_m) * BN + rank * BN_CTA;
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
           const uint32_t s = it % N_PK, ph = (it / N_PK) & 1;
-          if (!wait_bar(&bars->pk_empty[s], ph ^ 1, abort_flag)) {
+          if (!wait_bar(&bars->pk_empty[s], ph ^ 1, abort_flag, p.wait_clocks)) {
             ok = false;
             break;
           }
@@ -293,6 +293,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
           }
         }
       }
+      loads_issued = it;
       if (!ok) {
         bars->abort_flag = 1;
         pq::report(p.status, PQ_ERR_TIMEOUT);
@@ -310,7 +311,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
         const int m_row = (tile % p.tiles_m) * (2 * BM_CTA) + rank * BM_CTA;
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
           const uint32_t s = it % N_S8, ph = (it / N_S8) & 1;
-          if (!wait_bar(&bars->s8_empty[s], ph ^ 1, abort_flag)) {
+          if (!wait_bar(&bars->s8_empty[s], ph ^ 1, abort_flag, p.wait_clocks)) {
             ok = false;
             break;
           }
@@ -318,6 +319,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
           pq::tma_load_2d(s8_buf + s * S8_STAGE, &tmap_a, kb * BK, m_row, &bars->a_full[s]);
         }
       }
+      loads_issued = it;
       if (!ok) {
         bars->abort_flag = 1;
         pq::report(p.status, PQ_ERR_TIMEOUT);
@@ -333,7 +335,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
       bool ok = true;
       for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++tcount) {
         const uint32_t ab = tcount & 1, aph = (tcount >> 1) & 1;
-        if (!wait_bar(&bars->acc_empty[ab], aph ^ 1, abort_flag)) {
+        if (!wait_bar(&bars->acc_empty[ab], aph ^ 1, abort_flag, p.wait_clocks)) {
           ok = false;
           break;
         }
@@ -341,7 +343,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
         const uint32_t d_tmem = tmem_base + ab * BN;
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
           const uint32_t s = it % N_S8, ph = (it / N_S8) & 1;
-          if (!wait_bar(&bars->s8_full[s], ph, abort_flag)) {
+          if (!wait_bar(&bars->s8_full[s], ph, abort_flag, p.wait_clocks)) {
             ok = false;
             break;
           }
@@ -375,7 +377,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
       const uint32_t ps = it % N_PK, pph = (it / N_PK) & 1;
       const uint32_t ss = it % N_S8, sph = (it / N_S8) & 1;
       const bool stuck =
-          !wait_bar(&bars->pk_full[ps], pph, abort_flag) || !wait_bar(&bars->s8_empty[ss], sph ^ 1, abort_flag);
+          !wait_bar(&bars->pk_full[ps], pph, abort_flag, p.wait_clocks) || !wait_bar(&bars->s8_empty[ss], sph ^ 1, abort_flag, p.wait_clocks);
       if (__any_sync(0xffffffffu, stuck)) {  // warp-uniform decision
         ok = false;
         break;
@@ -406,7 +408,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
       }
       pq::fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async proxy
       if (A8) {  // the stage is complete only with this CTA's token box in place
-        const bool late = !wait_bar(&bars->a_full[ss], sph, abort_flag);
+        const bool late = !wait_bar(&bars->a_full[ss], sph, abort_flag, p.wait_clocks);
         if (__any_sync(0xffffffffu, late)) {
           ok = false;
           break;
@@ -445,7 +447,7 @@ __global__ void __launch_bounds__(N_THREADS, 1)
         if (ZP) my_zw[i * 32 + lane] = col < p.N ? zp8 * __ldg(p.wsum + col) : 0;
       }
       __syncwarp();
-      const bool stuck = !wait_bar(&bars->acc_full[ab], aph, abort_flag);
+      const bool stuck = !wait_bar(&bars->acc_full[ab], aph, abort_flag, p.wait_clocks);
       if (__any_sync(0xffffffffu, stuck)) {  // warp-uniform: the TMEM loads below are warp-collective
         ok = false;
         break;
@@ -525,6 +527,15 @@ __global__ void __launch_bounds__(N_THREADS, 1)
 
   pq::tc_fence_before();
   __syncthreads();
+  if (bars->abort_flag) {
+    // a role gave up: copies that nobody consumed must still have landed before the CTA may exit (they only wait
+    // for memory, hence the generous bound)
+    if (warp == 0 && lane == 0)
+      for (uint32_t j = loads_issued > N_PK ? loads_issued - N_PK : 0; j < loads_issued; ++j) pq::mbar_wait(&bars->pk_full[j % N_PK], (j / N_PK) & 1);
+    if (A8 && warp == 2 && lane == 0)
+      for (uint32_t j = loads_issued > N_S8 ? loads_issued - N_S8 : 0; j < loads_issued; ++j) pq::mbar_wait(&bars->a_full[j % N_S8], (j / N_S8) & 1);
+    __syncthreads();
+  }
   cluster_sync_all();  // neither CTA frees tensor memory or exits while the pair may still touch it
   if (warp == 1) {
     pq::tc_fence_after();
@@ -600,6 +611,7 @@ pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq,
   p.out = static_cast<__nv_bfloat16*>(out);
   p.acc_dbg = acc_dbg;
   p.status = ctx->d_status;
+  p.wait_clocks = ctx->wait_clocks;
   p.ldo = ldo;
   p.M = static_cast<int>(M);
   p.N = static_cast<int>(N);

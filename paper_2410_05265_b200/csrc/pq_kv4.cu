@@ -184,6 +184,7 @@ struct AttnParams {
   float* ws_ml;  // [B*Hkv, S, G, 2]   running maximum (log2 units) and denominator
   uint32_t* tickets;
   int32_t* status;  // device status word; null for the entry point that has no context
+  long long wait_clocks;  // bound of the waits for staged cache rows, in SM clocks
   float sm_scale;
   int B, Hq, Hkv, G, n_prefix, Tmax;
   // fused append (decode_attn_kernel<.., true>): the new token's k, v [B, Hkv, 128], the writable lengths and one
@@ -238,6 +239,7 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   __shared__ float sm_red[DA_WARPS][DA_ROWS];
   __shared__ int sm_full;
   __shared__ int is_last;
+  __shared__ volatile int sm_abort;  // a warp's wait for staged rows ran out: every warp leaves the key loop at the same round
 
   const int split = blockIdx.x, S = gridDim.x, h = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -280,6 +282,7 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   const bool has_extra = FUSED && split == S - 1;
   float k_new_d = 0.0f, v_new_d = 0.0f;  // this thread's head dim of the token being appended
   if (FUSED && threadIdx.x == 0) sm_full = 0;
+  if (threadIdx.x == 0) sm_abort = 0;
   // the operands of the first 16 (head, prefix key) pairs (all of them for a 4-token prefix under 4 heads)
   uint4 pre_q[2] = {}, pre_k[2] = {};
   auto load_pre = [&](bool want_q, bool want_k) {
@@ -300,7 +303,10 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   // is known when they lie inside the allocation as a whole.
   auto round_key0 = [&](int i) { return (split + i * S) * DA_ROUND; };
   auto speculated = [&](int i) { return round_key0(i) + DA_ROUND <= p.Tmax; };  // i < DA_EARLY only
+  int n_issued = 0;  // copies started on this warp's barrier (lane 0 of the warp; each warp owns exactly one barrier)
+  static_assert(DA_SLOTS * DA_CHUNKS == DA_WARPS, "one barrier per warp");
   auto issue_chunk = [&](int i, int c, int n_keys) {  // lane 0 of the owning warp
+    ++n_issued;
     const uint32_t slot = stage_addr + (i % DA_SLOTS) * DA_HALF_BYTES;
     const int k0 = round_key0(i) + c * DA_CHUNK;
     const uint32_t bytes = static_cast<uint32_t>(n_keys) * 64u;
@@ -487,14 +493,18 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
     // instruction streams to interleave. A block past the end of the sequence is computed all the
     // same on whatever the buffer holds (any code pattern is a finite fp16 value) with all its
     // probabilities forced to zero.
-    if (!pq::mbar_wait(&full[r % DA_SLOTS][0], parity) || (r0 + DA_CHUNK < t1 && !pq::mbar_wait(&full[r % DA_SLOTS][1], parity))) {
+    const bool round_ok = !__any_sync(0xffffffffu, !pq::mbar_wait_for(&full[r % DA_SLOTS][0], parity, p.wait_clocks) ||
+                                                        (r0 + DA_CHUNK < t1 && !pq::mbar_wait_for(&full[r % DA_SLOTS][1], parity, p.wait_clocks)));
+    if (!round_ok) {
+      sm_abort = 1;
       timed_out = true;
-      break;
+      if (r + DA_SLOTS >= n_rounds) break;  // no CTA barrier is left in the loop: this warp may leave on its own
     }
+    if (round_ok) {
     if (r == 0 && lane == 0) {  // the remaining slots are requested once the first data is here
-      for (int n = DA_EARLY * DA_CHUNKS + warp; n < DA_SLOTS * DA_CHUNKS; n += DA_WARPS) {
+      for (int n = warp; n < DA_SLOTS * DA_CHUNKS; n += DA_WARPS) {  // by the barrier's owner, like every other request
         const int i = n / DA_CHUNKS, k0 = round_key0(i) + (n % DA_CHUNKS) * DA_CHUNK;
-        if (i < n_rounds && k0 < t1) issue_chunk(i, n % DA_CHUNKS, min(DA_CHUNK, t1 - k0));
+        if (n >= DA_EARLY * DA_CHUNKS && i < n_rounds && k0 < t1) issue_chunk(i, n % DA_CHUNKS, min(DA_CHUNK, t1 - k0));
       }
     }
     float c[2][4];  // raw scores: [0], [1] = key g x heads 2t, 2t+1; [2], [3] = key g + 8 x the same heads
@@ -594,8 +604,13 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
                            hsub2_u32(and_xor<0x00F000F0u, 0x64806480u>(yb8), 0x64806480u), pb0, pb1);
       }
     }
+    }  // round_ok
     if (r + DA_SLOTS < n_rounds) {  // the slot is free once every warp is past it
       __syncthreads();
+      if (sm_abort) {  // the same verdict in every warp: nothing more is requested, the loop ends here
+        timed_out = true;
+        break;
+      }
       for (int c = 0; c < DA_CHUNKS; ++c) {
         const int k0 = round_key0(r + DA_SLOTS) + c * DA_CHUNK;
         if (lane == 0 && warp == ((r % DA_SLOTS) * DA_CHUNKS + c) % DA_WARPS && k0 < t1)
@@ -603,14 +618,10 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
       }
     }
   }
-  // a round requested ahead of the length and then not needed must still have landed before the
-  // staging area is reused
-#pragma unroll
-  for (int i = 0; i < DA_EARLY; ++i)
-    for (int c = 0; c < DA_CHUNKS; ++c)
-      if (speculated(i) && !timed_out && (i >= n_rounds || round_key0(i) + c * DA_CHUNK >= t1) &&
-          !pq::mbar_wait(&full[i][c], 0))
-        timed_out = true;
+  // every copy that was started must have landed before the staging area is reused: a round requested ahead of the
+  // length and then not needed, and whatever was in flight when a wait ran out (these only wait for memory, hence
+  // the generous bound)
+  if (lane == 0 && n_issued > 0 && !pq::mbar_wait(&full[0][0] + warp, (n_issued - 1) & 1)) timed_out = true;
   if (timed_out && lane == 0 && p.status) pq::report(p.status, PQ_ERR_TIMEOUT);
   __syncthreads();  // the staging area becomes the per-warp partial outputs
 
@@ -944,6 +955,7 @@ pq_status decode_attn_launch(pq_ctx* ctx, const pq_kv4_cache* cache, const void*
   p.ws_ml = p.ws_o + static_cast<size_t>(cache->B) * cache->Hkv * n_parts * G * 128;
   p.tickets = ctx->d_tickets;
   p.status = ctx->d_status;
+  p.wait_clocks = ctx->wait_clocks;
   p.sm_scale = sm_scale;
   p.B = cache->B, p.Hq = cache->Hq, p.Hkv = cache->Hkv, p.G = G, p.n_prefix = cache->n_prefix, p.Tmax = cache->Tmax;
   const bool fused = k_new != nullptr;
@@ -1092,6 +1104,7 @@ extern "C" pq_status pq_decode_attn_kv4_prefix_noalloc(const pq_kv4_cache* cache
   p.ws_ml = p.ws_o + static_cast<size_t>(bh) * S * G * 128;
   p.tickets = tickets;
   p.status = nullptr;
+  p.wait_clocks = PQ_DEFAULT_WAIT_CLOCKS;
   p.sm_scale = sm_scale;
   p.B = cache->B, p.Hq = cache->Hq, p.Hkv = cache->Hkv, p.G = G, p.n_prefix = cache->n_prefix, p.Tmax = cache->Tmax;
   dim3 grid(S, cache->Hkv, cache->B);

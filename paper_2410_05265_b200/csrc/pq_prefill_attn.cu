@@ -238,9 +238,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) prefill_attn_kernel(const Prefi
     if (pq::mbar_try_wait(bar, parity)) return true;
     const long long c0 = clock64();
     for (;;) {
-#pragma unroll 1
-      for (int i = 0; i < 32; ++i)
-        if (pq::mbar_try_wait(bar, parity)) return true;
+      if (pq::mbar_try_wait(bar, parity)) return true;
       if (*abort_flag) return false;
       if (clock64() - c0 > p.wait_clocks) return false;
     }

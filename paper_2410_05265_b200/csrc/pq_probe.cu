@@ -49,7 +49,25 @@ __global__ void __launch_bounds__(128, 1) probe_i8_mma_kernel(int iters, long lo
   }
 }
 
+// Failure-detection self-test: one thread waits on a barrier that nothing ever completes; the bounded wait runs out
+// after the context's limit, the status word takes PQ_ERR_TIMEOUT and the kernel returns.
+__global__ void selftest_wait_kernel(int32_t* status, long long wait_clocks, long long* waited) {
+  __shared__ __align__(8) uint64_t never;
+  pq::mbar_init(&never, 1);
+  pq::mbar_fence_init();
+  const long long t0 = clock64();
+  const bool ok = pq::mbar_wait_for(&never, 0, wait_clocks);
+  if (waited) *waited = clock64() - t0;
+  if (!ok) pq::report(status, PQ_ERR_TIMEOUT);
+}
+
 }  // namespace
+
+extern "C" pq_status pq_selftest_wait(pq_ctx* ctx, int64_t* waited_clocks, void* stream) {
+  if (!ctx) return PQ_ERR_INVALID_ARG;
+  selftest_wait_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(ctx->d_status, ctx->wait_clocks, reinterpret_cast<long long*>(waited_clocks));
+  return pq_launch_status();
+}
 
 extern "C" pq_status pq_probe_i8_mma(pq_ctx* ctx, int32_t iters, int64_t* cycles, int32_t n_ctas, void* stream) {
   if (!ctx || !cycles || iters <= 0 || iters > (1 << 20) || n_ctas <= 0 || n_ctas > ctx->sm_count) return PQ_ERR_INVALID_ARG;
