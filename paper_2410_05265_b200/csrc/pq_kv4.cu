@@ -88,8 +88,14 @@ constexpr float DA_HEADROOM = 15.0f;  // log2 units a score may exceed the refer
 constexpr int DA_ROUND = 128;                     // keys staged per round (one half of the staging buffer)
 constexpr int DA_CHUNK = 64;                      // keys per bulk copy and per barrier
 constexpr int DA_CHUNKS = DA_ROUND / DA_CHUNK;
-constexpr int DA_SLOTS = 2;                       // rounds of staging per CTA
-constexpr int DA_EARLY = 1;                       // rounds requested at kernel entry
+#ifndef PQ_DA_SLOTS
+#define PQ_DA_SLOTS 2
+#endif
+#ifndef PQ_DA_EARLY
+#define PQ_DA_EARLY 1
+#endif
+constexpr int DA_SLOTS = PQ_DA_SLOTS;             // rounds of staging per CTA
+constexpr int DA_EARLY = PQ_DA_EARLY;             // rounds requested at kernel entry
 constexpr int DA_HALF_BYTES = DA_ROUND * 64 * 2;  // one slot: packed K rows, then packed V rows
 constexpr int DA_SMEM_BYTES = DA_SLOTS * DA_HALF_BYTES;  // 32 KB
 static_assert(DA_CHUNK == 16 * DA_WARPS, "one 16-key block per warp per chunk");
@@ -303,10 +309,11 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   // is known when they lie inside the allocation as a whole.
   auto round_key0 = [&](int i) { return (split + i * S) * DA_ROUND; };
   auto speculated = [&](int i) { return round_key0(i) + DA_ROUND <= p.Tmax; };  // i < DA_EARLY only
-  int n_issued = 0;  // copies started on this warp's barrier (lane 0 of the warp; each warp owns exactly one barrier)
-  static_assert(DA_SLOTS * DA_CHUNKS == DA_WARPS, "one barrier per warp");
+  // copies started on the barriers this warp owns (barrier n belongs to warp n % DA_WARPS; lane 0 of the warp counts)
+  constexpr int DA_OWNED = (DA_SLOTS * DA_CHUNKS + DA_WARPS - 1) / DA_WARPS;
+  int n_issued[DA_OWNED] = {};
   auto issue_chunk = [&](int i, int c, int n_keys) {  // lane 0 of the owning warp
-    ++n_issued;
+    ++n_issued[((i % DA_SLOTS) * DA_CHUNKS + c) / DA_WARPS];
     const uint32_t slot = stage_addr + (i % DA_SLOTS) * DA_HALF_BYTES;
     const int k0 = round_key0(i) + c * DA_CHUNK;
     const uint32_t bytes = static_cast<uint32_t>(n_keys) * 64u;
@@ -621,7 +628,11 @@ __global__ void __launch_bounds__(DA_THREADS, 4) decode_attn_kernel(const AttnPa
   // every copy that was started must have landed before the staging area is reused: a round requested ahead of the
   // length and then not needed, and whatever was in flight when a wait ran out (these only wait for memory, hence
   // the generous bound)
-  if (lane == 0 && n_issued > 0 && !pq::mbar_wait(&full[0][0] + warp, (n_issued - 1) & 1)) timed_out = true;
+  if (lane == 0) {
+#pragma unroll
+    for (int o = 0; o < DA_OWNED; ++o)
+      if (n_issued[o] > 0 && !pq::mbar_wait(&full[0][0] + o * DA_WARPS + warp, (n_issued[o] - 1) & 1)) timed_out = true;
+  }
   if (timed_out && lane == 0 && p.status) pq::report(p.status, PQ_ERR_TIMEOUT);
   __syncthreads();  // the staging area becomes the per-warp partial outputs
 
