@@ -82,6 +82,8 @@ pq_status pq_check(pq_ctx* ctx, void* stream) {
   if (cudaMemcpyAsync(&h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return PQ_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return PQ_ERR_CUDA;
   if (h != 0) {
+    // a kernel that gave up may have left its "last block done" counters half-way: start the next one from zero
+    if (cudaMemsetAsync(ctx->d_tickets, 0, sizeof(uint32_t) * PQ_N_TICKETS, st) != cudaSuccess) return PQ_ERR_CUDA;
     if (cudaMemsetAsync(ctx->d_status, 0, sizeof(int32_t), st) != cudaSuccess) return PQ_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return PQ_ERR_CUDA;
   }
