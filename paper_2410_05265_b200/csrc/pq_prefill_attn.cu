@@ -73,6 +73,11 @@ __device__ __forceinline__ float ex2f(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
   const __half2 h = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
@@ -274,7 +279,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) prefill_attn_kernel(const Prefi
       if (lane == 0) pq::mbar_arrive(&bars->q_ready);
     }
     const float sk = DYN ? 1.0f : __ldg(p.s_k + h), sv = DYN ? 1.0f : __ldg(p.s_v + h);
-    const float scale_ctx = sk * p.sm_scale * l2e, scale_pre = p.sm_scale * l2e, inv_sv = 1.0f / sv;
+    const float scale_ctx = sk * p.sm_scale * l2e, scale_pre = p.sm_scale * l2e, log2_sv = log2f(sv);
     const float* skb = DYN ? p.sk_tok + static_cast<int64_t>(h) * p.Tmax : nullptr;
     const float* svb = DYN ? p.sv_tok + static_cast<int64_t>(h) * p.Tmax : nullptr;
     constexpr float LAZY = DYN ? 0.0f : PA_LAZY;
@@ -295,27 +300,35 @@ __global__ void __launch_bounds__(PA_THREADS, 1) prefill_attn_kernel(const Prefi
       const float scale = is_pre ? scale_pre : scale_ctx;
       const bool need_mask = is_pre ? (p.n_prefix < PA_MAX_PREFIX) : (key0 + PA_KEYS - 1 > tile_min_tok || key0 + PA_KEYS > n_ctx);
       const int limit = is_pre ? p.n_prefix : min(n_ctx - key0, tok - key0 + 1);  // columns below it are visible
-      // ---- pass 1: the row's maximum over the visible keys of this tile
-      float mx = -INFINITY;
-      for (int c = 0; c < n_chunks; ++c) {
-        uint32_t r[32];
-        pq::tmem_ld_32x32(s_addr + c * 32, r);
-        pq::tmem_ld_wait();
-        if (DYN && !is_pre) {
+      // ---- pass 1: the row's maximum over the visible keys of this tile. The next 32 columns are requested before
+      // the current ones are worked on (the last request is pass 2's first), and four partial maxima keep the
+      // comparisons from forming one chain.
+      uint32_t rr[2][32];
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      pq::tmem_ld_32x32(s_addr, rr[0]);
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const int col = c * 32 + e;
-            const float v = __uint_as_float(r[e]) * __ldg(skb + min(key0 + col, p.Tmax - 1));
-            mx = fmaxf(mx, col < limit ? v : -INFINITY);
+      for (int c = 0; c < PA_KEYS / 32; ++c) {
+        if (c < n_chunks) {
+          pq::tmem_ld_wait_for(rr[c & 1]);
+          pq::tmem_ld_32x32(s_addr + (c + 1 < n_chunks ? (c + 1) * 32 : 0), rr[(c + 1) & 1]);
+          const uint32_t(&r)[32] = rr[c & 1];
+          if (DYN && !is_pre) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const int col = c * 32 + e;
+              const float v = __uint_as_float(r[e]) * __ldg(skb + min(key0 + col, p.Tmax - 1));
+              mx4[e & 3] = fmaxf(mx4[e & 3], col < limit ? v : -INFINITY);
+            }
+          } else if (need_mask) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], c * 32 + e < limit ? __uint_as_float(r[e]) : -INFINITY);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) mx4[(e >> 1) & 3] = max3f(mx4[(e >> 1) & 3], __uint_as_float(r[e]), __uint_as_float(r[e + 1]));
           }
-        } else if (need_mask) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, c * 32 + e < limit ? __uint_as_float(r[e]) : -INFINITY);
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
         }
       }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       const float mx_s = mx * scale;
       const bool grow = mx_s > m_ref + LAZY;  // also the first visible key of a row (m_ref = -inf)
       if (__any_sync(0xffffffffu, grow)) {
@@ -334,30 +347,44 @@ __global__ void __launch_bounds__(PA_THREADS, 1) prefill_attn_kernel(const Prefi
         }
         m_ref = m_new;
       }
-      // ---- pass 2: P = 2^(s * scale - m), fp16, written over the first columns of S_i
+      // ---- pass 2: P = 2^(s * scale - m), fp16, written over the first columns of S_i. Prefix values are real
+      // values while O is kept in code units: their P carries 1 / s_v, as an offset of the exponent, and the tile's
+      // part of the denominator is multiplied back by s_v.
       const float m_use = m_ref == -INFINITY ? 0.0f : m_ref;  // such a row has every column masked
-      const float pscale = is_pre ? inv_sv : 1.0f;            // prefix values are real values, O is in code units
-      for (int c = 0; c < n_chunks; ++c) {
-        uint32_t r[32], pk[16];
-        pq::tmem_ld_32x32(s_addr + c * 32, r);
-        pq::tmem_ld_wait();
+      const float m_off = (!DYN && is_pre) ? m_use + log2_sv : m_use;
+      const float2 scale2 = make_float2(scale, scale), moff2 = make_float2(-m_off, -m_off);
+      float2 l4[4] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f)};
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          float s0 = __uint_as_float(r[e]), s1 = __uint_as_float(r[e + 1]), w0 = pscale, w1 = pscale;
-          if (DYN && !is_pre) {
-            const int j0 = min(key0 + c * 32 + e, p.Tmax - 1), j1 = min(key0 + c * 32 + e + 1, p.Tmax - 1);
-            s0 *= __ldg(skb + j0), s1 *= __ldg(skb + j1);
-            w0 = __ldg(svb + j0), w1 = __ldg(svb + j1);
+      for (int c = 0; c < PA_KEYS / 32; ++c) {  // n_chunks is even: pass 1 left the request for columns 0..31 in rr[0]
+        if (c < n_chunks) {
+          pq::tmem_ld_wait_for(rr[c & 1]);
+          if (c + 1 < n_chunks) pq::tmem_ld_32x32(s_addr + (c + 1) * 32, rr[(c + 1) & 1]);
+          const uint32_t(&r)[32] = rr[c & 1];
+          uint32_t pk[16];
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            float2 sc = make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1]));
+            float w0 = 1.0f, w1 = 1.0f;
+            if (DYN && !is_pre) {
+              const int j0 = min(key0 + c * 32 + e, p.Tmax - 1), j1 = min(key0 + c * 32 + e + 1, p.Tmax - 1);
+              sc.x *= __ldg(skb + j0), sc.y *= __ldg(skb + j1);
+              w0 = __ldg(svb + j0), w1 = __ldg(svb + j1);
+            }
+            const float2 x = __ffma2_rn(sc, scale2, moff2);
+            float2 pp = make_float2(ex2f(x.x), ex2f(x.y));
+            if (need_mask || DYN) {
+              pp.x = c * 32 + e < limit ? pp.x : 0.0f;
+              pp.y = c * 32 + e + 1 < limit ? pp.y : 0.0f;
+            }
+            l4[(e >> 1) & 3] = __fadd2_rn(l4[(e >> 1) & 3], pp);
+            pk[e >> 1] = DYN ? pack_h2(pp.x * w0, pp.y * w1) : pack_h2(pp.x, pp.y);
           }
-          float p0 = ex2f(fmaf(s0, scale, -m_use)), p1 = ex2f(fmaf(s1, scale, -m_use));
-          if (need_mask || DYN) {
-            p0 = c * 32 + e < limit ? p0 : 0.0f;
-            p1 = c * 32 + e + 1 < limit ? p1 : 0.0f;
-          }
-          l += p0 + p1;
-          pk[e >> 1] = pack_h2(p0 * w0, p1 * w1);
+          tmem_st_32x16(s_addr + c * 16, pk);
         }
-        tmem_st_32x16(s_addr + c * 16, pk);
+      }
+      {
+        const float lt = ((l4[0].x + l4[0].y) + (l4[1].x + l4[1].y)) + ((l4[2].x + l4[2].y) + (l4[3].x + l4[3].y));
+        l += (!DYN && is_pre) ? lt * sv : lt;
       }
       tmem_st_wait();
       pq::tc_fence_before();
