@@ -533,6 +533,48 @@ void orc_grid_search_act(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, i
   *s_out = cs[best], *z_out = cz[best];
 }
 
+// Grid search for the clipping factor of per-token dynamic quantization (Sec. 3, "Initialization of Quantization
+// Parameters": gamma is shared by all tokens of a layer and chosen by mean squared error). Symmetric form, as in
+// orc_dyn_act_scale: candidate i has gamma_i = 1 - i * (1 - lo) / (n - 1) (fp32 steps as in orc_grid_candidates), every
+// row takes its own step fp32(gamma_i * max |y_t| / 7), and sse[i] = sum over rows >= row_begin and columns of
+// (y - s_t q)^2 with q = clamp(round_half_even(y / s_t), -8, 7), in double. The smallest error wins, the first one in
+// index order among equals. gamma_out [1], cand_out (nullable) [n], sse_out (nullable) [n].
+void orc_grid_search_clip_dyn(const uint16_t* x, int64_t ldx, int64_t M, int64_t K, int B, int64_t row_begin, int n, float lo,
+                              float* gamma_out, float* cand_out, double* sse_out) {
+  volatile float step = n > 1 ? (1.0f - lo) / static_cast<float>(n - 1) : 0.0f;
+  int best = 0;
+  double best_sse = INFINITY;
+  float best_gamma = 1.0f;
+  for (int i = 0; i < n; ++i) {
+    volatile float fi = static_cast<float>(i) * step;
+    volatile float gamma = 1.0f - fi;
+    std::vector<float> s_tok(M, 1.0f);
+    orc_dyn_act_scale(x, ldx, M, K, B, row_begin, gamma, s_tok.data());
+    std::vector<double> row_sse(M, 0.0);
+    parallel_rows(M, [&](int64_t m) {
+      if (m < row_begin) return;
+      const double s = static_cast<double>(s_tok[m]);
+      std::vector<double> xr(K), yr(K);
+      for (int64_t j = 0; j < K; ++j) xr[j] = bf16_to_double(x[m * ldx + j]);
+      rotate_row(xr.data(), yr.data(), K, B);
+      double acc = 0.0;
+      for (int64_t j = 0; j < K; ++j) {
+        const long q = clampi(std::lrint(std::nearbyint(yr[j] / s)), -8, 7);
+        const double e = yr[j] - s * static_cast<double>(q);
+        acc += e * e;
+      }
+      row_sse[m] = acc;
+    });
+    double total = 0.0;
+    for (int64_t m = row_begin; m < M; ++m) total += row_sse[m];
+    if (cand_out) cand_out[i] = gamma;
+    if (sse_out) sse_out[i] = total;
+    if (total < best_sse) best_sse = total, best = i, best_gamma = gamma;
+  }
+  (void)best;
+  *gamma_out = best_gamma;
+}
+
 // acc[t,n] = sum_k (u[t,k] - z) * wq[n,k]: the dequantized activation (up to its step) times the weight codes,
 // written out as such (no correction-term algebra). Returns 1 if an accumulator does not fit int32.
 int orc_gemm_asym(const uint8_t* u, int32_t z, const uint8_t* wq, int64_t M, int64_t N, int64_t K, int32_t* acc) {

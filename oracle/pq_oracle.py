@@ -282,6 +282,17 @@ def grid_search_act(x_bits: np.ndarray, block: int, n: int, lo: float, row_begin
     return np.float32(s[0]), int(z[0]), sse
 
 
+def grid_search_clip_dyn(x_bits: np.ndarray, block: int, n: int, lo: float, row_begin: int = 0):
+    """MSE grid search for the clipping factor shared by the tokens of per-token dynamic quantization: returns the
+    chosen factor, the n candidates and their squared errors."""
+    x_bits = _u16(x_bits)
+    M, K = x_bits.shape
+    g, cand, sse = np.zeros(1, np.float32), np.zeros(n, np.float32), np.zeros(n, np.float64)
+    lib().orc_grid_search_clip_dyn(_p(x_bits, c_uint16), c_int64(K), c_int64(M), c_int64(K), c_int(block), c_int64(row_begin), c_int(n),
+                                   c_float(float(lo)), _p(g, c_float), _p(cand, c_float), _p(sse, c_double))
+    return np.float32(g[0]), cand, sse
+
+
 def gemm_asym(u: np.ndarray, z: int, wq: np.ndarray) -> np.ndarray:
     """sum_k (u[t,k] - z) * w[n,k] with unsigned activation codes and packed signed weight codes -> int32 [M,N]."""
     u = np.ascontiguousarray(u, np.uint8)

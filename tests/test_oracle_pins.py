@@ -523,6 +523,45 @@ def test_grid_search_for_s_and_z_brute_force_and_never_worse_than_max_min():
     assert orc.quant_sse_asym(xr, 256, s1, z1, row_begin=4) == pytest.approx(((yr - np.float64(s1) * (u - z1)) ** 2).sum(), rel=1e-12)
 
 
+def test_grid_search_for_the_dynamic_clipping_factor_brute_force():
+    # Sec. 3: for per-token dynamic quantization one clipping factor is shared by all tokens and chosen by squared error.
+    # Independent evaluation in numpy on a small tensor: no rotation first, then with an explicit Hadamard matrix.
+    n, lo = 9, 0.2
+    x = rng.standard_normal((6, 128))
+    x[:, 3] *= 12.0                                   # a heavy column: every row's maximum is far from its bulk
+    xb = bf16_bits(x)
+    y = orc.bf16_to_f64(xb)
+    g, cand, sse = orc.grid_search_clip_dyn(xb, 0, n, lo)
+    step = np.float32(np.float32(1.0 - np.float32(lo)) / np.float32(n - 1))
+    assert cand.tolist() == [float(np.float32(1.0) - np.float32(np.float32(i) * step)) for i in range(n)] and cand[0] == 1.0
+    ref = np.empty(n)
+    for i in range(n):
+        s = (np.float64(cand[i]) * np.abs(y.astype(np.float32).astype(np.float64)).max(axis=1) / 7.0).astype(np.float32).astype(np.float64)
+        q = np.clip(np.rint(y / s[:, None]), -8, 7)
+        ref[i] = ((y - s[:, None] * q) ** 2).sum()
+    assert np.allclose(sse, ref, rtol=1e-12) and g == cand[ref.argmin()]
+    assert ref.argmin() != 0, "with a heavy tail clipping pays: the unclipped step is not the best one"
+    # candidate 0 is the unclipped quantizer that orc_dyn_act_scale / orc_quant_act_rows define
+    s1 = orc.dyn_act_scale(xb, 0)
+    codes = orc.unpack_int4(orc.quant_act_rows(xb, 0, s1)).astype(np.float64)
+    assert sse[0] == pytest.approx(((y - s1.astype(np.float64)[:, None] * codes) ** 2).sum(), rel=1e-12)
+    # values already on the unclipped grid: no error at gamma = 1, which then wins as the first of the equals or alone
+    xg = bf16_bits(np.tile(np.arange(-7, 8, dtype=np.float64) * 0.5, (2, 8))[:, :64].repeat(2, axis=1))
+    gg, _, sse_g = orc.grid_search_clip_dyn(xg, 0, 4, 0.5)
+    assert sse_g[0] == 0.0 and gg == 1.0
+    # rotation and prefix rows: rotated rows at and after row_begin, against the explicit Sylvester matrix
+    H = np.array([[1.0]])
+    while H.shape[0] < 64:
+        H = np.block([[H, H], [H, -H]])
+    xr = inputs.bits(inputs.activations(9, 128, seed=3, n_prefix=4))
+    yr = (orc.bf16_to_f64(xr).reshape(9, 2, 64) @ H / 8.0).reshape(9, 128)[4:]
+    _, cand_r, sse_r = orc.grid_search_clip_dyn(xr, 64, 5, 0.5, row_begin=4)
+    for i in (0, 2, 4):
+        s = (np.float64(cand_r[i]) * np.abs(yr.astype(np.float32).astype(np.float64)).max(axis=1) / 7.0).astype(np.float32).astype(np.float64)
+        q = np.clip(np.rint(yr / s[:, None]), -8, 7)
+        assert sse_r[i] == pytest.approx(((yr - s[:, None] * q) ** 2).sum(), rel=1e-9)
+
+
 def test_gemm_asym_is_the_dequantized_product():
     M, N, K, z = 7, 11, 96, 5
     u = rng.integers(0, 16, (M, K)).astype(np.uint8)
