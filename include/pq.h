@@ -359,6 +359,19 @@ pq_status pq_grid_search_act_asym(pq_ctx* ctx, const void* x, int64_t M, int64_t
                                   int32_t n_grid, float lo, float* s_a, int32_t* z_a, float* cand_s, int32_t* cand_z, double* sse,
                                   void* stream);
 
+/* Grid search for the clipping factor of per-token dynamic quantization (same passage: gamma is shared by all tokens
+ * of a layer and chosen by mean squared error; symmetric form, as pq_dyn_act_scale takes it). Offline. Candidates
+ *     gamma_i = 1 - i * (1 - lo) / (n_grid - 1),  i = 0 .. n_grid - 1                 (gamma_0 = 1: no clipping)
+ * every row t >= row_begin takes the step gamma_i * s_tok[t] with s_tok[t] = max |y_t| / 7 its unclipped step (the
+ * product in fp32; pq_dyn_act_scale(clip = gamma) forms gamma * max / 7 and may differ from it in the last bit),
+ * sse[i] = sum (y - s q)^2 with q = clamp(round_half_even(y / s), -8, 7) over those rows, and the factor with the
+ * smallest error (the first among equals) is written to *gamma.
+ *   n_grid in [1, 256], lo in (0, 1]; s_tok f32 [M] (rows >= row_begin are overwritten with the unclipped steps),
+ *   cand f32 [n_grid], sse f64 [n_grid] (8-byte aligned): device buffers of the caller. Other arguments as in
+ *   pq_dyn_act_scale. */
+pq_status pq_grid_search_clip_dyn(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block, int64_t row_begin,
+                                  int32_t n_grid, float lo, float* gamma, float* s_tok, float* cand, double* sse, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Outlier tokens (Sec. 4.1, "Definition of Outlier Token", Eq. 2), the cheap part of the offline analysis
  * that decides which tokens are prefixed:

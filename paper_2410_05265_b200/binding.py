@@ -28,7 +28,7 @@ EXPORTS = [
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
     "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
     "pq_calib_act_asym", "pq_hadamard_quant_act_asym", "pq_weight_code_sums", "pq_w4a4_gemm_asym",
-    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma", "pq_grid_search_act_asym", "pq_rmsnorm_hadamard_quant_act", "pq_rope_kv4_append", "pq_selftest_wait",
+    "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma", "pq_grid_search_act_asym", "pq_grid_search_clip_dyn", "pq_rmsnorm_hadamard_quant_act", "pq_rope_kv4_append", "pq_selftest_wait",
 ]
 
 
@@ -104,6 +104,8 @@ def load_library() -> ctypes.CDLL:
                                                   c_void_p, c_void_p]
     lib.pq_rope_kv4_append.argtypes = [c_void_p, POINTER(KV4CacheStruct), c_int32, c_void_p, c_int64, c_int64, c_int64, c_double, c_int32,
                                        c_void_p]
+    lib.pq_grid_search_clip_dyn.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_int32, c_float, c_void_p,
+                                            c_void_p, c_void_p, c_void_p, c_void_p]
     lib.pq_grid_search_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_int32, c_float, c_void_p,
                                             c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.pq_hadamard_quant_act_asym.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_void_p, c_void_p,
@@ -317,6 +319,20 @@ class Context:
         _ok(self.lib.pq_grid_search_act_asym(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, int(n_grid), float(lo), _ptr(s_a),
                                              _ptr(z_a), _ptr(cand_s), _ptr(cand_z), _ptr(sse), _stream()), "pq_grid_search_act_asym")
         return s_a, z_a, cand_s, cand_z, sse
+
+    def grid_search_clip_dyn(self, x: torch.Tensor, had_block: int, n_grid: int, lo: float, row_begin: int = 0):
+        """MSE grid search for the clipping factor shared by the tokens of per-token dynamic quantization. Returns device
+        tensors gamma [1], s_tok [M] (unclipped steps), cand [n], sse [n]."""
+        _dev(x, torch.bfloat16, "x")
+        M, K = x.shape
+        n = max(1, n_grid)
+        gamma = torch.zeros((1,), dtype=torch.float32, device=x.device)
+        s_tok = torch.zeros((M,), dtype=torch.float32, device=x.device)
+        cand = torch.zeros((n,), dtype=torch.float32, device=x.device)
+        sse = torch.zeros((n,), dtype=torch.float64, device=x.device)
+        _ok(self.lib.pq_grid_search_clip_dyn(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, int(n_grid), float(lo), _ptr(gamma),
+                                             _ptr(s_tok), _ptr(cand), _ptr(sse), _stream()), "pq_grid_search_clip_dyn")
+        return gamma, s_tok, cand, sse
 
     def hadamard_quant_act_asym(self, x: torch.Tensor, had_block: int, s_a: torch.Tensor, z_a: torch.Tensor, row_begin: int = 0,
                                 out: torch.Tensor | None = None):

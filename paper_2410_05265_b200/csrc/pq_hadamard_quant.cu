@@ -44,7 +44,9 @@ __device__ __forceinline__ float swiglu_bf16(float g, float u) {
 
 // GRID (with CALIB and ZP; the grid search of Sec. 3 for the static s and z): s_a_in / zp_in hold n_cand candidate
 // (s, z) pairs, and the pass adds to s_a_out (n_cand doubles) the squared error of quantizing and dequantizing the
-// rotated values with each of them.
+// rotated values with each of them. With PER_TOKEN (the search for the clipping factor that the tokens of the dynamic
+// setting share) s_a_in holds every row's unclipped step, x2 (as floats) the n_cand candidate factors, and a row's
+// candidate step is factor * step; the codes are the symmetric ones (zero point 8).
 // NORM (the RMSNorm in front of a block's first linears, App. B figure): the row is one transform block; its values
 // become bf16(x * r * g) with r = 1 / sqrt(mean(x^2) + eps) before the transform, in the arithmetic and with the
 // rounding of the stand-alone call, so that fusing changes no bit. x2 is then the gain g [K], clip carries eps.
@@ -228,7 +230,13 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
         double* sse = reinterpret_cast<double*>(s_a_out);
 #pragma unroll 1
         for (int c = 0; c < n_cand; ++c) {
-          const float s = __ldg(s_a_in + c), z = static_cast<float>(__ldg(zp_in + c));
+          float s, z;
+          if (PER_TOKEN) {
+            const float s_row = __ldg(s_a_in + row);
+            s = s_row == 0.0f ? 1.0f : __fmul_rn(__ldg(reinterpret_cast<const float*>(x2) + c), s_row), z = 8.0f;
+          } else {
+            s = __ldg(s_a_in + c), z = static_cast<float>(__ldg(zp_in + c));
+          }
           const float inv_s = __fdiv_rn(1.0f, s);
           float acc = 0.0f;
           if (active) {
@@ -367,7 +375,7 @@ template <bool CALIB, int BITS, bool PER_TOKEN = false, bool ZP = false, bool SW
 pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block, int64_t row_begin,
                    const float* s_a_in, uint8_t* xq, float* s_a_out, void* stream, float clip = 1.0f,
                    const int32_t* zp_in = nullptr, const void* x2 = nullptr, int n_cand = 0) {
-  if (SWIGLU && (!x2 || (reinterpret_cast<uintptr_t>(x2) & 3))) return x2 ? PQ_ERR_ALIGN : PQ_ERR_INVALID_ARG;
+  if ((SWIGLU || (GRID && PER_TOKEN)) && (!x2 || (reinterpret_cast<uintptr_t>(x2) & 3))) return x2 ? PQ_ERR_ALIGN : PQ_ERR_INVALID_ARG;
   if (!ctx || !x || (!CALIB && (!s_a_in || !xq)) || (CALIB && !s_a_out)) return PQ_ERR_INVALID_ARG;
   if (M < 0 || K <= 0 || ldx < K || row_begin < 0 || had_block < 0) return PQ_ERR_INVALID_ARG;
   if (K % 128 != 0) return PQ_ERR_SHAPE;
@@ -380,13 +388,13 @@ pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx
   if (row_begin >= M) return PQ_OK;
   const int64_t n_rows = M - row_begin;
   const void* x0 = static_cast<const __nv_bfloat16*>(x) + row_begin * ldx;
-  const void* x20 = SWIGLU ? static_cast<const __nv_bfloat16*>(x2) + row_begin * ldx : nullptr;
+  const void* x20 = SWIGLU ? static_cast<const __nv_bfloat16*>(x2) + row_begin * ldx : ((GRID && PER_TOKEN) ? x2 : nullptr);
   uint8_t* xq0 = CALIB ? nullptr : xq + row_begin * (BITS == 4 ? K / 2 : K);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (PER_TOKEN) {  // the arrays are indexed by row
+  if (PER_TOKEN) {  // the arrays are indexed by row (not the error sums of the grid search)
     if (s_a_in) s_a_in += row_begin;
-    if (s_a_out) s_a_out += row_begin;
-    if (CALIB && cudaMemsetAsync(s_a_out, 0, static_cast<size_t>(n_rows) * sizeof(float), st) != cudaSuccess) return PQ_ERR_CUDA;
+    if (s_a_out && !GRID) s_a_out += row_begin;
+    if (CALIB && !GRID && cudaMemsetAsync(s_a_out, 0, static_cast<size_t>(n_rows) * sizeof(float), st) != cudaSuccess) return PQ_ERR_CUDA;
   }
   switch (had_block) {
     case 0: return launch<7, false, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID>(ctx, x0, ldx, n_rows, K, s_a_in, xq0, s_a_out, clip, zp_in, x20, st, n_cand);
@@ -523,6 +531,41 @@ extern "C" pq_status pq_grid_search_act_asym(pq_ctx* ctx, const void* x, int64_t
                                                    1.0f, cand_z, nullptr, n_cand);
   if (rc != PQ_OK) return rc;
   grid_argmin_kernel<<<1, 1, 0, st>>>(sse, cand_s, cand_z, n_cand, s_a, z_a);
+  return pq_launch_status();
+}
+
+namespace {
+__global__ void clip_candidates_kernel(int n, float lo, float* cand) {
+  const int i = threadIdx.x;
+  if (i >= n) return;
+  const float step = n > 1 ? __fdiv_rn(__fsub_rn(1.0f, lo), static_cast<float>(n - 1)) : 0.0f;
+  cand[i] = __fsub_rn(1.0f, __fmul_rn(static_cast<float>(i), step));
+}
+__global__ void clip_argmin_kernel(const double* sse, const float* cand, int n, float* gamma) {
+  int best = 0;
+  for (int c = 1; c < n; ++c)
+    if (sse[c] < sse[best]) best = c;
+  *gamma = cand[best];
+}
+}  // namespace
+
+extern "C" pq_status pq_grid_search_clip_dyn(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                             int64_t row_begin, int32_t n_grid, float lo, float* gamma, float* s_tok, float* cand,
+                                             double* sse, void* stream) {
+  if (!ctx || !gamma || !s_tok || !cand || !sse) return PQ_ERR_INVALID_ARG;
+  if (n_grid < 1 || n_grid > 256 || !(lo > 0.0f) || !(lo <= 1.0f)) return PQ_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(sse) & 7) || (reinterpret_cast<uintptr_t>(cand) & 3)) return PQ_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(sse, 0, sizeof(double) * n_grid, st) != cudaSuccess) return PQ_ERR_CUDA;
+  // every row's unclipped step, then one pass that quantizes with each candidate's multiple of it
+  pq_status rc = dispatch<true, 4, true>(ctx, x, M, K, ldx, had_block, row_begin, nullptr, nullptr, s_tok, stream, 1.0f);
+  if (rc != PQ_OK) return rc;
+  clip_candidates_kernel<<<1, 256, 0, st>>>(n_grid, lo, cand);
+  if (pq_launch_status() != PQ_OK) return PQ_ERR_CUDA;
+  rc = dispatch<true, 4, true, false, false, true>(ctx, x, M, K, ldx, had_block, row_begin, s_tok, nullptr, reinterpret_cast<float*>(sse), stream,
+                                                   1.0f, nullptr, cand, n_grid);
+  if (rc != PQ_OK) return rc;
+  clip_argmin_kernel<<<1, 1, 0, st>>>(sse, cand, n_grid, gamma);
   return pq_launch_status();
 }
 

@@ -127,3 +127,35 @@ def test_dynamic_linear_end_to_end(ctx):
     err_dyn = float((out[P:].double().cpu() - ref).pow(2).mean())
     err_sta = float((out_static[P:].double().cpu() - ref).pow(2).mean())
     assert err_dyn <= err_sta * 1.05
+
+
+@pytest.mark.parametrize("M,K,B,row_begin,n_grid,lo,heavy", [(40, 1024, 1024, 4, 9, 0.2, True), (33, 6144, 2048, 0, 5, 0.5, False),
+                                                            (64, 256, 0, 2, 16, 0.1, True), (5, 4096, 4096, 0, 1, 1.0, False),
+                                                            (300, 512, 128, 0, 33, 0.25, True)])
+def test_grid_search_for_the_shared_clipping_factor_matches_oracle(ctx, M, K, B, row_begin, n_grid, lo, heavy):
+    """Sec. 3: the clipping factor shared by the tokens of per-token dynamic quantization, by squared error. Candidates,
+    unclipped steps and every candidate's error against the oracle (whose step is gamma * max / 7 rounded once; the
+    kernel's gamma * (max / 7) differs in the last bit at most, far inside the tolerance of the error sums), and the
+    chosen factor: a candidate whose oracle error is the minimum up to that tolerance."""
+    x = inputs.activations(M, K, seed=2, n_prefix=row_begin)
+    if heavy:
+        x[row_begin:, 5] *= 25.0                  # a far value in every row: clipping pays
+    xb = inputs.bits(x)
+    gamma, s_tok, cand, sse = ctx.grid_search_clip_dyn(x.cuda(), B, n_grid, lo, row_begin)
+    ctx.check()
+    g_ref, cand_ref, sse_ref = orc.grid_search_clip_dyn(xb, B, n_grid, lo, row_begin)
+    assert np.array_equal(to_np(cand), cand_ref)
+    assert np.allclose(to_np(s_tok)[row_begin:], orc.dyn_act_scale(xb, B, 1.0, row_begin)[row_begin:], rtol=2e-6)
+    got = to_np(sse)
+    assert np.allclose(got, sse_ref, rtol=2e-4, atol=1e-9), f"worst {np.max(np.abs(got - sse_ref) / np.maximum(sse_ref, 1e-30))}"
+    pick = int(np.flatnonzero(cand_ref == float(gamma))[0])
+    assert sse_ref[pick] <= sse_ref.min() * (1 + 4e-4) and got[pick] == got.min()
+    assert sse_ref[pick] <= sse_ref[0], "never worse than no clipping"
+    if heavy:
+        assert pick != 0 and float(gamma) == float(g_ref)
+    # the factor is what pq_dyn_act_scale takes: the quantizer run with it reproduces the searched error
+    s_g = ctx.dyn_act_scale(x.cuda(), B, float(gamma), row_begin)
+    codes = orc.unpack_int4(to_np(ctx.hadamard_quant_act_rows(x.cuda(), B, s_g, row_begin))).astype(np.float64)[row_begin:]
+    y = orc.rotate_bf16(xb, B)[row_begin:]
+    err = ((y - to_np(s_g).astype(np.float64)[row_begin:, None] * codes) ** 2).sum()
+    assert err == pytest.approx(sse_ref[pick], rel=1e-3)
