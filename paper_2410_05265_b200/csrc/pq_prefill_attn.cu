@@ -263,16 +263,28 @@ __global__ void __launch_bounds__(PA_THREADS, 1) prefill_attn_kernel(const Prefi
     const int tok_raw = t0 + r_cta / G, head = h * G + r_cta % G;
     const int tok = min(tok_raw, p.T - 1);
     {
-      const uint4* src = reinterpret_cast<const uint4*>(p.q + static_cast<int64_t>(tok) * p.ldq + head * 128);
+      // Q staging: the warp brings its 32 rows in, two rows (512 contiguous bytes) per load instruction; a thread per
+      // row with 16-byte loads 256 bytes apart costs 32 tag look-ups per instruction and ~8000 clocks before the first MMA.
       const uint32_t dst = pq::smem_u32(q_buf + i * PA_TILE);
-#pragma unroll 4
-      for (int c16 = 0; c16 < 16; ++c16) {
-        const uint4 v = __ldg(src + c16);  // eight bf16: dims 8 c16 .. +7
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+      const int c16 = lane & 15, lg = __ffs(G) - 1;
+      uint4 qv[16];
+#pragma unroll
+      for (int it = 0; it < 16; ++it) {
+        const int rq = i * PA_ROWS + (warp & 3) * 32 + it * 2 + (lane >> 4);
+        const int tq = min(t0 + (rq >> lg), p.T - 1), hq = h * G + (rq & (G - 1));  // G is a power of two
+        const uint4* src = reinterpret_cast<const uint4*>(p.q + static_cast<int64_t>(tq) * p.ldq + hq * 128) + c16;  // eight bf16: dims 8 c16 .. +7
+        asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"  // volatile: the sixteen requests go out before the first use
+                     : "=r"(qv[it].x), "=r"(qv[it].y), "=r"(qv[it].z), "=r"(qv[it].w)
+                     : "l"(src));
+      }
+#pragma unroll
+      for (int it = 0; it < 16; ++it) {
+        const uint32_t w[4] = {qv[it].x, qv[it].y, qv[it].z, qv[it].w};
         float f[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) f[e] = __uint_as_float((e & 1) ? (w[e >> 1] & 0xFFFF0000u) : (w[e >> 1] << 16));
-        sts128(dst + tile_off(row, c16), make_uint4(pack_h2(f[0], f[4]), pack_h2(f[1], f[5]), pack_h2(f[2], f[6]), pack_h2(f[3], f[7])));
+        sts128(dst + tile_off((warp & 3) * 32 + it * 2 + (lane >> 4), c16),
+               make_uint4(pack_h2(f[0], f[4]), pack_h2(f[1], f[5]), pack_h2(f[2], f[6]), pack_h2(f[3], f[7])));
       }
       pq::fence_proxy_async_smem();
       __syncwarp();
