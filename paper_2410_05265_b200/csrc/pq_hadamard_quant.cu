@@ -90,11 +90,18 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
   float cal_max = 0.0f, cal_lo = INFINITY, cal_hi = -INFINITY;
   const int zp = (ZP && !CALIB) ? __ldg(zp_in) - 8 : 0;
 
-  for (int64_t sb = blockIdx.x; sb < n_super; sb += gridDim.x) {
-    const int64_t gb = sb * G + blk_local;
+  // (row, block inside the row) of this thread's transform block: divided once, then advanced by the grid's stride
+  // (a 64-bit division per iteration is a visible share of an instruction-bound kernel)
+  const int64_t gb_step = static_cast<int64_t>(gridDim.x) * G;
+  const int64_t row_step = gb_step / blocks_per_row, blk_step = gb_step % blocks_per_row;
+  int64_t gb = static_cast<int64_t>(blockIdx.x) * G + blk_local;
+  int64_t row_it = gb / blocks_per_row, blk_it = gb % blocks_per_row;
+  for (int64_t sb = blockIdx.x; sb < n_super; sb += gridDim.x, gb += gb_step) {
     const bool active = gb < total_blocks;
-    const int64_t row = active ? gb / blocks_per_row : 0;
-    const int64_t col0 = active ? (gb % blocks_per_row) * B : 0;
+    const int64_t row = active ? row_it : 0;
+    const int64_t col0 = active ? blk_it * B : 0;
+    row_it += row_step, blk_it += blk_step;
+    if (blk_it >= blocks_per_row) blk_it -= blocks_per_row, ++row_it;
     if (!CALIB && PER_TOKEN) {
       const float s_row = __ldg(s_a_in + row);
       inv = __fdiv_rn(norm, s_row == 0.0f ? 1.0f : s_row);  // an all-zero row has no step: any will do
