@@ -349,17 +349,384 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
   }
 }
 
+// ---- wide blocks (B = 2048, 4096, 8192) -------------------------------------------------------------
+// The first four stages of the transform run on the tensor cores: the inputs are bf16, the factor is +-1, so
+// X (16 x 16 bf16) times H_16 is exact apart from the fp32 accumulation. A warp owns 2048 elements of a block
+// (B / 2048 warps per block), 64 per thread, and loads them as 32-bit words so that every request of the warp
+// covers whole 32-byte sectors of as few 128-byte lines as the roles below allow. The bits of the block-local
+// element index play these roles (J = 13 - LOGB):
+//   bit 0                 the two halves of a loaded word (k0 of the MMA)
+//   lane % 4 (k1, k2)     bits 1, 2 (B = 2048), bits 1, 6 (B = 4096), bits 6, 7 (B = 8192)
+//   lane / 4              the next three bits below bit 6 (the MMA's row inside an 8-row half)
+//   warp inside the block the bits left below bit 6 (none, bit 5, bits 4 and 5)
+//   the thread's own      the five bits above: m3 (rows 0-7 or 8-15 of the A operand), k3 (columns 0-7 or 8-15)
+//                         and a 3-bit tile number tau
+// One m16n8k16 MMA per eight output columns transforms bits {0, k1, k2, k3}; m3 and tau are then combined in
+// registers as packed fp32 pairs (a pair spans bit 0, which is already done), the values cross shared memory
+// once (8-byte stores, 16-byte loads, both conflict-free thanks to the padding below) and come back with the
+// thread holding 64 consecutive elements, whose not yet transformed bits (lane / 4 and warp above) are combined in
+// registers again. Each thread therefore quantizes and stores 64 consecutive elements.
+constexpr int HQW_CTAS_PER_SM = 4;
+constexpr int HQW_SMEM_FLOATS = 2 * 4736;  // the widest of 4 x 2176, 2 x 4736 and 9088 padded floats per CTA
+
+__device__ __forceinline__ void mma_bf16_m16n8k16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%10, %10, %10, %10};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.0f));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+template <int LOGB, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU, bool GRID = false, int NORM = 0>
+__global__ void __launch_bounds__(HQ_THREADS, HQW_CTAS_PER_SM)
+    hadamard_quant_wide_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, int64_t n_rows, int64_t K,
+                               const float* __restrict__ s_a_in, uint8_t* __restrict__ xq, float* __restrict__ s_a_out,
+                               float clip, const int32_t* __restrict__ zp_in, const __nv_bfloat16* __restrict__ x2, int n_cand) {
+  static_assert(LOGB >= 11 && LOGB <= 13, "block width");
+  static_assert(BITS == 4 || BITS == 8, "code width");
+  constexpr int QMAX = BITS == 4 ? 7 : 127;
+  constexpr int B = 1 << LOGB;
+  constexpr int J = 13 - LOGB;
+  constexpr int T0S = J == 0 ? 6 : 1, T1S = J == 2 ? 2 : (J == 1 ? 6 : 7);   // index bits of lane % 4
+  constexpr int GS = J + 1;                                                   // lowest index bit of lane / 4
+  constexpr int WS = J + 4;                                                   // lowest index bit of the warp
+  constexpr int M3S = 8 - J, K3S = 9 - J, TAUS = 10 - J;                      // the thread's own bits
+  // padding of the exchange buffer: float i of a block lives at i + pad(i), with
+  //   pad = PADK * (i >> M3S) + 16 * bit 6 (B = 4096) or + 8 * bit 6 + 16 * bit 7 (B = 8192)
+  constexpr int PADK = J == 2 ? 4 : (J == 1 ? 20 : 28);
+  constexpr int BLKF = J == 2 ? 2176 : (J == 1 ? 4736 : 9088);               // floats per block, padding included
+  constexpr int WPB = B / 2048;                      // warps per block
+  constexpr int G = (HQ_THREADS / 32) / WPB;
+  extern __shared__ __align__(16) float sm[];
+  __shared__ float norm_red[HQ_THREADS / 32];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int blk_local = warp / WPB, wv = warp % WPB;
+  const int64_t blocks_per_row = K / B;
+  const int64_t total_blocks = n_rows * blocks_per_row;
+  const int64_t n_super = (total_blocks + G - 1) / G;
+  float* my = sm + blk_local * BLKF;
+  auto block_sync = [&]() {
+    if (WPB == 1) __syncwarp();
+    else if (WPB == 2) asm volatile("bar.sync %0, 64;" ::"r"(1 + blk_local) : "memory");
+    else __syncthreads();
+  };
+
+  // B operand of the MMA: H_16[k][n] = (-1)^popcount(k & n) for the columns n = lane / 4 (+ 8)
+  uint32_t hb[2][2];
+#pragma unroll
+  for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int k = 2 * t + 8 * h, n = g + 8 * nb;
+      hb[nb][h] = ((__popc(k & n) & 1) ? 0xBF80u : 0x3F80u) | ((__popc((k + 1) & n) & 1) ? 0xBF800000u : 0x3F800000u);
+    }
+
+  // element offset of this thread's loads inside the block, and its shared-memory offsets (in floats)
+  const int e_thr = ((t & 1) << T0S) | ((t >> 1) << T1S) | (g << GS) | (wv << WS);
+  const int wthr = e_thr + (J == 1 ? 16 * (t >> 1) : (J == 0 ? 8 * (t & 1) + 16 * (t >> 1) : 0));
+  const int hi = lane | (wv << 5);  // pass 2: this thread holds elements 64 hi .. 64 hi + 63 of the block
+  const int rthr = (hi << 6) + PADK * (hi >> (M3S - 6)) + (J == 1 ? 16 * (hi & 1) : (J == 0 ? 8 * (hi & 1) + 16 * ((hi >> 1) & 1) : 0));
+
+  const float norm = __fdiv_rn(1.0f, __fsqrt_rn(static_cast<float>(B)));
+  float inv = norm;
+  if (!CALIB && !PER_TOKEN) inv = __fdiv_rn(norm, __ldg(s_a_in));
+  float cal_max = 0.0f, cal_lo = INFINITY, cal_hi = -INFINITY;
+  const int zp = (ZP && !CALIB) ? __ldg(zp_in) - 8 : 0;
+
+  // words of a tensor with the element pitch of x, in the order the MMAs take them: wa[tau][m3 | k3 << 1]
+  auto load_words = [&](const __nv_bfloat16* base, bool on, uint32_t (&wa)[8][4]) {
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(base + e_thr);
+#pragma unroll
+    for (int tau = 0; tau < 8; ++tau)
+#pragma unroll
+      for (int v = 0; v < 4; ++v)
+        wa[tau][v] = on ? __ldg(src + ((tau << TAUS) | ((v & 1) << M3S) | ((v >> 1) << K3S)) / 2) : 0u;
+  };
+
+  const int64_t gb_step = static_cast<int64_t>(gridDim.x) * G;
+  const int64_t row_step = gb_step / blocks_per_row, blk_step = gb_step % blocks_per_row;
+  int64_t gb = static_cast<int64_t>(blockIdx.x) * G + blk_local;
+  int64_t row_it = gb / blocks_per_row, blk_it = gb % blocks_per_row;
+  // The words of an iteration are requested during the one before, as soon as its MMAs have taken theirs out of
+  // the same registers: the rest of that iteration (some 600 instructions) covers the latency.
+  uint32_t w[8][4];
+  if (static_cast<int64_t>(blockIdx.x) < n_super) load_words(x + row_it * ldx + blk_it * B, gb < total_blocks, w);
+  for (int64_t sb = blockIdx.x; sb < n_super; sb += gridDim.x) {
+    const bool active = gb < total_blocks;
+    const int64_t row = active ? row_it : 0;
+    const int64_t col0 = active ? blk_it * B : 0;
+    if (!CALIB && PER_TOKEN) {
+      const float s_row = __ldg(s_a_in + row);
+      inv = __fdiv_rn(norm, s_row == 0.0f ? 1.0f : s_row);
+    }
+    [[maybe_unused]] uint32_t u[8][4];
+    if (SWIGLU) load_words(x2 + row * ldx + col0, active, u);
+    gb += gb_step, row_it += row_step, blk_it += blk_step;
+    if (blk_it >= blocks_per_row) blk_it -= blocks_per_row, ++row_it;
+    const bool more = sb + gridDim.x < n_super;
+
+    if (SWIGLU) {
+#pragma unroll
+      for (int tau = 0; tau < 8; ++tau)
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+          w[tau][v] = pack_bf16x2(pq::silu_mul_f32(__uint_as_float(w[tau][v] << 16), __uint_as_float(u[tau][v] << 16)),
+                                  pq::silu_mul_f32(__uint_as_float(w[tau][v] & 0xFFFF0000u), __uint_as_float(u[tau][v] & 0xFFFF0000u)));
+    } else if (NORM) {
+      // sum of squares of the row in a fixed order: the thread's values, the warp's lanes, the block's warps
+      float ss = 0.0f;
+#pragma unroll
+      for (int tau = 0; tau < 8; ++tau)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const float a = __uint_as_float(w[tau][v] << 16), b = __uint_as_float(w[tau][v] & 0xFFFF0000u);
+          ss = __fmaf_rn(a, a, __fmaf_rn(b, b, ss));
+        }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      if (WPB > 1) {
+        if (lane == 0) norm_red[warp] = ss;
+        __syncthreads();
+        ss = 0.0f;
+#pragma unroll
+        for (int i = 0; i < WPB; ++i) ss += norm_red[blk_local * WPB + i];
+        __syncthreads();
+      }
+      const float rr = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(B)), clip)));
+      uint32_t g_w[8][4];
+      load_words(x2 + col0, true, g_w);
+#pragma unroll
+      for (int tau = 0; tau < 8; ++tau)
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+          w[tau][v] = pack_bf16x2(__fmul_rn(__fmul_rn(__uint_as_float(w[tau][v] << 16), rr), __uint_as_float(g_w[tau][v] << 16)),
+                                  __fmul_rn(__fmul_rn(__uint_as_float(w[tau][v] & 0xFFFF0000u), rr), __uint_as_float(g_w[tau][v] & 0xFFFF0000u)));
+      if (NORM == 2) {
+        if (active) {
+          uint32_t* drow = reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(xq) + row * n_cand + col0 + e_thr);
+#pragma unroll
+          for (int tau = 0; tau < 8; ++tau)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) drow[((tau << TAUS) | ((v & 1) << M3S) | ((v >> 1) << K3S)) / 2] = w[tau][v];
+        }
+        if (more) load_words(x + row_it * ldx + blk_it * B, gb < total_blocks, w);
+        continue;
+      }
+    }
+
+    // ---- tensor-core stage on bits {0, 6, 7, k3}; V[m3 | tau << 1][nb] = the pair (n0 = 0, 1) ---------------
+    float2 V[16][2];
+#pragma unroll
+    for (int tau = 0; tau < 8; ++tau)
+#pragma unroll
+      for (int nb = 0; nb < 2; ++nb) {
+        float d[4];
+        mma_bf16_m16n8k16(d, w[tau], hb[nb][0], hb[nb][1]);
+        V[2 * tau][nb] = make_float2(d[0], d[1]);
+        V[2 * tau + 1][nb] = make_float2(d[2], d[3]);
+      }
+    if (more) load_words(x + row_it * ldx + blk_it * B, gb < total_blocks, w);
+#pragma unroll
+    for (int s = 0; s < 4; ++s)
+#pragma unroll
+      for (int c = 0; c < 16; ++c)
+        if ((c & (1 << s)) == 0) {
+          const int c2 = c | (1 << s);
+#pragma unroll
+          for (int nb = 0; nb < 2; ++nb) {
+            const float2 a = V[c][nb], b = V[c2][nb];
+            V[c][nb] = __fadd2_rn(a, b);
+            V[c2][nb] = __ffma2_rn(b, make_float2(-1.0f, -1.0f), a);
+          }
+        }
+    // ---- exchange ----------------------------------------------------------------------------------------
+#pragma unroll
+    for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const int m3 = c & 1, tau = c >> 1;
+        *reinterpret_cast<float2*>(my + wthr + ((m3 << M3S) | (nb << K3S) | (tau << TAUS)) + PADK * (m3 | (nb << 1) | (tau << 2))) = V[c][nb];
+      }
+    block_sync();
+    // ---- pass 2: W[q] = elements 64 hi + 2q, 2q + 1; stages on bits J+1..5 ----------------------------------
+    float2 W[32];
+    {
+      const float* src = my + rthr;
+#pragma unroll
+      for (int cc = 0; cc < 16; ++cc) {
+        const float4 v = *reinterpret_cast<const float4*>(src + 4 * cc);
+        W[2 * cc] = make_float2(v.x, v.y);
+        W[2 * cc + 1] = make_float2(v.z, v.w);
+      }
+    }
+    block_sync();
+#pragma unroll
+    for (int j = J; j < 5; ++j)
+#pragma unroll
+      for (int q = 0; q < 32; ++q)
+        if ((q & (1 << j)) == 0) {
+          const int q2 = q | (1 << j);
+          const float2 a = W[q], b = W[q2];
+          W[q] = __fadd2_rn(a, b);
+          W[q2] = __ffma2_rn(b, make_float2(-1.0f, -1.0f), a);
+        }
+    const int64_t e0 = col0 + (hi << 6);  // first of this thread's 64 consecutive elements in the row
+    if (CALIB) {
+      float it_max = 0.0f;
+      if (active) {
+#pragma unroll
+        for (int q = 0; q < 32; ++q) it_max = fmaxf(it_max, fmaxf(fabsf(W[q].x * norm), fabsf(W[q].y * norm)));
+      }
+      if (GRID) {
+        double* sse = reinterpret_cast<double*>(s_a_out);
+#pragma unroll 1
+        for (int c = 0; c < n_cand; ++c) {
+          float s, z;
+          if (PER_TOKEN) {
+            const float s_row = __ldg(s_a_in + row);
+            s = s_row == 0.0f ? 1.0f : __fmul_rn(__ldg(reinterpret_cast<const float*>(x2) + c), s_row), z = 8.0f;
+          } else {
+            s = __ldg(s_a_in + c), z = static_cast<float>(__ldg(zp_in + c));
+          }
+          const float inv_s = __fdiv_rn(1.0f, s);
+          float acc = 0.0f;
+          if (active) {
+#pragma unroll
+            for (int q = 0; q < 32; ++q) {
+              const float a = W[q].x * norm, b = W[q].y * norm;
+              const float ua = fminf(fmaxf(rintf(a * inv_s) + z, 0.0f), 15.0f), ub = fminf(fmaxf(rintf(b * inv_s) + z, 0.0f), 15.0f);
+              const float ea = a - s * (ua - z), eb = b - s * (ub - z);
+              acc = fmaf(ea, ea, acc);
+              acc = fmaf(eb, eb, acc);
+            }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+          if (lane == 0 && acc != 0.0f) atomicAdd(sse + c, static_cast<double>(acc));
+        }
+      } else if (ZP) {
+        if (active) {
+#pragma unroll
+          for (int q = 0; q < 32; ++q) {
+            const float a = W[q].x * norm, b = W[q].y * norm;
+            cal_lo = fminf(cal_lo, fminf(a, b)), cal_hi = fmaxf(cal_hi, fmaxf(a, b));
+          }
+        }
+      } else if (PER_TOKEN) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) it_max = fmaxf(it_max, __shfl_xor_sync(0xffffffffu, it_max, o));
+        if (lane == 0 && active && it_max > 0.0f)
+          atomicMax(reinterpret_cast<int*>(s_a_out + row), __float_as_int(__fdiv_rn(it_max * clip, static_cast<float>(QMAX))));
+      } else {
+        cal_max = fmaxf(cal_max, it_max);
+      }
+    } else {
+      // ---- quantize and pack ---------------------------------------------------------------------------
+      // The offset code u = clamp(rne(y / s) + 2^(BITS-1), 0, 2^BITS - 1) is taken in two fused multiply-adds:
+      // f = sat(y * (inv / U) + 2^(BITS-1) / U) with U = 2^BITS - 1 is (y / s + 2^(BITS-1)) / U clamped to [0, 1] (the
+      // clamp of the code range, applied before the rounding, which gives the same code), and f * U + 1.5 * 2^23
+      // leaves rne(f * U) in the low mantissa bits. f carries one more rounding (2^-25 of the code range, i.e.
+      // 5e-7 of a step for 4 bits, 8e-6 for 8 bits), far inside the distance from a tie within which a code may
+      // differ from a double-precision evaluation. u ^ 2^(BITS-1) is the two's-complement code.
+      // With a zero point (odd z would move ties) the rounding comes first: y * inv + (1.5 * 2^23 + 8), the integer
+      // z - 8 added to the bit pattern, and an integer clamp.
+      constexpr int BASE = 0x4B400000;
+      constexpr float U = static_cast<float>(2 * QMAX + 1);
+      const float invU = __fdiv_rn(inv, U), offU = __fdiv_rn(static_cast<float>(QMAX + 1), U);
+      auto codes = [&](float2 y) -> uint2 {  // bit patterns whose low BITS bits are the two offset codes
+        if (ZP) {
+          const float2 tq = __ffma2_rn(y, make_float2(inv, inv), make_float2(12582920.0f, 12582920.0f));
+          return make_uint2(static_cast<uint32_t>(max(min(__float_as_int(tq.x) + zp, BASE + 15), BASE)),
+                            static_cast<uint32_t>(max(min(__float_as_int(tq.y) + zp, BASE + 15), BASE)));
+        }
+        float fx, fy;
+        asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(fx) : "f"(y.x), "f"(invU), "f"(offU));
+        asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(fy) : "f"(y.y), "f"(invU), "f"(offU));
+        const float2 tq = __ffma2_rn(make_float2(fx, fy), make_float2(U, U), make_float2(12582912.0f, 12582912.0f));
+        return make_uint2(__float_as_uint(tq.x), __float_as_uint(tq.y));
+      };
+      if (BITS == 4) {
+        uint32_t fin[8];
+#pragma unroll
+        for (int wd = 0; wd < 8; ++wd) {
+          uint32_t pb[4];  // low byte: the codes of two neighbouring elements
+#pragma unroll
+          for (int b = 0; b < 4; ++b) {
+            const uint2 c = codes(W[4 * wd + b]);
+            pb[b] = c.x + (c.y << 4);
+          }
+          fin[wd] = __byte_perm(__byte_perm(pb[0], pb[1], 0x0040), __byte_perm(pb[2], pb[3], 0x0040), 0x5410) ^ 0x88888888u;
+        }
+        if (active) {
+          uint8_t* dst = xq + row * (K / 2) + e0 / 2;  // one 32-byte sector per thread
+          asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(fin[0]), "r"(fin[1]), "r"(fin[2]),
+                       "r"(fin[3]), "r"(fin[4]), "r"(fin[5]), "r"(fin[6]), "r"(fin[7])
+                       : "memory");
+        }
+      } else {
+        uint32_t fin[16];
+#pragma unroll
+        for (int wd = 0; wd < 16; ++wd) {
+          const uint2 c0 = codes(W[2 * wd]), c1 = codes(W[2 * wd + 1]);
+          fin[wd] = __byte_perm(__byte_perm(c0.x, c0.y, 0x0040), __byte_perm(c1.x, c1.y, 0x0040), 0x5410) ^ 0x80808080u;
+        }
+        if (active) {
+          uint8_t* dst = xq + row * K + e0;
+#pragma unroll
+          for (int j = 0; j < 2; ++j)
+            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + 32 * j), "r"(fin[8 * j]), "r"(fin[8 * j + 1]),
+                         "r"(fin[8 * j + 2]), "r"(fin[8 * j + 3]), "r"(fin[8 * j + 4]), "r"(fin[8 * j + 5]), "r"(fin[8 * j + 6]), "r"(fin[8 * j + 7])
+                         : "memory");
+        }
+      }
+    }
+  }
+  if (CALIB && GRID) {
+  } else if (CALIB && ZP) {
+    for (int o = 16; o > 0; o >>= 1) {
+      cal_lo = fminf(cal_lo, __shfl_xor_sync(0xffffffffu, cal_lo, o));
+      cal_hi = fmaxf(cal_hi, __shfl_xor_sync(0xffffffffu, cal_hi, o));
+    }
+    if (lane == 0 && cal_hi >= cal_lo) {
+      atomicMax(reinterpret_cast<uint32_t*>(s_a_out), float_key(cal_hi));
+      atomicMin(reinterpret_cast<uint32_t*>(s_a_out) + 1, float_key(cal_lo));
+    }
+  } else if (CALIB && !PER_TOKEN) {
+    for (int o = 16; o > 0; o >>= 1) cal_max = fmaxf(cal_max, __shfl_xor_sync(0xffffffffu, cal_max, o));
+    if (lane == 0 && cal_max > 0.0f)
+      atomicMax(reinterpret_cast<int*>(s_a_out), __float_as_int(__fdiv_rn(cal_max, static_cast<float>(QMAX))));
+  }
+}
+
 template <int LOGB, bool ROTATE, bool CALIB, int BITS, bool PER_TOKEN, bool ZP, bool SWIGLU, bool GRID, int NORM = 0>
 pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_t K, const float* s_a_in, uint8_t* xq,
                  float* s_a_out, float clip, const int32_t* zp_in, const void* x2, cudaStream_t st, int n_cand) {
-  auto kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID, NORM>;
-  constexpr size_t smem = HQ_SMEM_FLOATS * sizeof(float);
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
-    return PQ_ERR_CUDA;
   constexpr int B = 1 << LOGB;
   constexpr int G = HQ_THREADS / (B / 64);
   int64_t n_super = (n_rows * (K / B) + G - 1) / G;
-  const int64_t resident = static_cast<int64_t>(HQ_CTAS_PER_SM) * ctx->sm_count;
+  // blocks of 2048 and wider take the kernel whose first stages run on the tensor cores
+  constexpr bool WIDE = LOGB >= 11 && (ROTATE || NORM == 2);
+  void (*kern)(const __nv_bfloat16*, int64_t, int64_t, int64_t, const float*, uint8_t*, float*, float, const int32_t*,
+               const __nv_bfloat16*, int);
+  size_t smem = HQ_SMEM_FLOATS * sizeof(float);
+  int ctas_per_sm = HQ_CTAS_PER_SM;
+  if constexpr (WIDE) {
+    kern = hadamard_quant_wide_kernel<LOGB, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID, NORM>;
+    smem = HQW_SMEM_FLOATS * sizeof(float);
+    ctas_per_sm = HQW_CTAS_PER_SM;
+  } else {
+    kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID, NORM>;
+  }
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+    return PQ_ERR_CUDA;
+  const int64_t resident = static_cast<int64_t>(ctas_per_sm) * ctx->sm_count;
   int64_t grid = n_super < resident ? n_super : resident;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(grid));
