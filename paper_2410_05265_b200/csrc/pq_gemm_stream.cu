@@ -239,9 +239,11 @@ pq_status pq_gemm_stream_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* w
                                 void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg,
                                 cudaStream_t st, bool per_token, bool a8, const int32_t* zp, const int32_t* wsum) {
   const int sa_stride = per_token ? 1 : 0;  // s_a is then an array of M per-token steps
-  // 16 channels per CTA when that still gives every SM several CTAs, else 8 (only for up to 8 tokens:
-  // with two token groups the narrower CTA repeats too much of the activation expansion)
-  const bool half = M <= 8 && (N + GS_CH - 1) / GS_CH < 4LL * ctx->sm_count;
+  // 8 channels per CTA when all those CTAs are resident at once (four 64-register CTAs per SM), else 16: CTAs of a
+  // second wave start after the programmatic launch's early weight requests have been spent (q|k|v with 768 CTAs of 8
+  // channels: 4.8 us, with 384 of 16: 3.2 us). Only for up to 8 tokens: with two token groups the narrower CTA repeats
+  // too much of the activation expansion.
+  const bool half = M <= 8 && (N + GS_CH / 2 - 1) / (GS_CH / 2) <= 4LL * ctx->sm_count;
   if (a8) {
     if (M <= 8)
       return half ? launch_stream<false, true, true>(xq, wq, s_a, s_w, out, ldo, M, N, K, acc_dbg, st, sa_stride, zp, wsum)

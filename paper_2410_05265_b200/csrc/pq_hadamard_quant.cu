@@ -439,6 +439,7 @@ __global__ void __launch_bounds__(HQ_THREADS, HQW_CTAS_PER_SM)
   if (!CALIB && !PER_TOKEN) inv = __fdiv_rn(norm, __ldg(s_a_in));
   float cal_max = 0.0f, cal_lo = INFINITY, cal_hi = -INFINITY;
   const int zp = (ZP && !CALIB) ? __ldg(zp_in) - 8 : 0;
+  [[maybe_unused]] const bool out32 = (reinterpret_cast<uintptr_t>(xq) & 31) == 0;
 
   // words of a tensor with the element pitch of x, in the order the MMAs take them: wa[tau][m3 | k3 << 1]
   auto load_words = [&](const __nv_bfloat16* base, bool on, uint32_t (&wa)[8][4]) {
@@ -652,6 +653,17 @@ __global__ void __launch_bounds__(HQ_THREADS, HQW_CTAS_PER_SM)
         const float2 tq = __ffma2_rn(make_float2(fx, fy), make_float2(U, U), make_float2(12582912.0f, 12582912.0f));
         return make_uint2(__float_as_uint(tq.x), __float_as_uint(tq.y));
       };
+      // a thread's 32 bytes leave as one sector when the output is 32-byte aligned (rows are whole kilobytes)
+      auto store32 = [&](uint8_t* dst, const uint32_t* v) {
+        if (out32) {
+          asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+                       "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                       : "memory");
+        } else {
+          reinterpret_cast<uint4*>(dst)[0] = make_uint4(v[0], v[1], v[2], v[3]);
+          reinterpret_cast<uint4*>(dst)[1] = make_uint4(v[4], v[5], v[6], v[7]);
+        }
+      };
       if (BITS == 4) {
         uint32_t fin[8];
 #pragma unroll
@@ -664,12 +676,7 @@ __global__ void __launch_bounds__(HQ_THREADS, HQW_CTAS_PER_SM)
           }
           fin[wd] = __byte_perm(__byte_perm(pb[0], pb[1], 0x0040), __byte_perm(pb[2], pb[3], 0x0040), 0x5410) ^ 0x88888888u;
         }
-        if (active) {
-          uint8_t* dst = xq + row * (K / 2) + e0 / 2;  // one 32-byte sector per thread
-          asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(fin[0]), "r"(fin[1]), "r"(fin[2]),
-                       "r"(fin[3]), "r"(fin[4]), "r"(fin[5]), "r"(fin[6]), "r"(fin[7])
-                       : "memory");
-        }
+        if (active) store32(xq + row * (K / 2) + e0 / 2, fin);
       } else {
         uint32_t fin[16];
 #pragma unroll
@@ -678,12 +685,8 @@ __global__ void __launch_bounds__(HQ_THREADS, HQW_CTAS_PER_SM)
           fin[wd] = __byte_perm(__byte_perm(c0.x, c0.y, 0x0040), __byte_perm(c1.x, c1.y, 0x0040), 0x5410) ^ 0x80808080u;
         }
         if (active) {
-          uint8_t* dst = xq + row * K + e0;
-#pragma unroll
-          for (int j = 0; j < 2; ++j)
-            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + 32 * j), "r"(fin[8 * j]), "r"(fin[8 * j + 1]),
-                         "r"(fin[8 * j + 2]), "r"(fin[8 * j + 3]), "r"(fin[8 * j + 4]), "r"(fin[8 * j + 5]), "r"(fin[8 * j + 6]), "r"(fin[8 * j + 7])
-                         : "memory");
+          store32(xq + row * K + e0, fin);
+          store32(xq + row * K + e0 + 32, fin + 8);
         }
       }
     }

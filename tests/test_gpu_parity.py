@@ -70,6 +70,23 @@ def test_hadamard_quant_act_matches_oracle(ctx, M, K, B, row_begin):
         assert torch.equal(out2, out[row_begin:])
 
 
+@pytest.mark.parametrize("K,B", [(4096, 2048), (4096, 4096)])
+def test_hadamard_quant_output_aligned_to_16_bytes_only(ctx, K, B):
+    """The header asks for a 16-byte aligned output: a base that is not 32-byte aligned gives the same codes."""
+    M = 9
+    x = inputs.activations(M, K, seed=0).cuda()
+    s_a = ctx.calib_act_scale(x, B)
+    ref = ctx.hadamard_quant_act(x, B, s_a)
+    buf = torch.zeros(M * (K // 2) + 64, dtype=torch.uint8, device="cuda")
+    off = (16 - buf.data_ptr() % 32) % 32
+    out = buf[off:off + M * (K // 2)].view(M, K // 2)
+    assert out.data_ptr() % 32 == 16
+    ctx.hadamard_quant_act(x, B, s_a, out=out)
+    ctx.check()
+    assert torch.equal(out, ref)
+    assert int(buf[:off].sum()) == 0 and int(buf[off + M * (K // 2):].sum()) == 0
+
+
 def test_hadamard_quant_prefix_outliers_never_set_scale(ctx):
     x = inputs.activations(64, 4096, seed=1, n_prefix=4)
     s1 = ctx.calib_act_scale(x.cuda(), 4096, 4)
