@@ -148,6 +148,24 @@ def test_gemm_decode_shapes_bit_exact(ctx, M, N, K):
     _gemm_case(ctx, M, N, K, seed=M * 7 + N)
 
 
+@pytest.mark.parametrize("M,N,K", [(1, 50, 1024), (2, 33, 2048), (3, 1000, 4096), (4, 264, 8192), (2, 72, 14336),
+                                   (1, 96, 28672), (4, 20, 28672), (3, 7, 3072)])
+def test_gemm_few_tokens_bit_exact(ctx, M, N, K):
+    """One to four tokens over short and long K, ragged channel counts."""
+    _gemm_case(ctx, M, N, K, seed=M * 13 + N)
+
+
+def test_gemm_few_tokens_extreme_codes_fit_int32(ctx):
+    N, K = 24, 28672
+    for M in (1, 4):
+        xq = np.full((M, K // 2), 0x88, np.uint8)   # every code -8
+        wq = np.full((N, K // 2), 0x88, np.uint8)
+        acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+        ctx.w4a4_gemm(dev(xq), dev(wq), torch.ones(1, device="cuda"), torch.ones(N, device="cuda"), acc_dbg=acc)
+        ctx.check()
+        assert int(acc.min()) == int(acc.max()) == 64 * K
+
+
 def test_gemm_extreme_codes_fit_int32(ctx):
     M, N, K = 128, 256, 28672
     xq = np.full((M, K // 2), 0x88, np.uint8)   # every code -8
