@@ -727,8 +727,15 @@ pq_status launch(pq_ctx* ctx, const void* x, int64_t ldx, int64_t n_rows, int64_
   } else {
     kern = hadamard_quant_kernel<LOGB, ROTATE, CALIB, BITS, PER_TOKEN, ZP, SWIGLU, GRID, NORM>;
   }
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
-    return PQ_ERR_CUDA;
+  // the shared-memory attribute is set once per device and instantiation (the call costs several microseconds of
+  // host time, a visible share of a decode-sized launch)
+  static bool attr_set[64] = {};
+  const int dev = ctx->device;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+      return PQ_ERR_CUDA;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
   const int64_t resident = static_cast<int64_t>(ctas_per_sm) * ctx->sm_count;
   int64_t grid = n_super < resident ? n_super : resident;
   cudaLaunchConfig_t cfg = {};
