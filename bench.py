@@ -221,6 +221,9 @@ def run_gpu(args):
 
     def step(gemm_events=None):
         for i, (name, N, K, had, inp) in enumerate(L):
+            if gemm_events is not None:
+                eh = torch.cuda.Event(enable_timing=True)
+                eh.record()
             ctx.hadamard_quant_act(acts[i], had, scales[i], N_PREFIX, out=xqs[i])
             if gemm_events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -229,6 +232,7 @@ def run_gpu(args):
             if gemm_events is not None:
                 e1.record()
                 gemm_events.append((i, e0, e1))
+                rot_events.append((i, eh, e0))
 
     def barrier():
         torch.cuda.synchronize()
@@ -240,20 +244,32 @@ def run_gpu(args):
         step()
     ctx.check()
     # ---- timed region: device-resident inputs -------------------------------------------------
+    # Two passes of the same K steps. The first has nothing but the eight launches of a step in the stream and gives
+    # `value`; the second brackets every launch with CUDA events for the per-kernel figures. An event record between
+    # two launches keeps the second from being placed while the first drains (programmatic dependent launch), so
+    # the bracketed pass is a few percent slower per step; its time is reported beside the other.
     sampler = ClockSampler(local)
     gemm_events = []
+    rot_events = []
     barrier()
     sampler.start()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
     for _ in range(args.steps):
-        step(gemm_events)
+        step()
     t1.record()
+    barrier()
+    t2, t3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t2.record()
+    for _ in range(args.steps):
+        step(gemm_events)
+    t3.record()
     barrier()
     clocks = sampler.stop()
     ctx.check()
     ms_per_step, ops_per_s = job_throughput(t0.elapsed_time(t1), args.steps, step_ops(m_rows), world, dist, device)
     value = ops_per_s / 1e12
+    bracketed_ms_per_step = t2.elapsed_time(t3) / args.steps
 
     gemm_ms = sum(e0.elapsed_time(e1) for _, e0, e1 in gemm_events)
     per_shape = {}
@@ -261,10 +277,19 @@ def run_gpu(args):
         per_shape.setdefault(L[i][0], []).append(e0.elapsed_time(e1))
     gemm_ops = args.steps * step_ops(m_rows)
     peaks = read_peaks()
+    # the rotate+quantize launch in front of every GEMM, between its own event and the GEMM's: 2.5 bytes per element
+    rot_shape = {}
+    for i, e0, e1 in rot_events:
+        rot_shape.setdefault(L[i][0], []).append(e0.elapsed_time(e1))
+    rotate_quant = {}
+    for k, v in rot_shape.items():
+        kk = next(kk for nm, n, kk, _, _ in L if nm == k)
+        gbs = 2.5 * m_rows * kk / (statistics.mean(v) * 1e-3) / 1e9
+        rotate_quant[k + " input"] = {"ms": round(statistics.mean(v), 4), "GB/s": round(gbs, 1), "frac_measured_hbm": round(gbs / peaks["hbm"], 3)}
     # Denominator: dense INT8 is nominally 2x dense bf16 (4.5 vs 2.25 PFLOP/s); of the two measured bf16 figures the
     # burst one applies to a timed region shorter than a second (the chip does not reach its power-capped clock in
     # that time), the sustained one to a longer region.
-    timed_s = t0.elapsed_time(t1) * 1e-3
+    timed_s = t2.elapsed_time(t3) * 1e-3  # the pass the per-launch events come from
     peak_kind = "burst" if timed_s < 1.0 else "sustained"
     int8_peak = 2.0 * (peaks["bf16"] if timed_s < 1.0 else peaks["bf16_sus"])
     achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
@@ -289,6 +314,7 @@ def run_gpu(args):
         "peak": round(int8_peak, 1), "unit": "TOPS", "frac": round(achieved / int8_peak, 4), "traffic": traffic, "traffic_note": traffic_note,
         "peak_source": f"2 x bf16 {peak_kind} GEMM of {peaks['src']} (timed region {timed_s:.2f} s)",
         "frac_of_nominal_4500": round(achieved / NOMINAL_INT8_TOPS, 4), "attainable_int8": attainable,
+        "per_launch_pass_ms_per_step": round(bracketed_ms_per_step, 4),
         "per_launch": {k: {"ms": round(statistics.mean(v), 4),
                            "tops": round(2.0 * m_rows * next(n * kk for nm, n, kk, _, _ in L if nm == k) /
                                          (statistics.mean(v) * 1e-3) / 1e12, 1)} for k, v in per_shape.items()},
@@ -373,6 +399,7 @@ def run_gpu(args):
             "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "pipeline": "uploads, library calls and downloads on three streams", "matches_device_step": e2e_ok},
             "gpu_launches": args.steps * 2 * len(L),
+            "rotate_quant_per_launch": rotate_quant,
         }
         if cpu_baseline:
             line["cpu_baseline"] = cpu_baseline
