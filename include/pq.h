@@ -165,6 +165,11 @@ pq_status pq_w4a8_gemm(pq_ctx* ctx, const int8_t* xq8, const uint8_t* wq, const 
  *   tensor-core kernel with the token operand in shared memory for every K (M - row_begin > 16). */
 pq_status pq_dyn_act_scale(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
                            int64_t row_begin, float clip, float* s_tok, void* stream);
+/* The first and the second pass in one call (same passage): s_tok [M] and xq [M, K/2] are both outputs, with the bits
+ * the two calls give. When a row is a single transform block of 2048 or more elements (had_block == K) the activations
+ * are read once and the call is one launch; otherwise it runs the two passes. */
+pq_status pq_dyn_hadamard_quant_act(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                    int64_t row_begin, float clip, float* s_tok, uint8_t* xq, void* stream);
 pq_status pq_hadamard_quant_act_rows(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
                                      int64_t row_begin, const float* s_tok, uint8_t* xq, void* stream);
 pq_status pq_w4a4_gemm_rows(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_tok, const float* s_w,

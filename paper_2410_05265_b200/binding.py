@@ -26,7 +26,7 @@ EXPORTS = [
     "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix", "pq_decode_attn_kv4_prefix_noalloc",
     "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add", "pq_prefill_attn_kv4_prefix", "pq_kv4_append_strided", "pq_calib_kv_scale",
     "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
-    "pq_dyn_act_scale", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
+    "pq_dyn_act_scale", "pq_dyn_hadamard_quant_act", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
     "pq_calib_act_asym", "pq_hadamard_quant_act_asym", "pq_weight_code_sums", "pq_w4a4_gemm_asym",
     "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma", "pq_grid_search_act_asym", "pq_grid_search_clip_dyn", "pq_rmsnorm_hadamard_quant_act", "pq_rope_kv4_append", "pq_selftest_wait",
 ]
@@ -96,6 +96,8 @@ def load_library() -> ctypes.CDLL:
                                  c_int64, c_void_p, c_void_p]
     lib.pq_dyn_act_scale.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_float, c_void_p, c_void_p]
     lib.pq_hadamard_quant_act_rows.argtypes = lib.pq_hadamard_quant_act.argtypes
+    lib.pq_dyn_hadamard_quant_act.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int64, c_float, c_void_p, c_void_p,
+                                              c_void_p]
     lib.pq_w4a4_gemm_rows.argtypes = lib.pq_w4a8_gemm.argtypes
     lib.pq_outlier_tokens.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_float, c_float, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p]
@@ -393,6 +395,21 @@ class Context:
         _ok(self.lib.pq_dyn_act_scale(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, float(clip), _ptr(out), _stream()),
             "pq_dyn_act_scale")
         return out
+
+    def dyn_hadamard_quant_act(self, x: torch.Tensor, had_block: int, clip: float = 1.0, row_begin: int = 0,
+                               s_tok: torch.Tensor | None = None, out: torch.Tensor | None = None):
+        """pq_dyn_act_scale followed by pq_hadamard_quant_act_rows in one call; returns (s_tok, xq)."""
+        _dev(x, torch.bfloat16, "x")
+        M, K = x.shape
+        assert x.stride(1) == 1
+        if s_tok is None:
+            s_tok = torch.zeros((M,), dtype=torch.float32, device=x.device)
+        if out is None:
+            out = torch.zeros((M, K // 2), dtype=torch.uint8, device=x.device)
+        _dev(s_tok, torch.float32, "s_tok"), _dev(out, torch.uint8, "out")
+        _ok(self.lib.pq_dyn_hadamard_quant_act(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, float(clip), _ptr(s_tok),
+                                               _ptr(out), _stream()), "pq_dyn_hadamard_quant_act")
+        return s_tok, out
 
     def hadamard_quant_act_rows(self, x: torch.Tensor, had_block: int, s_tok: torch.Tensor, row_begin: int = 0,
                                 out: torch.Tensor | None = None):

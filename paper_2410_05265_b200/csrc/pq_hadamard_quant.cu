@@ -463,7 +463,7 @@ __global__ void __launch_bounds__(HQ_THREADS, HQW_CTAS_PER_SM)
     const bool active = gb < total_blocks;
     const int64_t row = active ? row_it : 0;
     const int64_t col0 = active ? blk_it * B : 0;
-    if (!CALIB && PER_TOKEN) {
+    if (!CALIB && PER_TOKEN && s_a_out == nullptr) {
       const float s_row = __ldg(s_a_in + row);
       inv = __fdiv_rn(norm, s_row == 0.0f ? 1.0f : s_row);
     }
@@ -579,6 +579,27 @@ __global__ void __launch_bounds__(HQ_THREADS, HQW_CTAS_PER_SM)
           W[q2] = __ffma2_rn(b, make_float2(-1.0f, -1.0f), a);
         }
     const int64_t e0 = col0 + (hi << 6);  // first of this thread's 64 consecutive elements in the row
+    if (!CALIB && PER_TOKEN && s_a_out != nullptr) {
+      // One-pass dynamic form (the row is this one block): the token's step from the block's own maximum, in the
+      // operations of the two-pass form (max of |y| * norm, then clip * max / 7: monotone, so the maximum over the
+      // warps of the warps' steps is the step of the maximum), written out for the GEMM's epilogue.
+      float it_max = 0.0f;
+#pragma unroll
+      for (int q = 0; q < 32; ++q) it_max = fmaxf(it_max, fmaxf(fabsf(W[q].x * norm), fabsf(W[q].y * norm)));
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) it_max = fmaxf(it_max, __shfl_xor_sync(0xffffffffu, it_max, o));
+      if (WPB > 1) {
+        if (lane == 0) norm_red[warp] = it_max;
+        __syncthreads();
+        it_max = 0.0f;
+#pragma unroll
+        for (int i = 0; i < WPB; ++i) it_max = fmaxf(it_max, norm_red[blk_local * WPB + i]);
+        __syncthreads();
+      }
+      const float s_row = it_max > 0.0f ? __fdiv_rn(it_max * clip, static_cast<float>(QMAX)) : 0.0f;
+      if (active && hi == 0) s_a_out[row] = s_row;
+      inv = __fdiv_rn(norm, s_row == 0.0f ? 1.0f : s_row);
+    }
     if (CALIB) {
       float it_max = 0.0f;
       if (active) {
@@ -760,7 +781,7 @@ pq_status dispatch(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx
                    const float* s_a_in, uint8_t* xq, float* s_a_out, void* stream, float clip = 1.0f,
                    const int32_t* zp_in = nullptr, const void* x2 = nullptr, int n_cand = 0) {
   if ((SWIGLU || (GRID && PER_TOKEN)) && (!x2 || (reinterpret_cast<uintptr_t>(x2) & 3))) return x2 ? PQ_ERR_ALIGN : PQ_ERR_INVALID_ARG;
-  if (!ctx || !x || (!CALIB && (!s_a_in || !xq)) || (CALIB && !s_a_out)) return PQ_ERR_INVALID_ARG;
+  if (!ctx || !x || (!CALIB && ((!s_a_in && !s_a_out) || !xq)) || (CALIB && !s_a_out)) return PQ_ERR_INVALID_ARG;
   if (M < 0 || K <= 0 || ldx < K || row_begin < 0 || had_block < 0) return PQ_ERR_INVALID_ARG;
   if (K % 128 != 0) return PQ_ERR_SHAPE;
   if (had_block != 0) {
@@ -827,6 +848,18 @@ extern "C" pq_status pq_dyn_act_scale(pq_ctx* ctx, const void* x, int64_t M, int
 extern "C" pq_status pq_hadamard_quant_act_rows(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx,
                                                 int had_block, int64_t row_begin, const float* s_tok, uint8_t* xq,
                                                 void* stream) {
+  return dispatch<false, 4, true>(ctx, x, M, K, ldx, had_block, row_begin, s_tok, xq, nullptr, stream);
+}
+
+// Both in one call. When a row is one transform block of 2048 or more elements the step is formed and used in the
+// same pass over the activations (one launch); else the two passes above.
+extern "C" pq_status pq_dyn_hadamard_quant_act(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                               int64_t row_begin, float clip, float* s_tok, uint8_t* xq, void* stream) {
+  if (!(clip > 0.0f) || !(clip <= 1.0f) || !s_tok) return PQ_ERR_INVALID_ARG;
+  if (had_block == K && had_block >= 2048)
+    return dispatch<false, 4, true>(ctx, x, M, K, ldx, had_block, row_begin, nullptr, xq, s_tok, stream, clip);
+  pq_status rc = dispatch<true, 4, true>(ctx, x, M, K, ldx, had_block, row_begin, nullptr, nullptr, s_tok, stream, clip);
+  if (rc != PQ_OK) return rc;
   return dispatch<false, 4, true>(ctx, x, M, K, ldx, had_block, row_begin, s_tok, xq, nullptr, stream);
 }
 

@@ -57,6 +57,33 @@ def test_dynamic_scale_and_codes_match_oracle(ctx, M, K, B, row_begin, clip):
         assert np.all(np.abs(orc.unpack_int4(got[live])).max(axis=1) == 7)
 
 
+@pytest.mark.parametrize("M,K,B,row_begin,clip", [(37, 4096, 4096, 4, 1.0), (70, 2048, 2048, 0, 0.9), (5, 8192, 8192, 1, 0.75),
+                                                 (19, 14336, 2048, 0, 0.9), (70, 256, 128, 1, 1.0), (300, 4096, 4096, 4, 1.0)])
+def test_one_call_dynamic_quantizer_gives_the_bits_of_the_two_calls(ctx, M, K, B, row_begin, clip):
+    """pq_dyn_hadamard_quant_act: one pass over the activations when a row is one wide transform block, the two
+    passes otherwise; steps and codes equal those of pq_dyn_act_scale + pq_hadamard_quant_act_rows bit for bit
+    (which the test above compares with the oracle), prefix rows untouched, an all-zero token included."""
+    x = inputs.activations(M, K, seed=0, n_prefix=row_begin)
+    x[M - 1] = 0
+    xd = x.cuda()
+    s_two = torch.full((M,), -5.0, device="cuda")
+    ctx.dyn_act_scale(xd, B, clip, row_begin, out=s_two)
+    q_two = torch.full((M, K // 2), 0x5A, dtype=torch.uint8, device="cuda")
+    ctx.hadamard_quant_act_rows(xd, B, s_two, row_begin, out=q_two)
+    s_one = torch.full((M,), -5.0, device="cuda")
+    q_one = torch.full((M, K // 2), 0x5A, dtype=torch.uint8, device="cuda")
+    ctx.dyn_hadamard_quant_act(xd, B, clip, row_begin, s_tok=s_one, out=q_one)
+    ctx.check()
+    assert torch.equal(s_one, s_two) and torch.equal(q_one, q_two)
+    assert float(s_one[M - 1]) == 0.0 and int(q_one[M - 1].max()) == 0
+    # and against the oracle's steps directly
+    s_ref = orc.dyn_act_scale(inputs.bits(x), B, clip, row_begin)
+    live = np.arange(M) >= row_begin
+    live[M - 1] = False
+    s = to_np(s_one)
+    assert np.all(np.abs(s[live] - s_ref[live]) <= 2e-6 * s_ref[live])
+
+
 def test_dynamic_path_is_scale_free_per_token(ctx):
     M, K = 24, 4096
     x = inputs.activations(M, K, seed=2)
