@@ -161,8 +161,8 @@ pq_status pq_w4a8_gemm(pq_ctx* ctx, const int8_t* xq8, const uint8_t* wq, const 
  *     xq[t, :] = pack(clamp(rne(y[t, :] / s_tok[t]), -8, 7))   pq_hadamard_quant_act_rows (second pass)
  *     out[t, n] = bf16(acc[t, n] * s_tok[t] * s_w[n])          pq_w4a4_gemm_rows
  *   s_tok  f32 [M] on the device; rows below row_begin are neither read nor written; an all-zero row
- *   gets step 0 and codes 0. Every other argument as in the static calls. The GEMM uses the
- *   tensor-core kernel with the token operand in shared memory for every K (M - row_begin > 16). */
+ *   gets step 0 and codes 0. Every other argument as in the static calls; the GEMM picks its kernel as
+ *   pq_w4a4_gemm does. */
 pq_status pq_dyn_act_scale(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
                            int64_t row_begin, float clip, float* s_tok, void* stream);
 /* The first and the second pass in one call (same passage): s_tok [M] and xq [M, K/2] are both outputs, with the bits

@@ -6,7 +6,8 @@ pq_status pq_gemm_pair_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq,
                               void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st,
                               bool a8, const float* s_row, const int32_t* zp, const int32_t* wsum);
 pq_status pq_gemm_pair_ts_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a, const float* s_w,
-                                 void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st);
+                                 void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t* acc_dbg, cudaStream_t st,
+                                 const float* s_row, const int32_t* zp, const int32_t* wsum);
 pq_status pq_gemm_stream_launch(pq_ctx* ctx, const uint8_t* xq, const uint8_t* wq, const float* s_a,
                                 const float* s_w, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K,
                                 int32_t* acc_dbg, cudaStream_t st, bool per_token, bool a8, const int32_t* zp,
@@ -33,11 +34,11 @@ extern "C" pq_status pq_w4a4_gemm(pq_ctx* ctx, const uint8_t* xq, const uint8_t*
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (K == 0) return PQ_ERR_SHAPE;
   if (m <= 16) return pq_gemm_stream_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st, false, false, nullptr, nullptr);
-  // Two CTA-pair kernels: with the token operand in shared memory the accumulator is double-buffered
+  // Two CTA-pair kernels (every 4-bit setting takes the same choice): with the token operand in shared memory the accumulator is double-buffered
   // and the epilogue is free, which wins for short K; with the token operand in tensor memory the
   // expansion costs a third less shared-memory traffic, which wins once a tile's K loop is long enough
   // to hide the single accumulator's epilogue (measured crossover near K = 8192).
-  if (K >= 8192) return pq_gemm_pair_ts_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st);
+  if (K >= 8192) return pq_gemm_pair_ts_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st, nullptr, nullptr, nullptr);
   return pq_gemm_pair_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st, false, nullptr, nullptr, nullptr);
 }
 
@@ -81,6 +82,7 @@ extern "C" pq_status pq_w4a4_gemm_rows(pq_ctx* ctx, const uint8_t* xq, const uin
   int32_t* dbg0 = acc_dbg ? acc_dbg + row_begin * N : nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (m <= 16) return pq_gemm_stream_launch(ctx, xq0, wq, s0, s_w, out0, ldo, m, N, K, dbg0, st, true, false, nullptr, nullptr);
+  if (K >= 8192) return pq_gemm_pair_ts_launch(ctx, xq0, wq, nullptr, s_w, out0, ldo, m, N, K, dbg0, st, s0, nullptr, nullptr);
   return pq_gemm_pair_launch(ctx, xq0, wq, nullptr, s_w, out0, ldo, m, N, K, dbg0, st, false, s0, nullptr, nullptr);
 }
 
@@ -103,5 +105,6 @@ extern "C" pq_status pq_w4a4_gemm_asym(pq_ctx* ctx, const uint8_t* xq, const uin
   int32_t* dbg0 = acc_dbg ? acc_dbg + row_begin * N : nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (m <= 16) return pq_gemm_stream_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st, false, false, z_a, wsum);
+  if (K >= 8192) return pq_gemm_pair_ts_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st, nullptr, z_a, wsum);
   return pq_gemm_pair_launch(ctx, xq0, wq, s_a, s_w, out0, ldo, m, N, K, dbg0, st, false, nullptr, z_a, wsum);
 }

@@ -115,7 +115,7 @@ def _gemm_asym_case(ctx, M, N, K, z, seed, row_begin=0):
 
 
 @pytest.mark.parametrize("M,N,K,z", [(1, 256, 128, 3), (9, 96, 160, 15), (16, 1024, 4096, 0), (17, 96, 160, 8), (257, 300, 1184, 5),
-                                     (300, 520, 4096, 11), (130, 264, 14336, 2)])
+                                     (300, 520, 4096, 11), (130, 264, 14336, 2), (600, 520, 8192, 13)])
 def test_gemm_asym_bit_exact(ctx, M, N, K, z):
     _gemm_asym_case(ctx, M, N, K, z, seed=M + N + K)
 

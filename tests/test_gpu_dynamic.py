@@ -116,7 +116,7 @@ def _gemm_rows_case(ctx, M, N, K, seed, row_begin=0):
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 256, 128), (9, 96, 160), (16, 1024, 4096), (17, 96, 160), (257, 300, 1184), (300, 520, 4096),
-                                   (130, 264, 14336)])
+                                   (130, 264, 14336), (600, 520, 8192)])
 def test_gemm_rows_bit_exact_accumulators_and_per_token_epilogue(ctx, M, N, K):
     _gemm_rows_case(ctx, M, N, K, seed=M + N + K)
 
