@@ -77,8 +77,10 @@ def recorded_traffic():
         if ":" in line and not line.lstrip().startswith("#"):
             k, v = line.split(":", 1)
             kv[k.strip()] = v.strip()
-    src = os.path.join(ROOT, kv.get("source", ""))
-    if not os.path.isfile(src) or sha256_of(src) != kv.get("source_sha256"):
+    # the kernel's sources (comma-separated) and the SHA-256 of each, in the same order
+    srcs = [os.path.join(ROOT, t.strip()) for t in kv.get("source", "").split(",") if t.strip()]
+    shas = [t.strip() for t in kv.get("source_sha256", "").split(",") if t.strip()]
+    if not srcs or len(srcs) != len(shas) or any(not os.path.isfile(f) or sha256_of(f) != h for f, h in zip(srcs, shas)):
         return None, "kernel source changed since the ncu capture"
     return int(kv["dram_bytes_per_launch"]), f"ncu capture of the {kv.get('launch', '?')} launch (not measured by this run)"
 
