@@ -379,6 +379,7 @@ def run_gpu(args):
             sections["config0_single_linear_256x4096x4096"] = section_config0(ctx, device, peaks)
             sections["w4a8_prefill_linear_set"] = section_w4a8(ctx, device, peaks, acts, wqs, sws)
             sections["w4a4_dynamic_per_token_linear_set"] = section_dynamic(ctx, device, peaks, acts, wqs, sws)
+            sections["w4a4_byte_codes_linear_set"] = section_w4a4_byte_codes(ctx, device, peaks, acts, scales, wqs, sws)
             sections["decode_gemm"] = section_decode_gemm(ctx, device, peaks)
             sections["decode_attention"] = section_decode_attention(ctx, device, peaks)
             sections["block_llama3_70b_prefill4096"] = section_block(ctx, device, peaks)
@@ -645,6 +646,38 @@ def section_w4a8(ctx, device, peaks, acts, wqs, sws):
             "per_launch": {k: {"ms": round(statistics.mean(v), 4),
                                "tops": round(2.0 * m_rows * next(n * kk for nm, n, kk, _, _ in L if nm == k) / (statistics.mean(v) * 1e-3) / 1e12, 1)}
                            for k, v in per.items()}}
+
+
+def section_w4a4_byte_codes(ctx, device, peaks, acts, scales, wqs, sws):
+    """The linear set of configs[1] with the 4-bit activation codes stored one per byte (pq_hadamard_quant_act_c8 +
+    pq_w4a8_gemm): W4A4's codes, sums and outputs, without the expansion of the token operand in the GEMM and with
+    twice the activation bytes. Beside the packed path of the scope table, which the headline measures."""
+    import torch
+
+    L = linear_launches()
+    m_rows = M_TOKENS - N_PREFIX
+    xqs = [torch.zeros((M_TOKENS, K), dtype=torch.int8, device=device) for _, _, K, _, _ in L]
+    outs = [torch.zeros((M_TOKENS, N), dtype=torch.bfloat16, device=device) for _, N, _, _, _ in L]
+
+    def step():
+        for i, (name, N, K, had, inp) in enumerate(L):
+            ctx.hadamard_quant_act_c8(acts[i], had, scales[i], N_PREFIX, out=xqs[i])
+            ctx.w4a8_gemm(xqs[i], wqs[i], scales[i], sws[i], N_PREFIX, out=outs[i])
+
+    steps = 50
+    for _ in range(5):
+        step()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        step()
+    t1.record()
+    torch.cuda.synchronize()
+    ctx.check()
+    ms = t0.elapsed_time(t1) / steps
+    return {"ms_per_step": round(ms, 4), "TOPS": round(step_ops(m_rows) / (ms * 1e-3) / 1e12, 1),
+            "note": "same codes, sums and outputs as the packed path (asserted by the GPU tests); activations take M x K bytes instead of M x K / 2"}
 
 
 def section_dynamic(ctx, device, peaks, acts, wqs, sws):

@@ -150,6 +150,12 @@ pq_status pq_hadamard_quant_act8(pq_ctx* ctx, const void* x, int64_t M, int64_t 
                                  int64_t row_begin, const float* s_a, int8_t* xq8, void* stream);
 pq_status pq_calib_act_scale8(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
                               int64_t row_begin, float* s_a, void* stream);
+/* The 4-bit quantizer of pq_hadamard_quant_act (same step s_a = max|y| / 7, same codes in [-8, 7], bit for bit) with
+ * the codes stored one per byte in the layout of pq_hadamard_quant_act8: xq8 s8 [M, K], 16-byte aligned. Given to
+ * pq_w4a8_gemm with that s_a, the sums and outputs are those of pq_w4a4_gemm on the packed codes, and the prefill
+ * kernel skips the expansion of the token operand; the activation tensor is twice as large. */
+pq_status pq_hadamard_quant_act_c8(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,
+                                   int64_t row_begin, const float* s_a, int8_t* xq8, void* stream);
 pq_status pq_w4a8_gemm(pq_ctx* ctx, const int8_t* xq8, const uint8_t* wq, const float* s_a, const float* s_w, void* out,
                        int64_t ldo, int64_t M, int64_t N, int64_t K, int64_t row_begin, int32_t* acc_dbg, void* stream);
 

@@ -25,7 +25,7 @@ EXPORTS = [
     "pq_calib_act_scale", "pq_w4a4_gemm_workspace_bytes", "pq_w4a4_gemm", "pq_kv4_append",
     "pq_decode_attn_workspace_bytes", "pq_decode_attn_kv4_prefix", "pq_decode_attn_kv4_prefix_noalloc",
     "pq_rmsnorm", "pq_rope", "pq_silu_mul", "pq_residual_add", "pq_prefill_attn_kv4_prefix", "pq_kv4_append_strided", "pq_calib_kv_scale",
-    "pq_hadamard_quant_act8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
+    "pq_hadamard_quant_act8", "pq_hadamard_quant_act_c8", "pq_calib_act_scale8", "pq_w4a8_gemm", "pq_rope_rotate",
     "pq_dyn_act_scale", "pq_dyn_hadamard_quant_act", "pq_hadamard_quant_act_rows", "pq_w4a4_gemm_rows", "pq_outlier_tokens",
     "pq_calib_act_asym", "pq_hadamard_quant_act_asym", "pq_weight_code_sums", "pq_w4a4_gemm_asym",
     "pq_swiglu_hadamard_quant_act", "pq_kv4_append_decode_attn", "pq_set_wait_limit", "pq_probe_i8_mma", "pq_grid_search_act_asym", "pq_grid_search_clip_dyn", "pq_rmsnorm_hadamard_quant_act", "pq_rope_kv4_append", "pq_selftest_wait",
@@ -91,6 +91,7 @@ def load_library() -> ctypes.CDLL:
     lib.pq_silu_mul.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p]
     lib.pq_residual_add.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p]
     lib.pq_hadamard_quant_act8.argtypes = lib.pq_hadamard_quant_act.argtypes
+    lib.pq_hadamard_quant_act_c8.argtypes = lib.pq_hadamard_quant_act.argtypes
     lib.pq_calib_act_scale8.argtypes = lib.pq_calib_act_scale.argtypes
     lib.pq_w4a8_gemm.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int64,
                                  c_int64, c_void_p, c_void_p]
@@ -458,6 +459,19 @@ class Context:
         _dev(out, torch.int8, "out")
         _ok(self.lib.pq_hadamard_quant_act8(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, _ptr(s_a), _ptr(out),
                                             _stream()), "pq_hadamard_quant_act8")
+        return out
+
+    def hadamard_quant_act_c8(self, x: torch.Tensor, had_block: int, s_a: torch.Tensor, row_begin: int = 0,
+                              out: torch.Tensor | None = None):
+        """The 4-bit codes of hadamard_quant_act, one per byte (operand of w4a8_gemm)."""
+        _dev(x, torch.bfloat16, "x"), _dev(s_a, torch.float32, "s_a")
+        M, K = x.shape
+        assert x.stride(1) == 1
+        if out is None:
+            out = torch.zeros((M, K), dtype=torch.int8, device=x.device)
+        _dev(out, torch.int8, "out")
+        _ok(self.lib.pq_hadamard_quant_act_c8(self.h, _ptr(x), M, K, x.stride(0), had_block, row_begin, _ptr(s_a), _ptr(out),
+                                              _stream()), "pq_hadamard_quant_act_c8")
         return out
 
     def w4a8_gemm(self, xq8: torch.Tensor, wq: torch.Tensor, s_a: torch.Tensor, s_w: torch.Tensor, row_begin: int = 0,

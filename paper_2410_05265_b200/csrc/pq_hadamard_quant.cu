@@ -284,6 +284,8 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
       // y * inv + 1.5 * 2^23: the fp32 addition rounds half to even and leaves the integer in the low
       // mantissa bits; clamped as an integer, the low byte is the code as an s8.
       const float2 inv2 = make_float2(inv, inv), magic2 = make_float2(12582912.0f, 12582912.0f);
+      // byte stores with a narrower code range (4-bit codes, one per byte): the caller's largest code in n_cand
+      const int qmax = (BITS == 8 && n_cand > 0) ? n_cand : QMAX;
       uint32_t pw[16];  // word wd: codes of v[4wd .. 4wd+3], one nibble per byte
 #pragma unroll
       for (int wd = 0; wd < 8; ++wd) {
@@ -291,8 +293,8 @@ __global__ void __launch_bounds__(HQ_THREADS, HQ_CTAS_PER_SM)
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
           const float2 tq = __ffma2_rn(W[4 * wd + b], inv2, magic2);
-          lo[b] = max(min(__float_as_int(tq.x) + zp, 0x4B400000 + QMAX), 0x4B400000 - QMAX - 1);
-          hi[b] = max(min(__float_as_int(tq.y) + zp, 0x4B400000 + QMAX), 0x4B400000 - QMAX - 1);
+          lo[b] = max(min(__float_as_int(tq.x) + zp, 0x4B400000 + qmax), 0x4B400000 - qmax - 1);
+          hi[b] = max(min(__float_as_int(tq.y) + zp, 0x4B400000 + qmax), 0x4B400000 - qmax - 1);
         }
         pw[wd] = __byte_perm(__byte_perm(lo[0], lo[1], 0x0040), __byte_perm(lo[2], lo[3], 0x0040), 0x5410);
         pw[wd + 8] = __byte_perm(__byte_perm(hi[0], hi[1], 0x0040), __byte_perm(hi[2], hi[3], 0x0040), 0x5410);
@@ -660,8 +662,10 @@ __global__ void __launch_bounds__(HQ_THREADS, HQW_CTAS_PER_SM)
       // With a zero point (odd z would move ties) the rounding comes first: y * inv + (1.5 * 2^23 + 8), the integer
       // z - 8 added to the bit pattern, and an integer clamp.
       constexpr int BASE = 0x4B400000;
-      constexpr float U = static_cast<float>(2 * QMAX + 1);
-      const float invU = __fdiv_rn(inv, U), offU = __fdiv_rn(static_cast<float>(QMAX + 1), U);
+      // byte stores with a narrower code range (4-bit codes, one per byte): the caller's largest code in n_cand
+      const int qmax = (BITS == 8 && n_cand > 0) ? n_cand : QMAX;
+      const float U = static_cast<float>(2 * qmax + 1);
+      const float invU = __fdiv_rn(inv, U), offU = __fdiv_rn(static_cast<float>(qmax + 1), U);
       auto codes = [&](float2 y) -> uint2 {  // bit patterns whose low BITS bits are the two offset codes
         if (ZP) {
           const float2 tq = __ffma2_rn(y, make_float2(inv, inv), make_float2(12582920.0f, 12582920.0f));
@@ -703,7 +707,9 @@ __global__ void __launch_bounds__(HQ_THREADS, HQW_CTAS_PER_SM)
 #pragma unroll
         for (int wd = 0; wd < 16; ++wd) {
           const uint2 c0 = codes(W[2 * wd]), c1 = codes(W[2 * wd + 1]);
-          fin[wd] = __byte_perm(__byte_perm(c0.x, c0.y, 0x0040), __byte_perm(c1.x, c1.y, 0x0040), 0x5410) ^ 0x80808080u;
+          // offset codes u = n + qmax + 1 -> signed bytes n (for the full range this is u ^ 0x80)
+          fin[wd] = __vsub4(__byte_perm(__byte_perm(c0.x, c0.y, 0x0040), __byte_perm(c1.x, c1.y, 0x0040), 0x5410),
+                            static_cast<uint32_t>(qmax + 1) * 0x01010101u);
         }
         if (active) {
           store32(xq + row * K + e0, fin);
@@ -831,6 +837,14 @@ extern "C" pq_status pq_hadamard_quant_act8(pq_ctx* ctx, const void* x, int64_t 
                                             int had_block, int64_t row_begin, const float* s_a, int8_t* xq8,
                                             void* stream) {
   return dispatch<false, 8>(ctx, x, M, K, ldx, had_block, row_begin, s_a, reinterpret_cast<uint8_t*>(xq8), nullptr, stream);
+}
+
+// 4-bit codes stored one per byte (the range of pq_hadamard_quant_act, the layout of pq_hadamard_quant_act8).
+extern "C" pq_status pq_hadamard_quant_act_c8(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx,
+                                              int had_block, int64_t row_begin, const float* s_a, int8_t* xq8,
+                                              void* stream) {
+  return dispatch<false, 8>(ctx, x, M, K, ldx, had_block, row_begin, s_a, reinterpret_cast<uint8_t*>(xq8), nullptr, stream, 1.0f,
+                            nullptr, nullptr, 7);
 }
 
 extern "C" pq_status pq_calib_act_scale8(pq_ctx* ctx, const void* x, int64_t M, int64_t K, int64_t ldx, int had_block,

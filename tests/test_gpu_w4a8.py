@@ -106,6 +106,29 @@ def test_w4a8_gemm_decode_shapes_bit_exact(ctx, M, N, K):
         _gemm8_case(ctx, M + 4, N, K, seed=N, row_begin=4)
 
 
+@pytest.mark.parametrize("M,K,B,row_begin,N", [(70, 6144, 2048, 4, 264), (33, 4096, 4096, 0, 96), (9, 8192, 8192, 1, 40),
+                                               (37, 768, 256, 0, 64), (21, 384, 0, 2, 48), (300, 4096, 4096, 4, 520)])
+def test_four_bit_codes_one_per_byte_give_the_packed_path_bit_for_bit(ctx, M, K, B, row_begin, N):
+    """pq_hadamard_quant_act_c8: the codes of pq_hadamard_quant_act (which the parity tests compare with the oracle),
+    unpacked; pq_w4a8_gemm on them returns the sums and outputs of pq_w4a4_gemm on the packed codes."""
+    x = inputs.activations(M, K, seed=0, n_prefix=row_begin).cuda()
+    s_a = ctx.calib_act_scale(x, B, row_begin)
+    packed = ctx.hadamard_quant_act(x, B, s_a, row_begin)
+    bytes8 = torch.full((M, K), 0x5A, dtype=torch.int8, device="cuda")
+    ctx.hadamard_quant_act_c8(x, B, s_a, row_begin, out=bytes8)
+    ctx.check()
+    assert np.all(to_np(bytes8)[:row_begin] == 0x5A), "prefix rows must not be written"
+    assert np.array_equal(to_np(bytes8)[row_begin:], orc.unpack_int4(to_np(packed))[row_begin:])
+    wq = dev(rand_codes(np.random.default_rng(M + N), N, K))
+    s_w = torch.full((N,), 0.003, device="cuda")
+    acc4 = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    acc8 = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    out4 = ctx.w4a4_gemm(packed, wq, s_a, s_w, row_begin, acc_dbg=acc4)
+    out8 = ctx.w4a8_gemm(bytes8, wq, s_a, s_w, row_begin, acc_dbg=acc8)
+    ctx.check()
+    assert torch.equal(acc4[row_begin:], acc8[row_begin:]) and torch.equal(out4[row_begin:], out8[row_begin:])
+
+
 def test_w4a8_gemm_many_tiles_and_row_begin(ctx):
     _gemm8_case(ctx, 1024, 5120, 256, seed=5)       # 80 tiles on 74 CTA pairs: some pairs take a second tile
     _gemm8_case(ctx, 260, 256, 256, seed=11, row_begin=4)
